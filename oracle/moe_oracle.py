@@ -1,0 +1,246 @@
+"""Plain fp64 CPU oracle for the MoE expert-FFN hot path (forward and backward).
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, obviously-correct statement of what the
+CUDA library computes.  It shares no code with the CUDA path and must never be imported by the
+product package; only the tests, the smoke check and the CPU-baseline leg of the benchmark call it.
+
+Every function takes numpy arrays (any float dtype holding the exact input values, e.g. float32
+arrays whose values are bf16-representable), converts them to float64 and evaluates the plain
+mathematical definition with no intermediate rounding.  A library matmul / stable sort is used as
+a step; there is no blocking, fusion or reordering beyond the per-expert loop the packed layout
+itself implies.
+
+Notation: T tokens, H hidden, I per-expert intermediate, E experts, K = top-k, R = T*K routed rows.
+Pair id p = t*K + k (token-major).  Rows of the packed buffers are ordered by expert; the
+per-expert row ranges are [offsets[e], offsets[e+1]).
+
+What each step follows:
+  * packed-by-expert buffer + cumulative row counts: the paper's appendix on the dW1 kernel
+    ("What the kernel computes"); its inclusive cumulative-sum vector equals offsets[1:].
+  * weight gradient of the first projection, dW1_e = X_e^T G_e with G_e the gradient of the
+    pre-activation: the paper's section "Production Validation: VeOmni MoE" and the same appendix.
+  * an expert with no rows gets an all-zero weight-gradient tile: same appendix (routing model
+    paragraph, empty experts K_e = 0).
+  * everything else (SwiGLU, down projection, weighted combine, the remaining gradients): the
+    standard MoE FFN algebra and the chain rule.
+
+Pins (tests/test_oracle_*.py): brute-force counting sort, stable-sort library routine, dense
+SwiGLU MLP special cases evaluated with an independent library (torch, fp64), per-token loop,
+torch.autograd on a per-token formulation, central finite differences, identities of
+permute/unpermute, empty-expert zeros.  No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+def _f64(a):
+    return np.asarray(a).astype(F64, copy=False)
+
+
+# --------------------------------------------------------------------------------------------
+# O1  route-permute: stable sort of (token, slot) pairs by expert
+# --------------------------------------------------------------------------------------------
+def permute_indices(topk_idx, E):
+    """counts[E], offsets[E+1] (exclusive prefix, offsets[E]=R), row_to_pair[R], pair_to_row[R].
+
+    row_to_pair lists the pair ids p = t*K+k sorted by (expert(p), p): a stable sort by expert.
+    All int32.  The paper's inclusive cumulative-sum vector is offsets[1:].
+    """
+    idx = np.asarray(topk_idx)
+    e_of_p = idx.reshape(-1).astype(np.int64)
+    R = e_of_p.size
+    if R and (e_of_p.min() < 0 or e_of_p.max() >= E):
+        raise ValueError("expert id out of range")
+    counts = np.bincount(e_of_p, minlength=E).astype(np.int64)
+    offsets = np.zeros(E + 1, dtype=np.int64)
+    offsets[1:] = np.cumsum(counts)
+    row_to_pair = np.argsort(e_of_p, kind="stable")
+    pair_to_row = np.empty(R, dtype=np.int64)
+    pair_to_row[row_to_pair] = np.arange(R, dtype=np.int64)
+    return (counts.astype(np.int32), offsets.astype(np.int32),
+            row_to_pair.astype(np.int32), pair_to_row.astype(np.int32))
+
+
+def permute(X, topk_idx, E):
+    """X_perm[r,:] = X[row_to_pair[r] // K, :] plus the index arrays of permute_indices."""
+    X = _f64(X)
+    K = np.asarray(topk_idx).shape[1]
+    counts, offsets, row_to_pair, pair_to_row = permute_indices(topk_idx, E)
+    X_perm = X[row_to_pair.astype(np.int64) // K, :]
+    return X_perm, counts, offsets, row_to_pair, pair_to_row
+
+
+# --------------------------------------------------------------------------------------------
+# O2  grouped GEMM gate/up + SwiGLU
+# --------------------------------------------------------------------------------------------
+def gateup_swiglu(X_perm, W_gate, W_up, offsets):
+    """For rows r of expert e: g = Xp[r] @ Wg[e], u = Xp[r] @ Wu[e]; Hact = silu(g)*u.
+
+    Returns Hact [R,I] and the saved pre-activations GU [R,2I] = [g | u].
+    silu(g) = g / (1 + exp(-g)).
+    """
+    Xp = _f64(X_perm)
+    E, H, I = W_gate.shape
+    R = Xp.shape[0]
+    Hact = np.zeros((R, I), F64)
+    GU = np.zeros((R, 2 * I), F64)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        if r1 == r0:
+            continue
+        g = Xp[r0:r1] @ _f64(W_gate[e])
+        u = Xp[r0:r1] @ _f64(W_up[e])
+        GU[r0:r1, :I] = g
+        GU[r0:r1, I:] = u
+        Hact[r0:r1] = g / (1.0 + np.exp(-g)) * u
+    return Hact, GU
+
+
+# --------------------------------------------------------------------------------------------
+# O3  grouped GEMM down
+# --------------------------------------------------------------------------------------------
+def down(H_act, W_down, offsets):
+    """Yp[r,:] = Hact[r,:] @ Wd[e] for rows r of expert e."""
+    Hact = _f64(H_act)
+    E, I, H = W_down.shape
+    Yp = np.zeros((Hact.shape[0], H), F64)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        if r1 > r0:
+            Yp[r0:r1] = Hact[r0:r1] @ _f64(W_down[e])
+    return Yp
+
+
+# --------------------------------------------------------------------------------------------
+# O4  unpermute-combine
+# --------------------------------------------------------------------------------------------
+def unpermute_combine(Y_perm, topk_w, pair_to_row):
+    """Y[t,:] = sum_k w[t,k] * Yp[pair_to_row[t*K+k], :]."""
+    Yp = _f64(Y_perm)
+    w = _f64(topk_w)
+    T, K = w.shape
+    rows = np.asarray(pair_to_row).astype(np.int64).reshape(T, K)
+    Y = np.zeros((T, Yp.shape[1]), F64)
+    for k in range(K):
+        Y += w[:, k:k + 1] * Yp[rows[:, k]]
+    return Y
+
+
+# --------------------------------------------------------------------------------------------
+# O5  unpermute-combine backward
+# --------------------------------------------------------------------------------------------
+def unpermute_combine_bwd(dY, Y_perm, topk_w, pair_to_row):
+    """dYp[pair_to_row[p],:] = w(p) * dY[t(p),:];  dw[t,k] = <dY[t,:], Yp[pair_to_row[t*K+k],:]>."""
+    dY = _f64(dY)
+    Yp = _f64(Y_perm)
+    w = _f64(topk_w)
+    T, K = w.shape
+    rows = np.asarray(pair_to_row).astype(np.int64).reshape(T, K)
+    dYp = np.zeros((T * K, dY.shape[1]), F64)
+    dw = np.zeros((T, K), F64)
+    for k in range(K):
+        dYp[rows[:, k]] = w[:, k:k + 1] * dY
+        dw[:, k] = np.sum(dY * Yp[rows[:, k]], axis=1)
+    return dYp, dw
+
+
+# --------------------------------------------------------------------------------------------
+# O6  down backward: dgrad + wgrad
+# --------------------------------------------------------------------------------------------
+def down_bwd(dY_perm, H_act, W_down, offsets):
+    """dHact[r,:] = dYp[r,:] @ Wd[e]^T;  dWd[e] = Hact_e^T @ dYp_e  (zero for an empty expert)."""
+    dYp = _f64(dY_perm)
+    Hact = _f64(H_act)
+    E, I, H = W_down.shape
+    dHact = np.zeros((dYp.shape[0], I), F64)
+    dWd = np.zeros((E, I, H), F64)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        if r1 == r0:
+            continue
+        dHact[r0:r1] = dYp[r0:r1] @ _f64(W_down[e]).T
+        dWd[e] = Hact[r0:r1].T @ dYp[r0:r1]
+    return dHact, dWd
+
+
+# --------------------------------------------------------------------------------------------
+# O7  SwiGLU backward + gate/up backward: dgrad + wgrad (the paper's dW1)
+# --------------------------------------------------------------------------------------------
+def swiglu_bwd(dH_act, GU):
+    """dGU = [dg | du] with s = sigmoid(g): dg = dHact*u*s*(1+g*(1-s)), du = dHact*g*s."""
+    dHact = _f64(dH_act)
+    GU = _f64(GU)
+    I = dHact.shape[1]
+    g, u = GU[:, :I], GU[:, I:]
+    s = 1.0 / (1.0 + np.exp(-g))
+    dg = dHact * u * s * (1.0 + g * (1.0 - s))
+    du = dHact * g * s
+    return np.concatenate([dg, du], axis=1)
+
+
+def gateup_bwd_from_dgu(dGU, X_perm, W_gate, W_up, offsets):
+    """dXp[r,:] = dg[r,:] @ Wg[e]^T + du[r,:] @ Wu[e]^T;  dWg[e] = Xp_e^T @ dg_e;  dWu likewise."""
+    dGU = _f64(dGU)
+    Xp = _f64(X_perm)
+    E, H, I = W_gate.shape
+    dXp = np.zeros((Xp.shape[0], H), F64)
+    dWg = np.zeros((E, H, I), F64)
+    dWu = np.zeros((E, H, I), F64)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        if r1 == r0:
+            continue
+        dg, du = dGU[r0:r1, :I], dGU[r0:r1, I:]
+        dXp[r0:r1] = dg @ _f64(W_gate[e]).T + du @ _f64(W_up[e]).T
+        dWg[e] = Xp[r0:r1].T @ dg
+        dWu[e] = Xp[r0:r1].T @ du
+    return dXp, dWg, dWu
+
+
+def gateup_swiglu_bwd(dH_act, GU, X_perm, W_gate, W_up, offsets):
+    """Returns dGU [R,2I], dXp [R,H], dWg, dWu [E,H,I]."""
+    dGU = swiglu_bwd(dH_act, GU)
+    dXp, dWg, dWu = gateup_bwd_from_dgu(dGU, X_perm, W_gate, W_up, offsets)
+    return dGU, dXp, dWg, dWu
+
+
+# --------------------------------------------------------------------------------------------
+# O8  permute backward
+# --------------------------------------------------------------------------------------------
+def permute_bwd(dX_perm, pair_to_row, T, K):
+    """dX[t,:] = sum_k dXp[pair_to_row[t*K+k], :]."""
+    dXp = _f64(dX_perm)
+    rows = np.asarray(pair_to_row).astype(np.int64).reshape(T, K)
+    dX = np.zeros((T, dXp.shape[1]), F64)
+    for k in range(K):
+        dX += dXp[rows[:, k]]
+    return dX
+
+
+# --------------------------------------------------------------------------------------------
+# The whole layer, chained in fp64 with no intermediate rounding ("exact" mode)
+# --------------------------------------------------------------------------------------------
+def layer_fwd(X, topk_idx, topk_w, W_gate, W_up, W_down):
+    E = W_gate.shape[0]
+    Xp, counts, offsets, row_to_pair, pair_to_row = permute(X, topk_idx, E)
+    Hact, GU = gateup_swiglu(Xp, W_gate, W_up, offsets)
+    Yp = down(Hact, W_down, offsets)
+    Y = unpermute_combine(Yp, topk_w, pair_to_row)
+    return dict(X_perm=Xp, counts=counts, offsets=offsets, row_to_pair=row_to_pair,
+                pair_to_row=pair_to_row, H_act=Hact, GU=GU, Y_perm=Yp, Y=Y)
+
+
+def layer_fwd_bwd(X, topk_idx, topk_w, W_gate, W_up, W_down, dY):
+    """Forward then backward of L = sum(dY * Y) with the routing indices frozen."""
+    f = layer_fwd(X, topk_idx, topk_w, W_gate, W_up, W_down)
+    T, K = np.asarray(topk_idx).shape
+    dYp, dw = unpermute_combine_bwd(dY, f["Y_perm"], topk_w, f["pair_to_row"])
+    dHact, dWd = down_bwd(dYp, f["H_act"], W_down, f["offsets"])
+    dGU, dXp, dWg, dWu = gateup_swiglu_bwd(dHact, f["GU"], f["X_perm"], W_gate, W_up, f["offsets"])
+    dX = permute_bwd(dXp, f["pair_to_row"], T, K)
+    f.update(dY_perm=dYp, dtopk_w=dw, dH_act=dHact, dW_down=dWd, dGU=dGU, dX_perm=dXp,
+             dW_gate=dWg, dW_up=dWu, dX=dX)
+    return f
