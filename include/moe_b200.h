@@ -1,0 +1,173 @@
+/*
+ * moe_b200.h -- C ABI of libmoe_b200.so: the MoE expert FFN, forward and backward, on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The layer, for T tokens of width H routed to K of E experts with intermediate width I:
+ *
+ *   route-permute            stable sort of the (token, slot) pairs by expert into a packed,
+ *                            expert-ordered row buffer with per-expert offsets
+ *   grouped GEMM gate/up     per expert g = Xp.Wg[e], u = Xp.Wu[e]; Hact = silu(g) * u
+ *   grouped GEMM down        per expert Yp = Hact.Wd[e]
+ *   unpermute-combine        Y[t] = sum_k w[t,k] * Yp[row(t,k)]
+ *
+ * and the matching backward calls (dgrad and wgrad grouped GEMMs).  The packed-by-expert row
+ * buffer with cumulative row counts is the layout the paper describes in its appendix on the
+ * dW1 weight-gradient kernel ("What the kernel computes"); `offsets[1..E]` is that appendix's
+ * inclusive cumulative-sum vector.  The weight gradient of the first projection,
+ * dW1_e = X_e^T G_e over a ragged number of rows per expert, is the kernel of the paper's section
+ * "Production Validation: VeOmni MoE".
+ *
+ * Conventions for every call
+ *   - Notation: R = T*K routed rows; pair id p = t*K + k (token-major).
+ *   - All tensors are row-major with the last index contiguous.  `void*` tensors hold bf16
+ *     (bfloat16 as 16-bit words); all results are rounded once, to nearest even, from fp32.
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer to memory owned by the
+ *     caller, 16-byte aligned.  The library allocates nothing, keeps no pointer after a call
+ *     returns, and never synchronises: all work is enqueued on `stream` (a cudaStream_t) in
+ *     order.  Outputs are overwritten.  Inputs and outputs must not overlap.
+ *   - H and I must be multiples of 128; 1 <= K <= E <= 1024; K <= 32; T*K < 2^31.
+ *   - Return value: MOE_OK or an error code.  Argument errors are detected on the host before
+ *     anything is launched.  A kernel that gives up waiting (bounded waits, never a trap) records
+ *     MOE_ERR_TIMEOUT in a device status word readable with moe_device_status().
+ *   - `offsets` passed to a GEMM call must be the array moe_permute produced (non-decreasing,
+ *     offsets[0] = 0, offsets[E] = R).  Expert ids in topk_idx must lie in [0, E).
+ */
+#ifndef MOE_B200_H
+#define MOE_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+    int32_t T; /* tokens */
+    int32_t H; /* hidden width */
+    int32_t I; /* per-expert intermediate width */
+    int32_t E; /* experts */
+    int32_t K; /* experts per token (top-k) */
+} moe_dims_t;
+
+typedef enum {
+    MOE_OK = 0,
+    MOE_ERR_NULL = 1,              /* a required pointer is NULL */
+    MOE_ERR_DIMS = 2,              /* non-positive size, K > E, R overflow */
+    MOE_ERR_UNSUPPORTED_SHAPE = 3, /* H or I not a multiple of 128, E or K above the limits */
+    MOE_ERR_ALIGNMENT = 4,         /* a pointer is not 16-byte aligned */
+    MOE_ERR_WORKSPACE = 5,         /* workspace / arena too small */
+    MOE_ERR_CUDA = 6,              /* a CUDA runtime or driver call failed */
+    MOE_ERR_TIMEOUT = 8            /* device status only: a bounded wait inside a kernel ran out */
+} moe_status_t;
+
+typedef void* moe_stream_t; /* a cudaStream_t */
+
+/* Human-readable name of a status code (host; never NULL). */
+const char* moe_status_string(int status);
+
+/* Bytes of device workspace moe_permute needs for these sizes (host; 0 on invalid dims). */
+size_t moe_permute_workspace_bytes(const moe_dims_t* dims);
+
+/* Reads the device status word of the current device into *status_out (host pointer) and clears
+ * it.  Synchronises the device.  Returns MOE_OK or MOE_ERR_CUDA. */
+int moe_device_status(int* status_out);
+
+/* ---- a1: route-permute ----------------------------------------------------------------------
+ * counts[e]      number of pairs with topk_idx = e                               int32 [E]
+ * offsets        exclusive prefix of counts, offsets[E] = R                      int32 [E+1]
+ * row_to_pair    pair ids sorted by (expert, pair id): a stable sort by expert   int32 [R]
+ * pair_to_row    inverse of row_to_pair                                          int32 [R]
+ * x_perm[r,:]  = x[row_to_pair[r] / K, :]                                        bf16  [R,H]
+ * x [T,H] bf16, topk_idx [T,K] int32.  workspace: moe_permute_workspace_bytes(dims) bytes,
+ * contents undefined before and after.  x_perm may be NULL (indices only).
+ * Layout follows the paper's packed-by-expert buffer (appendix, "What the kernel computes"). */
+int moe_permute(const moe_dims_t* dims, const void* x, const int32_t* topk_idx, void* x_perm,
+                int32_t* counts, int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row,
+                void* workspace, size_t workspace_bytes, moe_stream_t stream);
+
+/* ---- a8: dx[t,:] = sum_k dx_perm[pair_to_row[t*K+k], :]   (fp32 sum in slot order) ---------- */
+int moe_permute_bwd(const moe_dims_t* dims, const void* dx_perm, const int32_t* pair_to_row,
+                    void* dx, moe_stream_t stream);
+
+/* ---- a2: grouped GEMM gate/up with fused SwiGLU ---------------------------------------------
+ * For rows r in [offsets[e], offsets[e+1]):  g = x_perm[r,:] . w_gate[e],  u = x_perm[r,:] . w_up[e]
+ * (bf16 operands, fp32 accumulation);  h_act[r,:] = g / (1 + exp(-g)) * u  from the fp32 values;
+ * gu_saved[r,:] = [g | u] rounded to bf16 (gate in columns [0,I), up in [I,2I)); may be NULL.
+ * x_perm [R,H], w_gate, w_up [E,H,I], h_act [R,I], gu_saved [R,2I].  The gate and up
+ * projections form one GEMM of width 2I as in the paper's gate_up_proj. */
+int moe_grouped_gemm_gateup_swiglu(const moe_dims_t* dims, const void* x_perm, const void* w_gate,
+                                   const void* w_up, const int32_t* offsets, void* h_act,
+                                   void* gu_saved, moe_stream_t stream);
+
+/* ---- a3: y_perm[r,:] = h_act[r,:] . w_down[e]      w_down [E,I,H], y_perm [R,H] -------------- */
+int moe_grouped_gemm_down(const moe_dims_t* dims, const void* h_act, const void* w_down,
+                          const int32_t* offsets, void* y_perm, moe_stream_t stream);
+
+/* ---- a4: y[t,:] = sum_k topk_w[t,k] * y_perm[pair_to_row[t*K+k], :] -------------------------
+ * topk_w [T,K] fp32; fp32 sum in slot order, one rounding.  y [T,H]. */
+int moe_unpermute_combine(const moe_dims_t* dims, const void* y_perm, const float* topk_w,
+                          const int32_t* pair_to_row, void* y, moe_stream_t stream);
+
+/* ---- a5: dy_perm[pair_to_row[p],:] = topk_w[p] * dy[t(p),:];
+ *          dtopk_w[t,k] = <dy[t,:], y_perm[pair_to_row[t*K+k],:]>   (fp32 [T,K]; may be NULL,
+ *          and then y_perm may be NULL too) */
+int moe_unpermute_combine_bwd(const moe_dims_t* dims, const void* dy, const void* y_perm,
+                              const float* topk_w, const int32_t* pair_to_row, void* dy_perm,
+                              float* dtopk_w, moe_stream_t stream);
+
+/* ---- a6: down projection backward ------------------------------------------------------------
+ * dgrad  dh_act[r,:] = dy_perm[r,:] . w_down[e]^T                      dh_act [R,I]
+ * wgrad  dw_down[e]  = sum over rows r of expert e of h_act[r,:]^T dy_perm[r,:]   [E,I,H]
+ *        (all zeros for an expert without rows; written for every expert).
+ * moe_grouped_gemm_down_bwd runs the dgrad then the wgrad. */
+int moe_grouped_gemm_down_dgrad(const moe_dims_t* dims, const void* dy_perm, const void* w_down,
+                                const int32_t* offsets, void* dh_act, moe_stream_t stream);
+int moe_grouped_gemm_down_wgrad(const moe_dims_t* dims, const void* h_act, const void* dy_perm,
+                                const int32_t* offsets, void* dw_down, moe_stream_t stream);
+int moe_grouped_gemm_down_bwd(const moe_dims_t* dims, const void* dy_perm, const void* h_act,
+                              const void* w_down, const int32_t* offsets, void* dh_act,
+                              void* dw_down, moe_stream_t stream);
+
+/* ---- a7: SwiGLU backward and gate/up projection backward ------------------------------------
+ * moe_swiglu_bwd   with s = 1/(1+exp(-g)):  dg = dh_act*u*s*(1+g*(1-s)),  du = dh_act*g*s;
+ *                  dgu [R,2I] = [dg | du] (bf16), g,u read from gu_saved.
+ * dgrad            dx_perm[r,:] = dg[r,:] . w_gate[e]^T + du[r,:] . w_up[e]^T          [R,H]
+ * wgrad            dw_gate[e] = sum_r x_perm[r,:]^T dg[r,:],  dw_up[e] likewise         [E,H,I]
+ *                  -- the paper's dW1_e = X_e^T G_e with the ragged contraction over the
+ *                  expert's rows; zeros for an expert without rows.
+ * moe_grouped_gemm_gateup_swiglu_bwd runs the three in this order; dgu is caller-provided
+ * scratch that also returns dGU. */
+int moe_swiglu_bwd(const moe_dims_t* dims, const void* dh_act, const void* gu_saved, void* dgu,
+                   moe_stream_t stream);
+int moe_grouped_gemm_gateup_dgrad(const moe_dims_t* dims, const void* dgu, const void* w_gate,
+                                  const void* w_up, const int32_t* offsets, void* dx_perm,
+                                  moe_stream_t stream);
+int moe_grouped_gemm_gateup_wgrad(const moe_dims_t* dims, const void* x_perm, const void* dgu,
+                                  const int32_t* offsets, void* dw_gate, void* dw_up,
+                                  moe_stream_t stream);
+int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_act,
+                                       const void* gu_saved, const void* x_perm,
+                                       const void* w_gate, const void* w_up,
+                                       const int32_t* offsets, void* dgu, void* dx_perm,
+                                       void* dw_gate, void* dw_up, moe_stream_t stream);
+
+/* ---- whole layer from HOST activations ------------------------------------------------------
+ * One training step of the layer for a caller whose per-step tensors live in host memory:
+ * copies x, topk_idx, topk_w, dy (HOST pointers; pinned memory makes the copies asynchronous)
+ * into the device arena, runs a1..a8, and copies y [T,H], dx [T,H] (bf16) and dtopk_w [T,K]
+ * (fp32) back to HOST pointers.  Weights w_* and weight gradients dw_* are DEVICE pointers (the
+ * parameters stay resident, as in training).  `arena` is device scratch of at least
+ * moe_layer_arena_bytes(dims) bytes holding every intermediate of the step.  Everything is
+ * enqueued on `stream`; the host results are valid after the caller synchronises the stream. */
+size_t moe_layer_arena_bytes(const moe_dims_t* dims);
+int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int32_t* topk_idx_host,
+                           const float* topk_w_host, const void* dy_host, const void* w_gate,
+                           const void* w_up, const void* w_down, void* y_host, void* dx_host,
+                           float* dtopk_w_host, void* dw_gate, void* dw_up, void* dw_down,
+                           void* arena, size_t arena_bytes, moe_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H */

@@ -1,0 +1,275 @@
+// C ABI of libmoe_b200.so: argument validation and dispatch to the kernels.  See include/moe_b200.h.
+#include "common.cuh"
+
+namespace moe {
+
+int sm_count() {
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    if (dev >= 0 && dev < 64 && cached[dev] > 0) return cached[dev];
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+    if (dev >= 0 && dev < 64) cached[dev] = n;
+    return n;
+}
+
+namespace {
+
+int check_dims(const moe_dims_t* d) {
+    if (d == nullptr) return MOE_ERR_NULL;
+    if (d->T <= 0 || d->H <= 0 || d->I <= 0 || d->E <= 0 || d->K <= 0 || d->K > d->E) return MOE_ERR_DIMS;
+    if ((long long)d->T * d->K >= (1ll << 31)) return MOE_ERR_DIMS;
+    if (d->H % 128 != 0 || d->I % 128 != 0 || d->E > 1024 || d->K > 32) return MOE_ERR_UNSUPPORTED_SHAPE;
+    return MOE_OK;
+}
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+// Validation helper: every pointer in `req` must be non-NULL and 16-byte aligned; pointers in `opt`
+// only need alignment when present.
+template <size_t NR, size_t NO>
+int check_ptrs(const void* const (&req)[NR], const void* const (&opt)[NO]) {
+    for (size_t i = 0; i < NR; ++i) {
+        if (req[i] == nullptr) return MOE_ERR_NULL;
+        if (misaligned(req[i])) return MOE_ERR_ALIGNMENT;
+    }
+    for (size_t i = 0; i < NO; ++i)
+        if (opt[i] != nullptr && misaligned(opt[i])) return MOE_ERR_ALIGNMENT;
+    return MOE_OK;
+}
+
+#define MOE_VALIDATE(dims, ...)                                \
+    do {                                                       \
+        int st_ = check_dims(dims);                            \
+        if (st_ != MOE_OK) return st_;                         \
+        st_ = check_ptrs(__VA_ARGS__);                         \
+        if (st_ != MOE_OK) return st_;                         \
+    } while (0)
+
+inline const bf16* cb(const void* p) { return static_cast<const bf16*>(p); }
+inline bf16* mb(void* p) { return static_cast<bf16*>(p); }
+inline cudaStream_t st(moe_stream_t s) { return static_cast<cudaStream_t>(s); }
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+}  // namespace moe
+
+using namespace moe;
+
+extern "C" {
+
+const char* moe_status_string(int status) {
+    switch (status) {
+        case MOE_OK: return "ok";
+        case MOE_ERR_NULL: return "a required pointer is NULL";
+        case MOE_ERR_DIMS: return "invalid dimensions";
+        case MOE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (H, I must be multiples of 128; E <= 1024; K <= 32)";
+        case MOE_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case MOE_ERR_WORKSPACE: return "workspace or arena too small";
+        case MOE_ERR_CUDA: return "CUDA call failed";
+        case MOE_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+size_t moe_permute_workspace_bytes(const moe_dims_t* dims) {
+    if (check_dims(dims) != MOE_OK) return 0;
+    return permute_workspace_bytes(*dims);
+}
+
+int moe_device_status(int* status_out) {
+    if (status_out == nullptr) return MOE_ERR_NULL;
+    return read_and_clear_device_status(status_out);
+}
+
+int moe_permute(const moe_dims_t* dims, const void* x, const int32_t* topk_idx, void* x_perm, int32_t* counts,
+                int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row, void* workspace,
+                size_t workspace_bytes, moe_stream_t stream) {
+    {
+        const void* const req[] = {topk_idx, counts, offsets, row_to_pair, pair_to_row, workspace};
+        const void* const opt[] = {x, x_perm};
+        MOE_VALIDATE(dims, req, opt);
+    }
+    if (x_perm != nullptr && x == nullptr) return MOE_ERR_NULL;
+    if (workspace_bytes < permute_workspace_bytes(*dims)) return MOE_ERR_WORKSPACE;
+    return launch_permute(*dims, cb(x), topk_idx, mb(x_perm), counts, offsets, row_to_pair, pair_to_row, workspace,
+                          st(stream));
+}
+
+int moe_permute_bwd(const moe_dims_t* dims, const void* dx_perm, const int32_t* pair_to_row, void* dx,
+                    moe_stream_t stream) {
+    const void* const req[] = {dx_perm, pair_to_row, dx};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_gather_sum(*dims, cb(dx_perm), nullptr, pair_to_row, mb(dx), st(stream));
+}
+
+int moe_grouped_gemm_gateup_swiglu(const moe_dims_t* dims, const void* x_perm, const void* w_gate, const void* w_up,
+                                   const int32_t* offsets, void* h_act, void* gu_saved, moe_stream_t stream) {
+    const void* const req[] = {x_perm, w_gate, w_up, offsets, h_act};
+    const void* const opt[] = {gu_saved};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_gateup_fwd(*dims, cb(x_perm), cb(w_gate), cb(w_up), offsets, mb(h_act), mb(gu_saved), st(stream));
+}
+
+int moe_grouped_gemm_down(const moe_dims_t* dims, const void* h_act, const void* w_down, const int32_t* offsets,
+                          void* y_perm, moe_stream_t stream) {
+    const void* const req[] = {h_act, w_down, offsets, y_perm};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_down_fwd(*dims, cb(h_act), cb(w_down), offsets, mb(y_perm), st(stream));
+}
+
+int moe_unpermute_combine(const moe_dims_t* dims, const void* y_perm, const float* topk_w, const int32_t* pair_to_row,
+                          void* y, moe_stream_t stream) {
+    const void* const req[] = {y_perm, topk_w, pair_to_row, y};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_gather_sum(*dims, cb(y_perm), topk_w, pair_to_row, mb(y), st(stream));
+}
+
+int moe_unpermute_combine_bwd(const moe_dims_t* dims, const void* dy, const void* y_perm, const float* topk_w,
+                              const int32_t* pair_to_row, void* dy_perm, float* dtopk_w, moe_stream_t stream) {
+    const void* const req[] = {dy, topk_w, pair_to_row, dy_perm};
+    const void* const opt[] = {y_perm, dtopk_w};
+    MOE_VALIDATE(dims, req, opt);
+    if (dtopk_w != nullptr && y_perm == nullptr) return MOE_ERR_NULL;
+    return launch_combine_bwd(*dims, cb(dy), cb(y_perm), topk_w, pair_to_row, mb(dy_perm), dtopk_w, st(stream));
+}
+
+int moe_grouped_gemm_down_dgrad(const moe_dims_t* dims, const void* dy_perm, const void* w_down,
+                                const int32_t* offsets, void* dh_act, moe_stream_t stream) {
+    const void* const req[] = {dy_perm, w_down, offsets, dh_act};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_down_dgrad(*dims, cb(dy_perm), cb(w_down), offsets, mb(dh_act), st(stream));
+}
+
+int moe_grouped_gemm_down_wgrad(const moe_dims_t* dims, const void* h_act, const void* dy_perm,
+                                const int32_t* offsets, void* dw_down, moe_stream_t stream) {
+    const void* const req[] = {h_act, dy_perm, offsets, dw_down};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_down_wgrad(*dims, cb(h_act), cb(dy_perm), offsets, mb(dw_down), st(stream));
+}
+
+int moe_grouped_gemm_down_bwd(const moe_dims_t* dims, const void* dy_perm, const void* h_act, const void* w_down,
+                              const int32_t* offsets, void* dh_act, void* dw_down, moe_stream_t stream) {
+    int s = moe_grouped_gemm_down_dgrad(dims, dy_perm, w_down, offsets, dh_act, stream);
+    if (s != MOE_OK) return s;
+    return moe_grouped_gemm_down_wgrad(dims, h_act, dy_perm, offsets, dw_down, stream);
+}
+
+int moe_swiglu_bwd(const moe_dims_t* dims, const void* dh_act, const void* gu_saved, void* dgu,
+                   moe_stream_t stream) {
+    const void* const req[] = {dh_act, gu_saved, dgu};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_swiglu_bwd(*dims, cb(dh_act), cb(gu_saved), mb(dgu), st(stream));
+}
+
+int moe_grouped_gemm_gateup_dgrad(const moe_dims_t* dims, const void* dgu, const void* w_gate, const void* w_up,
+                                  const int32_t* offsets, void* dx_perm, moe_stream_t stream) {
+    const void* const req[] = {dgu, w_gate, w_up, offsets, dx_perm};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_gateup_dgrad(*dims, cb(dgu), cb(w_gate), cb(w_up), offsets, mb(dx_perm), st(stream));
+}
+
+int moe_grouped_gemm_gateup_wgrad(const moe_dims_t* dims, const void* x_perm, const void* dgu,
+                                  const int32_t* offsets, void* dw_gate, void* dw_up, moe_stream_t stream) {
+    const void* const req[] = {x_perm, dgu, offsets, dw_gate, dw_up};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_gateup_wgrad(*dims, cb(x_perm), cb(dgu), offsets, mb(dw_gate), mb(dw_up), st(stream));
+}
+
+int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_act, const void* gu_saved,
+                                       const void* x_perm, const void* w_gate, const void* w_up,
+                                       const int32_t* offsets, void* dgu, void* dx_perm, void* dw_gate,
+                                       void* dw_up, moe_stream_t stream) {
+    int s = moe_swiglu_bwd(dims, dh_act, gu_saved, dgu, stream);
+    if (s != MOE_OK) return s;
+    s = moe_grouped_gemm_gateup_dgrad(dims, dgu, w_gate, w_up, offsets, dx_perm, stream);
+    if (s != MOE_OK) return s;
+    return moe_grouped_gemm_gateup_wgrad(dims, x_perm, dgu, offsets, dw_gate, dw_up, stream);
+}
+
+// Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).
+namespace {
+struct Arena {
+    size_t x, idx, w, dy, y, dx, dw, counts, offsets, r2p, p2r, ws, xp, hact, gu, yp, dyp, dhact, dgu, dxp, total;
+};
+Arena arena_layout(const moe_dims_t& d) {
+    const size_t T = d.T, H = d.H, I = d.I, E = d.E, K = d.K, R = T * K;
+    Arena a;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes, 256); return at; };
+    a.x = take(T * H * 2); a.idx = take(R * 4); a.w = take(R * 4); a.dy = take(T * H * 2);
+    a.y = take(T * H * 2); a.dx = take(T * H * 2); a.dw = take(R * 4);
+    a.counts = take(E * 4); a.offsets = take((E + 1) * 4); a.r2p = take(R * 4); a.p2r = take(R * 4);
+    a.ws = take(permute_workspace_bytes(d));
+    a.xp = take(R * H * 2); a.hact = take(R * I * 2); a.gu = take(R * 2 * I * 2); a.yp = take(R * H * 2);
+    a.dyp = take(R * H * 2); a.dhact = take(R * I * 2); a.dgu = take(R * 2 * I * 2); a.dxp = take(R * H * 2);
+    a.total = o;
+    return a;
+}
+}  // namespace
+
+size_t moe_layer_arena_bytes(const moe_dims_t* dims) {
+    if (check_dims(dims) != MOE_OK) return 0;
+    return arena_layout(*dims).total;
+}
+
+int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int32_t* topk_idx_host,
+                           const float* topk_w_host, const void* dy_host, const void* w_gate, const void* w_up,
+                           const void* w_down, void* y_host, void* dx_host, float* dtopk_w_host, void* dw_gate,
+                           void* dw_up, void* dw_down, void* arena, size_t arena_bytes, moe_stream_t stream) {
+    {
+        const void* const req[] = {w_gate, w_up, w_down, dw_gate, dw_up, dw_down, arena};
+        const void* const opt[] = {nullptr};
+        MOE_VALIDATE(dims, req, opt);
+    }
+    if (!x_host || !topk_idx_host || !topk_w_host || !dy_host || !y_host || !dx_host || !dtopk_w_host)
+        return MOE_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0) return MOE_ERR_ALIGNMENT;
+    const moe_dims_t& d = *dims;
+    const Arena a = arena_layout(d);
+    if (arena_bytes < a.total) return MOE_ERR_WORKSPACE;
+    uint8_t* base = static_cast<uint8_t*>(arena);
+    cudaStream_t s = st(stream);
+    const size_t T = d.T, H = d.H, R = T * d.K;
+    auto P = [&](size_t off) { return static_cast<void*>(base + off); };
+    auto Pi = [&](size_t off) { return reinterpret_cast<int32_t*>(base + off); };
+
+    if (cudaMemcpyAsync(P(a.x), x_host, T * H * 2, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(P(a.idx), topk_idx_host, R * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(P(a.w), topk_w_host, R * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(P(a.dy), dy_host, T * H * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return MOE_ERR_CUDA;
+
+    int rc;
+#define MOE_STEP(call) do { rc = (call); if (rc != MOE_OK) return rc; } while (0)
+    MOE_STEP(moe_permute(dims, P(a.x), Pi(a.idx), P(a.xp), Pi(a.counts), Pi(a.offsets), Pi(a.r2p), Pi(a.p2r), P(a.ws),
+                         a.xp - a.ws, stream));
+    MOE_STEP(moe_grouped_gemm_gateup_swiglu(dims, P(a.xp), w_gate, w_up, Pi(a.offsets), P(a.hact), P(a.gu), stream));
+    MOE_STEP(moe_grouped_gemm_down(dims, P(a.hact), w_down, Pi(a.offsets), P(a.yp), stream));
+    MOE_STEP(moe_unpermute_combine(dims, P(a.yp), reinterpret_cast<float*>(base + a.w), Pi(a.p2r), P(a.y), stream));
+    MOE_STEP(moe_unpermute_combine_bwd(dims, P(a.dy), P(a.yp), reinterpret_cast<float*>(base + a.w), Pi(a.p2r),
+                                       P(a.dyp), reinterpret_cast<float*>(base + a.dw), stream));
+    MOE_STEP(moe_grouped_gemm_down_bwd(dims, P(a.dyp), P(a.hact), w_down, Pi(a.offsets), P(a.dhact), dw_down, stream));
+    MOE_STEP(moe_grouped_gemm_gateup_swiglu_bwd(dims, P(a.dhact), P(a.gu), P(a.xp), w_gate, w_up, Pi(a.offsets),
+                                                P(a.dgu), P(a.dxp), dw_gate, dw_up, stream));
+    MOE_STEP(moe_permute_bwd(dims, P(a.dxp), Pi(a.p2r), P(a.dx), stream));
+#undef MOE_STEP
+
+    if (cudaMemcpyAsync(y_host, P(a.y), T * H * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(dx_host, P(a.dx), T * H * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(dtopk_w_host, P(a.dw), R * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    return MOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,48 @@
+// Shared declarations of the library's translation units (internal; not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/moe_b200.h"
+
+namespace moe {
+
+typedef __nv_bfloat16 bf16;
+
+// Device status word (one per device that loaded the library; lives in grouped_gemm.cu): kernels
+// record MOE_ERR_TIMEOUT there when a bounded wait runs out.  Synchronises the device.
+int read_and_clear_device_status(int* status_out);
+
+// Number of SMs of the current device (cached per device ordinal).
+int sm_count();
+
+inline int check_launch() { return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA; }
+
+// ---- data-movement kernels (movement.cu) ------------------------------------------------------
+int launch_permute(const moe_dims_t& d, const bf16* x, const int32_t* topk_idx, bf16* x_perm,
+                   int32_t* counts, int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row,
+                   void* workspace, cudaStream_t s);
+size_t permute_workspace_bytes(const moe_dims_t& d);
+int launch_gather_sum(const moe_dims_t& d, const bf16* src_perm, const float* topk_w,
+                      const int32_t* pair_to_row, bf16* dst, cudaStream_t s);  // topk_w may be NULL (unit weights)
+int launch_combine_bwd(const moe_dims_t& d, const bf16* dy, const bf16* y_perm, const float* topk_w,
+                       const int32_t* pair_to_row, bf16* dy_perm, float* dtopk_w, cudaStream_t s);
+int launch_swiglu_bwd(const moe_dims_t& d, const bf16* dh_act, const bf16* gu, bf16* dgu, cudaStream_t s);
+
+// ---- grouped GEMMs (grouped_gemm.cu) -----------------------------------------------------------
+int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gate, const bf16* w_up,
+                      const int32_t* offsets, bf16* h_act, bf16* gu, cudaStream_t s);
+int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, const int32_t* offsets,
+                    bf16* y_perm, cudaStream_t s);
+int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_down, const int32_t* offsets,
+                      bf16* dh_act, cudaStream_t s);
+int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_perm, const int32_t* offsets,
+                      bf16* dw_down, cudaStream_t s);
+int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate, const bf16* w_up,
+                        const int32_t* offsets, bf16* dx_perm, cudaStream_t s);
+int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu, const int32_t* offsets,
+                        bf16* dw_gate, bf16* dw_up, cudaStream_t s);
+
+}  // namespace moe

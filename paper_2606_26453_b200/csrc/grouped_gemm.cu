@@ -1,0 +1,661 @@
+// Grouped GEMMs of the MoE layer as persistent, warp-specialised tcgen05 kernels for sm_100a.
+//
+// One CTA per SM walks a tile list that every CTA derives by itself from the per-expert offsets
+// (no host round trip, no extra launch).  Per CTA:
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of 64-wide K blocks of A and B into a
+//               4-stage ring of 128-byte-swizzled shared-memory tiles, completion on mbarriers
+//   warp 1      MMA issuer: one lane issues tcgen05.mma (128 x 256 x 16, bf16 -> fp32) with the
+//               accumulator in tensor memory; tcgen05.commit releases ring stages and publishes
+//               finished accumulators
+//   warps 2..5  epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), apply the
+//               epilogue (plain / SwiGLU), round to bf16, store row segments with 16-byte stores
+// The accumulator is double buffered (2 x 256 of the 512 TMEM columns) so the epilogue of one tile
+// overlaps the main loop of the next.
+//
+// Two ragged shapes occur:
+//   row-ragged (forward, dgrad): output rows are the packed rows of an expert.  A tile starts at
+//     offsets[e] + 128*i; loading past the expert's last row is harmless, stores are clipped.
+//   contraction-ragged (wgrad; the paper's dW1_e = X_e^T G_e): the expert's rows are the
+//     contraction.  The last K block issues only ceil(rem/16) MMAs and the < 16 surplus rows
+//     are zeroed in shared memory first; an expert without rows gets a zero tile.
+//
+// All waits are bounded: a wait that runs out records MOE_ERR_TIMEOUT in the device status word,
+// raises a CTA-wide abort flag and every role leaves through the common teardown.
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include "common.cuh"
+
+namespace moe {
+
+__device__ int g_device_status = 0;
+
+int read_and_clear_device_status(int* status_out) {
+    int v = 0, zero = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)) != cudaSuccess) return MOE_ERR_CUDA;
+    if (v != 0 && cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return MOE_ERR_CUDA;
+    *status_out = v;
+    return MOE_OK;
+}
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;   // 16 KB
+constexpr int B_BYTES = BN * BK * 2;   // 32 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN-major box: 64 k-rows x 128 B = 8 KB
+constexpr int MAX_E = 1024;
+constexpr int NUM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3 };
+
+struct Params {
+    const int32_t* offsets;
+    int E;
+    int k_blocks;        // row-ragged kinds: contraction length / 64
+    int k_split;         // DGRAD: k blocks taken from the first B tensor (then the second); else k_blocks
+    int n_tiles;         // output column tiles
+    int m_tiles;         // WGRAD: output row tiles per expert
+    int n_cols;          // valid output columns (row-ragged) / total N (WGRAD)
+    int b_rows_per_e;    // rows per expert in B's 2-D view
+    int n_split;         // WGRAD / plain: columns >= n_split go to out1
+    long long ldo;       // output row pitch (elements)
+    long long out_e_stride;  // WGRAD: elements per expert in the outputs
+    bf16* out0;
+    bf16* out1;
+    bf16* gu;            // FWD_SWIGLU: [R, 2I] or null
+    int I;               // FWD_SWIGLU
+};
+
+struct SharedCtl {
+    unsigned long long full[STAGES];
+    unsigned long long empty[STAGES];
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    unsigned long long drain;
+    uint32_t tmem_base;
+    int abort_flag;
+    int32_t offs[MAX_E + 1];
+    int32_t tile_prefix[MAX_E + 1];
+};
+
+// ---- small PTX wrappers ------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait timed out, or another did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 0xFF) == 0) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                atomicExch(&g_device_status, (int)MOE_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                       uint32_t accumulate) {
+    asm volatile(
+        "{ .reg .pred p; setp.ne.u32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t v[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 version field set.
+//   K-major tile  [rows][64 k]  : 8-row groups 1024 B apart (stride byte offset); leading offset unused (1)
+//   MN-major tile [chunk][64 k-rows][64 mn]: 8-k-row groups 1024 B apart (stride byte offset),
+//                 64-wide mn chunks CHUNK_BYTES apart (leading byte offset)
+template <bool MN_MAJOR>
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+    const uint64_t lbo = MN_MAJOR ? (uint64_t)(CHUNK_BYTES >> 4) : 1ull;
+    const uint64_t sbo = 1024 >> 4;
+    return (uint64_t)((addr >> 4) & 0x3FFF) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, given N and operand major-ness.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn, bool b_mn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// ---- tile list ------------------------------------------------------------------------------------
+struct Tile {
+    int e;        // expert
+    int row0;     // row-ragged: first packed row of the tile; WGRAD: first output row (m)
+    int row_end;  // row-ragged: offsets[e+1]
+    int n0;       // first output column
+    int k_blocks; // contraction blocks of this tile
+    int k_row0;   // WGRAD: first packed row of the contraction
+    int k_rows;   // WGRAD: rows of the contraction
+};
+
+template <int KIND>
+__device__ __forceinline__ long long total_tiles(const Params& p, const SharedCtl* ctl) {
+    if (KIND == WGRAD) return (long long)p.E * p.m_tiles * p.n_tiles;
+    return (long long)ctl->tile_prefix[p.E] * p.n_tiles;
+}
+
+template <int KIND>
+__device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ctl, long long t) {
+    Tile tl;
+    if (KIND == WGRAD) {
+        const int per_e = p.m_tiles * p.n_tiles;
+        tl.e = (int)(t / per_e);
+        const int local = (int)(t - (long long)tl.e * per_e);
+        const int mt = local / p.n_tiles, nt = local - mt * p.n_tiles;
+        tl.row0 = mt * BM;
+        tl.n0 = nt * BN;
+        tl.k_row0 = ctl->offs[tl.e];
+        tl.k_rows = ctl->offs[tl.e + 1] - tl.k_row0;
+        tl.k_blocks = (tl.k_rows + BK - 1) / BK;
+        tl.row_end = 0;
+    } else {
+        // tile_prefix[e] = number of 128-row tiles of experts < e; tiles of an expert are ordered
+        // column tile major, row tile minor, so concurrently running CTAs share a weight tile.
+        const int mtile_flat = (int)(t / p.n_tiles);   // only used to bracket the expert
+        int lo = 0, hi = p.E;                          // largest e with tile_prefix[e]*n_tiles <= t
+        (void)mtile_flat;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if ((long long)ctl->tile_prefix[mid] * p.n_tiles <= t) lo = mid; else hi = mid;
+        }
+        tl.e = lo;
+        const int m_tiles_e = ctl->tile_prefix[lo + 1] - ctl->tile_prefix[lo];
+        const int local = (int)(t - (long long)ctl->tile_prefix[lo] * p.n_tiles);
+        const int nt = local / m_tiles_e, mt = local - nt * m_tiles_e;
+        tl.row0 = ctl->offs[lo] + mt * BM;
+        tl.row_end = ctl->offs[lo + 1];
+        tl.n0 = nt * BN;
+        tl.k_blocks = p.k_blocks;
+        tl.k_row0 = 0;
+        tl.k_rows = 0;
+    }
+    return tl;
+}
+
+// ---- the kernel -----------------------------------------------------------------------------------
+// Operand major-ness per kind:
+//   FWD_*  : A K-major (activations [R, K]),   B MN-major (weights [E*K, N], N contiguous)
+//   DGRAD  : A K-major,                        B K-major  (weights [E*N, K], K contiguous)
+//   WGRAD  : A MN-major (activations [R, M]),  B MN-major (gradients [R, N])
+template <int KIND>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
+                    const __grid_constant__ CUtensorMap map_b1, const Params p) {
+    constexpr bool A_MN = (KIND == WGRAD);
+    constexpr bool B_MN = (KIND != DGRAD);
+    constexpr uint32_t IDESC = make_idesc(BN, A_MN, B_MN);
+    constexpr uint32_t A_KSTEP = A_MN ? 2048 : 32;   // bytes per 16 k inside a stage
+    constexpr uint32_t B_KSTEP = B_MN ? 2048 : 32;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles_ptr + STAGES * STAGE_BYTES);
+    volatile int* abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- set-up: barriers, schedule tables, TMEM ----
+    for (int e = threadIdx.x; e <= p.E; e += NUM_THREADS) ctl->offs[e] = p.offsets[e];
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[a]), 4);
+        }
+        mbar_init(smem_u32(&ctl->drain), 1);
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tmap(&map_a);
+        prefetch_tmap(&map_b0);
+        prefetch_tmap(&map_b1);
+    }
+    __syncthreads();
+    if (KIND != WGRAD && threadIdx.x == 0) {
+        int run = 0;
+        for (int e = 0; e < p.E; ++e) {
+            ctl->tile_prefix[e] = run;
+            run += (ctl->offs[e + 1] - ctl->offs[e] + BM - 1) / BM;
+        }
+        ctl->tile_prefix[p.E] = run;
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                     "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const long long n_tiles_total = total_tiles<KIND>(p, ctl);
+
+    if (warp == 0) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t issued = 0;
+            bool ok = true;
+            for (long long t = blockIdx.x; ok && t < n_tiles_total; t += gridDim.x) {
+                const Tile tl = decode_tile<KIND>(p, ctl, t);
+                for (int kb = 0; kb < tl.k_blocks; ++kb) {
+                    if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t full = smem_u32(&ctl->full[stage]);
+                    mbar_arrive_expect_tx(full, STAGE_BYTES);
+                    const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
+                    const uint32_t b_dst = a_dst + A_BYTES;
+                    if (KIND == WGRAD) {
+                        const int krow = tl.k_row0 + kb * BK;
+#pragma unroll
+                        for (int c = 0; c < BM / 64; ++c)
+                            tma_load_2d(a_dst + c * CHUNK_BYTES, &map_a, tl.row0 + c * 64, krow, full);
+#pragma unroll
+                        for (int c = 0; c < BN / 64; ++c)
+                            tma_load_2d(b_dst + c * CHUNK_BYTES, &map_b0, tl.n0 + c * 64, krow, full);
+                    } else {
+                        tma_load_2d(a_dst, &map_a, kb * BK, tl.row0, full);
+                        if (KIND == DGRAD) {
+                            const bool second = kb >= p.k_split;
+                            const int kx = (second ? kb - p.k_split : kb) * BK;
+                            tma_load_2d(b_dst, second ? &map_b1 : &map_b0, kx, tl.e * p.b_rows_per_e + tl.n0, full);
+                        } else if (KIND == FWD_PLAIN) {
+                            const int ky = tl.e * p.b_rows_per_e + kb * BK;
+#pragma unroll
+                            for (int c = 0; c < BN / 64; ++c)
+                                tma_load_2d(b_dst + c * CHUNK_BYTES, &map_b0, tl.n0 + c * 64, ky, full);
+                        } else {  // FWD_SWIGLU: 128 gate columns then 128 up columns
+                            const int ky = tl.e * p.b_rows_per_e + kb * BK;
+                            const int ng = tl.n0 >> 1;   // n0 counts fused (gate+up) columns
+#pragma unroll
+                            for (int c = 0; c < 2; ++c) {
+                                tma_load_2d(b_dst + c * CHUNK_BYTES, &map_b0, ng + c * 64, ky, full);
+                                tma_load_2d(b_dst + (2 + c) * CHUNK_BYTES, &map_b1, ng + c * 64, ky, full);
+                            }
+                        }
+                    }
+                    ++issued;
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // leave no bulk copy in flight: wait (bounded) for the copies issued into each stage
+                const uint32_t n_wait = issued < (uint32_t)STAGES ? issued : (uint32_t)STAGES;
+                uint32_t s = stage, ph = phase;
+                for (uint32_t i = 0; i < n_wait; ++i) {
+                    if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
+                    const unsigned long long t0 = global_timer_ns();
+                    while (!mbar_try_wait(smem_u32(&ctl->full[s]), ph) && global_timer_ns() - t0 < WAIT_LIMIT_NS / 4) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        uint32_t stage = 0, phase = 0;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (long long t = blockIdx.x; ok && t < n_tiles_total; t += gridDim.x) {
+            const Tile tl = decode_tile<KIND>(p, ctl, t);
+            if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * BN;
+            for (int kb = 0; kb < tl.k_blocks; ++kb) {
+                if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
+                const uint32_t b_base = a_base + A_BYTES;
+                int n_mma = BK / 16;
+                if (KIND == WGRAD) {
+                    const int rem = tl.k_rows - kb * BK;
+                    if (rem < BK) {
+                        n_mma = (rem + 15) >> 4;
+                        const int z0 = rem, z1 = n_mma * 16;   // contraction rows to clear in A and B
+                        uint8_t* stage_ptr = tiles_ptr + stage * STAGE_BYTES;
+                        const int per_row = (BM / 64 + BN / 64) * 8;   // 16-byte pieces per k-row over all chunks
+                        for (int i = lane; i < (z1 - z0) * per_row; i += 32) {
+                            const int r = z0 + i / per_row, q = i % per_row;
+                            const int chunk = q >> 3, piece = q & 7;   // chunks 0..1 are A, 2..5 are B (contiguous)
+                            *reinterpret_cast<uint4*>(stage_ptr + chunk * CHUNK_BYTES + r * 128 + piece * 16) =
+                                make_uint4(0, 0, 0, 0);
+                        }
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
+                }
+                if (lane == 0) {
+                    const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
+                    const uint64_t b_desc = make_smem_desc<B_MN>(b_base);
+                    for (int kk = 0; kk < n_mma; ++kk) {
+                        tc_mma(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4), b_desc + (uint64_t)((kk * B_KSTEP) >> 4),
+                               IDESC, (kb | kk) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&ctl->empty[stage]));
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            if (lane == 0) tc_commit(smem_u32(&ctl->tmem_full[acc]));
+            __syncwarp();
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        // all issued MMAs must have retired before tensor memory is released
+        if (lane == 0) {
+            tc_commit(smem_u32(&ctl->drain));
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
+        }
+        __syncwarp();
+    } else {
+        // ================= epilogue (warps 2..5) =================
+        const int quarter = warp & 3;               // TMEM lanes [32*quarter, 32*quarter+32)
+        const int row_in_tile = quarter * 32 + lane;
+        uint32_t acc = 0, acc_phase = 0;
+        for (long long t = blockIdx.x; t < n_tiles_total; t += gridDim.x) {
+            const Tile tl = decode_tile<KIND>(p, ctl, t);
+            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+            if (KIND == FWD_SWIGLU) {
+                const long long row = (long long)tl.row0 + row_in_tile;
+                const bool row_ok = row < tl.row_end;
+                const int ng = tl.n0 >> 1;
+                bf16* h_row = p.out0 + row * p.I + ng;
+                bf16* g_row = p.gu ? p.gu + row * (2ll * p.I) + ng : nullptr;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t g[32], u[32];
+                    tc_ld32(taddr + c * 32, g);
+                    tc_ld32(taddr + 128 + c * 32, u);
+                    tc_wait_ld();
+                    if (row_ok) {
+                        uint32_t hp[16], gp[16], up[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float g0 = __uint_as_float(g[2 * j]), g1 = __uint_as_float(g[2 * j + 1]);
+                            const float u0 = __uint_as_float(u[2 * j]), u1 = __uint_as_float(u[2 * j + 1]);
+                            const float h0 = g0 / (1.f + __expf(-g0)) * u0;
+                            const float h1 = g1 / (1.f + __expf(-g1)) * u1;
+                            hp[j] = pack_bf16(h0, h1);
+                            gp[j] = pack_bf16(g0, g1);
+                            up[j] = pack_bf16(u0, u1);
+                        }
+                        uint4* hd = reinterpret_cast<uint4*>(h_row + c * 32);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) hd[j] = make_uint4(hp[4 * j], hp[4 * j + 1], hp[4 * j + 2], hp[4 * j + 3]);
+                        if (g_row) {
+                            uint4* gd = reinterpret_cast<uint4*>(g_row + c * 32);
+                            uint4* ud = reinterpret_cast<uint4*>(g_row + p.I + c * 32);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                gd[j] = make_uint4(gp[4 * j], gp[4 * j + 1], gp[4 * j + 2], gp[4 * j + 3]);
+                                ud[j] = make_uint4(up[4 * j], up[4 * j + 1], up[4 * j + 2], up[4 * j + 3]);
+                            }
+                        }
+                    }
+                }
+            } else {
+                long long row;
+                bool row_ok;
+                bf16 *o0, *o1;
+                if (KIND == WGRAD) {
+                    row = (long long)tl.row0 + row_in_tile;
+                    row_ok = true;
+                    o0 = p.out0 + (long long)tl.e * p.out_e_stride + row * p.ldo;
+                    o1 = p.out1 ? p.out1 + (long long)tl.e * p.out_e_stride + row * p.ldo : nullptr;
+                } else {
+                    row = (long long)tl.row0 + row_in_tile;
+                    row_ok = row < tl.row_end;
+                    o0 = p.out0 + row * p.ldo;
+                    o1 = nullptr;
+                }
+                const bool have_acc = tl.k_blocks > 0;
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t v[32];
+                    if (have_acc) {
+                        tc_ld32(taddr + c * 32, v);
+                        tc_wait_ld();
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = 0u;
+                    }
+                    const int n = tl.n0 + c * 32;
+                    if (row_ok && n < p.n_cols) {
+                        bf16* dst = (n < p.n_split) ? o0 + n : o1 + (n - p.n_split);
+                        uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            d4[j] = make_uint4(pack_bf16(__uint_as_float(v[8 * j]), __uint_as_float(v[8 * j + 1])),
+                                               pack_bf16(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3])),
+                                               pack_bf16(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5])),
+                                               pack_bf16(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7])));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+    }
+}
+
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + sizeof(SharedCtl);
+
+// ---- host side ------------------------------------------------------------------------------------
+PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    if (fn == nullptr) {
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(ptr);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [outer, inner] (inner contiguous), box [box_outer, box_inner], 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint32_t box_inner,
+              uint32_t box_outer) {
+    PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {inner * 2};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int KIND>
+int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const Params& p, cudaStream_t s) {
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
+    if (dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)SMEM_BYTES) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    const int grid = sm_count();
+    if (grid <= 0) return MOE_ERR_CUDA;
+    grouped_gemm_kernel<KIND><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(a, b0, b1, p);
+    return check_launch();
+}
+
+}  // namespace
+
+// Gate/up forward: A = x_perm [R,H]; B = w_gate, w_up viewed as [E*H, I]; fused width 2I in tiles of
+// 128 gate + 128 up columns.
+int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gate, const bf16* w_up,
+                      const int32_t* offsets, bf16* h_act, bf16* gu, cudaStream_t s) {
+    const uint64_t R = (uint64_t)d.T * d.K;
+    CUtensorMap a, b0, b1;
+    if (!make_map(&a, x_perm, d.H, R, BK, BM) || !make_map(&b0, w_gate, d.I, (uint64_t)d.E * d.H, 64, BK) ||
+        !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, 64, BK))
+        return MOE_ERR_CUDA;
+    Params p = {};
+    p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
+    p.n_tiles = d.I / 128; p.n_cols = 2 * d.I; p.b_rows_per_e = d.H;
+    p.out0 = h_act; p.gu = gu; p.I = d.I; p.ldo = d.I; p.n_split = 2 * d.I;
+    return launch<FWD_SWIGLU>(a, b0, b1, p, s);
+}
+
+// Down forward: A = h_act [R,I]; B = w_down viewed as [E*I, H].
+int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, const int32_t* offsets,
+                    bf16* y_perm, cudaStream_t s) {
+    const uint64_t R = (uint64_t)d.T * d.K;
+    CUtensorMap a, b0;
+    if (!make_map(&a, h_act, d.I, R, BK, BM) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, 64, BK))
+        return MOE_ERR_CUDA;
+    Params p = {};
+    p.offsets = offsets; p.E = d.E; p.k_blocks = d.I / BK; p.k_split = p.k_blocks;
+    p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.b_rows_per_e = d.I;
+    p.out0 = y_perm; p.ldo = d.H; p.n_split = d.H;
+    return launch<FWD_PLAIN>(a, b0, b0, p, s);
+}
+
+// Down dgrad: dh_act = dy_perm . w_down[e]^T.  A = dy_perm [R,H]; B = w_down viewed as [E*I, H] (rows are
+// output columns, K = H contiguous).
+int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_down, const int32_t* offsets,
+                      bf16* dh_act, cudaStream_t s) {
+    const uint64_t R = (uint64_t)d.T * d.K;
+    CUtensorMap a, b0;
+    if (!make_map(&a, dy_perm, d.H, R, BK, BM) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, BN))
+        return MOE_ERR_CUDA;
+    Params p = {};
+    p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
+    p.n_tiles = (d.I + BN - 1) / BN; p.n_cols = d.I; p.b_rows_per_e = d.I;
+    p.out0 = dh_act; p.ldo = d.I; p.n_split = d.I;
+    return launch<DGRAD>(a, b0, b0, p, s);
+}
+
+// Gate/up dgrad: dx_perm = dg . w_gate[e]^T + du . w_up[e]^T.  A = dgu [R,2I]; the contraction runs over the
+// gate half against w_gate viewed as [E*H, I], then over the up half against w_up.
+int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate, const bf16* w_up,
+                        const int32_t* offsets, bf16* dx_perm, cudaStream_t s) {
+    const uint64_t R = (uint64_t)d.T * d.K;
+    CUtensorMap a, b0, b1;
+    if (!make_map(&a, dgu, 2ull * d.I, R, BK, BM) || !make_map(&b0, w_gate, d.I, (uint64_t)d.E * d.H, BK, BN) ||
+        !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, BK, BN))
+        return MOE_ERR_CUDA;
+    Params p = {};
+    p.offsets = offsets; p.E = d.E; p.k_blocks = 2 * d.I / BK; p.k_split = d.I / BK;
+    p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.b_rows_per_e = d.H;
+    p.out0 = dx_perm; p.ldo = d.H; p.n_split = d.H;
+    return launch<DGRAD>(a, b0, b1, p, s);
+}
+
+// Down wgrad: dw_down[e] [I,H] = h_act_e^T . dy_perm_e.  A = h_act [R,I] (M = I), B = dy_perm [R,H] (N = H).
+int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_perm, const int32_t* offsets,
+                      bf16* dw_down, cudaStream_t s) {
+    const uint64_t R = (uint64_t)d.T * d.K;
+    CUtensorMap a, b0;
+    if (!make_map(&a, h_act, d.I, R, 64, BK) || !make_map(&b0, dy_perm, d.H, R, 64, BK)) return MOE_ERR_CUDA;
+    Params p = {};
+    p.offsets = offsets; p.E = d.E; p.m_tiles = d.I / BM; p.n_tiles = (d.H + BN - 1) / BN;
+    p.n_cols = d.H; p.n_split = d.H; p.ldo = d.H; p.out_e_stride = (long long)d.I * d.H;
+    p.out0 = dw_down; p.out1 = nullptr;
+    return launch<WGRAD>(a, b0, b0, p, s);
+}
+
+// Gate/up wgrad (the paper's dW1): [dw_gate[e] | dw_up[e]] = x_perm_e^T . dgu_e.  A = x_perm [R,H] (M = H),
+// B = dgu [R,2I] (N = 2I); output columns below I go to dw_gate, the rest to dw_up.
+int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu, const int32_t* offsets,
+                        bf16* dw_gate, bf16* dw_up, cudaStream_t s) {
+    const uint64_t R = (uint64_t)d.T * d.K;
+    CUtensorMap a, b0;
+    if (!make_map(&a, x_perm, d.H, R, 64, BK) || !make_map(&b0, dgu, 2ull * d.I, R, 64, BK)) return MOE_ERR_CUDA;
+    Params p = {};
+    p.offsets = offsets; p.E = d.E; p.m_tiles = d.H / BM; p.n_tiles = (2 * d.I + BN - 1) / BN;
+    p.n_cols = 2 * d.I; p.n_split = d.I; p.ldo = d.I; p.out_e_stride = (long long)d.H * d.I;
+    p.out0 = dw_gate; p.out1 = dw_up;
+    return launch<WGRAD>(a, b0, b0, p, s);
+}
+
+}  // namespace moe

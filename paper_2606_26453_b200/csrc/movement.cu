@@ -1,0 +1,425 @@
+// HBM-bound kernels of the MoE layer: route-permute (stable counting sort by expert + row
+// gather), unpermute-combine and its backward, permute backward, SwiGLU backward.
+//
+// Row movement is token-major: every source row is read once with 16-byte loads and written (or
+// gathered) K times, so the bytes moved are the algorithmic minimum.  The permutation indices
+// never depend on the order in which atomics land: ranks come from warp-level match/ballot
+// scans over pairs taken in ascending pair id, which makes the result the unique stable sort.
+#include "common.cuh"
+
+namespace moe {
+
+namespace {
+
+constexpr int kPairsPerWarp = 256;   // pairs ranked by one warp (8 rounds of 32)
+constexpr int kWarpsPerBlock = 8;
+constexpr int kThreads = kWarpsPerBlock * 32;
+
+__device__ __forceinline__ uint4 ldg16(const uint4* p) { return __ldg(p); }
+
+__device__ __forceinline__ void unpack8(const uint4& v, float f[8]) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float2 t = __bfloat1622float2(h[i]);
+        f[2 * i] = t.x;
+        f[2 * i + 1] = t.y;
+    }
+}
+
+__device__ __forceinline__ uint4 pack8(const float f[8]) {
+    uint4 v;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) h[i] = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+    return v;
+}
+
+// ------------------------------------------------------------------------------------------------
+// a1, index part.  Three small kernels over the R = T*K pairs, split into warp-chunks of
+// kPairsPerWarp consecutive pairs:
+//   hist : per warp-chunk, the number of pairs of each expert           -> ws[chunk][e]
+//   scan : per expert, exclusive prefix over the chunks (in place), total -> counts[e]
+//   rank : offsets = exclusive prefix of counts; row(p) = offsets[e] + ws[chunk][e] + number of
+//          earlier pairs of the same expert inside the chunk.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* __restrict__ topk_idx, int R, int E,
+                                                                int n_chunks, int32_t* __restrict__ ws) {
+    extern __shared__ int32_t smem_i[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int chunk = blockIdx.x * kWarpsPerBlock + warp;
+    if (chunk >= n_chunks) return;
+    int32_t* hist = smem_i + warp * E;
+    for (int e = lane; e < E; e += 32) hist[e] = 0;
+    __syncwarp();
+    const int p0 = chunk * kPairsPerWarp;
+#pragma unroll 1
+    for (int it = 0; it < kPairsPerWarp / 32; ++it) {
+        const int p = p0 + it * 32 + lane;
+        int e = (p < R) ? topk_idx[p] : -1;
+        if (e >= E) e = -1;
+        const unsigned mask = __match_any_sync(0xffffffffu, e);
+        if (e >= 0 && lane == __ffs(mask) - 1) hist[e] += __popc(mask);
+        __syncwarp();
+    }
+    int32_t* out = ws + (size_t)chunk * E;
+    for (int e = lane; e < E; e += 32) out[e] = hist[e];
+}
+
+__global__ void __launch_bounds__(kThreads) permute_scan_kernel(int32_t* __restrict__ ws, int n_chunks, int E,
+                                                                int32_t* __restrict__ counts) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int e = blockIdx.x * kWarpsPerBlock + warp;
+    if (e >= E) return;
+    const int per = (n_chunks + 31) / 32;
+    const int c0 = min(lane * per, n_chunks), c1 = min(c0 + per, n_chunks);
+    int sum = 0;
+    for (int c = c0; c < c1; ++c) sum += ws[(size_t)c * E + e];
+    int incl = sum;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    int run = incl - sum;
+    for (int c = c0; c < c1; ++c) {
+        const int v = ws[(size_t)c * E + e];
+        ws[(size_t)c * E + e] = run;
+        run += v;
+    }
+    if (lane == 31) counts[e] = incl;
+}
+
+__global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* __restrict__ topk_idx, int R, int E,
+                                                                int n_chunks, const int32_t* __restrict__ ws,
+                                                                const int32_t* __restrict__ counts,
+                                                                int32_t* __restrict__ offsets,
+                                                                int32_t* __restrict__ row_to_pair,
+                                                                int32_t* __restrict__ pair_to_row) {
+    extern __shared__ int32_t smem_i[];
+    int32_t* offs = smem_i;                 // [E+1]
+    int32_t* running_all = smem_i + E + 1;  // [warps][E]
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // offsets = exclusive prefix of counts, by warp 0 (each lane owns a contiguous run of experts)
+    if (warp == 0) {
+        const int per = (E + 31) / 32;
+        const int e0 = min(lane * per, E), e1 = min(e0 + per, E);
+        int sum = 0;
+        for (int e = e0; e < e1; ++e) sum += counts[e];
+        int incl = sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += v;
+        }
+        int run = incl - sum;
+        for (int e = e0; e < e1; ++e) {
+            offs[e] = run;
+            run += counts[e];
+        }
+        if (lane == 31) offs[E] = incl;
+    }
+    __syncthreads();
+    if (blockIdx.x == 0)
+        for (int e = threadIdx.x; e <= E; e += kThreads) offsets[e] = offs[e];
+
+    const int chunk = blockIdx.x * kWarpsPerBlock + warp;
+    if (chunk >= n_chunks) return;
+    int32_t* running = running_all + warp * E;
+    const int32_t* base = ws + (size_t)chunk * E;
+    for (int e = lane; e < E; e += 32) running[e] = offs[e] + base[e];
+    __syncwarp();
+    const int p0 = chunk * kPairsPerWarp;
+    const unsigned lt_mask = (1u << lane) - 1u;
+#pragma unroll 1
+    for (int it = 0; it < kPairsPerWarp / 32; ++it) {
+        const int p = p0 + it * 32 + lane;
+        int e = (p < R) ? topk_idx[p] : -1;
+        if (e >= E) e = -1;
+        const unsigned mask = __match_any_sync(0xffffffffu, e);
+        if (e >= 0) {
+            const int row = running[e] + __popc(mask & lt_mask);
+            row_to_pair[row] = p;
+            pair_to_row[p] = row;
+        }
+        __syncwarp();
+        if (e >= 0 && lane == __ffs(mask) - 1) running[e] += __popc(mask);
+        __syncwarp();
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// a1, row part: x_perm[pair_to_row[t*K+k], :] = x[t, :].  One thread per 16-byte piece of a token
+// row; the piece is loaded once and stored to the K destination rows.
+// ------------------------------------------------------------------------------------------------
+template <int KT>
+__global__ void __launch_bounds__(kThreads) permute_rows_kernel(const uint4* __restrict__ x,
+                                                                const int32_t* __restrict__ pair_to_row,
+                                                                uint4* __restrict__ x_perm, long long total,
+                                                                int hv, int K) {
+    const long long i = (long long)blockIdx.x * kThreads + threadIdx.x;
+    if (i >= total) return;
+    const int t = (int)(i / hv);
+    const int c = (int)(i - (long long)t * hv);
+    const uint4 v = ldg16(x + i);
+    const int32_t* rows = pair_to_row + (long long)t * K;
+    if (KT > 0) {
+        int r[KT > 0 ? KT : 1];
+#pragma unroll
+        for (int k = 0; k < KT; ++k) r[k] = __ldg(rows + k);
+#pragma unroll
+        for (int k = 0; k < KT; ++k) x_perm[(long long)r[k] * hv + c] = v;
+    } else {
+        for (int k = 0; k < K; ++k) x_perm[(long long)__ldg(rows + k) * hv + c] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// a4 / a8: dst[t,:] = sum_k w[t,k] * src[pair_to_row[t*K+k], :]  (w == NULL: unit weights).
+// fp32 accumulation in slot order, one rounding to bf16.
+// ------------------------------------------------------------------------------------------------
+template <int KT, bool WEIGHTED>
+__global__ void __launch_bounds__(kThreads) gather_sum_kernel(const uint4* __restrict__ src,
+                                                              const float* __restrict__ topk_w,
+                                                              const int32_t* __restrict__ pair_to_row,
+                                                              uint4* __restrict__ dst, long long total, int hv,
+                                                              int K) {
+    const long long i = (long long)blockIdx.x * kThreads + threadIdx.x;
+    if (i >= total) return;
+    const int t = (int)(i / hv);
+    const int c = (int)(i - (long long)t * hv);
+    const int32_t* rows = pair_to_row + (long long)t * K;
+    float acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+    if (KT > 0) {
+        uint4 v[KT > 0 ? KT : 1];
+        float w[KT > 0 ? KT : 1];
+#pragma unroll
+        for (int k = 0; k < KT; ++k) {
+            v[k] = ldg16(src + (long long)__ldg(rows + k) * hv + c);
+            w[k] = WEIGHTED ? __ldg(topk_w + (long long)t * K + k) : 1.f;
+        }
+#pragma unroll
+        for (int k = 0; k < KT; ++k) {
+            float f[8];
+            unpack8(v[k], f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = WEIGHTED ? fmaf(w[k], f[j], acc[j]) : acc[j] + f[j];
+        }
+    } else {
+        for (int k = 0; k < K; ++k) {
+            const uint4 v = ldg16(src + (long long)__ldg(rows + k) * hv + c);
+            const float w = WEIGHTED ? __ldg(topk_w + (long long)t * K + k) : 1.f;
+            float f[8];
+            unpack8(v, f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = WEIGHTED ? fmaf(w, f[j], acc[j]) : acc[j] + f[j];
+        }
+    }
+    dst[i] = pack8(acc);
+}
+
+// ------------------------------------------------------------------------------------------------
+// a5: one warp per token.  dy_perm[row_k, :] = w_k * dy[t, :]; dtopk_w[t,k] = <dy[t,:], y_perm[row_k,:]>.
+// ------------------------------------------------------------------------------------------------
+template <int KT, bool WITH_DW>
+__global__ void __launch_bounds__(kThreads) combine_bwd_kernel(const uint4* __restrict__ dy,
+                                                               const uint4* __restrict__ y_perm,
+                                                               const float* __restrict__ topk_w,
+                                                               const int32_t* __restrict__ pair_to_row,
+                                                               uint4* __restrict__ dy_perm,
+                                                               float* __restrict__ dtopk_w, int T, int hv, int K) {
+    constexpr int KA = KT > 0 ? KT : 32;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t = blockIdx.x * kWarpsPerBlock + warp;
+    if (t >= T) return;
+    const int kk = KT > 0 ? KT : K;
+    int rows[KA];
+    float w[KA], dot[KA];
+#pragma unroll
+    for (int k = 0; k < KA; ++k) {
+        if (k < kk) {
+            rows[k] = __ldg(pair_to_row + (long long)t * K + k);
+            w[k] = __ldg(topk_w + (long long)t * K + k);
+        }
+        dot[k] = 0.f;
+    }
+    for (int c = lane; c < hv; c += 32) {
+        const uint4 dv = ldg16(dy + (long long)t * hv + c);
+        float d[8];
+        unpack8(dv, d);
+        uint4 yv[KA];
+        if (WITH_DW) {
+#pragma unroll
+            for (int k = 0; k < KA; ++k)
+                if (k < kk) yv[k] = ldg16(y_perm + (long long)rows[k] * hv + c);
+        }
+#pragma unroll
+        for (int k = 0; k < KA; ++k) {
+            if (k < kk) {
+                float o[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) o[j] = w[k] * d[j];
+                dy_perm[(long long)rows[k] * hv + c] = pack8(o);
+                if (WITH_DW) {
+                    float y[8];
+                    unpack8(yv[k], y);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) dot[k] = fmaf(d[j], y[j], dot[k]);
+                }
+            }
+        }
+    }
+    if (WITH_DW) {
+#pragma unroll
+        for (int k = 0; k < KA; ++k) {
+            if (k < kk) {
+                float v = dot[k];
+#pragma unroll
+                for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
+                if (lane == 0) dtopk_w[(long long)t * K + k] = v;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// a7, elementwise part: dGU = [dg | du] from dHact and the saved pre-activations [g | u].
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) swiglu_bwd_kernel(const uint4* __restrict__ dh_act,
+                                                              const uint4* __restrict__ gu,
+                                                              uint4* __restrict__ dgu, long long total, int iv) {
+    const long long i = (long long)blockIdx.x * kThreads + threadIdx.x;
+    if (i >= total) return;
+    const long long r = i / iv;
+    const int c = (int)(i - r * iv);
+    const uint4 dhv = ldg16(dh_act + i);
+    const uint4 gv = ldg16(gu + r * (2 * iv) + c);
+    const uint4 uv = ldg16(gu + r * (2 * iv) + iv + c);
+    float dh[8], g[8], u[8], dg[8], du[8];
+    unpack8(dhv, dh);
+    unpack8(gv, g);
+    unpack8(uv, u);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float s = 1.f / (1.f + __expf(-g[j]));
+        dg[j] = dh[j] * u[j] * s * (1.f + g[j] * (1.f - s));
+        du[j] = dh[j] * g[j] * s;
+    }
+    dgu[r * (2 * iv) + c] = pack8(dg);
+    dgu[r * (2 * iv) + iv + c] = pack8(du);
+}
+
+inline unsigned blocks_for(long long total) { return (unsigned)((total + kThreads - 1) / kThreads); }
+
+}  // namespace
+
+size_t permute_workspace_bytes(const moe_dims_t& d) {
+    const long long R = (long long)d.T * d.K;
+    const long long n_chunks = (R + kPairsPerWarp - 1) / kPairsPerWarp;
+    return (size_t)(n_chunks * d.E) * sizeof(int32_t);
+}
+
+int launch_permute(const moe_dims_t& d, const bf16* x, const int32_t* topk_idx, bf16* x_perm, int32_t* counts,
+                   int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row, void* workspace,
+                   cudaStream_t s) {
+    const int R = d.T * d.K, E = d.E;
+    const int n_chunks = (R + kPairsPerWarp - 1) / kPairsPerWarp;
+    const int chunk_blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    int32_t* ws = static_cast<int32_t*>(workspace);
+    permute_hist_kernel<<<chunk_blocks, kThreads, kWarpsPerBlock * E * sizeof(int32_t), s>>>(topk_idx, R, E,
+                                                                                             n_chunks, ws);
+    permute_scan_kernel<<<(E + kWarpsPerBlock - 1) / kWarpsPerBlock, kThreads, 0, s>>>(ws, n_chunks, E, counts);
+    permute_rank_kernel<<<chunk_blocks, kThreads, ((kWarpsPerBlock + 1) * E + 1) * sizeof(int32_t), s>>>(
+        topk_idx, R, E, n_chunks, ws, counts, offsets, row_to_pair, pair_to_row);
+    if (x_perm != nullptr) {
+        const int hv = d.H / 8;
+        const long long total = (long long)d.T * hv;
+        const uint4* src = reinterpret_cast<const uint4*>(x);
+        uint4* dst = reinterpret_cast<uint4*>(x_perm);
+#define MOE_ROWS_CASE(KT)                                                                                  \
+    case KT:                                                                                               \
+        permute_rows_kernel<KT><<<blocks_for(total), kThreads, 0, s>>>(src, pair_to_row, dst, total, hv, d.K); \
+        break;
+        switch (d.K) {
+            MOE_ROWS_CASE(1) MOE_ROWS_CASE(2) MOE_ROWS_CASE(3) MOE_ROWS_CASE(4) MOE_ROWS_CASE(5) MOE_ROWS_CASE(6)
+            MOE_ROWS_CASE(7) MOE_ROWS_CASE(8)
+            default:
+                permute_rows_kernel<0><<<blocks_for(total), kThreads, 0, s>>>(src, pair_to_row, dst, total, hv, d.K);
+        }
+#undef MOE_ROWS_CASE
+    }
+    return check_launch();
+}
+
+template <bool WEIGHTED>
+static void gather_sum_dispatch(const moe_dims_t& d, const uint4* src, const float* w, const int32_t* p2r,
+                                uint4* dst, cudaStream_t s) {
+    const int hv = d.H / 8;
+    const long long total = (long long)d.T * hv;
+#define MOE_GS_CASE(KT)                                                                                          \
+    case KT:                                                                                                     \
+        gather_sum_kernel<KT, WEIGHTED><<<blocks_for(total), kThreads, 0, s>>>(src, w, p2r, dst, total, hv, d.K); \
+        break;
+    switch (d.K) {
+        MOE_GS_CASE(1) MOE_GS_CASE(2) MOE_GS_CASE(3) MOE_GS_CASE(4) MOE_GS_CASE(5) MOE_GS_CASE(6) MOE_GS_CASE(7)
+        MOE_GS_CASE(8)
+        default:
+            gather_sum_kernel<0, WEIGHTED><<<blocks_for(total), kThreads, 0, s>>>(src, w, p2r, dst, total, hv, d.K);
+    }
+#undef MOE_GS_CASE
+}
+
+int launch_gather_sum(const moe_dims_t& d, const bf16* src_perm, const float* topk_w, const int32_t* pair_to_row,
+                      bf16* dst, cudaStream_t s) {
+    const uint4* src = reinterpret_cast<const uint4*>(src_perm);
+    uint4* out = reinterpret_cast<uint4*>(dst);
+    if (topk_w != nullptr)
+        gather_sum_dispatch<true>(d, src, topk_w, pair_to_row, out, s);
+    else
+        gather_sum_dispatch<false>(d, src, nullptr, pair_to_row, out, s);
+    return check_launch();
+}
+
+template <bool WITH_DW>
+static void combine_bwd_dispatch(const moe_dims_t& d, const uint4* dy, const uint4* yp, const float* w,
+                                 const int32_t* p2r, uint4* dyp, float* dw, cudaStream_t s) {
+    const int hv = d.H / 8;
+    const unsigned blocks = (unsigned)((d.T + kWarpsPerBlock - 1) / kWarpsPerBlock);
+#define MOE_CB_CASE(KT)                                                                                     \
+    case KT:                                                                                                \
+        combine_bwd_kernel<KT, WITH_DW><<<blocks, kThreads, 0, s>>>(dy, yp, w, p2r, dyp, dw, d.T, hv, d.K); \
+        break;
+    switch (d.K) {
+        MOE_CB_CASE(1) MOE_CB_CASE(2) MOE_CB_CASE(3) MOE_CB_CASE(4) MOE_CB_CASE(5) MOE_CB_CASE(6) MOE_CB_CASE(7)
+        MOE_CB_CASE(8)
+        default:
+            combine_bwd_kernel<0, WITH_DW><<<blocks, kThreads, 0, s>>>(dy, yp, w, p2r, dyp, dw, d.T, hv, d.K);
+    }
+#undef MOE_CB_CASE
+}
+
+int launch_combine_bwd(const moe_dims_t& d, const bf16* dy, const bf16* y_perm, const float* topk_w,
+                       const int32_t* pair_to_row, bf16* dy_perm, float* dtopk_w, cudaStream_t s) {
+    const uint4* a = reinterpret_cast<const uint4*>(dy);
+    const uint4* b = reinterpret_cast<const uint4*>(y_perm);
+    uint4* o = reinterpret_cast<uint4*>(dy_perm);
+    if (dtopk_w != nullptr)
+        combine_bwd_dispatch<true>(d, a, b, topk_w, pair_to_row, o, dtopk_w, s);
+    else
+        combine_bwd_dispatch<false>(d, a, b, topk_w, pair_to_row, o, nullptr, s);
+    return check_launch();
+}
+
+int launch_swiglu_bwd(const moe_dims_t& d, const bf16* dh_act, const bf16* gu, bf16* dgu, cudaStream_t s) {
+    const int iv = d.I / 8;
+    const long long total = (long long)d.T * d.K * iv;
+    swiglu_bwd_kernel<<<blocks_for(total), kThreads, 0, s>>>(reinterpret_cast<const uint4*>(dh_act),
+                                                            reinterpret_cast<const uint4*>(gu),
+                                                            reinterpret_cast<uint4*>(dgu), total, iv);
+    return check_launch();
+}
+
+}  // namespace moe
