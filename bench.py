@@ -1,0 +1,437 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE expert-FFN layer (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+A step is one pass of the whole hot path (route-permute, gate/up GEMM + SwiGLU, down GEMM,
+unpermute-combine, and the four backward calls) over one batch of seeded synthetic input.  The
+metric is whole-layer throughput in TFLOP/s on the algorithmic work 18*R*H*I; the JSON line also
+carries the grouped-GEMM-only throughput, the permute bandwidth, a roofline object for the
+dominant kernel, an end-to-end number through the host-buffer entry point and the fp64 oracle
+timed on the host cores.  With N > 1 (torchrun) every rank runs an independent replica of the
+same workload: the layer is single-GPU by design, there is no collective on the data path.
+`--impl reference` times the CPU oracle alone on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2606_26453_b200 import workloads as W
+
+METRIC = "moe_layer_fwd_bwd_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------------------------
+# clock sampling during the timed region (read-only NVML queries)
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+
+    def __init__(self, device_index: int, period_s: float = 0.005):
+        self.samples, self.reasons, self.power = [], set(), []
+        self.period = period_s
+        self.stop_flag = threading.Event()
+        self.thread = None
+        self.max_mhz = None
+        self.handle = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = torch.cuda.get_device_properties(device_index).uuid
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.nv = pynvml
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.handle = None
+
+    def _run(self):
+        nv = self.nv
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.handle) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.handle is not None:
+            self.thread = threading.Thread(target=self._run, daemon=True)
+            self.thread.start()
+
+    def stop(self):
+        if self.thread is not None:
+            self.stop_flag.set()
+            self.thread.join()
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples),
+                "power_w_max": max(self.power) if self.power else None}
+
+
+# --------------------------------------------------------------------------------------------
+# one step of the CUDA path, as the fine-grained C-ABI calls (so every kernel can be timed)
+# --------------------------------------------------------------------------------------------
+CALLS = ["permute", "gateup_swiglu", "down", "combine", "combine_bwd", "down_dgrad", "down_wgrad", "swiglu_bwd",
+         "gateup_dgrad", "gateup_wgrad", "permute_bwd"]
+LAUNCHES_PER_CALL = {"permute": 4}
+GEMM_CALLS = ["gateup_swiglu", "down", "down_dgrad", "down_wgrad", "gateup_dgrad", "gateup_wgrad"]
+
+
+def call_flops(cfg):
+    rhi = float(cfg.R) * cfg.H * cfg.I
+    return {"gateup_swiglu": 4 * rhi, "down": 2 * rhi, "down_dgrad": 2 * rhi, "down_wgrad": 2 * rhi,
+            "gateup_dgrad": 4 * rhi, "gateup_wgrad": 4 * rhi}
+
+
+def call_bytes(cfg):
+    T, H, I, E, K, R = cfg.T, cfg.H, cfg.I, cfg.E, cfg.K, cfg.R
+    return {"permute": T * H * 2 + R * H * 2 + R * 4 + 2 * R * 4 + (2 * E + 1) * 4,
+            "combine": R * H * 2 + T * H * 2 + 2 * R * 4,
+            "combine_bwd": T * H * 2 + 2 * R * H * 2 + 2 * R * 4 + R * 4,
+            "swiglu_bwd": R * I * 2 * 5,
+            "permute_bwd": R * H * 2 + T * H * 2 + R * 4}
+
+
+def make_step(B, b, wl):
+    x, idx, w, dy = wl["X"], wl["topk_idx"], wl["topk_w"], wl["dY"]
+    wg, wu, wd = wl["W_gate"], wl["W_up"], wl["W_down"]
+    d = b.d
+    fns = [
+        lambda: B.moe_permute(d, x, idx, b.x_perm, b.counts, b.offsets, b.row_to_pair, b.pair_to_row, b.workspace),
+        lambda: B.moe_grouped_gemm_gateup_swiglu(d, b.x_perm, wg, wu, b.offsets, b.h_act, b.gu),
+        lambda: B.moe_grouped_gemm_down(d, b.h_act, wd, b.offsets, b.y_perm),
+        lambda: B.moe_unpermute_combine(d, b.y_perm, w, b.pair_to_row, b.y),
+        lambda: B.moe_unpermute_combine_bwd(d, dy, b.y_perm, w, b.pair_to_row, b.dy_perm, b.dtopk_w),
+        lambda: B.moe_grouped_gemm_down_dgrad(d, b.dy_perm, wd, b.offsets, b.dh_act),
+        lambda: B.moe_grouped_gemm_down_wgrad(d, b.h_act, b.dy_perm, b.offsets, b.dw_down),
+        lambda: B.moe_swiglu_bwd(d, b.dh_act, b.gu, b.dgu),
+        lambda: B.moe_grouped_gemm_gateup_dgrad(d, b.dgu, wg, wu, b.offsets, b.dx_perm),
+        lambda: B.moe_grouped_gemm_gateup_wgrad(d, b.x_perm, b.dgu, b.offsets, b.dw_gate, b.dw_up),
+        lambda: B.moe_permute_bwd(d, b.dx_perm, b.pair_to_row, b.dx),
+    ]
+
+    def step(events=None):
+        if events is None:
+            for f in fns:
+                f()
+            return
+        events[0].record()
+        for i, f in enumerate(fns):
+            f()
+            events[i + 1].record()
+
+    return step
+
+
+def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True):
+    wl = W.make_workload_device(cfg, device)
+    b = B.alloc_layer_buffers(cfg.T, cfg.H, cfg.I, cfg.E, cfg.K, device=device)
+    step = make_step(B, b, wl)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    if B.moe_device_status() != 0:
+        raise RuntimeError("device status word is set after warm-up")
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(steps)]
+    t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(device.index if device.index is not None else 0) if sample_clocks else None
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.start()
+    t_start.record()
+    for s in range(steps):
+        step(evs[s])
+    t_end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    if dist is not None:
+        dist.barrier()
+    total_ms = t_start.elapsed_time(t_end)
+    per_call = {}
+    for i, name in enumerate(CALLS):
+        per_call[name] = sum(evs[s][i].elapsed_time(evs[s][i + 1]) for s in range(steps)) / steps
+    if B.moe_device_status() != 0:
+        raise RuntimeError("device status word is set after the timed region")
+    return dict(wl=wl, buffers=b, total_ms=total_ms, per_call_ms=per_call, clocks=clocks)
+
+
+def summarize(cfg, res, steps, peaks):
+    ms_step = res["total_ms"] / steps
+    pc = res["per_call_ms"]
+    flops = call_flops(cfg)
+    nbytes = call_bytes(cfg)
+    gemm_ms = sum(pc[c] for c in GEMM_CALLS)
+    out = {
+        "workload": cfg.name, "ms_per_step": ms_step,
+        "layer_tflops": cfg.flops_fwd_bwd / (ms_step * 1e-3) / 1e12,
+        "gemm_tflops": cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12,
+        "gemm_frac_of_nominal_2250": cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS,
+        "gemm_frac_of_measured_burst": cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "gemm_frac_of_measured_sustained": cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+        "per_call_ms": {k: round(v, 5) for k, v in pc.items()},
+        "per_call_tflops": {c: round(flops[c] / (pc[c] * 1e-3) / 1e12, 1) for c in GEMM_CALLS},
+        "per_call_gbs": {c: round(nbytes[c] / (pc[c] * 1e-3) / 1e9, 1) for c in nbytes},
+        "permute_gbs": nbytes["permute"] / (pc["permute"] * 1e-3) / 1e9,
+        "permute_frac_of_nominal_8000": nbytes["permute"] / (pc["permute"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "permute_frac_of_measured": nbytes["permute"] / (pc["permute"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+    }
+    return out
+
+
+def roofline_object(cfg, res, peaks, peaks_kind):
+    pc = res["per_call_ms"]
+    flops = call_flops(cfg)
+    dom = max(GEMM_CALLS, key=lambda c: pc[c])
+    achieved = flops[dom] / (pc[dom] * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"]
+    return {"bound": "tensor", "kernel": "grouped_gemm_kernel[" + dom + "]", "achieved": achieved, "peak": peak,
+            "peak_kind": "bf16 cuBLAS burst, of " + peaks_kind, "unit": "TFLOP/s", "frac": achieved / peak,
+            "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+            "flops_per_launch": flops[dom], "avg_launch_ms": pc[dom],
+            "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, dom))}
+
+
+# --------------------------------------------------------------------------------------------
+# end to end through the host-buffer entry point
+# --------------------------------------------------------------------------------------------
+def time_e2e(B, cfg, wl, b, device, steps, warmup, dist=None):
+    d = b.d
+    arena = torch.empty(B.moe_layer_arena_bytes(d), dtype=torch.uint8, device=device)
+    pin = lambda t: t.cpu().pin_memory()
+    xh, ih, wh, dyh = pin(wl["X"]), pin(wl["topk_idx"]), pin(wl["topk_w"]), pin(wl["dY"])
+    yh = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16).pin_memory()
+    dxh = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16).pin_memory()
+    dwh = torch.empty((cfg.T, cfg.K), dtype=torch.float32).pin_memory()
+
+    def step():
+        B.moe_layer_fwd_bwd_host(d, xh, ih, wh, dyh, wl["W_gate"], wl["W_up"], wl["W_down"], yh, dxh, dwh,
+                                 b.dw_gate, b.dw_up, b.dw_down, arena)
+
+    for _ in range(warmup):
+        step()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    h2d = xh.numel() * 2 + ih.numel() * 4 + wh.numel() * 4 + dyh.numel() * 2
+    d2h = yh.numel() * 2 + dxh.numel() * 2 + dwh.numel() * 4
+    del arena
+    return ms, h2d, d2h
+
+
+# --------------------------------------------------------------------------------------------
+# the fp64 oracle on the host cores (baseline, not the target)
+# --------------------------------------------------------------------------------------------
+def oracle_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p["num_threads"] for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample_time(host, cfg, n_tokens):
+    """Runs the whole oracle chain on the first n_tokens tokens (all experts' weights); seconds."""
+    from oracle import moe_oracle as O
+    t0 = time.perf_counter()
+    O.layer_fwd_bwd(host["X"][:n_tokens], host["topk_idx"][:n_tokens], host["topk_w"][:n_tokens], host["W_gate"],
+                    host["W_up"], host["W_down"], host["dY"][:n_tokens])
+    return time.perf_counter() - t0
+
+
+def host_copy(wl):
+    return {k: (v.to(torch.float32).cpu().numpy() if v.dtype == torch.bfloat16 else v.cpu().numpy())
+            for k, v in wl.items()}
+
+
+def cpu_baseline(cfg, host, n_tokens):
+    oracle_sample_time(host, cfg, min(n_tokens, 16))          # first-touch / BLAS thread start-up, untimed
+    sec = oracle_sample_time(host, cfg, n_tokens)
+    fl = 18.0 * n_tokens * cfg.K * cfg.H * cfg.I
+    return {"value": fl / sec / 1e12, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"fp64 numpy oracle, whole fwd+bwd chain on the first {n_tokens} of {cfg.T} tokens of "
+                      f"'{cfg.name}' (all {cfg.E} experts' weights), {sec:.1f} s",
+            "seconds": sec}
+
+
+# --------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The oracle as the reference arm: rank 0 only, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = W.CONFIGS[args.config]
+    host = W.make_workload(cfg) if args.host_inputs == "numpy" else None
+    if host is None:
+        if torch.cuda.is_available():
+            host = host_copy(W.make_workload_device(cfg, torch.device("cuda", 0)))
+        else:
+            host = W.make_workload(cfg)
+    n_tok = min(args.ref_tokens, cfg.T)
+    budget = 240.0 / max(1, args.steps + args.warmup)
+    oracle_sample_time(host, cfg, 16)
+    while True:
+        t = oracle_sample_time(host, cfg, n_tok)
+        if t <= budget or n_tok <= 16:
+            break
+        n_tok //= 2
+    for _ in range(max(0, args.warmup - 1)):
+        oracle_sample_time(host, cfg, n_tok)
+    times = [oracle_sample_time(host, cfg, n_tok) for _ in range(args.steps)]
+    sec = sum(times) / len(times)
+    value = 18.0 * n_tok * cfg.K * cfg.H * cfg.I / sec / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E": cfg.E, "K": cfg.K,
+                       "sample_tokens_per_step": n_tok},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+                             "sample": f"each step = fp64 numpy oracle fwd+bwd chain on the first {n_tok} of {cfg.T} tokens"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback of the CUDA path)")
+    from paper_2606_26453_b200 import binding as B
+    B.load_library()
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group(backend="nccl", device_id=device)
+        dist = dist_mod
+    peaks, peaks_kind = load_peaks()
+    cfg = W.CONFIGS[args.config]
+
+    res = time_config(B, cfg, device, args.steps, args.warmup, dist)
+    e2e_ms, h2d, d2h = time_e2e(B, cfg, res["wl"], res["buffers"], device, args.steps, args.warmup, dist)
+
+    total_ms, e2e_ms_max = res["total_ms"], e2e_ms
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms_max = float(t[0]), float(t[1])
+    ms_step = total_ms / args.steps
+    value = world * cfg.flops_fwd_bwd / (ms_step * 1e-3) / 1e12
+    summary = summarize(cfg, res, args.steps, peaks)
+    launches_per_step = sum(LAUNCHES_PER_CALL.get(c, 1) for c in CALLS)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E": cfg.E, "K": cfg.K,
+                   "routing": cfg.routing, "parallelism": "replicas only (single-GPU layer)" if world > 1 else "1 GPU",
+                   "l2": "no flush: the step's working set (weights + activations) exceeds the 126 MB L2 many times"},
+        "clocks": res["clocks"],
+        "e2e": {"value": world * cfg.flops_fwd_bwd / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_max,
+                "note": "moe_layer_fwd_bwd_host: activations, routing and upstream gradient from pinned host "
+                        "memory each step; weights and weight gradients stay on the device"},
+        "gpu_launches": launches_per_step * args.steps,
+        "roofline": roofline_object(cfg, res, peaks, peaks_kind),
+        "pct_of_dense_bf16_peak_nominal": 100.0 * summary["gemm_frac_of_nominal_2250"],
+        "gemm_tflops": summary["gemm_tflops"], "permute_gbs": summary["permute_gbs"],
+        "detail": summary, "peaks": {"kind": peaks_kind, "hbm_gbs": peaks["hbm_gbs"], "bf16_tflops": peaks["bf16_tflops"],
+                                     "bf16_tflops_sustained": peaks["bf16_tflops_sustained"]},
+    }
+
+    if rank == 0 and world == 1:
+        extra = []
+        wl_host = host_copy(res["wl"]) if not args.no_cpu_baseline else None
+        del res
+        torch.cuda.empty_cache()
+        for name in args.also:
+            c2 = W.CONFIGS[name]
+            r2 = time_config(B, c2, device, max(3, args.steps // 4), 3, None, sample_clocks=True)
+            s2 = summarize(c2, r2, max(3, args.steps // 4), peaks)
+            s2["clocks"] = r2["clocks"]
+            extra.append(s2)
+            del r2
+            torch.cuda.empty_cache()
+        if extra:
+            line["other_configs"] = extra
+        if wl_host is not None:
+            line["cpu_baseline"] = cpu_baseline(cfg, wl_host, min(args.ref_tokens, cfg.T))
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--config", default="fine_grained", choices=list(W.CONFIGS))
+    ap.add_argument("--also", default="many_small,few_large,imbalanced",
+                    help="comma-separated other configurations to time briefly at N=1 ('' for none)")
+    ap.add_argument("--ref-tokens", type=int, default=512, help="tokens in the oracle's timed sample")
+    ap.add_argument("--host-inputs", default="device", choices=["device", "numpy"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    args.also = [s for s in args.also.split(",") if s]
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
