@@ -86,6 +86,31 @@ int moe_permute(const moe_dims_t* dims, const void* x, const int32_t* topk_idx, 
                 int32_t* counts, int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row,
                 void* workspace, size_t workspace_bytes, moe_stream_t stream);
 
+/* ---- route-permute for callers that cannot allocate device memory ----------------------------
+ * (The paper has no counterpart of this call; it exists for integration reasons only.)
+ * Same inputs, outputs and results as moe_permute, but without the workspace argument: the
+ * scratch table sits in a fixed array inside the library image, MOE_PERMUTE_STATIC_SCRATCH_BYTES
+ * large, which every GPU that loads the library holds until the process exits.  It is meant for
+ * code that runs where a device allocation is not possible or not allowed: inside a serving or
+ * training loop whose memory was handed out once at start-up and is owned by someone else's pool,
+ * in a plug-in that only receives the tensors it must fill, or on a latency-critical path where
+ * cudaMalloc's implicit device synchronisation is unacceptable.  The call itself makes no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - Limit: returns MOE_ERR_WORKSPACE (nothing launched) when
+ *     moe_permute_workspace_bytes(dims) > MOE_PERMUTE_STATIC_SCRATCH_BYTES, i.e. when
+ *     ceil(T*K/256) * E * 4 bytes exceeds 4 MiB (all five benchmark configurations need <= 256 KiB).
+ *   - The first call on each device looks up the array's device address (a one-time set-up on the
+ *     host, with that device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Its contents carry over from call to call, which
+ *     is harmless here because each call overwrites every entry before reading it; but two calls
+ *     whose kernels may overlap on the GPU (different streams without ordering, or different host
+ *     threads) race on it and give wrong indices.  Serialise them, or use moe_permute with
+ *     separate workspaces. */
+#define MOE_PERMUTE_STATIC_SCRATCH_BYTES (4u << 20)
+int moe_permute_static_scratch(const moe_dims_t* dims, const void* x, const int32_t* topk_idx,
+                               void* x_perm, int32_t* counts, int32_t* offsets,
+                               int32_t* row_to_pair, int32_t* pair_to_row, moe_stream_t stream);
+
 /* ---- a8: dx[t,:] = sum_k dx_perm[pair_to_row[t*K+k], :]   (fp32 sum in slot order) ---------- */
 int moe_permute_bwd(const moe_dims_t* dims, const void* dx_perm, const int32_t* pair_to_row,
                     void* dx, moe_stream_t stream);

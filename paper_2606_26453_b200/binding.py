@@ -16,7 +16,8 @@ _PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG_DIR, "libmoe_b200.so")
 
 EXPORTS = [
-    "moe_status_string", "moe_permute_workspace_bytes", "moe_device_status", "moe_permute", "moe_permute_bwd",
+    "moe_status_string", "moe_permute_workspace_bytes", "moe_device_status", "moe_permute", "moe_permute_static_scratch",
+    "moe_permute_bwd",
     "moe_grouped_gemm_gateup_swiglu", "moe_grouped_gemm_down", "moe_unpermute_combine",
     "moe_unpermute_combine_bwd", "moe_grouped_gemm_down_dgrad", "moe_grouped_gemm_down_wgrad",
     "moe_grouped_gemm_down_bwd", "moe_swiglu_bwd", "moe_grouped_gemm_gateup_dgrad",
@@ -58,6 +59,7 @@ def load_library() -> ctypes.CDLL:
         dp = ctypes.POINTER(MoeDims)
         sigs = {
             "moe_permute": [dp, p, p, p, p, p, p, p, p, ctypes.c_size_t, p],
+            "moe_permute_static_scratch": [dp, p, p, p, p, p, p, p, p],
             "moe_permute_bwd": [dp, p, p, p, p],
             "moe_grouped_gemm_gateup_swiglu": [dp, p, p, p, p, p, p, p],
             "moe_grouped_gemm_down": [dp, p, p, p, p, p],
@@ -128,6 +130,13 @@ def moe_permute(d, x, topk_idx, x_perm, counts, offsets, row_to_pair, pair_to_ro
     _call("moe_permute", ctypes.byref(d), _ptr(x), _ptr(topk_idx), _ptr(x_perm), _ptr(counts), _ptr(offsets),
           _ptr(row_to_pair), _ptr(pair_to_row), _ptr(workspace), ctypes.c_size_t(workspace.numel() * workspace.element_size()),
           _stream())
+
+
+def moe_permute_static_scratch(d, x, topk_idx, x_perm, counts, offsets, row_to_pair, pair_to_row):
+    """moe_permute for callers that may not allocate: the scratch is a fixed array inside the library
+    (shared by all calls on a device; see the header for the size limit and the no-overlap rule)."""
+    _call("moe_permute_static_scratch", ctypes.byref(d), _ptr(x), _ptr(topk_idx), _ptr(x_perm), _ptr(counts),
+          _ptr(offsets), _ptr(row_to_pair), _ptr(pair_to_row), _stream())
 
 
 def moe_permute_bwd(d, dx_perm, pair_to_row, dx):

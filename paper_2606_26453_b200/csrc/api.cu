@@ -98,6 +98,19 @@ int moe_permute(const moe_dims_t* dims, const void* x, const int32_t* topk_idx, 
                           st(stream));
 }
 
+int moe_permute_static_scratch(const moe_dims_t* dims, const void* x, const int32_t* topk_idx, void* x_perm,
+                               int32_t* counts, int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row,
+                               moe_stream_t stream) {
+    {
+        const void* const req[] = {topk_idx, counts, offsets, row_to_pair, pair_to_row};
+        const void* const opt[] = {x, x_perm};
+        MOE_VALIDATE(dims, req, opt);
+    }
+    if (x_perm != nullptr && x == nullptr) return MOE_ERR_NULL;
+    return launch_permute_static_scratch(*dims, cb(x), topk_idx, mb(x_perm), counts, offsets, row_to_pair,
+                                         pair_to_row, st(stream));
+}
+
 int moe_permute_bwd(const moe_dims_t* dims, const void* dx_perm, const int32_t* pair_to_row, void* dx,
                     moe_stream_t stream) {
     const void* const req[] = {dx_perm, pair_to_row, dx};

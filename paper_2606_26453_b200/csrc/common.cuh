@@ -25,6 +25,9 @@ int launch_permute(const moe_dims_t& d, const bf16* x, const int32_t* topk_idx, 
                    int32_t* counts, int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row,
                    void* workspace, cudaStream_t s);
 size_t permute_workspace_bytes(const moe_dims_t& d);
+int launch_permute_static_scratch(const moe_dims_t& d, const bf16* x, const int32_t* topk_idx, bf16* x_perm,
+                                  int32_t* counts, int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row,
+                                  cudaStream_t s);
 int launch_gather_sum(const moe_dims_t& d, const bf16* src_perm, const float* topk_w,
                       const int32_t* pair_to_row, bf16* dst, cudaStream_t s);  // topk_w may be NULL (unit weights)
 int launch_combine_bwd(const moe_dims_t& d, const bf16* dy, const bf16* y_perm, const float* topk_w,

@@ -413,6 +413,31 @@ int launch_combine_bwd(const moe_dims_t& d, const bf16* dy, const bf16* y_perm, 
     return check_launch();
 }
 
+// ------------------------------------------------------------------------------------------------
+// Route-permute without a caller-provided workspace.  The chunk-histogram table lives in a
+// file-scope device array instead, so that a caller who may not allocate device memory (see the
+// header) can still run the call.  The array's name is only a host-side handle in host code; the
+// device address is looked up once per device with cudaGetSymbolAddress and handed to the
+// ordinary permute launch.  Every entry the rank kernel reads is written by the histogram and
+// scan kernels of the same call first, so nothing has to be cleared between calls.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_permute_static_scratch[MOE_PERMUTE_STATIC_SCRATCH_BYTES];
+
+int launch_permute_static_scratch(const moe_dims_t& d, const bf16* x, const int32_t* topk_idx, bf16* x_perm,
+                                  int32_t* counts, int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row,
+                                  cudaStream_t s) {
+    if (permute_workspace_bytes(d) > (size_t)MOE_PERMUTE_STATIC_SCRATCH_BYTES) return MOE_ERR_WORKSPACE;
+    static void* scratch_of_device[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
+    if (scratch_of_device[dev] == nullptr) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_permute_static_scratch) != cudaSuccess || ptr == nullptr) return MOE_ERR_CUDA;
+        scratch_of_device[dev] = ptr;
+    }
+    return launch_permute(d, x, topk_idx, x_perm, counts, offsets, row_to_pair, pair_to_row, scratch_of_device[dev], s);
+}
+
 int launch_swiglu_bwd(const moe_dims_t& d, const bf16* dh_act, const bf16* gu, bf16* dgu, cudaStream_t s) {
     const int iv = d.I / 8;
     const long long total = (long long)d.T * d.K * iv;
