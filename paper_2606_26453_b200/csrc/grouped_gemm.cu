@@ -7,7 +7,7 @@
 //   warp 1      MMA issuer: one lane issues tcgen05.mma (128 x 256 x 16, bf16 -> fp32) with the
 //               accumulator in tensor memory; tcgen05.commit releases ring stages and publishes
 //               finished accumulators
-//   warps 2..5  epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), apply the
+//   warps 2..9  epilogue: tcgen05.ld the accumulator (32-lane quarter x half of the columns), apply the
 //               epilogue (plain / SwiGLU), round to bf16, store row segments with 16-byte stores
 // The accumulator is double buffered (2 x 256 of the 512 TMEM columns) so the epilogue of one tile
 // overlaps the main loop of the next.
@@ -46,8 +46,10 @@ constexpr int A_BYTES = BM * BK * 2;   // 16 KB
 constexpr int B_BYTES = BN * BK * 2;   // 32 KB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN-major box: 64 k-rows x 128 B = 8 KB
+constexpr int NUM_EPI_WARPS = 8;
+constexpr int STAGING_BYTES_PER_WARP = 32 * 32 * 2;   // one 32 x 32 bf16 output block
 constexpr int MAX_E = 1024;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;   // producer warp, MMA warp, 8 epilogue warps
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
@@ -135,6 +137,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x), "r"(y),
+                 "r"(src)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -196,6 +212,20 @@ struct Tile {
     int k_rows;   // WGRAD: rows of the contraction
 };
 
+// Order of an expert's m_tiles x n_tiles output tiles: bands of RASTER_BAND row tiles; inside a band
+// column tile major, row tile minor.  The CTAs that run at the same time (consecutive tile ids) then
+// touch about RASTER_BAND row-tile operands and gridDim/RASTER_BAND column-tile operands, a working
+// set of a few tens of MB that stays in L2 whatever the expert's size.
+constexpr int RASTER_BAND = 16;
+__device__ __forceinline__ void raster(int local, int m_tiles, int n_tiles, int& mt, int& nt) {
+    const int band = local / (RASTER_BAND * n_tiles);
+    const int m0 = band * RASTER_BAND;
+    const int rows = min(RASTER_BAND, m_tiles - m0);
+    const int in_band = local - band * RASTER_BAND * n_tiles;
+    nt = in_band / rows;
+    mt = m0 + (in_band - nt * rows);
+}
+
 template <int KIND>
 __device__ __forceinline__ long long total_tiles(const Params& p, const SharedCtl* ctl) {
     if (KIND == WGRAD) return (long long)p.E * p.m_tiles * p.n_tiles;
@@ -209,7 +239,8 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
         const int per_e = p.m_tiles * p.n_tiles;
         tl.e = (int)(t / per_e);
         const int local = (int)(t - (long long)tl.e * per_e);
-        const int mt = local / p.n_tiles, nt = local - mt * p.n_tiles;
+        int mt, nt;
+        raster(local, p.m_tiles, p.n_tiles, mt, nt);
         tl.row0 = mt * BM;
         tl.n0 = nt * BN;
         tl.k_row0 = ctl->offs[tl.e];
@@ -217,8 +248,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
         tl.k_blocks = (tl.k_rows + BK - 1) / BK;
         tl.row_end = 0;
     } else {
-        // tile_prefix[e] = number of 128-row tiles of experts < e; tiles of an expert are ordered
-        // column tile major, row tile minor, so concurrently running CTAs share a weight tile.
+        // tile_prefix[e] = number of 128-row tiles of experts < e
         const int mtile_flat = (int)(t / p.n_tiles);   // only used to bracket the expert
         int lo = 0, hi = p.E;                          // largest e with tile_prefix[e]*n_tiles <= t
         (void)mtile_flat;
@@ -229,7 +259,8 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
         tl.e = lo;
         const int m_tiles_e = ctl->tile_prefix[lo + 1] - ctl->tile_prefix[lo];
         const int local = (int)(t - (long long)ctl->tile_prefix[lo] * p.n_tiles);
-        const int nt = local / m_tiles_e, mt = local - nt * m_tiles_e;
+        int mt, nt;
+        raster(local, m_tiles_e, p.n_tiles, mt, nt);
         tl.row0 = ctl->offs[lo] + mt * BM;
         tl.row_end = ctl->offs[lo + 1];
         tl.n0 = nt * BN;
@@ -248,7 +279,8 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
 template <int KIND>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
-                    const __grid_constant__ CUtensorMap map_b1, const Params p) {
+                    const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_o0,
+                    const __grid_constant__ CUtensorMap map_o1, const Params p) {
     constexpr bool A_MN = (KIND == WGRAD);
     constexpr bool B_MN = (KIND != DGRAD);
     constexpr uint32_t IDESC = make_idesc(BN, A_MN, B_MN);
@@ -258,7 +290,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
-    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles_ptr + STAGES * STAGE_BYTES);
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles_ptr + STAGES * STAGE_BYTES + NUM_EPI_WARPS * STAGING_BYTES_PER_WARP);
     volatile int* abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -272,7 +304,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[a]), 4);
+            mbar_init(smem_u32(&ctl->tmem_empty[a]), 8);
         }
         mbar_init(smem_u32(&ctl->drain), 1);
         ctl->abort_flag = 0;
@@ -280,6 +312,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         prefetch_tmap(&map_a);
         prefetch_tmap(&map_b0);
         prefetch_tmap(&map_b1);
+        prefetch_tmap(&map_o0);
+        prefetch_tmap(&map_o1);
     }
     __syncthreads();
     if (KIND != WGRAD && threadIdx.x == 0) {
@@ -318,12 +352,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const uint32_t b_dst = a_dst + A_BYTES;
                     if (KIND == WGRAD) {
                         const int krow = tl.k_row0 + kb * BK;
-#pragma unroll
-                        for (int c = 0; c < BM / 64; ++c)
-                            tma_load_2d(a_dst + c * CHUNK_BYTES, &map_a, tl.row0 + c * 64, krow, full);
-#pragma unroll
-                        for (int c = 0; c < BN / 64; ++c)
-                            tma_load_2d(b_dst + c * CHUNK_BYTES, &map_b0, tl.n0 + c * 64, krow, full);
+                        // MN-major operands: one 3-D box = all 64-wide chunks of the tile, chunk-major in shared memory
+                        tma_load_3d(a_dst, &map_a, 0, krow, tl.row0 >> 6, full);
+                        tma_load_3d(b_dst, &map_b0, 0, krow, tl.n0 >> 6, full);
                     } else {
                         tma_load_2d(a_dst, &map_a, kb * BK, tl.row0, full);
                         if (KIND == DGRAD) {
@@ -332,17 +363,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                             tma_load_2d(b_dst, second ? &map_b1 : &map_b0, kx, tl.e * p.b_rows_per_e + tl.n0, full);
                         } else if (KIND == FWD_PLAIN) {
                             const int ky = tl.e * p.b_rows_per_e + kb * BK;
-#pragma unroll
-                            for (int c = 0; c < BN / 64; ++c)
-                                tma_load_2d(b_dst + c * CHUNK_BYTES, &map_b0, tl.n0 + c * 64, ky, full);
+                            tma_load_3d(b_dst, &map_b0, 0, ky, tl.n0 >> 6, full);
                         } else {  // FWD_SWIGLU: 128 gate columns then 128 up columns
                             const int ky = tl.e * p.b_rows_per_e + kb * BK;
                             const int ng = tl.n0 >> 1;   // n0 counts fused (gate+up) columns
-#pragma unroll
-                            for (int c = 0; c < 2; ++c) {
-                                tma_load_2d(b_dst + c * CHUNK_BYTES, &map_b0, ng + c * 64, ky, full);
-                                tma_load_2d(b_dst + (2 + c) * CHUNK_BYTES, &map_b1, ng + c * 64, ky, full);
-                            }
+                            tma_load_3d(b_dst, &map_b0, 0, ky, ng >> 6, full);
+                            tma_load_3d(b_dst + 2 * CHUNK_BYTES, &map_b1, 0, ky, ng >> 6, full);
                         }
                     }
                     ++issued;
@@ -418,71 +444,93 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         __syncwarp();
     } else {
-        // ================= epilogue (warps 2..5) =================
+        // ================= epilogue (warps 2..9) =================
+        // Each warp owns a 32-row slab (its TMEM lane quarter) and half of the tile's columns.  A
+        // 32 x 32 block is rounded to bf16, written to the warp's 2 KB staging buffer in the 64-byte
+        // swizzle pattern and sent to global memory by one bulk tensor store, so the LSU never issues
+        // scattered global stores next to the TMA fills of the operand ring.  A slab that is only partly
+        // inside its expert (row-ragged kinds) falls back to predicated 16-byte row stores.
         const int quarter = warp & 3;               // TMEM lanes [32*quarter, 32*quarter+32)
-        const int row_in_tile = quarter * 32 + lane;
+        const int half = (warp - 2) >> 2;           // which half of the tile's columns this warp handles
+        uint8_t* stage_ptr = tiles_ptr + STAGES * STAGE_BYTES + (warp - 2) * STAGING_BYTES_PER_WARP;
+        const uint32_t stage_addr = smem_u32(stage_ptr);
+        uint8_t* my_row = stage_ptr + lane * 64;
+        const int sw = (lane >> 1) & 3;             // 64-byte swizzle: 16-byte piece j of row r sits at j ^ ((r>>1)&3)
+        bool store_pending = false;
+
+        // stage one 32x32 bf16 block (this thread: 16 packed words of its row) and issue its bulk store
+        auto stage_and_store = [&](const uint32_t (&w)[16], const CUtensorMap* map, int x, int y) {
+            if (store_pending) {
+                if (lane == 0) bulk_wait_read0();
+                __syncwarp();
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                *reinterpret_cast<uint4*>(my_row + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(map, x, y, stage_addr);
+                bulk_commit();
+            }
+            store_pending = true;
+        };
+        auto direct_store = [&](const uint32_t (&w)[16], bf16* dst) {
+            uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) d4[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+        };
+
         uint32_t acc = 0, acc_phase = 0;
         for (long long t = blockIdx.x; t < n_tiles_total; t += gridDim.x) {
             const Tile tl = decode_tile<KIND>(p, ctl, t);
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
+            const int slab0 = tl.row0 + quarter * 32;                 // first row of this warp's slab
+            // rows of the slab that belong to the expert (row-ragged kinds); 32 = whole slab
+            const int rows_valid = (KIND == WGRAD) ? 32 : max(0, min(32, tl.row_end - slab0));
+            const int slab_y = (KIND == WGRAD) ? tl.e * (p.m_tiles * BM) + slab0 : slab0;
+            const long long row = (long long)slab0 + lane;
             if (KIND == FWD_SWIGLU) {
-                const long long row = (long long)tl.row0 + row_in_tile;
-                const bool row_ok = row < tl.row_end;
                 const int ng = tl.n0 >> 1;
-                bf16* h_row = p.out0 + row * p.I + ng;
-                bf16* g_row = p.gu ? p.gu + row * (2ll * p.I) + ng : nullptr;
 #pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 2 * half; c < 2 * half + 2; ++c) {
                     uint32_t g[32], u[32];
                     tc_ld32(taddr + c * 32, g);
                     tc_ld32(taddr + 128 + c * 32, u);
                     tc_wait_ld();
-                    if (row_ok) {
-                        uint32_t hp[16], gp[16], up[16];
+                    if (rows_valid == 0) continue;
+                    uint32_t hp[16], gp[16], up[16];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const float g0 = __uint_as_float(g[2 * j]), g1 = __uint_as_float(g[2 * j + 1]);
-                            const float u0 = __uint_as_float(u[2 * j]), u1 = __uint_as_float(u[2 * j + 1]);
-                            const float h0 = g0 / (1.f + __expf(-g0)) * u0;
-                            const float h1 = g1 / (1.f + __expf(-g1)) * u1;
-                            hp[j] = pack_bf16(h0, h1);
-                            gp[j] = pack_bf16(g0, g1);
-                            up[j] = pack_bf16(u0, u1);
+                    for (int j = 0; j < 16; ++j) {
+                        const float g0 = __uint_as_float(g[2 * j]), g1 = __uint_as_float(g[2 * j + 1]);
+                        const float u0 = __uint_as_float(u[2 * j]), u1 = __uint_as_float(u[2 * j + 1]);
+                        const float h0 = g0 / (1.f + __expf(-g0)) * u0;
+                        const float h1 = g1 / (1.f + __expf(-g1)) * u1;
+                        hp[j] = pack_bf16(h0, h1);
+                        gp[j] = pack_bf16(g0, g1);
+                        up[j] = pack_bf16(u0, u1);
+                    }
+                    const int x = ng + c * 32;
+                    if (rows_valid == 32) {
+                        stage_and_store(hp, &map_o0, x, slab_y);
+                        if (p.gu) {
+                            stage_and_store(gp, &map_o1, x, slab_y);
+                            stage_and_store(up, &map_o1, p.I + x, slab_y);
                         }
-                        uint4* hd = reinterpret_cast<uint4*>(h_row + c * 32);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) hd[j] = make_uint4(hp[4 * j], hp[4 * j + 1], hp[4 * j + 2], hp[4 * j + 3]);
-                        if (g_row) {
-                            uint4* gd = reinterpret_cast<uint4*>(g_row + c * 32);
-                            uint4* ud = reinterpret_cast<uint4*>(g_row + p.I + c * 32);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) {
-                                gd[j] = make_uint4(gp[4 * j], gp[4 * j + 1], gp[4 * j + 2], gp[4 * j + 3]);
-                                ud[j] = make_uint4(up[4 * j], up[4 * j + 1], up[4 * j + 2], up[4 * j + 3]);
-                            }
+                    } else if (lane < rows_valid) {
+                        direct_store(hp, p.out0 + row * p.I + x);
+                        if (p.gu) {
+                            direct_store(gp, p.gu + row * (2ll * p.I) + x);
+                            direct_store(up, p.gu + row * (2ll * p.I) + p.I + x);
                         }
                     }
                 }
             } else {
-                long long row;
-                bool row_ok;
-                bf16 *o0, *o1;
-                if (KIND == WGRAD) {
-                    row = (long long)tl.row0 + row_in_tile;
-                    row_ok = true;
-                    o0 = p.out0 + (long long)tl.e * p.out_e_stride + row * p.ldo;
-                    o1 = p.out1 ? p.out1 + (long long)tl.e * p.out_e_stride + row * p.ldo : nullptr;
-                } else {
-                    row = (long long)tl.row0 + row_in_tile;
-                    row_ok = row < tl.row_end;
-                    o0 = p.out0 + row * p.ldo;
-                    o1 = nullptr;
-                }
                 const bool have_acc = tl.k_blocks > 0;
 #pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
+                for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
                     uint32_t v[32];
                     if (have_acc) {
                         tc_ld32(taddr + c * 32, v);
@@ -492,16 +540,16 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         for (int j = 0; j < 32; ++j) v[j] = 0u;
                     }
                     const int n = tl.n0 + c * 32;
-                    if (row_ok && n < p.n_cols) {
-                        bf16* dst = (n < p.n_split) ? o0 + n : o1 + (n - p.n_split);
-                        uint4* d4 = reinterpret_cast<uint4*>(dst);
+                    if (rows_valid == 0 || n >= p.n_cols) continue;
+                    uint32_t w[16];
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            d4[j] = make_uint4(pack_bf16(__uint_as_float(v[8 * j]), __uint_as_float(v[8 * j + 1])),
-                                               pack_bf16(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3])),
-                                               pack_bf16(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5])),
-                                               pack_bf16(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7])));
-                        }
+                    for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                    const bool first = n < p.n_split;
+                    const int x = first ? n : n - p.n_split;
+                    if (rows_valid == 32) {
+                        stage_and_store(w, first ? &map_o0 : &map_o1, x, slab_y);
+                    } else if (lane < rows_valid) {
+                        direct_store(w, p.out0 + row * p.ldo + x);     // row-ragged kinds have a single output
                     }
                 }
             }
@@ -510,6 +558,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
+        // the staging buffer must have been read, and the stores completed, before the CTA exits
+        if (store_pending && lane == 0) bulk_wait_all0();
+        __syncwarp();
     }
 
     // ---- teardown ----
@@ -522,7 +573,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     }
 }
 
-constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + sizeof(SharedCtl);
+constexpr size_t SMEM_BYTES =
+    (size_t)STAGES * STAGE_BYTES + NUM_EPI_WARPS * STAGING_BYTES_PER_WARP + 1024 + sizeof(SharedCtl);
+static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA can opt in to");
 
 // ---- host side ------------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
@@ -539,7 +592,7 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
 
 // 2-D bf16 tensor [outer, inner] (inner contiguous), box [box_outer, box_inner], 128-byte swizzle.
 bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint32_t box_inner,
-              uint32_t box_outer) {
+              uint32_t box_outer, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
     if (fn == nullptr) return false;
     cuuint64_t dims[2] = {inner, outer};
@@ -547,12 +600,33 @@ bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer
     cuuint32_t box[2] = {box_inner, box_outer};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// MN-major operand [rows, cols] (cols contiguous) seen as {64 columns, rows, cols/64 chunks}: one box of
+// {64, BK rows, n_chunks} lands chunk-major in shared memory, i.e. as n_chunks consecutive 64 x BK swizzled
+// blocks -- the layout the MN-major UMMA descriptors expect.
+bool make_map_mn(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows, uint32_t n_chunks) {
+    PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[3] = {64, rows, cols / 64};
+    cuuint64_t strides[2] = {cols * 2, 128};
+    cuuint32_t box[3] = {64, (cuuint32_t)BK, n_chunks};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Output map: [rows, cols] bf16, 32 x 32 blocks in the 64-byte swizzle pattern of the staging buffers.
+bool make_out_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t rows) {
+    return make_map(map, base, cols, rows, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+}
+
 template <int KIND>
-int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const Params& p, cudaStream_t s) {
+int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const CUtensorMap& o0,
+           const CUtensorMap& o1, const Params& p, cudaStream_t s) {
     static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
@@ -564,7 +638,7 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
     }
     const int grid = sm_count();
     if (grid <= 0) return MOE_ERR_CUDA;
-    grouped_gemm_kernel<KIND><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(a, b0, b1, p);
+    grouped_gemm_kernel<KIND><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(a, b0, b1, o0, o1, p);
     return check_launch();
 }
 
@@ -575,29 +649,31 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
 int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gate, const bf16* w_up,
                       const int32_t* offsets, bf16* h_act, bf16* gu, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    CUtensorMap a, b0, b1;
-    if (!make_map(&a, x_perm, d.H, R, BK, BM) || !make_map(&b0, w_gate, d.I, (uint64_t)d.E * d.H, 64, BK) ||
-        !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, 64, BK))
+    CUtensorMap a, b0, b1, o0, o1;
+    if (!make_map(&a, x_perm, d.H, R, BK, BM) || !make_map_mn(&b0, w_gate, d.I, (uint64_t)d.E * d.H, 2) ||
+        !make_map_mn(&b1, w_up, d.I, (uint64_t)d.E * d.H, 2) || !make_out_map(&o0, h_act, d.I, R) ||
+        !make_out_map(&o1, gu ? gu : h_act, gu ? 2ull * d.I : d.I, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
     p.n_tiles = d.I / 128; p.n_cols = 2 * d.I; p.b_rows_per_e = d.H;
     p.out0 = h_act; p.gu = gu; p.I = d.I; p.ldo = d.I; p.n_split = 2 * d.I;
-    return launch<FWD_SWIGLU>(a, b0, b1, p, s);
+    return launch<FWD_SWIGLU>(a, b0, b1, o0, o1, p, s);
 }
 
 // Down forward: A = h_act [R,I]; B = w_down viewed as [E*I, H].
 int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, const int32_t* offsets,
                     bf16* y_perm, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    CUtensorMap a, b0;
-    if (!make_map(&a, h_act, d.I, R, BK, BM) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, 64, BK))
+    CUtensorMap a, b0, o0;
+    if (!make_map(&a, h_act, d.I, R, BK, BM) || !make_map_mn(&b0, w_down, d.H, (uint64_t)d.E * d.I, BN / 64) ||
+        !make_out_map(&o0, y_perm, d.H, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.I / BK; p.k_split = p.k_blocks;
     p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.b_rows_per_e = d.I;
     p.out0 = y_perm; p.ldo = d.H; p.n_split = d.H;
-    return launch<FWD_PLAIN>(a, b0, b0, p, s);
+    return launch<FWD_PLAIN>(a, b0, b0, o0, o0, p, s);
 }
 
 // Down dgrad: dh_act = dy_perm . w_down[e]^T.  A = dy_perm [R,H]; B = w_down viewed as [E*I, H] (rows are
@@ -605,14 +681,15 @@ int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, 
 int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_down, const int32_t* offsets,
                       bf16* dh_act, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    CUtensorMap a, b0;
-    if (!make_map(&a, dy_perm, d.H, R, BK, BM) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, BN))
+    CUtensorMap a, b0, o0;
+    if (!make_map(&a, dy_perm, d.H, R, BK, BM) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, BN) ||
+        !make_out_map(&o0, dh_act, d.I, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
     p.n_tiles = (d.I + BN - 1) / BN; p.n_cols = d.I; p.b_rows_per_e = d.I;
     p.out0 = dh_act; p.ldo = d.I; p.n_split = d.I;
-    return launch<DGRAD>(a, b0, b0, p, s);
+    return launch<DGRAD>(a, b0, b0, o0, o0, p, s);
 }
 
 // Gate/up dgrad: dx_perm = dg . w_gate[e]^T + du . w_up[e]^T.  A = dgu [R,2I]; the contraction runs over the
@@ -620,28 +697,30 @@ int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_do
 int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate, const bf16* w_up,
                         const int32_t* offsets, bf16* dx_perm, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    CUtensorMap a, b0, b1;
+    CUtensorMap a, b0, b1, o0;
     if (!make_map(&a, dgu, 2ull * d.I, R, BK, BM) || !make_map(&b0, w_gate, d.I, (uint64_t)d.E * d.H, BK, BN) ||
-        !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, BK, BN))
+        !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, BK, BN) || !make_out_map(&o0, dx_perm, d.H, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = 2 * d.I / BK; p.k_split = d.I / BK;
     p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.b_rows_per_e = d.H;
     p.out0 = dx_perm; p.ldo = d.H; p.n_split = d.H;
-    return launch<DGRAD>(a, b0, b1, p, s);
+    return launch<DGRAD>(a, b0, b1, o0, o0, p, s);
 }
 
 // Down wgrad: dw_down[e] [I,H] = h_act_e^T . dy_perm_e.  A = h_act [R,I] (M = I), B = dy_perm [R,H] (N = H).
 int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_perm, const int32_t* offsets,
                       bf16* dw_down, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    CUtensorMap a, b0;
-    if (!make_map(&a, h_act, d.I, R, 64, BK) || !make_map(&b0, dy_perm, d.H, R, 64, BK)) return MOE_ERR_CUDA;
+    CUtensorMap a, b0, o0;
+    if (!make_map_mn(&a, h_act, d.I, R, BM / 64) || !make_map_mn(&b0, dy_perm, d.H, R, BN / 64) ||
+        !make_out_map(&o0, dw_down, d.H, (uint64_t)d.E * d.I))
+        return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.m_tiles = d.I / BM; p.n_tiles = (d.H + BN - 1) / BN;
     p.n_cols = d.H; p.n_split = d.H; p.ldo = d.H; p.out_e_stride = (long long)d.I * d.H;
     p.out0 = dw_down; p.out1 = nullptr;
-    return launch<WGRAD>(a, b0, b0, p, s);
+    return launch<WGRAD>(a, b0, b0, o0, o0, p, s);
 }
 
 // Gate/up wgrad (the paper's dW1): [dw_gate[e] | dw_up[e]] = x_perm_e^T . dgu_e.  A = x_perm [R,H] (M = H),
@@ -649,13 +728,15 @@ int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_per
 int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu, const int32_t* offsets,
                         bf16* dw_gate, bf16* dw_up, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    CUtensorMap a, b0;
-    if (!make_map(&a, x_perm, d.H, R, 64, BK) || !make_map(&b0, dgu, 2ull * d.I, R, 64, BK)) return MOE_ERR_CUDA;
+    CUtensorMap a, b0, o0, o1;
+    if (!make_map_mn(&a, x_perm, d.H, R, BM / 64) || !make_map_mn(&b0, dgu, 2ull * d.I, R, BN / 64) ||
+        !make_out_map(&o0, dw_gate, d.I, (uint64_t)d.E * d.H) || !make_out_map(&o1, dw_up, d.I, (uint64_t)d.E * d.H))
+        return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.m_tiles = d.H / BM; p.n_tiles = (2 * d.I + BN - 1) / BN;
     p.n_cols = 2 * d.I; p.n_split = d.I; p.ldo = d.I; p.out_e_stride = (long long)d.H * d.I;
     p.out0 = dw_gate; p.out1 = dw_up;
-    return launch<WGRAD>(a, b0, b0, p, s);
+    return launch<WGRAD>(a, b0, b0, o0, o1, p, s);
 }
 
 }  // namespace moe
