@@ -432,6 +432,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", default="fine_grained", choices=list(W.CONFIGS))
+    ap.add_argument("--custom", default="", help="T,H,I,E,K of an ad-hoc softmax-routed workload (profiling aid)")
     ap.add_argument("--also", default="many_small,few_large,imbalanced",
                     help="comma-separated other configurations to time briefly at N=1 ('' for none)")
     ap.add_argument("--ref-tokens", type=int, default=512, help="tokens in the oracle's timed sample")
@@ -441,6 +442,10 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     args.also = [s for s in args.also.split(",") if s]
+    if args.custom:
+        T, H, I, E, K = (int(v) for v in args.custom.split(","))
+        W.CONFIGS["custom"] = W.MoeConfig("custom", T=T, H=H, I=I, E=E, K=K, routing="softmax", cfg_id=9)
+        args.config = "custom"
     if args.impl == "reference":
         run_reference(args)
     else:

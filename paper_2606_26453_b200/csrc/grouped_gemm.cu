@@ -3,18 +3,30 @@
 // One CTA per SM walks a tile list that every CTA derives by itself from the per-expert offsets
 // (no host round trip, no extra launch).  Per CTA:
 //   warp 0      TMA producer: cp.async.bulk.tensor loads of 64-wide K blocks of A and B into a
-//               4-stage ring of 128-byte-swizzled shared-memory tiles, completion on mbarriers
-//   warp 1      MMA issuer: one lane issues tcgen05.mma (128 x 256 x 16, bf16 -> fp32) with the
-//               accumulator in tensor memory; tcgen05.commit releases ring stages and publishes
-//               finished accumulators
-//   warps 2..9  epilogue: tcgen05.ld the accumulator (32-lane quarter x half of the columns), apply the
-//               epilogue (plain / SwiGLU), round to bf16, store row segments with 16-byte stores
+//               ring of 128-byte-swizzled shared-memory stages, completion on mbarriers
+//   warp 1      MMA issuer: one lane issues tcgen05.mma (bf16 -> fp32) with the accumulator in
+//               tensor memory; tcgen05.commit releases ring stages and publishes finished
+//               accumulators
+//   warps 2..9  epilogue: tcgen05.ld the accumulator (32-lane quarter x half of the columns), apply
+//               the epilogue (plain / SwiGLU), round to bf16, stage 32x32 blocks in swizzled shared
+//               memory and write them with bulk tensor stores
 // The accumulator is double buffered (2 x 256 of the 512 TMEM columns) so the epilogue of one tile
 // overlaps the main loop of the next.
 //
+// Two launch shapes of the same kernel:
+//   single  one CTA computes a 128 x 256 tile (tcgen05.mma.cta_group::1, 4 stages of 48 KB).
+//   pair    a cluster of two CTAs computes a 256 x 256 tile with tcgen05.mma.cta_group::2: each CTA
+//           loads its 128 rows of A and HALF of B (6 stages of 32 KB), the tensor cores of both SMs
+//           read both halves.  That cuts the bytes each SM must pull from L2 per flop by a third
+//           and deepens the ring, which is what the L2 -> SM path needs at full MMA rate.  Only
+//           plain (non-multicast) TMA loads are used: each CTA's loads complete on its own
+//           barrier, a relay warp in the second CTA forwards "my half has landed" to the first
+//           CTA's barrier with a remote mbarrier arrive, and the first CTA's MMA warp releases
+//           stages / publishes accumulators in both CTAs with a multicast tcgen05.commit.
+//
 // Two ragged shapes occur:
 //   row-ragged (forward, dgrad): output rows are the packed rows of an expert.  A tile starts at
-//     offsets[e] + 128*i; loading past the expert's last row is harmless, stores are clipped.
+//     offsets[e] + TILE_M*i; loading past the expert's last row is harmless, stores are clipped.
 //   contraction-ragged (wgrad; the paper's dW1_e = X_e^T G_e): the expert's rows are the
 //     contraction.  The last K block issues only ceil(rem/16) MMAs and the < 16 surplus rows
 //     are zeroed in shared memory first; an expert without rows gets a zero tile.
@@ -41,17 +53,27 @@ int read_and_clear_device_status(int* status_out) {
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2;   // 16 KB
-constexpr int B_BYTES = BN * BK * 2;   // 32 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN-major box: 64 k-rows x 128 B = 8 KB
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN-major block: 64 k-rows x 128 B = 8 KB
 constexpr int NUM_EPI_WARPS = 8;
 constexpr int STAGING_BYTES_PER_WARP = 32 * 32 * 2;   // one 32 x 32 bf16 output block
 constexpr int MAX_E = 1024;
+constexpr int MAX_STAGES = 6;
 constexpr int NUM_THREADS = 320;   // producer warp, MMA warp, 8 epilogue warps
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+// Ring geometry of the two launch shapes.
+template <bool PAIR>
+struct Geo {
+    static constexpr int STAGES = PAIR ? 6 : 4;
+    static constexpr int TILE_M = PAIR ? 2 * BM : BM;        // output rows per tile (whole pair)
+    static constexpr int BN_LOCAL = PAIR ? BN / 2 : BN;      // B columns this CTA keeps in shared memory
+    static constexpr int A_BYTES = BM * BK * 2;              // 16 KB
+    static constexpr int B_BYTES = BN_LOCAL * BK * 2;        // 16 / 32 KB
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;    // 32 / 48 KB
+    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;  // 192 KB either way
+};
 
 enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3 };
 
@@ -61,12 +83,12 @@ struct Params {
     int k_blocks;        // row-ragged kinds: contraction length / 64
     int k_split;         // DGRAD: k blocks taken from the first B tensor (then the second); else k_blocks
     int n_tiles;         // output column tiles
-    int m_tiles;         // WGRAD: output row tiles per expert
+    int m_tiles;         // WGRAD: output row tiles (of TILE_M rows) per expert
+    int m_rows;          // WGRAD: output rows per expert (M)
     int n_cols;          // valid output columns (row-ragged) / total N (WGRAD)
     int b_rows_per_e;    // rows per expert in B's 2-D view
-    int n_split;         // WGRAD / plain: columns >= n_split go to out1
+    int n_split;         // columns >= n_split go to the second output
     long long ldo;       // output row pitch (elements)
-    long long out_e_stride;  // WGRAD: elements per expert in the outputs
     bf16* out0;
     bf16* out1;
     bf16* gu;            // FWD_SWIGLU: [R, 2I] or null
@@ -74,8 +96,8 @@ struct Params {
 };
 
 struct SharedCtl {
-    unsigned long long full[STAGES];
-    unsigned long long empty[STAGES];
+    unsigned long long full[MAX_STAGES];
+    unsigned long long empty[MAX_STAGES];
     unsigned long long tmem_full[2];
     unsigned long long tmem_empty[2];
     unsigned long long drain;
@@ -88,12 +110,37 @@ struct SharedCtl {
 // ---- small PTX wrappers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of `local_addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(bar) : "memory");
 }
+// Arrive on a barrier of another CTA of the cluster (address from map_to_cta).  Default semantics: a
+// cluster-scope release on every ring stage would serialise the pipeline on a fence; the data the arrival
+// announces was written by the TMA unit and is consumed by the tensor cores, both ordered by the barriers
+// themselves.  Generic-proxy writes that must be visible to the other CTA are fenced explicitly
+// (cluster_fence) at the one place they occur.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__device__ __forceinline__ void cluster_fence() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes)
                  : "memory");
@@ -157,15 +204,42 @@ __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// arrive on `bar` once all tcgen05 operations issued so far by this thread have completed; in pair mode
+// the arrival goes to the barrier at the same offset in BOTH CTAs
+template <bool PAIR>
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    if (PAIR) {
+        asm volatile(
+            "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+            "h"((uint16_t)3)
+            : "memory");
+    } else {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    }
 }
+// same, but only this CTA's barrier is signalled
+template <bool PAIR>
+__device__ __forceinline__ void tc_commit_local(uint32_t bar) {
+    if (PAIR)
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+template <bool PAIR>
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                        uint32_t accumulate) {
-    asm volatile(
-        "{ .reg .pred p; setp.ne.u32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
+    if (PAIR) {
+        asm volatile(
+            "{ .reg .pred p; setp.ne.u32 p, %4, 0; tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
+            "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    } else {
+        asm volatile(
+            "{ .reg .pred p; setp.ne.u32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
+            "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t v[32]) {
     asm volatile(
@@ -190,10 +264,11 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
     const uint64_t sbo = 1024 >> 4;
     return (uint64_t)((addr >> 4) & 0x3FFF) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, given N and operand major-ness.
-__host__ __device__ constexpr uint32_t make_idesc(int n, bool a_mn, bool b_mn) {
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, given M (128, or 256 over a CTA pair), N and
+// operand major-ness.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n, bool a_mn, bool b_mn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -232,7 +307,7 @@ __device__ __forceinline__ long long total_tiles(const Params& p, const SharedCt
     return (long long)ctl->tile_prefix[p.E] * p.n_tiles;
 }
 
-template <int KIND>
+template <int KIND, int TILE_M>
 __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ctl, long long t) {
     Tile tl;
     if (KIND == WGRAD) {
@@ -241,17 +316,15 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
         const int local = (int)(t - (long long)tl.e * per_e);
         int mt, nt;
         raster(local, p.m_tiles, p.n_tiles, mt, nt);
-        tl.row0 = mt * BM;
+        tl.row0 = mt * TILE_M;
         tl.n0 = nt * BN;
         tl.k_row0 = ctl->offs[tl.e];
         tl.k_rows = ctl->offs[tl.e + 1] - tl.k_row0;
         tl.k_blocks = (tl.k_rows + BK - 1) / BK;
         tl.row_end = 0;
     } else {
-        // tile_prefix[e] = number of 128-row tiles of experts < e
-        const int mtile_flat = (int)(t / p.n_tiles);   // only used to bracket the expert
+        // tile_prefix[e] = number of TILE_M-row tiles of experts < e
         int lo = 0, hi = p.E;                          // largest e with tile_prefix[e]*n_tiles <= t
-        (void)mtile_flat;
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
             if ((long long)ctl->tile_prefix[mid] * p.n_tiles <= t) lo = mid; else hi = mid;
@@ -261,7 +334,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
         const int local = (int)(t - (long long)ctl->tile_prefix[lo] * p.n_tiles);
         int mt, nt;
         raster(local, m_tiles_e, p.n_tiles, mt, nt);
-        tl.row0 = ctl->offs[lo] + mt * BM;
+        tl.row0 = ctl->offs[lo] + mt * TILE_M;
         tl.row_end = ctl->offs[lo + 1];
         tl.n0 = nt * BN;
         tl.k_blocks = p.k_blocks;
@@ -271,40 +344,60 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
     return tl;
 }
 
+// WGRAD: clear contraction rows [z0, z1) of a stage (A chunks and this CTA's B chunks are contiguous)
+__device__ __forceinline__ void zero_k_rows(uint8_t* stage_ptr, int n_chunks, int z0, int z1, int lane) {
+    const int per_row = n_chunks * 8;   // 16-byte pieces per k-row over all chunks
+    for (int i = lane; i < (z1 - z0) * per_row; i += 32) {
+        const int r = z0 + i / per_row, q = i % per_row;
+        const int chunk = q >> 3, piece = q & 7;
+        *reinterpret_cast<uint4*>(stage_ptr + chunk * CHUNK_BYTES + r * 128 + piece * 16) = make_uint4(0, 0, 0, 0);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 // ---- the kernel -----------------------------------------------------------------------------------
 // Operand major-ness per kind:
 //   FWD_*  : A K-major (activations [R, K]),   B MN-major (weights [E*K, N], N contiguous)
 //   DGRAD  : A K-major,                        B K-major  (weights [E*N, K], K contiguous)
 //   WGRAD  : A MN-major (activations [R, M]),  B MN-major (gradients [R, N])
-template <int KIND>
+template <int KIND, bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
                     const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_o0,
                     const __grid_constant__ CUtensorMap map_o1, const Params p) {
+    using G = Geo<PAIR>;
+    constexpr int STAGES = G::STAGES;
+    constexpr int STAGE_BYTES = G::STAGE_BYTES;
     constexpr bool A_MN = (KIND == WGRAD);
     constexpr bool B_MN = (KIND != DGRAD);
-    constexpr uint32_t IDESC = make_idesc(BN, A_MN, B_MN);
+    constexpr uint32_t IDESC = make_idesc(G::TILE_M, BN, A_MN, B_MN);
     constexpr uint32_t A_KSTEP = A_MN ? 2048 : 32;   // bytes per 16 k inside a stage
     constexpr uint32_t B_KSTEP = B_MN ? 2048 : 32;
+    constexpr int STAGE_CHUNKS = BM / 64 + G::BN_LOCAL / 64;   // 64-wide MN-major blocks per stage (WGRAD)
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
-    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles_ptr + STAGES * STAGE_BYTES + NUM_EPI_WARPS * STAGING_BYTES_PER_WARP);
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles_ptr + G::RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES_PER_WARP);
     volatile int* abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;          // 0 = the CTA that issues the MMAs
+    const long long first_tile = PAIR ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
+    const long long tile_stride = PAIR ? (long long)(gridDim.x >> 1) : (long long)gridDim.x;
+    const int my_rows = rank * BM;                                 // this CTA's row offset inside the tile
 
     // ---- set-up: barriers, schedule tables, TMEM ----
     for (int e = threadIdx.x; e <= p.E; e += NUM_THREADS) ctl->offs[e] = p.offsets[e];
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
+            // pair mode, first CTA: own producer's arrive + the relay's remote arrive
+            mbar_init(smem_u32(&ctl->full[s]), (PAIR && rank == 0) ? 2 : 1);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[a]), 8);
+            mbar_init(smem_u32(&ctl->tmem_empty[a]), PAIR ? 2 * NUM_EPI_WARPS : NUM_EPI_WARPS);
         }
         mbar_init(smem_u32(&ctl->drain), 1);
         ctl->abort_flag = 0;
@@ -320,55 +413,68 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         int run = 0;
         for (int e = 0; e < p.E; ++e) {
             ctl->tile_prefix[e] = run;
-            run += (ctl->offs[e + 1] - ctl->offs[e] + BM - 1) / BM;
+            run += (ctl->offs[e + 1] - ctl->offs[e] + G::TILE_M - 1) / G::TILE_M;
         }
         ctl->tile_prefix[p.E] = run;
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
-                     "r"((uint32_t)TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                         "r"((uint32_t)TMEM_COLS)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                         "r"((uint32_t)TMEM_COLS)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();   // the other CTA's barriers and tensor memory exist from here on
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
     const long long n_tiles_total = total_tiles<KIND>(p, ctl);
 
     if (warp == 0) {
-        // ================= TMA producer =================
+        // ================= TMA producer (both CTAs of a pair; each fills its own ring) =================
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0;
             bool ok = true;
-            for (long long t = blockIdx.x; ok && t < n_tiles_total; t += gridDim.x) {
-                const Tile tl = decode_tile<KIND>(p, ctl, t);
+            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+                const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
                 for (int kb = 0; kb < tl.k_blocks; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t full = smem_u32(&ctl->full[stage]);
                     mbar_arrive_expect_tx(full, STAGE_BYTES);
                     const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
-                    const uint32_t b_dst = a_dst + A_BYTES;
+                    const uint32_t b_dst = a_dst + G::A_BYTES;
+                    const int n_local = tl.n0 + (PAIR ? my_rows : 0);   // first B column this CTA loads
                     if (KIND == WGRAD) {
                         const int krow = tl.k_row0 + kb * BK;
-                        // MN-major operands: one 3-D box = all 64-wide chunks of the tile, chunk-major in shared memory
-                        tma_load_3d(a_dst, &map_a, 0, krow, tl.row0 >> 6, full);
-                        tma_load_3d(b_dst, &map_b0, 0, krow, tl.n0 >> 6, full);
+                        // MN-major operands: one 3-D box = all 64-wide chunks, chunk-major in shared memory
+                        tma_load_3d(a_dst, &map_a, 0, krow, (tl.row0 + my_rows) >> 6, full);
+                        tma_load_3d(b_dst, &map_b0, 0, krow, n_local >> 6, full);
                     } else {
-                        tma_load_2d(a_dst, &map_a, kb * BK, tl.row0, full);
+                        tma_load_2d(a_dst, &map_a, kb * BK, tl.row0 + my_rows, full);
                         if (KIND == DGRAD) {
                             const bool second = kb >= p.k_split;
                             const int kx = (second ? kb - p.k_split : kb) * BK;
-                            tma_load_2d(b_dst, second ? &map_b1 : &map_b0, kx, tl.e * p.b_rows_per_e + tl.n0, full);
+                            tma_load_2d(b_dst, second ? &map_b1 : &map_b0, kx, tl.e * p.b_rows_per_e + n_local, full);
                         } else if (KIND == FWD_PLAIN) {
                             const int ky = tl.e * p.b_rows_per_e + kb * BK;
-                            tma_load_3d(b_dst, &map_b0, 0, ky, tl.n0 >> 6, full);
+                            tma_load_3d(b_dst, &map_b0, 0, ky, n_local >> 6, full);
                         } else {  // FWD_SWIGLU: 128 gate columns then 128 up columns
                             const int ky = tl.e * p.b_rows_per_e + kb * BK;
                             const int ng = tl.n0 >> 1;   // n0 counts fused (gate+up) columns
-                            tma_load_3d(b_dst, &map_b0, 0, ky, ng >> 6, full);
-                            tma_load_3d(b_dst + 2 * CHUNK_BYTES, &map_b1, 0, ky, ng >> 6, full);
+                            if (PAIR) {                  // first CTA holds the gate half of B, second the up half
+                                tma_load_3d(b_dst, rank == 0 ? &map_b0 : &map_b1, 0, ky, ng >> 6, full);
+                            } else {
+                                tma_load_3d(b_dst, &map_b0, 0, ky, ng >> 6, full);
+                                tma_load_3d(b_dst + 2 * CHUNK_BYTES, &map_b1, 0, ky, ng >> 6, full);
+                            }
                         }
                     }
                     ++issued;
@@ -381,18 +487,19 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 uint32_t s = stage, ph = phase;
                 for (uint32_t i = 0; i < n_wait; ++i) {
                     if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
+                    if (PAIR && rank == 0) continue;   // completion there also needs the relay; the copies were bounded by it
                     const unsigned long long t0 = global_timer_ns();
                     while (!mbar_try_wait(smem_u32(&ctl->full[s]), ph) && global_timer_ns() - t0 < WAIT_LIMIT_NS / 4) {}
                 }
             }
         }
-    } else if (warp == 1) {
-        // ================= MMA issuer =================
+    } else if (warp == 1 && rank == 0) {
+        // ================= MMA issuer (first CTA of a pair) =================
         uint32_t stage = 0, phase = 0;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
-        for (long long t = blockIdx.x; ok && t < n_tiles_total; t += gridDim.x) {
-            const Tile tl = decode_tile<KIND>(p, ctl, t);
+        for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+            const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
             if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + acc * BN;
@@ -400,49 +507,74 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
-                const uint32_t b_base = a_base + A_BYTES;
+                const uint32_t b_base = a_base + G::A_BYTES;
                 int n_mma = BK / 16;
                 if (KIND == WGRAD) {
                     const int rem = tl.k_rows - kb * BK;
                     if (rem < BK) {
                         n_mma = (rem + 15) >> 4;
-                        const int z0 = rem, z1 = n_mma * 16;   // contraction rows to clear in A and B
-                        uint8_t* stage_ptr = tiles_ptr + stage * STAGE_BYTES;
-                        const int per_row = (BM / 64 + BN / 64) * 8;   // 16-byte pieces per k-row over all chunks
-                        for (int i = lane; i < (z1 - z0) * per_row; i += 32) {
-                            const int r = z0 + i / per_row, q = i % per_row;
-                            const int chunk = q >> 3, piece = q & 7;   // chunks 0..1 are A, 2..5 are B (contiguous)
-                            *reinterpret_cast<uint4*>(stage_ptr + chunk * CHUNK_BYTES + r * 128 + piece * 16) =
-                                make_uint4(0, 0, 0, 0);
+                        if (n_mma * 16 > rem) {
+                            zero_k_rows(tiles_ptr + stage * STAGE_BYTES, STAGE_CHUNKS, rem, n_mma * 16, lane);
+                            if (PAIR) cluster_fence();   // pairs with the relay's fence: its cleared rows are visible too
                         }
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
                     }
                 }
                 if (lane == 0) {
                     const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
                     const uint64_t b_desc = make_smem_desc<B_MN>(b_base);
-                    for (int kk = 0; kk < n_mma; ++kk) {
-                        tc_mma(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4), b_desc + (uint64_t)((kk * B_KSTEP) >> 4),
-                               IDESC, (kb | kk) != 0 ? 1u : 0u);
+                    if (n_mma == BK / 16) {   // full block: fully unrolled issue (a runtime trip count costs ~15 % here)
+#pragma unroll
+                        for (int kk = 0; kk < BK / 16; ++kk)
+                            tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
+                                         b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, (kb | kk) != 0 ? 1u : 0u);
+                    } else {
+                        for (int kk = 0; kk < n_mma; ++kk)
+                            tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
+                                         b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, (kb | kk) != 0 ? 1u : 0u);
                     }
-                    tc_commit(smem_u32(&ctl->empty[stage]));
+                    tc_commit<PAIR>(smem_u32(&ctl->empty[stage]));
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
             if (!ok) break;
-            if (lane == 0) tc_commit(smem_u32(&ctl->tmem_full[acc]));
+            if (lane == 0) tc_commit<PAIR>(smem_u32(&ctl->tmem_full[acc]));
             __syncwarp();
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
         // all issued MMAs must have retired before tensor memory is released
         if (lane == 0) {
-            tc_commit(smem_u32(&ctl->drain));
+            tc_commit_local<PAIR>(smem_u32(&ctl->drain));
             const unsigned long long t0 = global_timer_ns();
             while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
         }
         __syncwarp();
+    } else if (warp == 1) {
+        // ================= relay (second CTA of a pair) =================
+        // Waits until this CTA's loads of a stage have landed, clears the surplus contraction rows
+        // (WGRAD) and then tells the first CTA's barrier that this half of the stage is ready.
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+            const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
+            for (int kb = 0; kb < tl.k_blocks; ++kb) {
+                if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+                if (KIND == WGRAD) {
+                    const int rem = tl.k_rows - kb * BK;
+                    if (rem < BK) {
+                        const int z1 = ((rem + 15) >> 4) * 16;
+                        if (z1 > rem) {
+                            zero_k_rows(tiles_ptr + stage * STAGE_BYTES, STAGE_CHUNKS, rem, z1, lane);
+                            cluster_fence();
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&ctl->full[stage]), 0));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
     } else {
         // ================= epilogue (warps 2..9) =================
         // Each warp owns a 32-row slab (its TMEM lane quarter) and half of the tile's columns.  A
@@ -452,7 +584,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // inside its expert (row-ragged kinds) falls back to predicated 16-byte row stores.
         const int quarter = warp & 3;               // TMEM lanes [32*quarter, 32*quarter+32)
         const int half = (warp - 2) >> 2;           // which half of the tile's columns this warp handles
-        uint8_t* stage_ptr = tiles_ptr + STAGES * STAGE_BYTES + (warp - 2) * STAGING_BYTES_PER_WARP;
+        uint8_t* stage_ptr = tiles_ptr + G::RING_BYTES + (warp - 2) * STAGING_BYTES_PER_WARP;
         const uint32_t stage_addr = smem_u32(stage_ptr);
         uint8_t* my_row = stage_ptr + lane * 64;
         const int sw = (lane >> 1) & 3;             // 64-byte swizzle: 16-byte piece j of row r sits at j ^ ((r>>1)&3)
@@ -480,17 +612,19 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
             for (int j = 0; j < 4; ++j) d4[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         };
+        const uint32_t tmem_empty_remote0 = PAIR ? map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0) : 0u;
+        const uint32_t tmem_empty_remote1 = PAIR ? map_to_cta(smem_u32(&ctl->tmem_empty[1]), 0) : 0u;
 
         uint32_t acc = 0, acc_phase = 0;
-        for (long long t = blockIdx.x; t < n_tiles_total; t += gridDim.x) {
-            const Tile tl = decode_tile<KIND>(p, ctl, t);
+        for (long long t = first_tile; t < n_tiles_total; t += tile_stride) {
+            const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
-            const int slab0 = tl.row0 + quarter * 32;                 // first row of this warp's slab
-            // rows of the slab that belong to the expert (row-ragged kinds); 32 = whole slab
-            const int rows_valid = (KIND == WGRAD) ? 32 : max(0, min(32, tl.row_end - slab0));
-            const int slab_y = (KIND == WGRAD) ? tl.e * (p.m_tiles * BM) + slab0 : slab0;
+            const int slab0 = tl.row0 + my_rows + quarter * 32;       // first row of this warp's slab
+            // rows of the slab that are owed: inside the expert (row-ragged kinds) / inside M (WGRAD); 32 = whole slab
+            const int rows_valid = (KIND == WGRAD) ? (slab0 < p.m_rows ? 32 : 0) : max(0, min(32, tl.row_end - slab0));
+            const int slab_y = (KIND == WGRAD) ? tl.e * p.m_rows + slab0 : slab0;
             const long long row = (long long)slab0 + lane;
             if (KIND == FWD_SWIGLU) {
                 const int ng = tl.n0 >> 1;
@@ -555,7 +689,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+            if (lane == 0) {
+                if (PAIR && rank != 0)
+                    mbar_arrive_remote(acc == 0 ? tmem_empty_remote0 : tmem_empty_remote1);
+                else
+                    mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+            }
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
         // the staging buffer must have been read, and the stores completed, before the CTA exits
@@ -566,15 +705,20 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ---- teardown ----
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();   // neither CTA's shared memory / barriers may go away while the other still uses them
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
-                     : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+                         : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS)
+                         : "memory");
     }
 }
 
-constexpr size_t SMEM_BYTES =
-    (size_t)STAGES * STAGE_BYTES + NUM_EPI_WARPS * STAGING_BYTES_PER_WARP + 1024 + sizeof(SharedCtl);
+constexpr size_t SMEM_BYTES = (size_t)Geo<false>::RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES_PER_WARP + 1024 + sizeof(SharedCtl);
+static_assert(Geo<false>::RING_BYTES == Geo<true>::RING_BYTES, "both launch shapes use the same ring size");
 static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA can opt in to");
 
 // ---- host side ------------------------------------------------------------------------------------
@@ -590,7 +734,7 @@ PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
     return fn;
 }
 
-// 2-D bf16 tensor [outer, inner] (inner contiguous), box [box_outer, box_inner], 128-byte swizzle.
+// 2-D bf16 tensor [outer, inner] (inner contiguous), box [box_outer, box_inner].
 bool make_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint32_t box_inner,
               uint32_t box_outer, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     PFN_cuTensorMapEncodeTiled_v12000 fn = get_encode_fn();
@@ -624,23 +768,54 @@ bool make_out_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t ro
     return make_map(map, base, cols, rows, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
-template <int KIND>
+// Grid of a launch: one CTA per SM (single), or as many CTA pairs as can be resident at once (pair).
+// A pair that could not be co-scheduled would run after the others and double the kernel's duration,
+// so the pair grid is sized from the occupancy query, per device and kernel.
+template <int KIND, bool PAIR>
 int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const CUtensorMap& o0,
            const CUtensorMap& o1, const Params& p, cudaStream_t s) {
-    static bool attr_set[64] = {};
+    static int grid_of_device[64] = {};
     int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ERR_CUDA;
-    if (dev < 64 && !attr_set[dev]) {
-        if (cudaFuncSetAttribute(grouped_gemm_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)SMEM_BYTES) != cudaSuccess)
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
+    auto kernel = grouped_gemm_kernel<KIND, PAIR>;
+    if (grid_of_device[dev] == 0) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
             return MOE_ERR_CUDA;
-        attr_set[dev] = true;
+        const int sms = sm_count();
+        if (sms <= 0) return MOE_ERR_CUDA;
+        if (PAIR) {
+            cudaLaunchConfig_t qc = {};
+            cudaLaunchAttribute qa[1];
+            qa[0].id = cudaLaunchAttributeClusterDimension;
+            qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+            qc.gridDim = dim3(2 * (sms / 2)); qc.blockDim = dim3(NUM_THREADS); qc.dynamicSmemBytes = SMEM_BYTES;
+            qc.attrs = qa; qc.numAttrs = 1;
+            int clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &qc) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
+            if (clusters > sms / 2) clusters = sms / 2;
+            grid_of_device[dev] = 2 * clusters;
+        } else {
+            grid_of_device[dev] = sms;
+        }
     }
-    const int grid = sm_count();
-    if (grid <= 0) return MOE_ERR_CUDA;
-    grouped_gemm_kernel<KIND><<<grid, NUM_THREADS, SMEM_BYTES, s>>>(a, b0, b1, o0, o1, p);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3(grid_of_device[dev]);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = s;
+    if (PAIR) {
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+    }
+    if (cudaLaunchKernelEx(&cfg, kernel, a, b0, b1, o0, o1, p) != cudaSuccess) return MOE_ERR_CUDA;
     return check_launch();
 }
+
+// Row-ragged kinds use CTA pairs (256-row tiles) when experts are large enough on average that the extra
+// padding of the last tile of each expert costs less than the pair's better operand reuse buys.
+bool use_pairs_for_rows(const moe_dims_t& d) { return (long long)d.T * d.K >= 512ll * d.E; }
 
 }  // namespace
 
@@ -658,22 +833,24 @@ int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gat
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
     p.n_tiles = d.I / 128; p.n_cols = 2 * d.I; p.b_rows_per_e = d.H;
     p.out0 = h_act; p.gu = gu; p.I = d.I; p.ldo = d.I; p.n_split = 2 * d.I;
-    return launch<FWD_SWIGLU>(a, b0, b1, o0, o1, p, s);
+    return use_pairs_for_rows(d) ? launch<FWD_SWIGLU, true>(a, b0, b1, o0, o1, p, s)
+                                 : launch<FWD_SWIGLU, false>(a, b0, b1, o0, o1, p, s);
 }
 
 // Down forward: A = h_act [R,I]; B = w_down viewed as [E*I, H].
 int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, const int32_t* offsets,
                     bf16* y_perm, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
+    const bool pair = use_pairs_for_rows(d);
     CUtensorMap a, b0, o0;
-    if (!make_map(&a, h_act, d.I, R, BK, BM) || !make_map_mn(&b0, w_down, d.H, (uint64_t)d.E * d.I, BN / 64) ||
-        !make_out_map(&o0, y_perm, d.H, R))
+    if (!make_map(&a, h_act, d.I, R, BK, BM) ||
+        !make_map_mn(&b0, w_down, d.H, (uint64_t)d.E * d.I, pair ? BN / 128 : BN / 64) || !make_out_map(&o0, y_perm, d.H, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.I / BK; p.k_split = p.k_blocks;
     p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.b_rows_per_e = d.I;
     p.out0 = y_perm; p.ldo = d.H; p.n_split = d.H;
-    return launch<FWD_PLAIN>(a, b0, b0, o0, o0, p, s);
+    return pair ? launch<FWD_PLAIN, true>(a, b0, b0, o0, o0, p, s) : launch<FWD_PLAIN, false>(a, b0, b0, o0, o0, p, s);
 }
 
 // Down dgrad: dh_act = dy_perm . w_down[e]^T.  A = dy_perm [R,H]; B = w_down viewed as [E*I, H] (rows are
@@ -681,15 +858,16 @@ int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, 
 int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_down, const int32_t* offsets,
                       bf16* dh_act, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
+    const bool pair = use_pairs_for_rows(d);
     CUtensorMap a, b0, o0;
-    if (!make_map(&a, dy_perm, d.H, R, BK, BM) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, BN) ||
-        !make_out_map(&o0, dh_act, d.I, R))
+    if (!make_map(&a, dy_perm, d.H, R, BK, BM) ||
+        !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, pair ? BN / 2 : BN) || !make_out_map(&o0, dh_act, d.I, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
     p.n_tiles = (d.I + BN - 1) / BN; p.n_cols = d.I; p.b_rows_per_e = d.I;
     p.out0 = dh_act; p.ldo = d.I; p.n_split = d.I;
-    return launch<DGRAD>(a, b0, b0, o0, o0, p, s);
+    return pair ? launch<DGRAD, true>(a, b0, b0, o0, o0, p, s) : launch<DGRAD, false>(a, b0, b0, o0, o0, p, s);
 }
 
 // Gate/up dgrad: dx_perm = dg . w_gate[e]^T + du . w_up[e]^T.  A = dgu [R,2I]; the contraction runs over the
@@ -697,30 +875,34 @@ int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_do
 int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate, const bf16* w_up,
                         const int32_t* offsets, bf16* dx_perm, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
+    const bool pair = use_pairs_for_rows(d);
+    const uint32_t bn = pair ? BN / 2 : BN;
     CUtensorMap a, b0, b1, o0;
-    if (!make_map(&a, dgu, 2ull * d.I, R, BK, BM) || !make_map(&b0, w_gate, d.I, (uint64_t)d.E * d.H, BK, BN) ||
-        !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, BK, BN) || !make_out_map(&o0, dx_perm, d.H, R))
+    if (!make_map(&a, dgu, 2ull * d.I, R, BK, BM) || !make_map(&b0, w_gate, d.I, (uint64_t)d.E * d.H, BK, bn) ||
+        !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, BK, bn) || !make_out_map(&o0, dx_perm, d.H, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = 2 * d.I / BK; p.k_split = d.I / BK;
     p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.b_rows_per_e = d.H;
     p.out0 = dx_perm; p.ldo = d.H; p.n_split = d.H;
-    return launch<DGRAD>(a, b0, b1, o0, o0, p, s);
+    return pair ? launch<DGRAD, true>(a, b0, b1, o0, o0, p, s) : launch<DGRAD, false>(a, b0, b1, o0, o0, p, s);
 }
 
+// Weight gradients always run as CTA pairs: their tile grid is static (M x N per expert), 256 x 256 tiles
+// waste nothing unless M is an odd multiple of 128 (then the last pair's second CTA idles).
 // Down wgrad: dw_down[e] [I,H] = h_act_e^T . dy_perm_e.  A = h_act [R,I] (M = I), B = dy_perm [R,H] (N = H).
 int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_perm, const int32_t* offsets,
                       bf16* dw_down, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
     CUtensorMap a, b0, o0;
-    if (!make_map_mn(&a, h_act, d.I, R, BM / 64) || !make_map_mn(&b0, dy_perm, d.H, R, BN / 64) ||
+    if (!make_map_mn(&a, h_act, d.I, R, BM / 64) || !make_map_mn(&b0, dy_perm, d.H, R, BN / 128) ||
         !make_out_map(&o0, dw_down, d.H, (uint64_t)d.E * d.I))
         return MOE_ERR_CUDA;
     Params p = {};
-    p.offsets = offsets; p.E = d.E; p.m_tiles = d.I / BM; p.n_tiles = (d.H + BN - 1) / BN;
-    p.n_cols = d.H; p.n_split = d.H; p.ldo = d.H; p.out_e_stride = (long long)d.I * d.H;
+    p.offsets = offsets; p.E = d.E; p.m_rows = d.I; p.m_tiles = (d.I + 2 * BM - 1) / (2 * BM);
+    p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.n_split = d.H; p.ldo = d.H;
     p.out0 = dw_down; p.out1 = nullptr;
-    return launch<WGRAD>(a, b0, b0, o0, o0, p, s);
+    return launch<WGRAD, true>(a, b0, b0, o0, o0, p, s);
 }
 
 // Gate/up wgrad (the paper's dW1): [dw_gate[e] | dw_up[e]] = x_perm_e^T . dgu_e.  A = x_perm [R,H] (M = H),
@@ -729,14 +911,14 @@ int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu
                         bf16* dw_gate, bf16* dw_up, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
     CUtensorMap a, b0, o0, o1;
-    if (!make_map_mn(&a, x_perm, d.H, R, BM / 64) || !make_map_mn(&b0, dgu, 2ull * d.I, R, BN / 64) ||
+    if (!make_map_mn(&a, x_perm, d.H, R, BM / 64) || !make_map_mn(&b0, dgu, 2ull * d.I, R, BN / 128) ||
         !make_out_map(&o0, dw_gate, d.I, (uint64_t)d.E * d.H) || !make_out_map(&o1, dw_up, d.I, (uint64_t)d.E * d.H))
         return MOE_ERR_CUDA;
     Params p = {};
-    p.offsets = offsets; p.E = d.E; p.m_tiles = d.H / BM; p.n_tiles = (2 * d.I + BN - 1) / BN;
-    p.n_cols = 2 * d.I; p.n_split = d.I; p.ldo = d.I; p.out_e_stride = (long long)d.H * d.I;
+    p.offsets = offsets; p.E = d.E; p.m_rows = d.H; p.m_tiles = (d.H + 2 * BM - 1) / (2 * BM);
+    p.n_tiles = (2 * d.I + BN - 1) / BN; p.n_cols = 2 * d.I; p.n_split = d.I; p.ldo = d.I;
     p.out0 = dw_gate; p.out1 = dw_up;
-    return launch<WGRAD>(a, b0, b0, o0, o1, p, s);
+    return launch<WGRAD, true>(a, b0, b0, o0, o1, p, s);
 }
 
 }  // namespace moe
