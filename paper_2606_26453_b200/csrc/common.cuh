@@ -14,6 +14,7 @@ typedef __nv_bfloat16 bf16;
 // Device status word (one per device that loaded the library; lives in grouped_gemm.cu): kernels
 // record MOE_ERR_TIMEOUT there when a bounded wait runs out.  Synchronises the device.
 int read_and_clear_device_status(int* status_out);
+int movement_read_and_clear_status(int* status_out);   // the data-movement kernels' word (movement.cu)
 
 // Number of SMs of the current device (cached per device ordinal).
 int sm_count();

@@ -47,7 +47,9 @@ int read_and_clear_device_status(int* status_out) {
     if (cudaDeviceSynchronize() != cudaSuccess) return MOE_ERR_CUDA;
     if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(int)) != cudaSuccess) return MOE_ERR_CUDA;
     if (v != 0 && cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return MOE_ERR_CUDA;
-    *status_out = v;
+    int m = 0;
+    if (movement_read_and_clear_status(&m) != MOE_OK) return MOE_ERR_CUDA;
+    *status_out = v != 0 ? v : m;
     return MOE_OK;
 }
 

@@ -11,7 +11,7 @@ namespace moe {
 
 namespace {
 
-constexpr int kPairsPerWarp = 256;   // pairs ranked by one warp (8 rounds of 32)
+constexpr int kPairsPerWarp = 256;   // workspace is sized for one histogram row per 256 pairs (an upper bound)
 constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
 
@@ -36,77 +36,66 @@ __device__ __forceinline__ uint4 pack8(const float f[8]) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// a1, index part.  Three small kernels over the R = T*K pairs, split into warp-chunks of
-// kPairsPerWarp consecutive pairs:
-//   hist : per warp-chunk, the number of pairs of each expert           -> ws[chunk][e]
-//   scan : per expert, exclusive prefix over the chunks (in place), total -> counts[e]
-//   rank : offsets = exclusive prefix of counts; row(p) = offsets[e] + ws[chunk][e] + number of
-//          earlier pairs of the same expert inside the chunk.
+// a1, index part.  Two small kernels over the R = T*K pairs, split into block-chunks of `chunk`
+// consecutive pairs (a multiple of 256; one block per chunk, one eighth of it per warp):
+//   hist : per block-chunk, the number of pairs of each expert                  -> ws[block][e]
+//   rank : every block sums the histogram rows before it (its base) and all rows (the counts),
+//          turns the counts into offsets, ranks its warps' pairs with match/popc scans:
+//          row(p) = offsets[e] + base[e] + pairs of e in earlier warps of the block + earlier
+//          pairs of e in the same warp.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* __restrict__ topk_idx, int R, int E,
-                                                                int n_chunks, int32_t* __restrict__ ws) {
+                                                                int chunk, int32_t* __restrict__ ws) {
     extern __shared__ int32_t smem_i[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int chunk = blockIdx.x * kWarpsPerBlock + warp;
-    if (chunk >= n_chunks) return;
-    int32_t* hist = smem_i + warp * E;
-    for (int e = lane; e < E; e += 32) hist[e] = 0;
-    __syncwarp();
-    const int p0 = chunk * kPairsPerWarp;
-#pragma unroll 1
-    for (int it = 0; it < kPairsPerWarp / 32; ++it) {
-        const int p = p0 + it * 32 + lane;
+    int32_t* hist = smem_i;   // [E]
+    const int lane = threadIdx.x & 31;
+    for (int e = threadIdx.x; e < E; e += kThreads) hist[e] = 0;
+    __syncthreads();
+    const long long p0 = (long long)blockIdx.x * chunk;
+    for (int i = threadIdx.x; i < chunk; i += kThreads) {   // chunk is a multiple of kThreads: whole warps stay together
+        const long long p = p0 + i;
         int e = (p < R) ? topk_idx[p] : -1;
         if (e >= E) e = -1;
         const unsigned mask = __match_any_sync(0xffffffffu, e);
-        if (e >= 0 && lane == __ffs(mask) - 1) hist[e] += __popc(mask);
-        __syncwarp();
+        if (e >= 0 && lane == __ffs(mask) - 1) atomicAdd(&hist[e], __popc(mask));   // counts only: order-free
     }
-    int32_t* out = ws + (size_t)chunk * E;
-    for (int e = lane; e < E; e += 32) out[e] = hist[e];
-}
-
-__global__ void __launch_bounds__(kThreads) permute_scan_kernel(int32_t* __restrict__ ws, int n_chunks, int E,
-                                                                int32_t* __restrict__ counts) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int e = blockIdx.x * kWarpsPerBlock + warp;
-    if (e >= E) return;
-    const int per = (n_chunks + 31) / 32;
-    const int c0 = min(lane * per, n_chunks), c1 = min(c0 + per, n_chunks);
-    int sum = 0;
-    for (int c = c0; c < c1; ++c) sum += ws[(size_t)c * E + e];
-    int incl = sum;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += v;
-    }
-    int run = incl - sum;
-    for (int c = c0; c < c1; ++c) {
-        const int v = ws[(size_t)c * E + e];
-        ws[(size_t)c * E + e] = run;
-        run += v;
-    }
-    if (lane == 31) counts[e] = incl;
+    __syncthreads();
+    int32_t* out = ws + (size_t)blockIdx.x * E;
+    for (int e = threadIdx.x; e < E; e += kThreads) out[e] = hist[e];
 }
 
 __global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* __restrict__ topk_idx, int R, int E,
-                                                                int n_chunks, const int32_t* __restrict__ ws,
-                                                                const int32_t* __restrict__ counts,
+                                                                int chunk, int n_blocks,
+                                                                const int32_t* __restrict__ ws,
+                                                                int32_t* __restrict__ counts,
                                                                 int32_t* __restrict__ offsets,
                                                                 int32_t* __restrict__ row_to_pair,
                                                                 int32_t* __restrict__ pair_to_row) {
     extern __shared__ int32_t smem_i[];
-    int32_t* offs = smem_i;                 // [E+1]
-    int32_t* running_all = smem_i + E + 1;  // [warps][E]
+    int32_t* offs = smem_i;                       // [E+1] exclusive prefix of the counts
+    int32_t* total = smem_i + (E + 1);            // [E]   counts
+    int32_t* base = total + E;                    // [E]   pairs of e in earlier blocks
+    int32_t* whist = base + E;                    // [warps][E] per-warp counts, then running row cursors
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+    for (int e = threadIdx.x; e < E; e += kThreads) {
+        int before = 0, all = 0;
+        for (int b = 0; b < n_blocks; ++b) {
+            const int v = ws[(size_t)b * E + e];
+            all += v;
+            if (b < (int)blockIdx.x) before += v;
+        }
+        total[e] = all;
+        base[e] = before;
+    }
+    for (int i = threadIdx.x; i < kWarpsPerBlock * E; i += kThreads) whist[i] = 0;
+    __syncthreads();
     // offsets = exclusive prefix of counts, by warp 0 (each lane owns a contiguous run of experts)
     if (warp == 0) {
         const int per = (E + 31) / 32;
         const int e0 = min(lane * per, E), e1 = min(e0 + per, E);
         int sum = 0;
-        for (int e = e0; e < e1; ++e) sum += counts[e];
+        for (int e = e0; e < e1; ++e) sum += total[e];
         int incl = sum;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -116,63 +105,141 @@ __global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* _
         int run = incl - sum;
         for (int e = e0; e < e1; ++e) {
             offs[e] = run;
-            run += counts[e];
+            run += total[e];
         }
         if (lane == 31) offs[E] = incl;
     }
+    // pass 1: this warp's histogram over its eighth of the chunk
+    const int per_warp = chunk / kWarpsPerBlock;
+    const long long p0 = (long long)blockIdx.x * chunk + (long long)warp * per_warp;
+    int32_t* mine = whist + warp * E;
+#pragma unroll 1
+    for (int i = lane; i < per_warp; i += 32) {
+        const long long p = p0 + i;
+        int e = (p < R) ? topk_idx[p] : -1;
+        if (e >= E) e = -1;
+        const unsigned mask = __match_any_sync(0xffffffffu, e);
+        if (e >= 0 && lane == __ffs(mask) - 1) mine[e] += __popc(mask);
+        __syncwarp();
+    }
     __syncthreads();
-    if (blockIdx.x == 0)
+    if (blockIdx.x == 0) {
         for (int e = threadIdx.x; e <= E; e += kThreads) offsets[e] = offs[e];
-
-    const int chunk = blockIdx.x * kWarpsPerBlock + warp;
-    if (chunk >= n_chunks) return;
-    int32_t* running = running_all + warp * E;
-    const int32_t* base = ws + (size_t)chunk * E;
-    for (int e = lane; e < E; e += 32) running[e] = offs[e] + base[e];
-    __syncwarp();
-    const int p0 = chunk * kPairsPerWarp;
+        for (int e = threadIdx.x; e < E; e += kThreads) counts[e] = total[e];
+    }
+    // per-warp counts -> first row of each (warp, expert)
+    for (int e = threadIdx.x; e < E; e += kThreads) {
+        int run = offs[e] + base[e];
+#pragma unroll
+        for (int w = 0; w < kWarpsPerBlock; ++w) {
+            const int v = whist[w * E + e];
+            whist[w * E + e] = run;
+            run += v;
+        }
+    }
+    __syncthreads();
+    // pass 2: stable ranks
     const unsigned lt_mask = (1u << lane) - 1u;
 #pragma unroll 1
-    for (int it = 0; it < kPairsPerWarp / 32; ++it) {
-        const int p = p0 + it * 32 + lane;
+    for (int i = lane; i < per_warp; i += 32) {
+        const long long p = p0 + i;
         int e = (p < R) ? topk_idx[p] : -1;
         if (e >= E) e = -1;
         const unsigned mask = __match_any_sync(0xffffffffu, e);
         if (e >= 0) {
-            const int row = running[e] + __popc(mask & lt_mask);
-            row_to_pair[row] = p;
+            const int row = mine[e] + __popc(mask & lt_mask);
+            row_to_pair[row] = (int32_t)p;
             pair_to_row[p] = row;
         }
         __syncwarp();
-        if (e >= 0 && lane == __ffs(mask) - 1) running[e] += __popc(mask);
+        if (e >= 0 && lane == __ffs(mask) - 1) mine[e] += __popc(mask);
         __syncwarp();
     }
 }
 
 // ------------------------------------------------------------------------------------------------
-// a1, row part: x_perm[pair_to_row[t*K+k], :] = x[t, :].  One thread per 16-byte piece of a token
-// row; the piece is loaded once and stored to the K destination rows.
+// a1, row part: x_perm[pair_to_row[t*K+k], :] = x[t, :] with the bulk-copy engine.  One warp per CTA
+// runs a ring of NBUF shared-memory buffers: a token row (or a <= 16 KB segment of it) is pulled in
+// with one cp.async.bulk load and pushed to its K destination rows with K cp.async.bulk stores
+// (lane k issues store k), so the row is read from HBM once and no data passes through registers.
+// Loads run kRowLookahead units ahead of the stores.
 // ------------------------------------------------------------------------------------------------
-template <int KT>
-__global__ void __launch_bounds__(kThreads) permute_rows_kernel(const uint4* __restrict__ x,
-                                                                const int32_t* __restrict__ pair_to_row,
-                                                                uint4* __restrict__ x_perm, long long total,
-                                                                int hv, int K) {
-    const long long i = (long long)blockIdx.x * kThreads + threadIdx.x;
-    if (i >= total) return;
-    const int t = (int)(i / hv);
-    const int c = (int)(i - (long long)t * hv);
-    const uint4 v = ldg16(x + i);
-    const int32_t* rows = pair_to_row + (long long)t * K;
-    if (KT > 0) {
-        int r[KT > 0 ? KT : 1];
-#pragma unroll
-        for (int k = 0; k < KT; ++k) r[k] = __ldg(rows + k);
-#pragma unroll
-        for (int k = 0; k < KT; ++k) x_perm[(long long)r[k] * hv + c] = v;
-    } else {
-        for (int k = 0; k < K; ++k) x_perm[(long long)__ldg(rows + k) * hv + c] = v;
+constexpr int kRowBufs = 4, kRowLookahead = 2, kRowMaxSeg = 16384;
+__device__ int g_movement_status = 0;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__global__ void __launch_bounds__(32) permute_rows_bulk_kernel(const uint8_t* __restrict__ x,
+                                                               const int32_t* __restrict__ pair_to_row,
+                                                               uint8_t* __restrict__ x_perm, int T, int K,
+                                                               int row_bytes, int seg_bytes, int n_seg) {
+    extern __shared__ __align__(128) uint8_t bufs[];   // [kRowBufs][seg_bytes]
+    __shared__ unsigned long long bars[kRowBufs];
+    __shared__ int32_t dest[kRowBufs][32];
+    const int lane = threadIdx.x;
+    if (lane == 0) {
+        for (int s = 0; s < kRowBufs; ++s)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[s])) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    __syncwarp();
+    const long long n_units_all = (long long)T * n_seg;
+    const long long first = blockIdx.x, stride = gridDim.x;
+    const long long n_mine = first < n_units_all ? (n_units_all - first + stride - 1) / stride : 0;
+    bool ok = true;
+    for (long long it = 0; ok && it < n_mine + kRowLookahead; ++it) {
+        if (it < n_mine) {
+            const int s = (int)(it % kRowBufs);
+            const long long u = first + it * stride;
+            const int t = (int)(u / n_seg), seg = (int)(u - (long long)t * n_seg);
+            const int bytes = min(seg_bytes, row_bytes - seg * seg_bytes);
+            // the stores that last read this buffer were committed kRowLookahead iterations ago
+            if (it >= kRowBufs) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kRowLookahead - 1) : "memory");
+            if (lane < K) dest[s][lane] = __ldg(pair_to_row + (long long)t * K + lane);
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t bar = smem_addr(&bars[s]);
+                asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes)
+                             : "memory");
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                                 smem_addr(bufs + (size_t)s * seg_bytes)),
+                             "l"(x + (long long)t * row_bytes + (long long)seg * seg_bytes), "r"(bytes), "r"(bar)
+                             : "memory");
+            }
+        }
+        const long long j = it - kRowLookahead;
+        if (j >= 0) {
+            const int s = (int)(j % kRowBufs);
+            const uint32_t parity = (uint32_t)((j / kRowBufs) & 1);
+            const long long u = first + j * stride;
+            const int t = (int)(u / n_seg), seg = (int)(u - (long long)t * n_seg);
+            const int bytes = min(seg_bytes, row_bytes - seg * seg_bytes);
+            const uint32_t bar = smem_addr(&bars[s]);
+            uint32_t done = 0;
+            for (uint32_t spin = 0; !done; ++spin) {
+                asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                             : "=r"(done)
+                             : "r"(bar), "r"(parity)
+                             : "memory");
+                if (!done && spin > (1u << 24)) {   // bounded: give up, report, leave
+                    atomicExch(&g_movement_status, (int)MOE_ERR_TIMEOUT);
+                    ok = false;
+                    break;
+                }
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (lane < K) {
+                uint8_t* dst = x_perm + (long long)dest[s][lane] * row_bytes + (long long)seg * seg_bytes;
+                asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
+                             "r"(smem_addr(bufs + (size_t)s * seg_bytes)), "r"(bytes)
+                             : "memory");
+            }
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+    }
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __syncwarp();
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -322,34 +389,54 @@ size_t permute_workspace_bytes(const moe_dims_t& d) {
     return (size_t)(n_chunks * d.E) * sizeof(int32_t);
 }
 
+// pairs per block-chunk: 2048, or more (a multiple of 256) when R is so large that the rank kernel's
+// per-block sum over all histogram rows would otherwise grow past 512 rows
+static int permute_chunk(long long R) {
+    long long chunk = 2048;
+    const long long need = (R + 511) / 512;
+    if (need > chunk) chunk = (need + kThreads - 1) / kThreads * kThreads;
+    return (int)chunk;
+}
+
+int movement_read_and_clear_status(int* status_out) {
+    int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_movement_status, sizeof(int)) != cudaSuccess) return MOE_ERR_CUDA;
+    if (v != 0 && cudaMemcpyToSymbol(g_movement_status, &zero, sizeof(int)) != cudaSuccess) return MOE_ERR_CUDA;
+    *status_out = v;
+    return MOE_OK;
+}
+
 int launch_permute(const moe_dims_t& d, const bf16* x, const int32_t* topk_idx, bf16* x_perm, int32_t* counts,
                    int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row, void* workspace,
                    cudaStream_t s) {
     const int R = d.T * d.K, E = d.E;
-    const int n_chunks = (R + kPairsPerWarp - 1) / kPairsPerWarp;
-    const int chunk_blocks = (n_chunks + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const int chunk = permute_chunk(R);
+    const int n_blocks = (R + chunk - 1) / chunk;
     int32_t* ws = static_cast<int32_t*>(workspace);
-    permute_hist_kernel<<<chunk_blocks, kThreads, kWarpsPerBlock * E * sizeof(int32_t), s>>>(topk_idx, R, E,
-                                                                                             n_chunks, ws);
-    permute_scan_kernel<<<(E + kWarpsPerBlock - 1) / kWarpsPerBlock, kThreads, 0, s>>>(ws, n_chunks, E, counts);
-    permute_rank_kernel<<<chunk_blocks, kThreads, ((kWarpsPerBlock + 1) * E + 1) * sizeof(int32_t), s>>>(
-        topk_idx, R, E, n_chunks, ws, counts, offsets, row_to_pair, pair_to_row);
+    permute_hist_kernel<<<n_blocks, kThreads, E * sizeof(int32_t), s>>>(topk_idx, R, E, chunk, ws);
+    permute_rank_kernel<<<n_blocks, kThreads, ((kWarpsPerBlock + 3) * E + 1) * sizeof(int32_t), s>>>(
+        topk_idx, R, E, chunk, n_blocks, ws, counts, offsets, row_to_pair, pair_to_row);
     if (x_perm != nullptr) {
-        const int hv = d.H / 8;
-        const long long total = (long long)d.T * hv;
-        const uint4* src = reinterpret_cast<const uint4*>(x);
-        uint4* dst = reinterpret_cast<uint4*>(x_perm);
-#define MOE_ROWS_CASE(KT)                                                                                  \
-    case KT:                                                                                               \
-        permute_rows_kernel<KT><<<blocks_for(total), kThreads, 0, s>>>(src, pair_to_row, dst, total, hv, d.K); \
-        break;
-        switch (d.K) {
-            MOE_ROWS_CASE(1) MOE_ROWS_CASE(2) MOE_ROWS_CASE(3) MOE_ROWS_CASE(4) MOE_ROWS_CASE(5) MOE_ROWS_CASE(6)
-            MOE_ROWS_CASE(7) MOE_ROWS_CASE(8)
-            default:
-                permute_rows_kernel<0><<<blocks_for(total), kThreads, 0, s>>>(src, pair_to_row, dst, total, hv, d.K);
+        const int row_bytes = d.H * 2;
+        const int n_seg = (row_bytes + kRowMaxSeg - 1) / kRowMaxSeg;
+        const int seg_bytes = ((row_bytes + n_seg - 1) / n_seg + 15) / 16 * 16;
+        const size_t smem = (size_t)kRowBufs * seg_bytes;
+        static bool attr_set[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
+        if (!attr_set[dev]) {
+            if (cudaFuncSetAttribute(permute_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     kRowBufs * kRowMaxSeg) != cudaSuccess)
+                return MOE_ERR_CUDA;
+            attr_set[dev] = true;
         }
-#undef MOE_ROWS_CASE
+        const long long units = (long long)d.T * n_seg;
+        const int per_sm = (int)(196608 / (smem + 1024) < 8 ? 196608 / (smem + 1024) : 8);
+        long long grid = (long long)sm_count() * (per_sm < 1 ? 1 : per_sm);
+        if (grid > units) grid = units;
+        permute_rows_bulk_kernel<<<(unsigned)grid, 32, smem, s>>>(reinterpret_cast<const uint8_t*>(x), pair_to_row,
+                                                                  reinterpret_cast<uint8_t*>(x_perm), d.T, d.K, row_bytes,
+                                                                  seg_bytes, n_seg);
     }
     return check_launch();
 }
