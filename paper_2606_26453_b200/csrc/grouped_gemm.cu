@@ -35,6 +35,7 @@
 // raises a CTA-wide abort flag and every role leaves through the common teardown.
 #include <cuda.h>
 #include <cudaTypedefs.h>
+#include <cstdlib>
 
 #include "common.cuh"
 
@@ -58,24 +59,12 @@ namespace {
 constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int CHUNK_BYTES = 64 * BK * 2;   // one 64-wide MN-major block: 64 k-rows x 128 B = 8 KB
 constexpr int NUM_EPI_WARPS = 8;
-constexpr int STAGING_BYTES_PER_WARP = 32 * 32 * 2;   // one 32 x 32 bf16 output block
+constexpr int STAGING_BLOCK_BYTES = 32 * 32 * 2;   // one 32 x 32 bf16 output block
 constexpr int MAX_E = 1024;
 constexpr int MAX_STAGES = 6;
 constexpr int NUM_THREADS = 320;   // producer warp, MMA warp, 8 epilogue warps
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
-
-// Ring geometry of the two launch shapes.
-template <bool PAIR>
-struct Geo {
-    static constexpr int STAGES = PAIR ? 6 : 4;
-    static constexpr int TILE_M = PAIR ? 2 * BM : BM;        // output rows per tile (whole pair)
-    static constexpr int BN_LOCAL = PAIR ? BN / 2 : BN;      // B columns this CTA keeps in shared memory
-    static constexpr int A_BYTES = BM * BK * 2;              // 16 KB
-    static constexpr int B_BYTES = BN_LOCAL * BK * 2;        // 16 / 32 KB
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;    // 32 / 48 KB
-    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;  // 192 KB either way
-};
 
 enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3 };
 
@@ -107,6 +96,27 @@ struct SharedCtl {
     int abort_flag;
     int32_t offs[MAX_E + 1];
     int32_t tile_prefix[MAX_E + 1];
+};
+
+// Ring geometry of the two launch shapes.
+template <bool PAIR>
+struct Geo {
+#ifndef MOE_PAIR_STAGES
+#define MOE_PAIR_STAGES 6
+#endif
+#ifndef MOE_PAIR_STAGING
+#define MOE_PAIR_STAGING 1
+#endif
+    static constexpr int STAGES = PAIR ? MOE_PAIR_STAGES : 4;
+    static constexpr int STAGING_BLOCKS = PAIR ? MOE_PAIR_STAGING : 1;   // staging blocks per epilogue warp (2 = ping-pong)
+    static constexpr int TILE_M = PAIR ? 2 * BM : BM;        // output rows per tile (whole pair)
+    static constexpr int BN_LOCAL = PAIR ? BN / 2 : BN;      // B columns this CTA keeps in shared memory
+    static constexpr int A_BYTES = BM * BK * 2;              // 16 KB
+    static constexpr int B_BYTES = BN_LOCAL * BK * 2;        // 16 / 32 KB
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;    // 32 / 48 KB
+    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;  // 160 / 192 KB
+    static constexpr int STAGING_BYTES = NUM_EPI_WARPS * STAGING_BLOCKS * STAGING_BLOCK_BYTES;   // 32 / 16 KB
+    static constexpr int SMEM_BYTES = RING_BYTES + STAGING_BYTES + 1024 + (int)sizeof(SharedCtl);
 };
 
 // ---- small PTX wrappers ------------------------------------------------------------------------
@@ -162,6 +172,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait timed out, or another did).
+// Every lane of a waiting warp polls: electing one lane and broadcasting the verdict measured 5-10 % slower.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
@@ -179,7 +190,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
 }
-
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -199,6 +209,7 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int 
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
@@ -380,7 +391,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
-    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles_ptr + G::RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES_PER_WARP);
+    SharedCtl* ctl = reinterpret_cast<SharedCtl*>(tiles_ptr + G::RING_BYTES + G::STAGING_BYTES);
     volatile int* abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -586,28 +597,31 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // inside its expert (row-ragged kinds) falls back to predicated 16-byte row stores.
         const int quarter = warp & 3;               // TMEM lanes [32*quarter, 32*quarter+32)
         const int half = (warp - 2) >> 2;           // which half of the tile's columns this warp handles
-        uint8_t* stage_ptr = tiles_ptr + G::RING_BYTES + (warp - 2) * STAGING_BYTES_PER_WARP;
-        const uint32_t stage_addr = smem_u32(stage_ptr);
-        uint8_t* my_row = stage_ptr + lane * 64;
+        uint8_t* stage_ptr = tiles_ptr + G::RING_BYTES + (warp - 2) * (G::STAGING_BLOCKS * STAGING_BLOCK_BYTES);
         const int sw = (lane >> 1) & 3;             // 64-byte swizzle: 16-byte piece j of row r sits at j ^ ((r>>1)&3)
-        bool store_pending = false;
+        uint32_t n_stores = 0;                      // bulk stores issued so far by this warp
 
-        // stage one 32x32 bf16 block (this thread: 16 packed words of its row) and issue its bulk store
+        // stage one 32x32 bf16 block (this thread: 16 packed words of its row) and issue its bulk store;
+        // with two staging blocks the warp only waits for the store issued two blocks ago
         auto stage_and_store = [&](const uint32_t (&w)[16], const CUtensorMap* map, int x, int y) {
-            if (store_pending) {
-                if (lane == 0) bulk_wait_read0();
+            uint8_t* blk = stage_ptr + (n_stores % G::STAGING_BLOCKS) * STAGING_BLOCK_BYTES;
+            if (n_stores >= (uint32_t)G::STAGING_BLOCKS) {
+                if (lane == 0) {
+                    if (G::STAGING_BLOCKS == 2) bulk_wait_read1(); else bulk_wait_read0();
+                }
                 __syncwarp();
             }
+            uint8_t* my_row = blk + lane * 64;
 #pragma unroll
             for (int j = 0; j < 4; ++j)
                 *reinterpret_cast<uint4*>(my_row + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
-                tma_store_2d(map, x, y, stage_addr);
+                tma_store_2d(map, x, y, smem_u32(blk));
                 bulk_commit();
             }
-            store_pending = true;
+            ++n_stores;
         };
         auto direct_store = [&](const uint32_t (&w)[16], bf16* dst) {
             uint4* d4 = reinterpret_cast<uint4*>(dst);
@@ -700,7 +714,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
         // the staging buffer must have been read, and the stores completed, before the CTA exits
-        if (store_pending && lane == 0) bulk_wait_all0();
+        if (n_stores != 0 && lane == 0) bulk_wait_all0();
         __syncwarp();
     }
 
@@ -719,9 +733,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     }
 }
 
-constexpr size_t SMEM_BYTES = (size_t)Geo<false>::RING_BYTES + NUM_EPI_WARPS * STAGING_BYTES_PER_WARP + 1024 + sizeof(SharedCtl);
-static_assert(Geo<false>::RING_BYTES == Geo<true>::RING_BYTES, "both launch shapes use the same ring size");
-static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB of shared memory a CTA can opt in to");
+static_assert(Geo<false>::SMEM_BYTES <= 232448 && Geo<true>::SMEM_BYTES <= 232448,
+              "exceeds the 227 KB of shared memory a CTA can opt in to");
 
 // ---- host side ------------------------------------------------------------------------------------
 PFN_cuTensorMapEncodeTiled_v12000 get_encode_fn() {
@@ -781,7 +794,7 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
     auto kernel = grouped_gemm_kernel<KIND, PAIR>;
     if (grid_of_device[dev] == 0) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<PAIR>::SMEM_BYTES) != cudaSuccess)
             return MOE_ERR_CUDA;
         const int sms = sm_count();
         if (sms <= 0) return MOE_ERR_CUDA;
@@ -790,7 +803,7 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
             cudaLaunchAttribute qa[1];
             qa[0].id = cudaLaunchAttributeClusterDimension;
             qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
-            qc.gridDim = dim3(2 * (sms / 2)); qc.blockDim = dim3(NUM_THREADS); qc.dynamicSmemBytes = SMEM_BYTES;
+            qc.gridDim = dim3(2 * (sms / 2)); qc.blockDim = dim3(NUM_THREADS); qc.dynamicSmemBytes = Geo<PAIR>::SMEM_BYTES;
             qc.attrs = qa; qc.numAttrs = 1;
             int clusters = 0;
             if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &qc) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
@@ -804,7 +817,7 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
     cudaLaunchAttribute attr[1];
     cfg.gridDim = dim3(grid_of_device[dev]);
     cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.dynamicSmemBytes = Geo<PAIR>::SMEM_BYTES;
     cfg.stream = s;
     if (PAIR) {
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -817,7 +830,11 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
 
 // Row-ragged kinds use CTA pairs (256-row tiles) when experts are large enough on average that the extra
 // padding of the last tile of each expert costs less than the pair's better operand reuse buys.
-bool use_pairs_for_rows(const moe_dims_t& d) { return (long long)d.T * d.K >= 512ll * d.E; }
+bool use_pairs_for_rows(const moe_dims_t& d) {
+    const char* e = getenv("MOE_DBG_PAIR_MIN");
+    const long long thr = e ? atoll(e) : 512;
+    return (long long)d.T * d.K >= thr * d.E;
+}
 
 }  // namespace
 
@@ -890,21 +907,24 @@ int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate
     return pair ? launch<DGRAD, true>(a, b0, b1, o0, o0, p, s) : launch<DGRAD, false>(a, b0, b1, o0, o0, p, s);
 }
 
-// Weight gradients always run as CTA pairs: their tile grid is static (M x N per expert), 256 x 256 tiles
-// waste nothing unless M is an odd multiple of 128 (then the last pair's second CTA idles).
+// Weight gradients: the tile grid is static (M x N per expert).  Pairs (256 x 256 tiles) pay off once an
+// expert's contraction is long enough to amortise the pair's per-tile hand-shakes; with few rows per expert
+// the independent 128 x 256 tiles are faster.
 // Down wgrad: dw_down[e] [I,H] = h_act_e^T . dy_perm_e.  A = h_act [R,I] (M = I), B = dy_perm [R,H] (N = H).
 int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_perm, const int32_t* offsets,
                       bf16* dw_down, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
+    const bool pair = use_pairs_for_rows(d);
+    const int tile_m = pair ? 2 * BM : BM;
     CUtensorMap a, b0, o0;
-    if (!make_map_mn(&a, h_act, d.I, R, BM / 64) || !make_map_mn(&b0, dy_perm, d.H, R, BN / 128) ||
+    if (!make_map_mn(&a, h_act, d.I, R, BM / 64) || !make_map_mn(&b0, dy_perm, d.H, R, pair ? BN / 128 : BN / 64) ||
         !make_out_map(&o0, dw_down, d.H, (uint64_t)d.E * d.I))
         return MOE_ERR_CUDA;
     Params p = {};
-    p.offsets = offsets; p.E = d.E; p.m_rows = d.I; p.m_tiles = (d.I + 2 * BM - 1) / (2 * BM);
+    p.offsets = offsets; p.E = d.E; p.m_rows = d.I; p.m_tiles = (d.I + tile_m - 1) / tile_m;
     p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.n_split = d.H; p.ldo = d.H;
     p.out0 = dw_down; p.out1 = nullptr;
-    return launch<WGRAD, true>(a, b0, b0, o0, o0, p, s);
+    return pair ? launch<WGRAD, true>(a, b0, b0, o0, o0, p, s) : launch<WGRAD, false>(a, b0, b0, o0, o0, p, s);
 }
 
 // Gate/up wgrad (the paper's dW1): [dw_gate[e] | dw_up[e]] = x_perm_e^T . dgu_e.  A = x_perm [R,H] (M = H),
@@ -912,15 +932,17 @@ int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_per
 int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu, const int32_t* offsets,
                         bf16* dw_gate, bf16* dw_up, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
+    const bool pair = use_pairs_for_rows(d);
+    const int tile_m = pair ? 2 * BM : BM;
     CUtensorMap a, b0, o0, o1;
-    if (!make_map_mn(&a, x_perm, d.H, R, BM / 64) || !make_map_mn(&b0, dgu, 2ull * d.I, R, BN / 128) ||
+    if (!make_map_mn(&a, x_perm, d.H, R, BM / 64) || !make_map_mn(&b0, dgu, 2ull * d.I, R, pair ? BN / 128 : BN / 64) ||
         !make_out_map(&o0, dw_gate, d.I, (uint64_t)d.E * d.H) || !make_out_map(&o1, dw_up, d.I, (uint64_t)d.E * d.H))
         return MOE_ERR_CUDA;
     Params p = {};
-    p.offsets = offsets; p.E = d.E; p.m_rows = d.H; p.m_tiles = (d.H + 2 * BM - 1) / (2 * BM);
+    p.offsets = offsets; p.E = d.E; p.m_rows = d.H; p.m_tiles = (d.H + tile_m - 1) / tile_m;
     p.n_tiles = (2 * d.I + BN - 1) / BN; p.n_cols = 2 * d.I; p.n_split = d.I; p.ldo = d.I;
     p.out0 = dw_gate; p.out1 = dw_up;
-    return launch<WGRAD, true>(a, b0, b0, o0, o1, p, s);
+    return pair ? launch<WGRAD, true>(a, b0, b0, o0, o1, p, s) : launch<WGRAD, false>(a, b0, b0, o0, o1, p, s);
 }
 
 }  // namespace moe
