@@ -35,8 +35,16 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); None = not captured.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of each grouped-GEMM kernel, from the
+# ncu captures summarised in profiles/ncu_full_<workload>.md.  Workloads without a capture report null.
+NCU_TRAFFIC_BYTES = {
+    ("fine_grained", "gateup_swiglu"): 1030.4e6, ("fine_grained", "down"): 523.0e6,
+    ("fine_grained", "down_dgrad"): 528.6e6, ("fine_grained", "down_wgrad"): 486.7e6,
+    ("fine_grained", "gateup_dgrad"): 977.1e6, ("fine_grained", "gateup_wgrad"): 923.7e6,
+    ("many_small", "gateup_swiglu"): 2596.4e6, ("many_small", "down"): 1159.9e6,
+    ("many_small", "down_dgrad"): 1374.8e6, ("many_small", "down_wgrad"): 1239.7e6,
+    ("many_small", "gateup_dgrad"): 2192.4e6, ("many_small", "gateup_wgrad"): 2158.9e6,
+}
 
 
 def load_peaks():
@@ -109,7 +117,7 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 CALLS = ["permute", "gateup_swiglu", "down", "combine", "combine_bwd", "down_dgrad", "down_wgrad", "swiglu_bwd",
          "gateup_dgrad", "gateup_wgrad", "permute_bwd"]
-LAUNCHES_PER_CALL = {"permute": 4}
+LAUNCHES_PER_CALL = {"permute": 3}
 GEMM_CALLS = ["gateup_swiglu", "down", "down_dgrad", "down_wgrad", "gateup_dgrad", "gateup_wgrad"]
 
 
@@ -337,6 +345,34 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def stream_calibration(device):
+    """Read-only, write-only and copy stream rates of this GPU right now (torch library kernels on a 2 GiB
+    buffer).  Context for the data-movement kernels: their traffic mixes reads and writes very unevenly and
+    the write-only rate of this part is far below its copy rate."""
+    n = 1 << 30
+    a = torch.empty(n, dtype=torch.bfloat16, device=device)
+    b = torch.empty(n, dtype=torch.bfloat16, device=device)
+    a.zero_()
+
+    def rate(fn, nbytes, reps=10):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return nbytes * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+    out = {"write_only_gbs": rate(lambda: a.fill_(1.0), 2 * n), "read_only_gbs": rate(lambda: a.sum(), 2 * n),
+           "copy_gbs": rate(lambda: b.copy_(a), 4 * n)}
+    del a, b
+    torch.cuda.empty_cache()
+    return out
+
+
 def max_over_ranks(values, dist, device):
     """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
     if dist is None:
@@ -416,6 +452,7 @@ def run_ours(args):
             torch.cuda.empty_cache()
         if extra:
             line["other_configs"] = extra
+        line["stream_calibration"] = stream_calibration(device)
         if wl_host is not None:
             line["cpu_baseline"] = cpu_baseline(cfg, wl_host, min(args.ref_tokens, cfg.T))
     if rank == 0:

@@ -35,7 +35,6 @@
 // raises a CTA-wide abort flag and every role leaves through the common teardown.
 #include <cuda.h>
 #include <cudaTypedefs.h>
-#include <cstdlib>
 
 #include "common.cuh"
 
@@ -828,13 +827,11 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
     return check_launch();
 }
 
-// Row-ragged kinds use CTA pairs (256-row tiles) when experts are large enough on average that the extra
-// padding of the last tile of each expert costs less than the pair's better operand reuse buys.
-bool use_pairs_for_rows(const moe_dims_t& d) {
-    const char* e = getenv("MOE_DBG_PAIR_MIN");
-    const long long thr = e ? atoll(e) : 512;
-    return (long long)d.T * d.K >= thr * d.E;
-}
+// CTA pairs (256-row tiles) are used when experts hold at least 512 rows on average: below that the extra
+// padding of each expert's last tile (row-ragged kinds) and the pair's per-tile hand-shakes (short
+// contractions in the weight gradients) cost more than the halved operand traffic buys.  Measured: at 384
+// rows per expert single tiles are 8-25 % faster, from 1024 rows per expert on pairs are 5-15 % faster.
+bool use_pairs_for_rows(const moe_dims_t& d) { return (long long)d.T * d.K >= 512ll * d.E; }
 
 }  // namespace
 
