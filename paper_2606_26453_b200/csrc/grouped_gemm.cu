@@ -171,7 +171,8 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
     return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait timed out, or another did).
-// Every lane of a waiting warp polls: electing one lane and broadcasting the verdict measured 5-10 % slower.
+// Every lane of a waiting warp polls: electing one lane and broadcasting the verdict measured 5-10 % slower,
+// and suspend-time hints on the long waits changed nothing.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
@@ -367,6 +368,41 @@ __device__ __forceinline__ void zero_k_rows(uint8_t* stage_ptr, int n_chunks, in
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// The TMA loads of one ring stage: k-block `kb` of tile `tl`, for the CTA with row offset `my_rows` inside
+// the tile (and, in pair mode, its half of B).  (Prefetching the same boxes into L2 a few k-blocks ahead was
+// tried and cost 10-15 %: the L2 -> SM path, not DRAM latency, is what these kernels saturate.)
+template <int KIND, bool PAIR>
+__device__ __forceinline__ void stage_loads(const Tile& tl, int kb, const Params& p, const CUtensorMap* map_a,
+                                         const CUtensorMap* map_b0, const CUtensorMap* map_b1, uint32_t a_dst,
+                                         uint32_t b_dst, uint32_t full, uint32_t rank, int my_rows) {
+    const int n_local = tl.n0 + (PAIR ? my_rows : 0);   // first B column this CTA loads
+    if (KIND == WGRAD) {
+        const int krow = tl.k_row0 + kb * BK;
+        // MN-major operands: one 3-D box = all 64-wide chunks, chunk-major in shared memory
+        tma_load_3d(a_dst, map_a, 0, krow, (tl.row0 + my_rows) >> 6, full);
+        tma_load_3d(b_dst, map_b0, 0, krow, n_local >> 6, full);
+    } else {
+        tma_load_2d(a_dst, map_a, kb * BK, tl.row0 + my_rows, full);
+        if (KIND == DGRAD) {
+            const bool second = kb >= p.k_split;
+            const int kx = (second ? kb - p.k_split : kb) * BK;
+            tma_load_2d(b_dst, second ? map_b1 : map_b0, kx, tl.e * p.b_rows_per_e + n_local, full);
+        } else if (KIND == FWD_PLAIN) {
+            const int ky = tl.e * p.b_rows_per_e + kb * BK;
+            tma_load_3d(b_dst, map_b0, 0, ky, n_local >> 6, full);
+        } else {  // FWD_SWIGLU: 128 gate columns then 128 up columns
+            const int ky = tl.e * p.b_rows_per_e + kb * BK;
+            const int ng = tl.n0 >> 1;   // n0 counts fused (gate+up) columns
+            if (PAIR) {                  // first CTA holds the gate half of B, second the up half
+                tma_load_3d(b_dst, rank == 0 ? map_b0 : map_b1, 0, ky, ng >> 6, full);
+            } else {
+                tma_load_3d(b_dst, map_b0, 0, ky, ng >> 6, full);
+                tma_load_3d(b_dst + 2 * CHUNK_BYTES, map_b1, 0, ky, ng >> 6, full);
+            }
+        }
+    }
+}
+
 // ---- the kernel -----------------------------------------------------------------------------------
 // Operand major-ness per kind:
 //   FWD_*  : A K-major (activations [R, K]),   B MN-major (weights [E*K, N], N contiguous)
@@ -462,33 +498,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const uint32_t full = smem_u32(&ctl->full[stage]);
                     mbar_arrive_expect_tx(full, STAGE_BYTES);
                     const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
-                    const uint32_t b_dst = a_dst + G::A_BYTES;
-                    const int n_local = tl.n0 + (PAIR ? my_rows : 0);   // first B column this CTA loads
-                    if (KIND == WGRAD) {
-                        const int krow = tl.k_row0 + kb * BK;
-                        // MN-major operands: one 3-D box = all 64-wide chunks, chunk-major in shared memory
-                        tma_load_3d(a_dst, &map_a, 0, krow, (tl.row0 + my_rows) >> 6, full);
-                        tma_load_3d(b_dst, &map_b0, 0, krow, n_local >> 6, full);
-                    } else {
-                        tma_load_2d(a_dst, &map_a, kb * BK, tl.row0 + my_rows, full);
-                        if (KIND == DGRAD) {
-                            const bool second = kb >= p.k_split;
-                            const int kx = (second ? kb - p.k_split : kb) * BK;
-                            tma_load_2d(b_dst, second ? &map_b1 : &map_b0, kx, tl.e * p.b_rows_per_e + n_local, full);
-                        } else if (KIND == FWD_PLAIN) {
-                            const int ky = tl.e * p.b_rows_per_e + kb * BK;
-                            tma_load_3d(b_dst, &map_b0, 0, ky, n_local >> 6, full);
-                        } else {  // FWD_SWIGLU: 128 gate columns then 128 up columns
-                            const int ky = tl.e * p.b_rows_per_e + kb * BK;
-                            const int ng = tl.n0 >> 1;   // n0 counts fused (gate+up) columns
-                            if (PAIR) {                  // first CTA holds the gate half of B, second the up half
-                                tma_load_3d(b_dst, rank == 0 ? &map_b0 : &map_b1, 0, ky, ng >> 6, full);
-                            } else {
-                                tma_load_3d(b_dst, &map_b0, 0, ky, ng >> 6, full);
-                                tma_load_3d(b_dst + 2 * CHUNK_BYTES, &map_b1, 0, ky, ng >> 6, full);
-                            }
-                        }
-                    }
+                    stage_loads<KIND, PAIR>(tl, kb, p, &map_a, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES, full, rank, my_rows);
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }

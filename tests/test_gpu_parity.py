@@ -314,3 +314,42 @@ def test_host_entry_point_matches_device_chain(B):
     torch.cuda.synchronize()
     assert torch.equal(yh, b.y.cpu()) and torch.equal(dxh, b.dx.cpu()) and torch.equal(dwh, b.dtopk_w.cpu())
     assert torch.equal(dwg, b.dw_gate) and torch.equal(dwu, b.dw_up) and torch.equal(dwd, b.dw_down)
+
+
+# ------------------------------------------------------------------------------------------------
+# degenerate shapes: a single expert, top-1, fewer rows than one tile, one token, many experts
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("T,H,I,E,K", [(1, 128, 128, 1, 1), (3, 128, 128, 4, 2), (130, 256, 128, 1, 1),
+                                       (64, 128, 256, 300, 4), (40, 384, 128, 33, 32), (513, 128, 128, 2, 1)])
+def test_degenerate_shapes_end_to_end(B, T, H, I, E, K):
+    cfg = W.MoeConfig("deg", T=T, H=H, I=I, E=E, K=K, routing="softmax", cfg_id=70 + T % 7)
+    host = W.make_workload(cfg)
+    ref = O.layer_fwd_bwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"],
+                          host["W_down"], host["dY"])
+    b = Hh.run_cuda_layer(Hh.device_workload(host), E)
+    for name in ("counts", "offsets", "row_to_pair", "pair_to_row"):
+        assert np.array_equal(getattr(b, name).cpu().numpy(), ref[name]), name
+    for attr, key in FLOAT_OUTPUTS:
+        Hh.assert_close(Hh.to_np64(getattr(b, attr)), ref[key], key)
+    Hh.assert_close(b.dtopk_w.cpu().numpy().astype(np.float64), ref["dtopk_w"], "dtopk_w")
+
+
+def test_pair_and_single_tile_shapes_agree(B):
+    """The same experts' rows run through the CTA-pair kernels (>= 512 rows per expert on average) and, split
+    over twice as many experts with duplicated weights, through the single-CTA kernels: equal outputs."""
+    counts = [700, 650, 520, 690]
+    cfg, host = Hh.ragged_workload(counts, K=2, H=256, I=256, seed=5)
+    ref = O.layer_fwd_bwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"],
+                          host["W_down"], host["dY"])
+    b = Hh.run_cuda_layer(Hh.device_workload(host), cfg.E)            # 640 rows per expert: pair kernels
+    for attr, key in FLOAT_OUTPUTS:
+        Hh.assert_close(Hh.to_np64(getattr(b, attr)), ref[key], key)
+    # pad with 4 experts that get no rows: 320 rows per expert on average -> single-CTA kernels
+    pad = lambda w: np.concatenate([w, np.zeros_like(w)], axis=0)
+    host2 = dict(host, W_gate=pad(host["W_gate"]), W_up=pad(host["W_up"]), W_down=pad(host["W_down"]))
+    b2 = Hh.run_cuda_layer(Hh.device_workload(host2), 2 * cfg.E)
+    for attr in ("y", "dx", "h_act", "gu", "y_perm", "dh_act", "dgu", "dx_perm"):
+        assert torch.equal(getattr(b, attr), getattr(b2, attr)), attr   # same arithmetic order per element
+    for attr in ("dw_gate", "dw_up", "dw_down"):
+        assert torch.equal(getattr(b, attr), getattr(b2, attr)[:cfg.E]), attr
+        assert not bool(getattr(b2, attr)[cfg.E:].any())
