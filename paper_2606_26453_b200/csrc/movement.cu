@@ -289,52 +289,57 @@ __global__ void __launch_bounds__(kThreads) gather_sum_kernel(const uint4* __res
 }
 
 // ------------------------------------------------------------------------------------------------
-// a5: one warp per token.  dy_perm[row_k, :] = w_k * dy[t, :]; dtopk_w[t,k] = <dy[t,:], y_perm[row_k,:]>.
+// a5: one block per token, one thread per 16-byte piece of the row.
+// dy_perm[row_k, :] = w_k * dy[t, :]; dtopk_w[t,k] = <dy[t,:], y_perm[row_k,:]> (warp shuffles, then a
+// fixed-order sum over the block's warps: deterministic).  y_perm pieces are fetched four slots at a time
+// to keep the register count low enough for five blocks per SM.
 // ------------------------------------------------------------------------------------------------
 template <int KT, bool WITH_DW>
-__global__ void __launch_bounds__(kThreads) combine_bwd_kernel(const uint4* __restrict__ dy,
-                                                               const uint4* __restrict__ y_perm,
-                                                               const float* __restrict__ topk_w,
-                                                               const int32_t* __restrict__ pair_to_row,
-                                                               uint4* __restrict__ dy_perm,
-                                                               float* __restrict__ dtopk_w, int T, int hv, int K) {
+__global__ void __launch_bounds__(kThreads, 5) combine_bwd_kernel(const uint4* __restrict__ dy,
+                                                                  const uint4* __restrict__ y_perm,
+                                                                  const float* __restrict__ topk_w,
+                                                                  const int32_t* __restrict__ pair_to_row,
+                                                                  uint4* __restrict__ dy_perm,
+                                                                  float* __restrict__ dtopk_w, int T, int hv, int K) {
     constexpr int KA = KT > 0 ? KT : 32;
+    __shared__ float partial[kWarpsPerBlock][32];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t = blockIdx.x * kWarpsPerBlock + warp;
-    if (t >= T) return;
+    const int t = blockIdx.x;
     const int kk = KT > 0 ? KT : K;
-    int rows[KA];
-    float w[KA], dot[KA];
+    const int32_t* rows = pair_to_row + (long long)t * K;
+    const float* wt = topk_w + (long long)t * K;
+    float dot[KA];
 #pragma unroll
-    for (int k = 0; k < KA; ++k) {
-        if (k < kk) {
-            rows[k] = __ldg(pair_to_row + (long long)t * K + k);
-            w[k] = __ldg(topk_w + (long long)t * K + k);
-        }
-        dot[k] = 0.f;
-    }
-    for (int c = lane; c < hv; c += 32) {
+    for (int k = 0; k < KA; ++k) dot[k] = 0.f;
+    for (int c = threadIdx.x; c < hv; c += kThreads) {
         const uint4 dv = ldg16(dy + (long long)t * hv + c);
         float d[8];
         unpack8(dv, d);
-        uint4 yv[KA];
-        if (WITH_DW) {
 #pragma unroll
-            for (int k = 0; k < KA; ++k)
-                if (k < kk) yv[k] = ldg16(y_perm + (long long)rows[k] * hv + c);
-        }
+        for (int k0 = 0; k0 < KA; k0 += 4) {
+            uint4 yv[4];
+            long long row[4];
 #pragma unroll
-        for (int k = 0; k < KA; ++k) {
-            if (k < kk) {
-                float o[8];
+            for (int q = 0; q < 4; ++q) {
+                if (k0 + q < kk) {
+                    row[q] = __ldg(rows + k0 + q);
+                    if (WITH_DW) yv[q] = ldg16(y_perm + row[q] * hv + c);
+                }
+            }
 #pragma unroll
-                for (int j = 0; j < 8; ++j) o[j] = w[k] * d[j];
-                dy_perm[(long long)rows[k] * hv + c] = pack8(o);
-                if (WITH_DW) {
-                    float y[8];
-                    unpack8(yv[k], y);
+            for (int q = 0; q < 4; ++q) {
+                if (k0 + q < kk) {
+                    const float w = __ldg(wt + k0 + q);
+                    float o[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) dot[k] = fmaf(d[j], y[j], dot[k]);
+                    for (int j = 0; j < 8; ++j) o[j] = w * d[j];
+                    dy_perm[row[q] * hv + c] = pack8(o);
+                    if (WITH_DW) {
+                        float y[8];
+                        unpack8(yv[q], y);
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) dot[k0 + q] = fmaf(d[j], y[j], dot[k0 + q]);
+                    }
                 }
             }
         }
@@ -346,8 +351,15 @@ __global__ void __launch_bounds__(kThreads) combine_bwd_kernel(const uint4* __re
                 float v = dot[k];
 #pragma unroll
                 for (int s = 16; s > 0; s >>= 1) v += __shfl_xor_sync(0xffffffffu, v, s);
-                if (lane == 0) dtopk_w[(long long)t * K + k] = v;
+                if (lane == 0) partial[warp][k] = v;
             }
+        }
+        __syncthreads();
+        if (threadIdx.x < kk) {
+            float v = 0.f;
+#pragma unroll
+            for (int wq = 0; wq < kWarpsPerBlock; ++wq) v += partial[wq][threadIdx.x];
+            dtopk_w[(long long)t * K + threadIdx.x] = v;
         }
     }
 }
@@ -474,7 +486,7 @@ template <bool WITH_DW>
 static void combine_bwd_dispatch(const moe_dims_t& d, const uint4* dy, const uint4* yp, const float* w,
                                  const int32_t* p2r, uint4* dyp, float* dw, cudaStream_t s) {
     const int hv = d.H / 8;
-    const unsigned blocks = (unsigned)((d.T + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    const unsigned blocks = (unsigned)d.T;
 #define MOE_CB_CASE(KT)                                                                                     \
     case KT:                                                                                                \
         combine_bwd_kernel<KT, WITH_DW><<<blocks, kThreads, 0, s>>>(dy, yp, w, p2r, dyp, dw, d.T, hv, d.K); \
