@@ -24,7 +24,10 @@
  *   - Unless a parameter says "host", every pointer is a DEVICE pointer to memory owned by the
  *     caller, 16-byte aligned.  The library allocates nothing, keeps no pointer after a call
  *     returns, and never synchronises: all work is enqueued on `stream` (a cudaStream_t) in
- *     order.  Outputs are overwritten.  Inputs and outputs must not overlap.
+ *     order.  Outputs are overwritten.  Inputs and outputs must not overlap.  Nothing a call does depends
+ *     on data that must first travel to the host, so a sequence of calls can be captured in a CUDA
+ *     graph and replayed; run each kind of call once on the device before capturing (the first call of a
+ *     kernel sets its launch attributes and queries occupancy).
  *   - H and I must be multiples of 128; 1 <= K <= E <= 1024; K <= 32; T*K < 2^31.
  *   - Return value: MOE_OK or an error code.  Argument errors are detected on the host before
  *     anything is launched.  A kernel that gives up waiting (bounded waits, never a trap) records

@@ -353,3 +353,34 @@ def test_pair_and_single_tile_shapes_agree(B):
     for attr in ("dw_gate", "dw_up", "dw_down"):
         assert torch.equal(getattr(b, attr), getattr(b2, attr)[:cfg.E]), attr
         assert not bool(getattr(b2, attr)[cfg.E:].any())
+
+
+def test_layer_can_be_captured_in_a_cuda_graph_and_replayed(B):
+    """All work is enqueued on the caller's stream with no host synchronisation or allocation, so a whole
+    forward + backward can be captured once and replayed on new inputs written into the same buffers."""
+    cfg, host = Hh.ragged_workload([300, 0, 77, 200, 1, 190], K=2, H=256, I=256, seed=7)
+    dev = Hh.device_workload(host)
+    b = Hh.run_cuda_layer(dev, cfg.E)                       # first calls (attribute set-up) outside capture
+    want = {a: getattr(b, a).clone() for a, _ in FLOAT_OUTPUTS}
+    x_static, dy_static = dev["X"].clone(), dev["dY"].clone()
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            B.layer_forward(b, x_static, dev["topk_idx"], dev["topk_w"], dev["W_gate"], dev["W_up"], dev["W_down"])
+            B.layer_backward(b, dy_static, dev["topk_w"], dev["W_gate"], dev["W_up"], dev["W_down"])
+    for a, _ in FLOAT_OUTPUTS:
+        getattr(b, a).fill_(float("nan"))
+    graph.replay()
+    torch.cuda.synchronize()
+    for a, _ in FLOAT_OUTPUTS:
+        assert torch.equal(getattr(b, a), want[a]), a
+    # new inputs in the captured buffers: doubling X and dY doubles X_perm and dY_perm exactly (powers of two)
+    x_static.mul_(2.0)
+    dy_static.mul_(2.0)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(b.x_perm, want["x_perm"] * 2) if "x_perm" in want else True
+    assert torch.equal(b.dy_perm, want["dy_perm"] * 2)
+    assert B.moe_device_status() == 0
