@@ -144,14 +144,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(bar) : "memory");
 }
 // Arrive on a barrier of another CTA of the cluster (address from map_to_cta).  Default semantics: a
-// cluster-scope release on every ring stage would serialise the pipeline on a fence; the data the arrival
-// announces was written by the TMA unit and is consumed by the tensor cores, both ordered by the barriers
-// themselves.  Generic-proxy writes that must be visible to the other CTA are fenced explicitly
-// (cluster_fence) at the one place they occur.
+// cluster-scope release/acquire pair on every ring stage serialises the pipeline on fences (measured: half
+// the throughput; even one fence per tile costs 10-20 % on short contractions).  None is needed: the data
+// the arrival announces sits in the ARRIVING CTA's own shared memory -- written there by the TMA unit
+// (complete before the local barrier wait returns) or by this warp's generic stores (each lane runs
+// fence.proxy.async after its stores and the warp synchronises before the arrive is issued) -- and is
+// read from there by that CTA's own tensor core once the first CTA, having seen the arrival, issues the MMA.
 __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_bar) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
-__device__ __forceinline__ void cluster_fence() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes)
                  : "memory");
@@ -569,10 +570,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const int rem = tl.k_rows - kb * BK;
                     if (rem < BK) {
                         n_mma = (rem + 15) >> 4;
-                        if (n_mma * 16 > rem) {
-                            zero_k_rows(tiles_ptr + stage * STAGE_BYTES, STAGE_CHUNKS, rem, n_mma * 16, lane);
-                            if (PAIR) cluster_fence();   // pairs with the relay's fence: its cleared rows are visible too
-                        }
+                        if (n_mma * 16 > rem) zero_k_rows(tiles_ptr + stage * STAGE_BYTES, STAGE_CHUNKS, rem, n_mma * 16, lane);
                         __syncwarp();
                     }
                 }
@@ -622,10 +620,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const int rem = tl.k_rows - kb * BK;
                     if (rem < BK) {
                         const int z1 = ((rem + 15) >> 4) * 16;
-                        if (z1 > rem) {
-                            zero_k_rows(tiles_ptr + stage * STAGE_BYTES, STAGE_CHUNKS, rem, z1, lane);
-                            cluster_fence();
-                        }
+                        if (z1 > rem) zero_k_rows(tiles_ptr + stage * STAGE_BYTES, STAGE_CHUNKS, rem, z1, lane);
                     }
                 }
                 __syncwarp();
@@ -880,6 +875,8 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
 // contractions in the weight gradients) cost more than the halved operand traffic buys.  Measured: at 384
 // rows per expert single tiles are 8-25 % faster, from 1024 rows per expert on pairs are 5-15 % faster.
 bool use_pairs_for_rows(const moe_dims_t& d) { return (long long)d.T * d.K >= 512ll * d.E; }
+// Weight gradients have no row padding to lose, so pairs already win from 256 rows per expert.
+bool use_pairs_for_wgrad(const moe_dims_t& d) { return (long long)d.T * d.K >= 256ll * d.E; }
 
 }  // namespace
 
@@ -959,7 +956,7 @@ int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate
 int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_perm, const int32_t* offsets,
                       bf16* dw_down, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    const bool pair = use_pairs_for_rows(d);
+    const bool pair = use_pairs_for_wgrad(d);
     const int tile_m = pair ? 2 * BM : BM;
     CUtensorMap a, b0, o0;
     if (!make_map_mn(&a, h_act, d.I, R, BM / 64) || !make_map_mn(&b0, dy_perm, d.H, R, pair ? BN / 128 : BN / 64) ||
@@ -977,7 +974,7 @@ int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_per
 int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu, const int32_t* offsets,
                         bf16* dw_gate, bf16* dw_up, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    const bool pair = use_pairs_for_rows(d);
+    const bool pair = use_pairs_for_wgrad(d);
     const int tile_m = pair ? 2 * BM : BM;
     CUtensorMap a, b0, o0, o1;
     if (!make_map_mn(&a, x_perm, d.H, R, BM / 64) || !make_map_mn(&b0, dgu, 2ull * d.I, R, pair ? BN / 128 : BN / 64) ||
