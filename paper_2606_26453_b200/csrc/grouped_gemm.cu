@@ -18,11 +18,12 @@
 //   pair    a cluster of two CTAs computes a 256 x 256 tile with tcgen05.mma.cta_group::2: each CTA
 //           loads its 128 rows of A and HALF of B (6 stages of 32 KB), the tensor cores of both SMs
 //           read both halves.  That cuts the bytes each SM must pull from L2 per flop by a third
-//           and deepens the ring, which is what the L2 -> SM path needs at full MMA rate.  Only
-//           plain (non-multicast) TMA loads are used: each CTA's loads complete on its own
+//           and deepens the ring, which is what the L2 -> SM path needs at full MMA rate.  Every
+//           TMA load has a single destination CTA: each CTA's loads complete on its own
 //           barrier, a relay warp in the second CTA forwards "my half has landed" to the first
 //           CTA's barrier with a remote mbarrier arrive, and the first CTA's MMA warp releases
-//           stages / publishes accumulators in both CTAs with a multicast tcgen05.commit.
+//           stages / publishes accumulators in both CTAs with one tcgen05.commit that arrives on
+//           the barriers of both CTAs.
 //
 // Two ragged shapes occur:
 //   row-ragged (forward, dgrad): output rows are the packed rows of an expert.  A tile starts at
