@@ -38,12 +38,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of each grouped-GEMM kernel, from the
 # ncu captures summarised in profiles/ncu_full_<workload>.md.  Workloads without a capture report null.
 NCU_TRAFFIC_BYTES = {
-    ("fine_grained", "gateup_swiglu"): 1030.4e6, ("fine_grained", "down"): 523.0e6,
-    ("fine_grained", "down_dgrad"): 528.6e6, ("fine_grained", "down_wgrad"): 486.7e6,
-    ("fine_grained", "gateup_dgrad"): 977.1e6, ("fine_grained", "gateup_wgrad"): 923.7e6,
-    ("many_small", "gateup_swiglu"): 2596.4e6, ("many_small", "down"): 1159.9e6,
-    ("many_small", "down_dgrad"): 1374.8e6, ("many_small", "down_wgrad"): 1239.7e6,
-    ("many_small", "gateup_dgrad"): 2192.4e6, ("many_small", "gateup_wgrad"): 2158.9e6,
+    ("fine_grained", "gateup_swiglu"): 1029.1e6, ("fine_grained", "down"): 523.5e6,
+    ("fine_grained", "down_dgrad"): 527.5e6, ("fine_grained", "down_wgrad"): 498.1e6,
+    ("fine_grained", "gateup_dgrad"): 975.0e6, ("fine_grained", "gateup_wgrad"): 945.3e6,
+    ("many_small", "gateup_swiglu"): 2594.3e6, ("many_small", "down"): 1166.9e6,
+    ("many_small", "down_dgrad"): 1405.9e6, ("many_small", "down_wgrad"): 1215.6e6,
+    ("many_small", "gateup_dgrad"): 2195.9e6, ("many_small", "gateup_wgrad"): 2124.7e6,
 }
 
 
