@@ -1,8 +1,8 @@
 // HBM-bound kernels of the MoE layer: route-permute (stable counting sort by expert + row
 // gather), unpermute-combine and its backward, permute backward, SwiGLU backward.
 //
-// Row movement is token-major: every source row is read once with 16-byte loads and written (or
-// gathered) K times, so the bytes moved are the algorithmic minimum.  The permutation indices
+// Row movement is token-major: every source row is read once and written (bulk copies) or gathered
+// (16-byte loads) K times, so the bytes moved are the algorithmic minimum.  The permutation indices
 // never depend on the order in which atomics land: ranks come from warp-level match/ballot
 // scans over pairs taken in ascending pair id, which makes the result the unique stable sort.
 #include "common.cuh"
@@ -11,7 +11,7 @@ namespace moe {
 
 namespace {
 
-constexpr int kPairsPerWarp = 256;   // workspace is sized for one histogram row per 256 pairs (an upper bound)
+constexpr int kWorkspacePairsPerRow = 256;   // the workspace holds one histogram row per 256 pairs (an upper bound on what is used)
 constexpr int kWarpsPerBlock = 8;
 constexpr int kThreads = kWarpsPerBlock * 32;
 
@@ -397,7 +397,7 @@ inline unsigned blocks_for(long long total) { return (unsigned)((total + kThread
 
 size_t permute_workspace_bytes(const moe_dims_t& d) {
     const long long R = (long long)d.T * d.K;
-    const long long n_chunks = (R + kPairsPerWarp - 1) / kPairsPerWarp;
+    const long long n_chunks = (R + kWorkspacePairsPerRow - 1) / kWorkspacePairsPerRow;
     return (size_t)(n_chunks * d.E) * sizeof(int32_t);
 }
 
