@@ -470,7 +470,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--config", default="fine_grained", choices=list(W.CONFIGS))
     ap.add_argument("--custom", default="", help="T,H,I,E,K of an ad-hoc softmax-routed workload (profiling aid)")
-    ap.add_argument("--also", default="many_small,few_large,imbalanced",
+    ap.add_argument("--also", default="many_small,few_large,imbalanced,paper_dw1",
                     help="comma-separated other configurations to time briefly at N=1 ('' for none)")
     ap.add_argument("--ref-tokens", type=int, default=512, help="tokens in the oracle's timed sample")
     ap.add_argument("--host-inputs", default="device", choices=["device", "numpy"])

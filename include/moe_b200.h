@@ -28,7 +28,7 @@
  *     on data that must first travel to the host, so a sequence of calls can be captured in a CUDA
  *     graph and replayed; run each kind of call once on the device before capturing (the first call of a
  *     kernel sets its launch attributes and queries occupancy).
- *   - H and I must be multiples of 128; 1 <= K <= E <= 1024; K <= 32; T*K < 2^31.
+ *   - H and I must be multiples of 64; 1 <= K <= E <= 1024; K <= 32; T*K < 2^31.
  *   - Return value: MOE_OK or an error code.  Argument errors are detected on the host before
  *     anything is launched.  A kernel that gives up waiting (bounded waits, never a trap) records
  *     MOE_ERR_TIMEOUT in a device status word readable with moe_device_status().
@@ -57,7 +57,7 @@ typedef enum {
     MOE_OK = 0,
     MOE_ERR_NULL = 1,              /* a required pointer is NULL */
     MOE_ERR_DIMS = 2,              /* non-positive size, K > E, R overflow */
-    MOE_ERR_UNSUPPORTED_SHAPE = 3, /* H or I not a multiple of 128, E or K above the limits */
+    MOE_ERR_UNSUPPORTED_SHAPE = 3, /* H or I not a multiple of 64, E or K above the limits */
     MOE_ERR_ALIGNMENT = 4,         /* a pointer is not 16-byte aligned */
     MOE_ERR_WORKSPACE = 5,         /* workspace / arena too small */
     MOE_ERR_CUDA = 6,              /* a CUDA runtime or driver call failed */

@@ -20,7 +20,7 @@ int check_dims(const moe_dims_t* d) {
     if (d == nullptr) return MOE_ERR_NULL;
     if (d->T <= 0 || d->H <= 0 || d->I <= 0 || d->E <= 0 || d->K <= 0 || d->K > d->E) return MOE_ERR_DIMS;
     if ((long long)d->T * d->K >= (1ll << 31)) return MOE_ERR_DIMS;
-    if (d->H % 128 != 0 || d->I % 128 != 0 || d->E > 1024 || d->K > 32) return MOE_ERR_UNSUPPORTED_SHAPE;
+    if (d->H % 64 != 0 || d->I % 64 != 0 || d->E > 1024 || d->K > 32) return MOE_ERR_UNSUPPORTED_SHAPE;
     return MOE_OK;
 }
 
@@ -65,7 +65,7 @@ const char* moe_status_string(int status) {
         case MOE_OK: return "ok";
         case MOE_ERR_NULL: return "a required pointer is NULL";
         case MOE_ERR_DIMS: return "invalid dimensions";
-        case MOE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (H, I must be multiples of 128; E <= 1024; K <= 32)";
+        case MOE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape (H, I must be multiples of 64; E <= 1024; K <= 32)";
         case MOE_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
         case MOE_ERR_WORKSPACE: return "workspace or arena too small";
         case MOE_ERR_CUDA: return "CUDA call failed";

@@ -693,7 +693,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     tc_ld32(taddr + c * 32, g);
                     tc_ld32(taddr + 128 + c * 32, u);
                     tc_wait_ld();
-                    if (rows_valid == 0) continue;
+                    if (rows_valid == 0 || ng + c * 32 >= p.I) continue;   // past the expert's rows / past column I
                     uint32_t hp[16], gp[16], up[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
@@ -893,7 +893,7 @@ int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gat
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
-    p.n_tiles = d.I / 128; p.n_cols = 2 * d.I; p.b_rows_per_e = d.H;
+    p.n_tiles = (d.I + 127) / 128; p.n_cols = 2 * d.I; p.b_rows_per_e = d.H;
     p.out0 = h_act; p.gu = gu; p.I = d.I; p.ldo = d.I; p.n_split = 2 * d.I;
     return use_pairs_for_rows(d) ? launch<FWD_SWIGLU, true>(a, b0, b1, o0, o1, p, s)
                                  : launch<FWD_SWIGLU, false>(a, b0, b1, o0, o1, p, s);

@@ -38,7 +38,7 @@ class MoeConfig:
     I: int
     E: int
     K: int
-    routing: str = "softmax"      # "softmax" | "skew" | "zipf"
+    routing: str = "softmax"      # "softmax" | "skew" | "zipf" | "dirichlet_multinomial"
     n_empty: int = 0              # zipf only: ranks that get probability zero
     cfg_id: int = 0
 
@@ -60,6 +60,12 @@ CONFIGS = {
     "imbalanced": MoeConfig("imbalanced", T=32768, H=4096, I=1536, E=64, K=8, routing="zipf", n_empty=4, cfg_id=5),
 }
 CONFIG_ORDER = ["tiny", "fine_grained", "many_small", "few_large", "imbalanced"]
+
+# The paper's own weight-gradient workload (section "Production Validation: VeOmni MoE" and its appendix):
+# hidden 2880, gate_up width 5760 (I = 2880), 128 experts, top-4, R = 57 768 routed rows whose per-expert counts
+# follow Dirichlet(0.24)-multinomial (heavy tail, several empty experts).  14 442 tokens x 4 = 57 768.
+CONFIGS["paper_dw1"] = MoeConfig("paper_dw1", T=14442, H=2880, I=2880, E=128, K=4, routing="dirichlet_multinomial",
+                                 cfg_id=6)
 
 
 def round_to_bf16(x) -> np.ndarray:
@@ -103,6 +109,9 @@ def make_routing(cfg: MoeConfig, seed: int = 0):
         gumbel = _rng(seed, cfg.cfg_id, 5).gumbel(size=(T, E))
         idx = _topk_desc(logq[None, :] + gumbel, K)
         w = _rng(seed, cfg.cfg_id, 7).dirichlet(np.ones(K), size=T)
+    elif cfg.routing == "dirichlet_multinomial":
+        counts = dirichlet_multinomial_counts(E, T * K, alpha=0.24, seed=seed + cfg.cfg_id)
+        return make_routing_from_counts(counts, K, seed)
     else:
         raise ValueError(cfg.routing)
     return idx.astype(np.int32), round_to_bf16(w.astype(np.float32))

@@ -29,6 +29,9 @@ CASES = {
     "tiny": lambda: (W.CONFIGS["tiny"], W.make_workload(W.CONFIGS["tiny"])),
     "ragged": lambda: Hh.ragged_workload(RAGGED_COUNTS, K=2, H=256, I=384, seed=1),
     "ragged_k5": lambda: Hh.ragged_workload([65, 0, 250, 33, 17, 640], K=5, H=384, I=128, seed=2),
+    # H and I multiples of 64 only (the paper's 2880 = 45 * 64): partial column tiles everywhere
+    "ragged_64": lambda: Hh.ragged_workload([200, 0, 31, 290, 1], K=2, H=192, I=320, seed=4),
+    "pair_64": lambda: Hh.ragged_workload([600, 540, 0, 700], K=2, H=320, I=192, seed=6),
 }
 
 

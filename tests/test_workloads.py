@@ -84,3 +84,15 @@ def test_flop_accounting():
     cfg = W.CONFIGS["few_large"]
     assert cfg.R == 16384
     assert abs(cfg.flops_fwd_bwd / 1e12 - 17.3173) < 1e-3
+
+
+def test_paper_workload_routing_matches_its_load_model():
+    g = read_golden()
+    cfg = W.CONFIGS["paper_dw1"]
+    assert (cfg.H, 2 * cfg.I, cfg.E, cfg.K, cfg.R) == (int(g["M"]), int(g["N"]), int(g["E"]), int(g["top_k"]), int(g["R"]))
+    idx, w = W.make_routing(cfg)
+    counts = np.bincount(idx.reshape(-1), minlength=cfg.E)
+    assert counts.sum() == cfg.R and (counts == 0).sum() >= 3
+    cv = counts.std() / counts.mean()
+    assert 1.3 < cv < 3.0                                  # heavy tail like the paper's measured 2.13
+    assert abs(4.0 * cfg.R * cfg.H * cfg.I / 1e12 - 1.917) < 1e-3   # the dW1 call: 2*R*M*N
