@@ -186,8 +186,13 @@ int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_ac
  * into the device arena, runs a1..a8, and copies y [T,H], dx [T,H] (bf16) and dtopk_w [T,K]
  * (fp32) back to HOST pointers.  Weights w_* and weight gradients dw_* are DEVICE pointers (the
  * parameters stay resident, as in training).  `arena` is device scratch of at least
- * moe_layer_arena_bytes(dims) bytes holding every intermediate of the step.  Everything is
- * enqueued on `stream`; the host results are valid after the caller synchronises the stream. */
+ * moe_layer_arena_bytes(dims) bytes holding every intermediate of the step.  The kernels and
+ * most copies are enqueued on `stream`; the upload of dy and the download of y run on one internal
+ * copy stream per device (created on the first call, the only CUDA object the library ever
+ * creates) so that they overlap the forward and the backward pass, and are tied to `stream` with
+ * events in both directions: the call behaves as if everything were on `stream`, and the host
+ * results are valid after the caller synchronises it.  Not safe to call from two host threads at
+ * once on the same device. */
 size_t moe_layer_arena_bytes(const moe_dims_t* dims);
 int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int32_t* topk_idx_host,
                            const float* topk_w_host, const void* dy_host, const void* w_gate,

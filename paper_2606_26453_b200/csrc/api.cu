@@ -212,6 +212,27 @@ int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_ac
 
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).
 namespace {
+// One side stream and four events per device for moe_layer_fwd_bwd_host, created on first use and kept for
+// the life of the process (the one place where the library creates CUDA objects of its own).
+struct HostCopyLane {
+    cudaStream_t stream;
+    cudaEvent_t begin, dy_up, y_ready, y_down;
+    bool ready;
+};
+HostCopyLane* host_copy_lane() {
+    static HostCopyLane lanes[64] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostCopyLane& l = lanes[dev];
+    if (!l.ready) {
+        if (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        cudaEvent_t* evs[4] = {&l.begin, &l.dy_up, &l.y_ready, &l.y_down};
+        for (cudaEvent_t* e : evs)
+            if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        l.ready = true;
+    }
+    return &l;
+}
 struct Arena {
     size_t x, idx, w, dy, y, dx, dw, counts, offsets, r2p, p2r, ws, xp, hact, gu, yp, dyp, dhact, dgu, dxp, total;
 };
@@ -257,10 +278,18 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
     auto P = [&](size_t off) { return static_cast<void*>(base + off); };
     auto Pi = [&](size_t off) { return reinterpret_cast<int32_t*>(base + off); };
 
+    // Side stream for the copies that can overlap compute: dy goes up while the forward pass runs, y comes
+    // down while the backward pass runs.  Everything is ordered against the caller's stream with events.
+    HostCopyLane* lane = host_copy_lane();
+    if (lane == nullptr) return MOE_ERR_CUDA;
+    cudaStream_t c = lane->stream;
+    if (cudaEventRecord(lane->begin, s) != cudaSuccess || cudaStreamWaitEvent(c, lane->begin, 0) != cudaSuccess ||
+        cudaMemcpyAsync(P(a.dy), dy_host, T * H * 2, cudaMemcpyHostToDevice, c) != cudaSuccess ||
+        cudaEventRecord(lane->dy_up, c) != cudaSuccess)
+        return MOE_ERR_CUDA;
     if (cudaMemcpyAsync(P(a.x), x_host, T * H * 2, cudaMemcpyHostToDevice, s) != cudaSuccess ||
         cudaMemcpyAsync(P(a.idx), topk_idx_host, R * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(P(a.w), topk_w_host, R * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(P(a.dy), dy_host, T * H * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        cudaMemcpyAsync(P(a.w), topk_w_host, R * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
         return MOE_ERR_CUDA;
 
     int rc;
@@ -270,6 +299,10 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
     MOE_STEP(moe_grouped_gemm_gateup_swiglu(dims, P(a.xp), w_gate, w_up, Pi(a.offsets), P(a.hact), P(a.gu), stream));
     MOE_STEP(moe_grouped_gemm_down(dims, P(a.hact), w_down, Pi(a.offsets), P(a.yp), stream));
     MOE_STEP(moe_unpermute_combine(dims, P(a.yp), reinterpret_cast<float*>(base + a.w), Pi(a.p2r), P(a.y), stream));
+    if (cudaEventRecord(lane->y_ready, s) != cudaSuccess || cudaStreamWaitEvent(c, lane->y_ready, 0) != cudaSuccess ||
+        cudaMemcpyAsync(y_host, P(a.y), T * H * 2, cudaMemcpyDeviceToHost, c) != cudaSuccess ||
+        cudaEventRecord(lane->y_down, c) != cudaSuccess || cudaStreamWaitEvent(s, lane->dy_up, 0) != cudaSuccess)
+        return MOE_ERR_CUDA;
     MOE_STEP(moe_unpermute_combine_bwd(dims, P(a.dy), P(a.yp), reinterpret_cast<float*>(base + a.w), Pi(a.p2r),
                                        P(a.dyp), reinterpret_cast<float*>(base + a.dw), stream));
     MOE_STEP(moe_grouped_gemm_down_bwd(dims, P(a.dyp), P(a.hact), w_down, Pi(a.offsets), P(a.dhact), dw_down, stream));
@@ -278,9 +311,9 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
     MOE_STEP(moe_permute_bwd(dims, P(a.dxp), Pi(a.p2r), P(a.dx), stream));
 #undef MOE_STEP
 
-    if (cudaMemcpyAsync(y_host, P(a.y), T * H * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaMemcpyAsync(dx_host, P(a.dx), T * H * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaMemcpyAsync(dtopk_w_host, P(a.dw), R * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    if (cudaMemcpyAsync(dx_host, P(a.dx), T * H * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(dtopk_w_host, P(a.dw), R * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamWaitEvent(s, lane->y_down, 0) != cudaSuccess)   // the caller's stream also covers the side copies
         return MOE_ERR_CUDA;
     return MOE_OK;
 }
