@@ -187,9 +187,10 @@ int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_ac
  * (fp32) back to HOST pointers.  Weights w_* and weight gradients dw_* are DEVICE pointers (the
  * parameters stay resident, as in training).  `arena` is device scratch of at least
  * moe_layer_arena_bytes(dims) bytes holding every intermediate of the step.  The kernels and
- * most copies are enqueued on `stream`; the upload of dy and the download of y run on one internal
- * copy stream per device (created on the first call, the only CUDA object the library ever
- * creates) so that they overlap the forward and the backward pass, and are tied to `stream` with
+ * most copies are enqueued on `stream`; the upload of dy and the downloads of y, dx and dtopk_w run on
+ * one internal copy stream per device (created on the first call, the only CUDA object the
+ * library ever creates) so that they overlap the forward pass, the backward pass and the last
+ * weight-gradient GEMM, and are tied to `stream` with
  * events in both directions: the call behaves as if everything were on `stream`, and the host
  * results are valid after the caller synchronises it.  Not safe to call from two host threads at
  * once on the same device. */

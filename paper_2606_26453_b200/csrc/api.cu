@@ -212,11 +212,11 @@ int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_ac
 
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).
 namespace {
-// One side stream and four events per device for moe_layer_fwd_bwd_host, created on first use and kept for
+// One side stream and five events per device for moe_layer_fwd_bwd_host, created on first use and kept for
 // the life of the process (the one place where the library creates CUDA objects of its own).
 struct HostCopyLane {
     cudaStream_t stream;
-    cudaEvent_t begin, dy_up, y_ready, y_down;
+    cudaEvent_t begin, dy_up, y_ready, dx_ready, down_done;
     bool ready;
 };
 HostCopyLane* host_copy_lane() {
@@ -226,7 +226,7 @@ HostCopyLane* host_copy_lane() {
     HostCopyLane& l = lanes[dev];
     if (!l.ready) {
         if (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-        cudaEvent_t* evs[4] = {&l.begin, &l.dy_up, &l.y_ready, &l.y_down};
+        cudaEvent_t* evs[5] = {&l.begin, &l.dy_up, &l.y_ready, &l.dx_ready, &l.down_done};
         for (cudaEvent_t* e : evs)
             if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         l.ready = true;
@@ -279,7 +279,7 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
     auto Pi = [&](size_t off) { return reinterpret_cast<int32_t*>(base + off); };
 
     // Side stream for the copies that can overlap compute: dy goes up while the forward pass runs, y comes
-    // down while the backward pass runs.  Everything is ordered against the caller's stream with events.
+    // down while the backward pass runs, dx and dtopk_w come down under the last weight-gradient GEMM.  Everything is ordered against the caller's stream with events.
     HostCopyLane* lane = host_copy_lane();
     if (lane == nullptr) return MOE_ERR_CUDA;
     cudaStream_t c = lane->stream;
@@ -301,20 +301,26 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
     MOE_STEP(moe_unpermute_combine(dims, P(a.yp), reinterpret_cast<float*>(base + a.w), Pi(a.p2r), P(a.y), stream));
     if (cudaEventRecord(lane->y_ready, s) != cudaSuccess || cudaStreamWaitEvent(c, lane->y_ready, 0) != cudaSuccess ||
         cudaMemcpyAsync(y_host, P(a.y), T * H * 2, cudaMemcpyDeviceToHost, c) != cudaSuccess ||
-        cudaEventRecord(lane->y_down, c) != cudaSuccess || cudaStreamWaitEvent(s, lane->dy_up, 0) != cudaSuccess)
+        cudaStreamWaitEvent(s, lane->dy_up, 0) != cudaSuccess)
         return MOE_ERR_CUDA;
     MOE_STEP(moe_unpermute_combine_bwd(dims, P(a.dy), P(a.yp), reinterpret_cast<float*>(base + a.w), Pi(a.p2r),
                                        P(a.dyp), reinterpret_cast<float*>(base + a.dw), stream));
     MOE_STEP(moe_grouped_gemm_down_bwd(dims, P(a.dyp), P(a.hact), w_down, Pi(a.offsets), P(a.dhact), dw_down, stream));
-    MOE_STEP(moe_grouped_gemm_gateup_swiglu_bwd(dims, P(a.dhact), P(a.gu), P(a.xp), w_gate, w_up, Pi(a.offsets),
-                                                P(a.dgu), P(a.dxp), dw_gate, dw_up, stream));
+    // gate/up backward in pieces: dgrad and permute-bwd first, so that dx can travel to the host while the
+    // weight-gradient GEMM (which nothing downstream waits for) is still running
+    MOE_STEP(moe_swiglu_bwd(dims, P(a.dhact), P(a.gu), P(a.dgu), stream));
+    MOE_STEP(moe_grouped_gemm_gateup_dgrad(dims, P(a.dgu), w_gate, w_up, Pi(a.offsets), P(a.dxp), stream));
     MOE_STEP(moe_permute_bwd(dims, P(a.dxp), Pi(a.p2r), P(a.dx), stream));
+    if (cudaEventRecord(lane->dx_ready, s) != cudaSuccess || cudaStreamWaitEvent(c, lane->dx_ready, 0) != cudaSuccess ||
+        cudaMemcpyAsync(dx_host, P(a.dx), T * H * 2, cudaMemcpyDeviceToHost, c) != cudaSuccess ||
+        cudaMemcpyAsync(dtopk_w_host, P(a.dw), R * 4, cudaMemcpyDeviceToHost, c) != cudaSuccess ||
+        cudaEventRecord(lane->down_done, c) != cudaSuccess)
+        return MOE_ERR_CUDA;
+    MOE_STEP(moe_grouped_gemm_gateup_wgrad(dims, P(a.xp), P(a.dgu), Pi(a.offsets), dw_gate, dw_up, stream));
 #undef MOE_STEP
 
-    if (cudaMemcpyAsync(dx_host, P(a.dx), T * H * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaMemcpyAsync(dtopk_w_host, P(a.dw), R * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
-        cudaStreamWaitEvent(s, lane->y_down, 0) != cudaSuccess)   // the caller's stream also covers the side copies
-        return MOE_ERR_CUDA;
+    // the caller's stream also covers the side copies (y, then dx and dtopk_w, in stream order on the side stream)
+    if (cudaStreamWaitEvent(s, lane->down_done, 0) != cudaSuccess) return MOE_ERR_CUDA;
     return MOE_OK;
 }
 
