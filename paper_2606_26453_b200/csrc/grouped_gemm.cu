@@ -641,6 +641,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         uint8_t* stage_ptr = tiles_ptr + G::RING_BYTES + (warp - 2) * (G::STAGING_BLOCKS * STAGING_BLOCK_BYTES);
         const int sw = (lane >> 1) & 3;             // 64-byte swizzle: 16-byte piece j of row r sits at j ^ ((r>>1)&3)
         uint32_t n_stores = 0;                      // bulk stores issued so far by this warp
+        bool drain_first = false;                   // the next staging write must wait for ALL earlier stores
 
         // stage one 32x32 bf16 block (this thread: 16 packed words of its row) and issue its bulk store;
         // with two staging blocks the warp only waits for the store issued two blocks ago
@@ -648,9 +649,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             uint8_t* blk = stage_ptr + (n_stores % G::STAGING_BLOCKS) * STAGING_BLOCK_BYTES;
             if (n_stores >= (uint32_t)G::STAGING_BLOCKS) {
                 if (lane == 0) {
-                    if (G::STAGING_BLOCKS == 2) bulk_wait_read1(); else bulk_wait_read0();
+                    if (G::STAGING_BLOCKS == 2 && !drain_first) bulk_wait_read1(); else bulk_wait_read0();
                 }
                 __syncwarp();
+                drain_first = false;
             }
             uint8_t* my_row = blk + lane * 64;
 #pragma unroll
@@ -722,6 +724,30 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 }
             } else {
                 const bool have_acc = tl.k_blocks > 0;
+                if (!have_acc && rows_valid == 32) {
+                    // expert without rows (WGRAD): a zero tile.  Clear the staging block once and send it to
+                    // all of this warp's 32 x 32 output blocks back to back.
+                    uint8_t* blk = stage_ptr;
+                    if (n_stores != 0) {
+                        if (lane == 0) bulk_wait_read0();
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(blk + lane * 64 + j * 16) = make_uint4(0, 0, 0, 0);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
+                            const int n = tl.n0 + c * 32;
+                            if (n >= p.n_cols) continue;
+                            const bool first = n < p.n_split;
+                            tma_store_2d(first ? &map_o0 : &map_o1, first ? n : n - p.n_split, slab_y, smem_u32(blk));
+                        }
+                        bulk_commit();
+                    }
+                    n_stores += G::STAGING_BLOCKS;   // keeps the block rotation; the next staging write drains first
+                    drain_first = true;
+                } else
 #pragma unroll 1
                 for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
                     uint32_t v[32];
