@@ -748,27 +748,44 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     n_stores += G::STAGING_BLOCKS;   // keeps the block rotation; the next staging write drains first
                     drain_first = true;
                 } else
-#pragma unroll 1
-                for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
-                    uint32_t v[32];
+                {
+                    // software pipeline over the warp's four 32-column blocks: the TMEM load of the next block
+                    // is in flight while the current one is converted, staged and stored
+                    constexpr int NC = BN / 64;
+                    const int c0 = half * NC;
+                    auto emit = [&](const uint32_t (&v)[32], int c) {
+                        const int n = tl.n0 + c * 32;
+                        if (rows_valid == 0 || n >= p.n_cols) return;
+                        uint32_t w[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                        const bool first = n < p.n_split;
+                        const int x = first ? n : n - p.n_split;
+                        if (rows_valid == 32) {
+                            stage_and_store(w, first ? &map_o0 : &map_o1, x, slab_y);
+                        } else if (lane < rows_valid) {
+                            direct_store(w, p.out0 + row * p.ldo + x);     // row-ragged kinds have a single output
+                        }
+                    };
+                    uint32_t va[32], vb[32];
                     if (have_acc) {
-                        tc_ld32(taddr + c * 32, v);
-                        tc_wait_ld();
-                    } else {
+                        tc_ld32(taddr + c0 * 32, va);
+                    } else {   // only reached for a partial zero slab, which cannot occur; kept total
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = 0u;
+                        for (int j = 0; j < 32; ++j) va[j] = vb[j] = 0u;
                     }
-                    const int n = tl.n0 + c * 32;
-                    if (rows_valid == 0 || n >= p.n_cols) continue;
-                    uint32_t w[16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-                    const bool first = n < p.n_split;
-                    const int x = first ? n : n - p.n_split;
-                    if (rows_valid == 32) {
-                        stage_and_store(w, first ? &map_o0 : &map_o1, x, slab_y);
-                    } else if (lane < rows_valid) {
-                        direct_store(w, p.out0 + row * p.ldo + x);     // row-ragged kinds have a single output
+                    for (int i = 0; i < NC; i += 2) {
+                        if (have_acc) {
+                            tc_wait_ld();
+                            tc_ld32(taddr + (c0 + i + 1) * 32, vb);
+                        }
+                        emit(va, c0 + i);
+                        if (have_acc) {
+                            tc_wait_ld();
+                            if (i + 2 < NC) tc_ld32(taddr + (c0 + i + 2) * 32, va);
+                        }
+                        emit(vb, c0 + i + 1);
                     }
                 }
             }
