@@ -313,10 +313,23 @@ def test_host_entry_point_matches_device_chain(B):
     dxh = torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16).pin_memory()
     dwh = torch.empty((cfg.T, cfg.K), dtype=torch.float32).pin_memory()
     dwg, dwu, dwd = torch.empty_like(b.dw_gate), torch.empty_like(b.dw_up), torch.empty_like(b.dw_down)
-    B.moe_layer_fwd_bwd_host(d, xh, ih, wh, dyh, dev["W_gate"], dev["W_up"], dev["W_down"], yh, dxh, dwh, dwg, dwu, dwd, arena)
+    # three calls back to back without host synchronisation in between (the internal copy stream and its
+    # events are reused): the last one must still give the device chain's results
+    for _ in range(3):
+        B.moe_layer_fwd_bwd_host(d, xh, ih, wh, dyh, dev["W_gate"], dev["W_up"], dev["W_down"], yh, dxh, dwh, dwg, dwu, dwd,
+                                 arena)
     torch.cuda.synchronize()
     assert torch.equal(yh, b.y.cpu()) and torch.equal(dxh, b.dx.cpu()) and torch.equal(dwh, b.dtopk_w.cpu())
     assert torch.equal(dwg, b.dw_gate) and torch.equal(dwu, b.dw_up) and torch.equal(dwd, b.dw_down)
+    # different inputs through the same arena: exact scaling by a power of two
+    xh2, dyh2 = (xh.float() * 2).to(torch.bfloat16).pin_memory(), (dyh.float() * 0.5).to(torch.bfloat16).pin_memory()
+    B.moe_layer_fwd_bwd_host(d, xh2, ih, wh, dyh2, dev["W_gate"], dev["W_up"], dev["W_down"], yh, dxh, dwh, dwg, dwu, dwd,
+                             arena)
+    torch.cuda.synchronize()
+    dev2 = dict(dev, X=xh2.cuda(), dY=dyh2.cuda())
+    b2 = Hh.run_cuda_layer(dev2, cfg.E)
+    assert torch.equal(yh, b2.y.cpu()) and torch.equal(dxh, b2.dx.cpu()) and torch.equal(dwh, b2.dtopk_w.cpu())
+    assert torch.equal(dwg, b2.dw_gate) and torch.equal(dwd, b2.dw_down)
 
 
 # ------------------------------------------------------------------------------------------------
