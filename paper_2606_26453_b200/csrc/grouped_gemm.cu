@@ -10,6 +10,9 @@
 //   warps 2..9  epilogue: tcgen05.ld the accumulator (32-lane quarter x half of the columns), apply
 //               the epilogue (plain / SwiGLU), round to bf16, stage 32x32 blocks in swizzled shared
 //               memory and write them with bulk tensor stores
+//   warp 10     (WGRAD only) tail-fix warp: clears the surplus rows of an expert's last K block once its
+//               loads have landed and only then signals the stage as full, so that the MMA warp's issue
+//               loop carries no tail handling
 // The accumulator is double buffered (2 x 256 of the 512 TMEM columns) so the epilogue of one tile
 // overlaps the main loop of the next.
 //
@@ -29,8 +32,9 @@
 //   row-ragged (forward, dgrad): output rows are the packed rows of an expert.  A tile starts at
 //     offsets[e] + TILE_M*i; loading past the expert's last row is harmless, stores are clipped.
 //   contraction-ragged (wgrad; the paper's dW1_e = X_e^T G_e): the expert's rows are the
-//     contraction.  The last K block issues only ceil(rem/16) MMAs and the < 16 surplus rows
-//     are zeroed in shared memory first; an expert without rows gets a zero tile.
+//     contraction.  The last K block issues only ceil(rem/16) MMAs (guard predicates) and the < 16
+//     surplus rows are zeroed in shared memory first, by the tail-fix warp (first CTA) and the relay
+//     warp (second CTA); an expert without rows gets a zero tile.
 //
 // All waits are bounded: a wait that runs out records MOE_ERR_TIMEOUT in the device status word,
 // raises a CTA-wide abort flag and every role leaves through the common teardown.
@@ -62,7 +66,8 @@ constexpr int NUM_EPI_WARPS = 8;
 constexpr int STAGING_BLOCK_BYTES = 32 * 32 * 2;   // one 32 x 32 bf16 output block
 constexpr int MAX_E = 1024;
 constexpr int MAX_STAGES = 6;
-constexpr int NUM_THREADS = 320;   // producer warp, MMA warp, 8 epilogue warps
+constexpr int NUM_THREADS = 352;   // producer warp, MMA warp, 8 epilogue warps, tail-fix warp (WGRAD)
+constexpr int FIX_WARP = 2 + NUM_EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
@@ -89,6 +94,7 @@ struct Params {
 struct SharedCtl {
     unsigned long long full[MAX_STAGES];
     unsigned long long empty[MAX_STAGES];
+    unsigned long long landed[MAX_STAGES];   // WGRAD, MMA-issuing CTA: the stage's loads have arrived (not yet tail-fixed)
     unsigned long long tmem_full[2];
     unsigned long long tmem_empty[2];
     unsigned long long drain;
@@ -96,6 +102,7 @@ struct SharedCtl {
     int abort_flag;
     int32_t offs[MAX_E + 1];
     int32_t tile_prefix[MAX_E + 1];
+    int32_t sorted_rows[MAX_E];   // WGRAD: row count of the expert at each position of the largest-first order
 };
 
 // Ring geometry of the two launch shapes.
@@ -253,6 +260,24 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
         asm volatile(
             "{ .reg .pred p; setp.ne.u32 p, %4, 0; tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
             "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+            : "memory");
+    }
+}
+// same, issued only when `doit` is non-zero (a guard predicate instead of a branch keeps the issue loop straight-line)
+template <bool PAIR>
+__device__ __forceinline__ void tc_mma_if(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate, uint32_t doit) {
+    if (PAIR) {
+        asm volatile(
+            "{ .reg .pred p, q; setp.ne.u32 p, %4, 0; setp.ne.u32 q, %5, 0;"
+            " @q tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
+            "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(doit)
+            : "memory");
+    } else {
+        asm volatile(
+            "{ .reg .pred p, q; setp.ne.u32 p, %4, 0; setp.ne.u32 q, %5, 0;"
+            " @q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }" ::"r"(d_tmem),
+            "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(doit)
             : "memory");
     }
 }
@@ -455,14 +480,18 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const long long first_tile = PAIR ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
     const long long tile_stride = PAIR ? (long long)(gridDim.x >> 1) : (long long)gridDim.x;
     const int my_rows = rank * BM;                                 // this CTA's row offset inside the tile
+    // WGRAD, MMA-issuing CTA: loads complete on landed[]; the tail-fix warp clears surplus contraction rows
+    // and only then arrives on full[], so the MMA warp's loop has no tail branch at all
+    const bool local_fix = (KIND == WGRAD) && rank == 0;
 
     // ---- set-up: barriers, schedule tables, TMEM ----
     for (int e = threadIdx.x; e <= p.E; e += NUM_THREADS) ctl->offs[e] = p.offsets[e];
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            // pair mode, first CTA: own producer's arrive + the relay's remote arrive
+            // pair mode, first CTA: own producer's (WGRAD: own tail-fix warp's) arrive + the relay's remote arrive
             mbar_init(smem_u32(&ctl->full[s]), (PAIR && rank == 0) ? 2 : 1);
             mbar_init(smem_u32(&ctl->empty[s]), 1);
+            mbar_init(smem_u32(&ctl->landed[s]), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
@@ -488,6 +517,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 rank += (n_f > n_e || (n_f == n_e && f < e)) ? 1 : 0;
             }
             ctl->tile_prefix[rank] = e;
+            ctl->sorted_rows[rank] = n_e;
         }
     } else if (threadIdx.x == 0) {
         int run = 0;
@@ -529,10 +559,10 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
                 for (int kb = 0; kb < tl.k_blocks; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t full = smem_u32(&ctl->full[stage]);
-                    mbar_arrive_expect_tx(full, STAGE_BYTES);
+                    const uint32_t land = smem_u32(local_fix ? &ctl->landed[stage] : &ctl->full[stage]);
+                    mbar_arrive_expect_tx(land, STAGE_BYTES);
                     const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
-                    stage_loads<KIND, PAIR>(tl, kb, p, &map_a, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES, full, rank, my_rows);
+                    stage_loads<KIND, PAIR>(tl, kb, p, &map_a, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES, land, rank, my_rows);
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -543,61 +573,75 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 uint32_t s = stage, ph = phase;
                 for (uint32_t i = 0; i < n_wait; ++i) {
                     if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
-                    if (PAIR && rank == 0) continue;   // completion there also needs the relay; the copies were bounded by it
+                    if (PAIR && rank == 0 && !local_fix) continue;   // completion there also needs the relay; the copies were bounded by it
                     const unsigned long long t0 = global_timer_ns();
-                    while (!mbar_try_wait(smem_u32(&ctl->full[s]), ph) && global_timer_ns() - t0 < WAIT_LIMIT_NS / 4) {}
+                    const uint32_t land = smem_u32(local_fix ? &ctl->landed[s] : &ctl->full[s]);
+                    while (!mbar_try_wait(land, ph) && global_timer_ns() - t0 < WAIT_LIMIT_NS / 4) {}
                 }
             }
         }
     } else if (warp == 1 && rank == 0) {
-        // ================= MMA issuer (first CTA of a pair) =================
-        uint32_t stage = 0, phase = 0;
-        uint32_t acc = 0, acc_phase = 0;
-        bool ok = true;
-        for (long long it = 0; ok; ++it) {
-            const long long t = tile_of<KIND>(it, first_tile, tile_stride, n_tiles_total);
-            if (t < 0) break;
-            const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
-            if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + acc * BN;
-            for (int kb = 0; kb < tl.k_blocks; ++kb) {
-                if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
-                const uint32_t b_base = a_base + G::A_BYTES;
-                int n_mma = BK / 16;
+        // ================= MMA issuer (first CTA of a pair): one thread =================
+        // Measured on this part: the issuing thread spends ~85 cycles on each tcgen05.mma and the tensor pipe
+        // queues about two of them, so per 64-wide K block (4 MMAs, 512 pipe cycles) the thread has only
+        // ~170 cycles for everything else before the pipe runs dry.  The role is therefore a single thread (no
+        // warp synchronisation, no divergence), its loop holds nothing but wait / MMAs / commit, the ragged
+        // last block of a WGRAD tile is peeled out of the loop, and the per-tile bookkeeping is reduced to an
+        // incrementally advanced position in the expert order plus one shared-memory load.
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            uint32_t acc = 0, acc_phase = 0;
+            bool ok = true;
+            const long long per_e = (long long)p.m_tiles * p.n_tiles;   // WGRAD: tiles per expert
+            int e_pos = 0;                                              // WGRAD: position in the largest-first order
+            long long e_end = per_e;
+            for (long long it = 0; ok; ++it) {
+                const long long t = tile_of<KIND>(it, first_tile, tile_stride, n_tiles_total);
+                if (t < 0) break;
+                int n_full = p.k_blocks, n_tail = 0;   // whole K blocks; MMAs of the ragged last block
                 if (KIND == WGRAD) {
-                    const int rem = tl.k_rows - kb * BK;
-                    if (rem < BK) {
-                        n_mma = (rem + 15) >> 4;
-                        if (n_mma * 16 > rem) zero_k_rows(tiles_ptr + stage * STAGE_BYTES, STAGE_CHUNKS, rem, n_mma * 16, lane);
-                        __syncwarp();
-                    }
+                    while (t >= e_end) { ++e_pos; e_end += per_e; }   // tile ids of one CTA only grow
+                    const int k_rows = ctl->sorted_rows[e_pos];
+                    n_full = k_rows >> 6;
+                    n_tail = ((k_rows & (BK - 1)) + 15) >> 4;
                 }
-                if (lane == 0) {
+                if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < n_full; ++kb) {
+                    if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
                     const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
-                    const uint64_t b_desc = make_smem_desc<B_MN>(b_base);
-                    if (n_mma == BK / 16) {   // full block: fully unrolled issue (a runtime trip count costs ~15 % here)
+                    const uint64_t b_desc = make_smem_desc<B_MN>(a_base + G::A_BYTES);
 #pragma unroll
-                        for (int kk = 0; kk < BK / 16; ++kk)
-                            tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
-                                         b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, (kb | kk) != 0 ? 1u : 0u);
-                    } else {
-                        for (int kk = 0; kk < n_mma; ++kk)
-                            tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
-                                         b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, (kb | kk) != 0 ? 1u : 0u);
-                    }
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
+                                     b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, (kb | kk) != 0 ? 1u : 0u);
                     tc_commit<PAIR>(smem_u32(&ctl->empty[stage]));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                if (!ok) break;
+                if (KIND == WGRAD && n_tail != 0) {
+                    // ragged last block: ceil(rem/16) MMAs; its surplus rows were cleared before full[] was signalled
+                    if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
+                    const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
+                    const uint64_t b_desc = make_smem_desc<B_MN>(a_base + G::A_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; ++kk)
+                        tc_mma_if<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
+                                        b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, (n_full | kk) != 0 ? 1u : 0u,
+                                        kk < n_tail ? 1u : 0u);
+                    tc_commit<PAIR>(smem_u32(&ctl->empty[stage]));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                tc_commit<PAIR>(smem_u32(&ctl->tmem_full[acc]));
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
             }
-            if (!ok) break;
-            if (lane == 0) tc_commit<PAIR>(smem_u32(&ctl->tmem_full[acc]));
-            __syncwarp();
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
+        __syncwarp();
         // all issued MMAs must have retired before tensor memory is released
         if (lane == 0) {
             tc_commit_local<PAIR>(smem_u32(&ctl->drain));
@@ -605,10 +649,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ================= relay (second CTA of a pair) =================
+    } else if (warp == 1 || (warp == FIX_WARP && local_fix)) {
+        // ================= relay (second CTA of a pair) / tail-fix warp (WGRAD, MMA-issuing CTA) =================
         // Waits until this CTA's loads of a stage have landed, clears the surplus contraction rows
-        // (WGRAD) and then tells the first CTA's barrier that this half of the stage is ready.
+        // (WGRAD) and then tells the first CTA's full[] barrier that this CTA's part of the stage is ready:
+        // with a remote arrive from the second CTA, with a local one in the first.
+        const bool remote = rank != 0;
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         for (long long it = 0; ok; ++it) {
@@ -616,7 +662,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (t < 0) break;
             const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
             for (int kb = 0; kb < tl.k_blocks; ++kb) {
-                if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+                const uint32_t land = smem_u32(remote ? &ctl->full[stage] : &ctl->landed[stage]);
+                if (!mbar_wait(land, phase, abort_flag)) { ok = false; break; }
                 if (KIND == WGRAD) {
                     const int rem = tl.k_rows - kb * BK;
                     if (rem < BK) {
@@ -625,11 +672,14 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     }
                 }
                 __syncwarp();
-                if (lane == 0) mbar_arrive_remote(map_to_cta(smem_u32(&ctl->full[stage]), 0));
+                if (lane == 0) {
+                    if (remote) mbar_arrive_remote(map_to_cta(smem_u32(&ctl->full[stage]), 0));
+                    else mbar_arrive(smem_u32(&ctl->full[stage]));
+                }
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-    } else {
+    } else if (warp < FIX_WARP) {
         // ================= epilogue (warps 2..9) =================
         // Each warp owns a 32-row slab (its TMEM lane quarter) and half of the tile's columns.  A
         // 32 x 32 block is rounded to bf16, written to the warp's 2 KB staging buffer in the 64-byte
