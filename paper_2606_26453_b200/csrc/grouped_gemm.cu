@@ -174,6 +174,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return done != 0;
 }
+// non-blocking test of a barrier phase (acquire on success)
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
 __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -584,10 +594,13 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // ================= MMA issuer (first CTA of a pair): one thread =================
         // Measured on this part: the issuing thread spends ~85 cycles on each tcgen05.mma and the tensor pipe
         // queues about two of them, so per 64-wide K block (4 MMAs, 512 pipe cycles) the thread has only
-        // ~170 cycles for everything else before the pipe runs dry.  The role is therefore a single thread (no
-        // warp synchronisation, no divergence), its loop holds nothing but wait / MMAs / commit, the ragged
-        // last block of a WGRAD tile is peeled out of the loop, and the per-tile bookkeeping is reduced to an
-        // incrementally advanced position in the expert order plus one shared-memory load.
+        // ~170 cycles for everything else before the pipe runs dry; shared-memory loads and barrier polls
+        // take 100+ cycles each here because TMA fills and operand reads keep the shared-memory pipe busy.
+        // The role is therefore a single thread (no warp synchronisation, no divergence) whose loop holds
+        // nothing but wait / MMAs / commit.  Per tile: the id and row count of the NEXT tile are fetched
+        // before the K loop (the load's latency passes under the MMAs), the last block is peeled out of the
+        // loop (guard predicates for the ragged last block of a WGRAD tile), and whether the next accumulator
+        // buffer is free is tested, without blocking, just before that last block.
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             uint32_t acc = 0, acc_phase = 0;
@@ -595,50 +608,60 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const long long per_e = (long long)p.m_tiles * p.n_tiles;   // WGRAD: tiles per expert
             int e_pos = 0;                                              // WGRAD: position in the largest-first order
             long long e_end = per_e;
-            for (long long it = 0; ok; ++it) {
-                const long long t = tile_of<KIND>(it, first_tile, tile_stride, n_tiles_total);
-                if (t < 0) break;
-                int n_full = p.k_blocks, n_tail = 0;   // whole K blocks; MMAs of the ragged last block
-                if (KIND == WGRAD) {
-                    while (t >= e_end) { ++e_pos; e_end += per_e; }   // tile ids of one CTA only grow
-                    const int k_rows = ctl->sorted_rows[e_pos];
-                    n_full = k_rows >> 6;
-                    n_tail = ((k_rows & (BK - 1)) + 15) >> 4;
+            auto rows_of = [&](long long tile) -> int {                 // WGRAD; tile ids of one CTA only grow
+                while (tile >= e_end) { ++e_pos; e_end += per_e; }
+                return ctl->sorted_rows[e_pos];
+            };
+            // one K block: n_mma MMAs from ring stage `stage`, then the stage is released
+            auto issue_block = [&](uint32_t d_tmem, bool first_block, int n_mma, bool partial) -> bool {
+                if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
+                const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
+                const uint64_t b_desc = make_smem_desc<B_MN>(a_base + G::A_BYTES);
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; ++kk) {
+                    const uint32_t accumulate = (!first_block || kk != 0) ? 1u : 0u;
+                    if (partial)
+                        tc_mma_if<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
+                                        b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, accumulate, kk < n_mma ? 1u : 0u);
+                    else
+                        tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
+                                     b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, accumulate);
                 }
-                if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_commit<PAIR>(smem_u32(&ctl->empty[stage]));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                return true;
+            };
+            long long t = tile_of<KIND>(0, first_tile, tile_stride, n_tiles_total);
+            int k_rows = (KIND == WGRAD && t >= 0) ? rows_of(t) : 0;
+            bool acc_free = false;   // the accumulator buffer of the current tile is already known to be free
+            for (long long it = 0; ok && t >= 0; ++it) {
+                const long long t_next = tile_of<KIND>(it + 1, first_tile, tile_stride, n_tiles_total);
+                const int k_rows_next = (KIND == WGRAD && t_next >= 0) ? rows_of(t_next) : 0;
+                // whole K blocks, and MMAs of the ragged last block (WGRAD; its surplus rows were cleared
+                // before full[] was signalled)
+                const int n_full = (KIND == WGRAD) ? (k_rows >> 6) : p.k_blocks;
+                const int n_tail = (KIND == WGRAD) ? (((k_rows & (BK - 1)) + 15) >> 4) : 0;
+                if (!acc_free && !mbar_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < n_full; ++kb) {
-                    if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
-                    const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
-                    const uint64_t b_desc = make_smem_desc<B_MN>(a_base + G::A_BYTES);
-#pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
-                                     b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, (kb | kk) != 0 ? 1u : 0u);
-                    tc_commit<PAIR>(smem_u32(&ctl->empty[stage]));
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
+                const int n_main = n_tail != 0 ? n_full : n_full - 1;   // blocks before the peeled last one
+                for (int kb = 0; kb < n_main; ++kb)
+                    if (!issue_block(d_tmem, kb == 0, BK / 16, false)) { ok = false; break; }
                 if (!ok) break;
-                if (KIND == WGRAD && n_tail != 0) {
-                    // ragged last block: ceil(rem/16) MMAs; its surplus rows were cleared before full[] was signalled
-                    if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
-                    const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
-                    const uint64_t b_desc = make_smem_desc<B_MN>(a_base + G::A_BYTES);
-#pragma unroll
-                    for (int kk = 0; kk < BK / 16; ++kk)
-                        tc_mma_if<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
-                                        b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, (n_full | kk) != 0 ? 1u : 0u,
-                                        kk < n_tail ? 1u : 0u);
-                    tc_commit<PAIR>(smem_u32(&ctl->empty[stage]));
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                // the next tile's accumulator buffer was handed to the epilogue one tile ago: usually free by now
+                const uint32_t acc_n = acc ^ 1u, acc_phase_n = acc_phase ^ acc;
+                acc_free = mbar_test_wait(smem_u32(&ctl->tmem_empty[acc_n]), acc_phase_n ^ 1u);
+                if (n_main >= 0) {
+                    if (n_tail != 0) { if (!issue_block(d_tmem, n_main == 0, n_tail, true)) { ok = false; break; } }
+                    else             { if (!issue_block(d_tmem, n_main == 0, BK / 16, false)) { ok = false; break; } }
                 }
                 tc_commit<PAIR>(smem_u32(&ctl->tmem_full[acc]));
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+                acc = acc_n;
+                acc_phase = acc_phase_n;
+                t = t_next;
+                k_rows = k_rows_next;
             }
         }
         __syncwarp();
