@@ -27,7 +27,8 @@ What each step follows:
 Pins (tests/test_oracle_*.py): brute-force counting sort, stable-sort library routine, dense
 SwiGLU MLP special cases evaluated with an independent library (torch, fp64), per-token loop,
 torch.autograd on a per-token formulation, central finite differences, identities of
-permute/unpermute, empty-expert zeros.  No function here is "parity unpinned".
+permute/unpermute, empty-expert zeros; for the router: a per-row selection loop, a library softmax,
+shift invariance, the all-ties closed form, finite differences.  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -244,3 +245,37 @@ def layer_fwd_bwd(X, topk_idx, topk_w, W_gate, W_up, W_down, dY):
     f.update(dY_perm=dYp, dtopk_w=dw, dH_act=dHact, dW_down=dWd, dGU=dGU, dX_perm=dXp,
              dW_gate=dWg, dW_up=dWu, dX=dX)
     return f
+
+
+# ---- router in front of the layer (the step before route-permute) ------------------------------
+def router_topk(logits, K):
+    """Top-k routing as the spec workloads describe it: softmax over the router logits, the K
+    largest per token kept and renormalised to sum 1.
+
+    logits [T,E] float32.  Selection is decided on the float32 values as given: the K largest per
+    row in descending order, equal values ordered by lower expert id (the comparison of two float32
+    numbers is exact in any precision).  Renormalising softmax(z) over the selected set cancels the
+    full denominator, so  w_k = exp(z_k) / sum_{j selected} exp(z_j),  evaluated in fp64 with the
+    row maximum subtracted.  Returns topk_idx [T,K] int32, topk_w [T,K] float64.  Logits must be finite."""
+    z32 = np.asarray(logits, dtype=np.float32)
+    T, E = z32.shape
+    assert 1 <= K <= E
+    z = z32.astype(F64)
+    ids = np.broadcast_to(np.arange(E), (T, E))
+    order = np.lexsort((ids, -z), axis=1)          # primary key: value descending; secondary: id ascending
+    idx = order[:, :K]
+    zs = np.take_along_axis(z, idx, axis=1)
+    ex = np.exp(zs - zs[:, :1])
+    return idx.astype(np.int32), ex / ex.sum(axis=1, keepdims=True)
+
+
+def router_topk_bwd(topk_idx, topk_w, dtopk_w, E):
+    """Gradient of the renormalised top-k weights with respect to the logits, selection frozen:
+    dz[t, idx[t,k]] = w_k * (dw_k - sum_j w_j dw_j); zero for experts that were not selected."""
+    idx = np.asarray(topk_idx).astype(np.int64)
+    w, dw = _f64(topk_w), _f64(dtopk_w)
+    T, K = idx.shape
+    inner = (w * dw).sum(axis=1, keepdims=True)
+    dz = np.zeros((T, E), dtype=F64)
+    np.put_along_axis(dz, idx, w * (dw - inner), axis=1)
+    return dz

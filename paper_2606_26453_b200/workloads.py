@@ -117,6 +117,18 @@ def make_routing(cfg: MoeConfig, seed: int = 0):
     return idx.astype(np.int32), round_to_bf16(w.astype(np.float32))
 
 
+def make_router_logits(cfg: MoeConfig, seed: int = 0):
+    """Router logits [T,E] float32 for the "softmax" / "skew" workloads: the float32 image of the
+    values make_routing draws.  An input for the router entry points only: selection and weights are
+    the business of the code under test (and of the oracle), not of this module."""
+    if cfg.routing not in ("softmax", "skew"):
+        raise ValueError("router logits are defined for the softmax / skew routings only")
+    z = _rng(seed, cfg.cfg_id, 5).standard_normal((cfg.T, cfg.E))
+    if cfg.routing == "skew":
+        z = z + 0.5 * _rng(seed, cfg.cfg_id, 6).standard_normal(cfg.E)[None, :]
+    return z.astype(np.float32)
+
+
 def make_routing_from_counts(counts, K: int, seed: int = 0):
     """A routing with prescribed per-expert row counts (sum must be a multiple of K, and no
     count may exceed the number of tokens): used for adversarial load tests (empty experts at the

@@ -345,3 +345,96 @@ def test_down_bwd_einsum():
     np.testing.assert_allclose(dHact, np.einsum("rh,rih->ri", dYp, Wd[e_of_row]), rtol=1e-12, atol=1e-12)
     onehot = (e_of_row[:, None] == np.arange(E)[None, :]).astype(np.float64)
     np.testing.assert_allclose(dWd, np.einsum("re,ri,rh->eih", onehot, Hact, dYp), rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------------------------------------
+# router (softmax, top-k, renormalise) and its backward
+# ------------------------------------------------------------------------------------------
+def _router_loop(z32, K):
+    """Per-row selection by repeated arg-max with the tie rule, weights by the textbook formula."""
+    T, E = z32.shape
+    idx = np.zeros((T, K), dtype=np.int32)
+    w = np.zeros((T, K))
+    for t in range(T):
+        taken = set()
+        for k in range(K):
+            best = None
+            for e in range(E):
+                if e in taken:
+                    continue
+                if best is None or z32[t, e] > z32[t, best]:
+                    best = e
+            taken.add(best)
+            idx[t, k] = best
+        p = np.exp(z32[t].astype(np.float64))
+        p /= p.sum()                                  # full softmax ...
+        w[t] = p[idx[t]] / p[idx[t]].sum()            # ... renormalised over the kept experts
+    return idx, w
+
+
+@pytest.mark.parametrize("T,E,K,seed", [(17, 8, 2, 0), (9, 33, 5, 1), (5, 4, 4, 2), (11, 64, 1, 3)])
+def test_router_matches_selection_loop(T, E, K, seed):
+    z = np.random.default_rng(seed).standard_normal((T, E)).astype(np.float32)
+    z[0, :] = np.round(z[0, :])                        # a row with many exact ties
+    idx, w = O.router_topk(z, K)
+    ridx, rw = _router_loop(z, K)
+    assert np.array_equal(idx, ridx)
+    np.testing.assert_allclose(w, rw, rtol=1e-12, atol=0)
+    np.testing.assert_allclose(w.sum(axis=1), 1.0, rtol=1e-14)
+
+
+def test_router_full_k_is_library_softmax_and_ties_closed_form():
+    from scipy.special import softmax
+    z = np.random.default_rng(4).standard_normal((13, 12)).astype(np.float32)
+    idx, w = O.router_topk(z, 12)
+    full = softmax(z.astype(np.float64), axis=1)
+    np.testing.assert_allclose(w, np.take_along_axis(full, idx.astype(np.int64), axis=1), rtol=1e-12)
+    assert np.all(np.diff(np.take_along_axis(z, idx.astype(np.int64), axis=1), axis=1) <= 0)
+    # all logits equal: the first K experts in id order, equal weights
+    idx, w = O.router_topk(np.full((3, 10), 0.25, dtype=np.float32), 4)
+    assert np.array_equal(idx, np.tile(np.arange(4, dtype=np.int32), (3, 1)))
+    np.testing.assert_allclose(w, 0.25, rtol=1e-15)
+
+
+def test_router_shift_invariance_and_generator_agreement():
+    rng = np.random.default_rng(5)
+    z = rng.integers(-8, 9, size=(20, 16)).astype(np.float32)       # shifts stay exact in float32
+    i0, w0 = O.router_topk(z, 3)
+    i1, w1 = O.router_topk(z + np.float32(5.0), 3)
+    assert np.array_equal(i0, i1)
+    np.testing.assert_allclose(w0, w1, rtol=1e-12)
+    # the workload generator's own routing (written separately) from the same logits
+    cfg = W.CONFIGS["tiny"]
+    gen_idx, gen_w = W.make_routing(cfg)
+    idx, w = O.router_topk(W.make_router_logits(cfg), cfg.K)
+    assert np.array_equal(idx, gen_idx)
+    np.testing.assert_allclose(w, gen_w, rtol=2.0 ** -8)          # the generator rounds its weights to bf16
+
+
+def test_router_bwd_matches_finite_differences():
+    rng = np.random.default_rng(6)
+    T, E, K = 6, 9, 4
+    z = rng.standard_normal((T, E)).astype(np.float32)
+    c = rng.standard_normal((T, K))
+    idx, w = O.router_topk(z, K)
+    dz = O.router_topk_bwd(idx, w, c, E)
+
+    def f(zz):                                       # selection frozen: weights of the same experts
+        zs = np.take_along_axis(zz, idx.astype(np.int64), axis=1)
+        ex = np.exp(zs - zs.max(axis=1, keepdims=True))
+        return float((c * ex / ex.sum(axis=1, keepdims=True)).sum())
+
+    z64 = z.astype(np.float64)
+    num = np.zeros_like(z64)
+    h = 1e-6
+    for t in range(T):
+        for e in range(E):
+            zp, zm = z64.copy(), z64.copy()
+            zp[t, e] += h
+            zm[t, e] -= h
+            num[t, e] = (f(zp) - f(zm)) / (2 * h)
+    np.testing.assert_allclose(dz, num, rtol=1e-6, atol=1e-9)
+    np.testing.assert_allclose(dz.sum(axis=1), 0.0, atol=1e-14)
+    unselected = np.ones((T, E), dtype=bool)
+    np.put_along_axis(unselected, idx.astype(np.int64), False, axis=1)
+    assert np.all(dz[unselected] == 0.0)
