@@ -201,6 +201,36 @@ def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True):
     return dict(wl=wl, buffers=b, total_ms=total_ms, per_call_ms=per_call, clocks=clocks)
 
 
+def time_router(B, cfg, device, reps=30):
+    """The router in front of the layer (outside the step the headline metric times): logits of the workload's own
+    draw -> top-k indices and weights, and the backward to the logits.  Timed alone with CUDA events after
+    3 warm-ups; the logits of the benchmark workloads are a few MB, so this measures launch plus a few microseconds."""
+    if cfg.routing not in ("softmax", "skew"):
+        return None
+    z = torch.from_numpy(W.make_router_logits(cfg)).to(device)
+    d = B.dims(cfg.T, cfg.H, cfg.I, cfg.E, cfg.K)
+    idx = torch.empty((cfg.T, cfg.K), dtype=torch.int32, device=device)
+    w = torch.empty((cfg.T, cfg.K), dtype=torch.float32, device=device)
+    dw = torch.randn((cfg.T, cfg.K), dtype=torch.float32, device=device)
+    dz = torch.empty_like(z)
+    out = {}
+    for name, fn in (("fwd", lambda: B.moe_router_topk(d, z, idx, w)), ("bwd", lambda: B.moe_router_topk_bwd(d, idx, w, dw, dz))):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name + "_ms"] = e0.elapsed_time(e1) / reps
+    nbytes = cfg.T * cfg.E * 4 + cfg.T * cfg.K * 8
+    out["fwd_gbs"] = nbytes / (out["fwd_ms"] * 1e-3) / 1e9
+    out["bwd_gbs"] = (cfg.T * cfg.E * 4 + cfg.T * cfg.K * 12) / (out["bwd_ms"] * 1e-3) / 1e9
+    out["note"] = "back-to-back launches, inputs L2-resident at these sizes"
+    return out
+
+
 def summarize(cfg, res, steps, peaks):
     ms_step = res["total_ms"] / steps
     pc = res["per_call_ms"]
@@ -452,6 +482,9 @@ def run_ours(args):
             torch.cuda.empty_cache()
         if extra:
             line["other_configs"] = extra
+        router = time_router(B, cfg, device)
+        if router is not None:
+            line["router"] = router
         line["stream_calibration"] = stream_calibration(device)
         if wl_host is not None:
             line["cpu_baseline"] = cpu_baseline(cfg, wl_host, min(args.ref_tokens, cfg.T))

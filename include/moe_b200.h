@@ -180,6 +180,23 @@ int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_ac
                                        const int32_t* offsets, void* dgu, void* dx_perm,
                                        void* dw_gate, void* dw_up, moe_stream_t stream);
 
+/* ---- router in front of a1 ---------------------------------------------------------------------
+ * The step that produces a1's routing inputs; the north-star workloads describe it as "softmax
+ * over router logits, top-k renormalised" (the paper itself has no counterpart: its kernel starts
+ * from the packed buffer).  Uses dims->T, E, K.
+ * moe_router_topk      logits [T,E] fp32 (device, no NaN).  Per token the K largest logits, slots in
+ *                      descending order, equal values ordered by lower expert id, decided on the
+ *                      fp32 values as given -> topk_idx [T,K] int32.  topk_w [T,K] fp32 =
+ *                      exp(z_k) / sum over the kept j of exp(z_j), i.e. softmax(z) renormalised over
+ *                      the kept experts (fp32 arithmetic, row maximum subtracted).
+ * moe_router_topk_bwd  selection frozen: dlogits[t, topk_idx[t,k]] = w_k (dw_k - sum_j w_j dw_j),
+ *                      zero for the other experts; dlogits [T,E] fp32 is written in full.
+ * All pointers device, 16-byte aligned, caller-owned; status codes as everywhere else. */
+int moe_router_topk(const moe_dims_t* dims, const float* logits, int32_t* topk_idx, float* topk_w,
+                    moe_stream_t stream);
+int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const float* topk_w,
+                        const float* dtopk_w, float* dlogits, moe_stream_t stream);
+
 /* ---- whole layer from HOST activations ------------------------------------------------------
  * One training step of the layer for a caller whose per-step tensors live in host memory:
  * copies x, topk_idx, topk_w, dy (HOST pointers; pinned memory makes the copies asynchronous)

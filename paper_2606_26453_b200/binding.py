@@ -22,7 +22,7 @@ EXPORTS = [
     "moe_unpermute_combine_bwd", "moe_grouped_gemm_down_dgrad", "moe_grouped_gemm_down_wgrad",
     "moe_grouped_gemm_down_bwd", "moe_swiglu_bwd", "moe_grouped_gemm_gateup_dgrad",
     "moe_grouped_gemm_gateup_wgrad", "moe_grouped_gemm_gateup_swiglu_bwd", "moe_layer_arena_bytes",
-    "moe_layer_fwd_bwd_host",
+    "moe_layer_fwd_bwd_host", "moe_router_topk", "moe_router_topk_bwd",
 ]
 
 
@@ -69,6 +69,8 @@ def load_library() -> ctypes.CDLL:
             "moe_grouped_gemm_down_wgrad": [dp, p, p, p, p, p],
             "moe_grouped_gemm_down_bwd": [dp, p, p, p, p, p, p, p],
             "moe_swiglu_bwd": [dp, p, p, p, p],
+            "moe_router_topk": [dp, p, p, p, p],
+            "moe_router_topk_bwd": [dp, p, p, p, p, p],
             "moe_grouped_gemm_gateup_dgrad": [dp, p, p, p, p, p, p],
             "moe_grouped_gemm_gateup_wgrad": [dp, p, p, p, p, p, p],
             "moe_grouped_gemm_gateup_swiglu_bwd": [dp, p, p, p, p, p, p, p, p, p, p, p],
@@ -174,6 +176,14 @@ def moe_grouped_gemm_down_wgrad(d, h_act, dy_perm, offsets, dw_down):
 def moe_grouped_gemm_down_bwd(d, dy_perm, h_act, w_down, offsets, dh_act, dw_down):
     _call("moe_grouped_gemm_down_bwd", ctypes.byref(d), _ptr(dy_perm), _ptr(h_act), _ptr(w_down), _ptr(offsets),
           _ptr(dh_act), _ptr(dw_down), _stream())
+
+
+def moe_router_topk(d, logits, topk_idx, topk_w):
+    _call("moe_router_topk", ctypes.byref(d), _ptr(logits), _ptr(topk_idx), _ptr(topk_w), _stream())
+
+
+def moe_router_topk_bwd(d, topk_idx, topk_w, dtopk_w, dlogits):
+    _call("moe_router_topk_bwd", ctypes.byref(d), _ptr(topk_idx), _ptr(topk_w), _ptr(dtopk_w), _ptr(dlogits), _stream())
 
 
 def moe_swiglu_bwd(d, dh_act, gu_saved, dgu):

@@ -8,7 +8,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libmoe_b200.so")
-SOURCES = ["api.cu", "movement.cu", "grouped_gemm.cu"]
+SOURCES = ["api.cu", "movement.cu", "router.cu", "grouped_gemm.cu"]
 HEADERS = ["common.cuh", os.path.join("..", "..", "include", "moe_b200.h")]
 
 

@@ -210,6 +210,22 @@ int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_ac
     return moe_grouped_gemm_gateup_wgrad(dims, x_perm, dgu, offsets, dw_gate, dw_up, stream);
 }
 
+int moe_router_topk(const moe_dims_t* dims, const float* logits, int32_t* topk_idx, float* topk_w,
+                    moe_stream_t stream) {
+    const void* const req[] = {logits, topk_idx, topk_w};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_router_topk(*dims, logits, topk_idx, topk_w, st(stream));
+}
+
+int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const float* topk_w, const float* dtopk_w,
+                        float* dlogits, moe_stream_t stream) {
+    const void* const req[] = {topk_idx, topk_w, dtopk_w, dlogits};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_router_topk_bwd(*dims, topk_idx, topk_w, dtopk_w, dlogits, st(stream));
+}
+
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).
 namespace {
 // One side stream and five events per device for moe_layer_fwd_bwd_host, created on first use and kept for

@@ -35,6 +35,11 @@ int launch_combine_bwd(const moe_dims_t& d, const bf16* dy, const bf16* y_perm, 
                        const int32_t* pair_to_row, bf16* dy_perm, float* dtopk_w, cudaStream_t s);
 int launch_swiglu_bwd(const moe_dims_t& d, const bf16* dh_act, const bf16* gu, bf16* dgu, cudaStream_t s);
 
+// ---- router (router.cu) ------------------------------------------------------------------------
+int launch_router_topk(const moe_dims_t& d, const float* logits, int32_t* topk_idx, float* topk_w, cudaStream_t s);
+int launch_router_topk_bwd(const moe_dims_t& d, const int32_t* topk_idx, const float* topk_w, const float* dtopk_w,
+                           float* dlogits, cudaStream_t s);
+
 // ---- grouped GEMMs (grouped_gemm.cu) -----------------------------------------------------------
 int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gate, const bf16* w_up,
                       const int32_t* offsets, bf16* h_act, bf16* gu, cudaStream_t s);
