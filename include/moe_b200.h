@@ -206,8 +206,8 @@ int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const f
  * moe_layer_arena_bytes(dims) bytes holding every intermediate of the step.  The kernels and
  * most copies are enqueued on `stream`; the upload of dy and the downloads of y, dx and dtopk_w run on
  * one internal copy stream per device (created on the first call, the only CUDA object the
- * library ever creates) so that they overlap the forward pass, the backward pass and the last
- * weight-gradient GEMM, and are tied to `stream` with
+ * library ever creates) so that they overlap the forward pass, the backward pass and the two
+ * weight-gradient GEMMs (which run last: nothing downstream waits for them), and are tied to `stream` with
  * events in both directions: the call behaves as if everything were on `stream`, and the host
  * results are valid after the caller synchronises it.  Not safe to call from two host threads at
  * once on the same device. */

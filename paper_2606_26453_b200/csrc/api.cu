@@ -321,9 +321,9 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
         return MOE_ERR_CUDA;
     MOE_STEP(moe_unpermute_combine_bwd(dims, P(a.dy), P(a.yp), reinterpret_cast<float*>(base + a.w), Pi(a.p2r),
                                        P(a.dyp), reinterpret_cast<float*>(base + a.dw), stream));
-    MOE_STEP(moe_grouped_gemm_down_bwd(dims, P(a.dyp), P(a.hact), w_down, Pi(a.offsets), P(a.dhact), dw_down, stream));
-    // gate/up backward in pieces: dgrad and permute-bwd first, so that dx can travel to the host while the
-    // weight-gradient GEMM (which nothing downstream waits for) is still running
+    // backward in pieces: the whole data-gradient chain first, so that dx can travel to the host while the two
+    // weight-gradient GEMMs (which nothing downstream waits for) are still running
+    MOE_STEP(moe_grouped_gemm_down_dgrad(dims, P(a.dyp), w_down, Pi(a.offsets), P(a.dhact), stream));
     MOE_STEP(moe_swiglu_bwd(dims, P(a.dhact), P(a.gu), P(a.dgu), stream));
     MOE_STEP(moe_grouped_gemm_gateup_dgrad(dims, P(a.dgu), w_gate, w_up, Pi(a.offsets), P(a.dxp), stream));
     MOE_STEP(moe_permute_bwd(dims, P(a.dxp), Pi(a.p2r), P(a.dx), stream));
@@ -332,6 +332,7 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
         cudaMemcpyAsync(dtopk_w_host, P(a.dw), R * 4, cudaMemcpyDeviceToHost, c) != cudaSuccess ||
         cudaEventRecord(lane->down_done, c) != cudaSuccess)
         return MOE_ERR_CUDA;
+    MOE_STEP(moe_grouped_gemm_down_wgrad(dims, P(a.hact), P(a.dyp), Pi(a.offsets), dw_down, stream));
     MOE_STEP(moe_grouped_gemm_gateup_wgrad(dims, P(a.xp), P(a.dgu), Pi(a.offsets), dw_gate, dw_up, stream));
 #undef MOE_STEP
 
