@@ -4,8 +4,9 @@
 // how their routing inputs are made; the paper has no counterpart.
 //
 // One warp per token.  The E <= 1024 logits of a row sit in registers, element e = j*32 + lane (coalesced
-// loads).  Selection is K rounds of: per-lane best among the not-yet-taken elements, then a warp arg-max on
-// (value, id) by shuffles.  All comparisons are on the float32 values as given, so the indices are exact.
+// loads).  Selection is K rounds of: per-lane best among the not-yet-taken elements, then a warp arg-max with
+// two integer redux instructions (maximum of an order-preserving key, then the lowest id among its holders).
+// All comparisons are on the float32 values as given, so the indices are exact.
 // HBM-bound in principle (T*E*4 bytes in, 8*T*K out), in practice a few microseconds.
 #include <limits.h>
 #include <math.h>
@@ -17,8 +18,15 @@ namespace {
 
 constexpr int kWarpsPerBlock = 8;
 
-// (value, id) ordering of the selection: larger value first, equal values: lower id first
-__device__ __forceinline__ bool better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
+// Order-preserving map of a float onto unsigned integers (larger float <=> larger key; -inf maps above 0, which
+// stands for "no candidate"), and its inverse.  Lets the warp arg-max run on the integer redux instructions.
+__device__ __forceinline__ uint32_t key_of(float v) {
+    const uint32_t u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float value_of(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
 
 template <int VPL>   // logits per lane, E <= 32 * VPL
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
@@ -28,31 +36,31 @@ router_topk_kernel(const float* __restrict__ logits, int T, int E, int K, int32_
     const int t = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     if (t >= T) return;
     const float* row = logits + (size_t)t * E;
-    float v[VPL];
+    uint32_t key[VPL];
 #pragma unroll
     for (int j = 0; j < VPL; ++j) {
         const int e = j * 32 + lane;
-        v[j] = e < E ? row[e] : -INFINITY;
+        key[j] = e < E ? key_of(row[e] + 0.0f) : 0u;   // + 0.0f: -0.0 and +0.0 compare equal, so they share a key
     }
-    uint32_t taken = 0;                 // bit j: element j of this lane was selected
     float my_val = 0.f;                 // lane k keeps the k-th selection
     int my_idx = 0;
     for (int k = 0; k < K; ++k) {
-        float bv = -INFINITY;
-        int bi = INT_MAX;               // INT_MAX = no candidate in this lane
+        // this lane's best remaining element (ascending j = ascending id, strict > keeps the lower id on ties)
+        uint32_t bk = 0u;
+        int bj = 0;
 #pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-            const int e = j * 32 + lane;
-            if (e < E && !((taken >> j) & 1u) && better(v[j], e, bv, bi)) { bv = v[j]; bi = e; }
-        }
+        for (int j = 0; j < VPL; ++j)
+            if (key[j] > bk) { bk = key[j]; bj = j; }
+        const uint32_t kmax = __reduce_max_sync(0xffffffffu, bk);
+        // among the lanes that hold the maximum: the lowest expert id
+        const uint32_t cand = (bk == kmax && bk != 0u) ? (uint32_t)(bj * 32 + lane) : 0xffffffffu;
+        const uint32_t imin = __reduce_min_sync(0xffffffffu, cand);
+        if ((int)(imin & 31u) == lane && imin != 0xffffffffu) {
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, off);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-            if (oi != INT_MAX && (bi == INT_MAX || better(ov, oi, bv, bi))) { bv = ov; bi = oi; }
+            for (int j = 0; j < VPL; ++j)
+                if (j == (int)(imin >> 5)) key[j] = 0u;   // taken
         }
-        if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
-        if (k == lane) { my_val = bv; my_idx = bi; }
+        if (k == lane) { my_val = value_of(kmax); my_idx = (int)imin; }
     }
     // softmax over the kept logits; the first selection is the row maximum
     const float m = __shfl_sync(0xffffffffu, my_val, 0);
