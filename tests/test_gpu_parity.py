@@ -32,6 +32,9 @@ CASES = {
     # H and I multiples of 64 only (the paper's 2880 = 45 * 64): partial column tiles everywhere
     "ragged_64": lambda: Hh.ragged_workload([200, 0, 31, 290, 1], K=2, H=192, I=320, seed=4),
     "pair_64": lambda: Hh.ragged_workload([600, 540, 0, 700], K=2, H=320, I=192, seed=6),
+    # CTA-pair kernels whose last 256-row tile per expert holds 100, exactly 128, 65 and 129 rows (the second CTA's
+    # half of the tile partly or wholly past the expert's end), plus one expert of several full tiles
+    "pair_half": lambda: Hh.ragged_workload([356, 640, 321, 900, 385], K=2, H=256, I=320, seed=8),
 }
 
 
