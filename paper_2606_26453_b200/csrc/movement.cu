@@ -44,6 +44,8 @@ __device__ __forceinline__ uint4 pack8(const float f[8]) {
 //          row(p) = offsets[e] + base[e] + pairs of e in earlier warps of the block + earlier
 //          pairs of e in the same warp.
 // ------------------------------------------------------------------------------------------------
+constexpr int kIdxGroup = 8;   // index loads in flight per thread in the permute index kernels
+
 __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* __restrict__ topk_idx, int R, int E,
                                                                 int chunk, int32_t* __restrict__ ws) {
     extern __shared__ int32_t smem_i[];
@@ -52,12 +54,24 @@ __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* _
     for (int e = threadIdx.x; e < E; e += kThreads) hist[e] = 0;
     __syncthreads();
     const long long p0 = (long long)blockIdx.x * chunk;
-    for (int i = threadIdx.x; i < chunk; i += kThreads) {   // chunk is a multiple of kThreads: whole warps stay together
-        const long long p = p0 + i;
-        int e = (p < R) ? topk_idx[p] : -1;
-        if (e >= E) e = -1;
-        const unsigned mask = __match_any_sync(0xffffffffu, e);
-        if (e >= 0 && lane == __ffs(mask) - 1) atomicAdd(&hist[e], __popc(mask));   // counts only: order-free
+    // chunk is a multiple of kThreads: whole warps stay together.  The indices of kIdxGroup iterations are loaded
+    // first, so that their global-memory latencies overlap instead of adding up in front of every match.
+    for (int i0 = threadIdx.x; i0 < chunk; i0 += kThreads * kIdxGroup) {
+        int ev[kIdxGroup];
+#pragma unroll
+        for (int g = 0; g < kIdxGroup; ++g) {
+            const int i = i0 + g * kThreads;
+            const long long p = p0 + i;
+            int e = (i < chunk && p < R) ? topk_idx[p] : -1;
+            ev[g] = e >= E ? -1 : e;
+        }
+#pragma unroll
+        for (int g = 0; g < kIdxGroup; ++g) {
+            if (i0 - (int)threadIdx.x + g * kThreads >= chunk) break;   // block-uniform
+            const int e = ev[g];
+            const unsigned mask = __match_any_sync(0xffffffffu, e);
+            if (e >= 0 && lane == __ffs(mask) - 1) atomicAdd(&hist[e], __popc(mask));   // counts only: order-free
+        }
     }
     __syncthreads();
     int32_t* out = ws + (size_t)blockIdx.x * E;
@@ -114,13 +128,23 @@ __global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* _
     const long long p0 = (long long)blockIdx.x * chunk + (long long)warp * per_warp;
     int32_t* mine = whist + warp * E;
 #pragma unroll 1
-    for (int i = lane; i < per_warp; i += 32) {
-        const long long p = p0 + i;
-        int e = (p < R) ? topk_idx[p] : -1;
-        if (e >= E) e = -1;
-        const unsigned mask = __match_any_sync(0xffffffffu, e);
-        if (e >= 0 && lane == __ffs(mask) - 1) mine[e] += __popc(mask);
-        __syncwarp();
+    for (int i0 = 0; i0 < per_warp; i0 += 32 * kIdxGroup) {   // indices of kIdxGroup iterations loaded up front
+        int ev[kIdxGroup];
+#pragma unroll
+        for (int g = 0; g < kIdxGroup; ++g) {
+            const int i = i0 + g * 32 + lane;
+            const long long p = p0 + i;
+            int e = (i < per_warp && p < R) ? topk_idx[p] : -1;
+            ev[g] = e >= E ? -1 : e;
+        }
+#pragma unroll
+        for (int g = 0; g < kIdxGroup; ++g) {
+            if (i0 + g * 32 >= per_warp) break;   // warp-uniform
+            const int e = ev[g];
+            const unsigned mask = __match_any_sync(0xffffffffu, e);
+            if (e >= 0 && lane == __ffs(mask) - 1) mine[e] += __popc(mask);
+            __syncwarp();
+        }
     }
     __syncthreads();
     if (blockIdx.x == 0) {
@@ -141,19 +165,30 @@ __global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* _
     // pass 2: stable ranks
     const unsigned lt_mask = (1u << lane) - 1u;
 #pragma unroll 1
-    for (int i = lane; i < per_warp; i += 32) {
-        const long long p = p0 + i;
-        int e = (p < R) ? topk_idx[p] : -1;
-        if (e >= E) e = -1;
-        const unsigned mask = __match_any_sync(0xffffffffu, e);
-        if (e >= 0) {
-            const int row = mine[e] + __popc(mask & lt_mask);
-            row_to_pair[row] = (int32_t)p;
-            pair_to_row[p] = row;
+    for (int i0 = 0; i0 < per_warp; i0 += 32 * kIdxGroup) {
+        int ev[kIdxGroup];
+#pragma unroll
+        for (int g = 0; g < kIdxGroup; ++g) {
+            const int i = i0 + g * 32 + lane;
+            const long long p = p0 + i;
+            int e = (i < per_warp && p < R) ? topk_idx[p] : -1;
+            ev[g] = e >= E ? -1 : e;
         }
-        __syncwarp();
-        if (e >= 0 && lane == __ffs(mask) - 1) mine[e] += __popc(mask);
-        __syncwarp();
+#pragma unroll
+        for (int g = 0; g < kIdxGroup; ++g) {
+            if (i0 + g * 32 >= per_warp) break;   // warp-uniform
+            const int e = ev[g];
+            const long long p = p0 + i0 + g * 32 + lane;
+            const unsigned mask = __match_any_sync(0xffffffffu, e);
+            if (e >= 0) {
+                const int row = mine[e] + __popc(mask & lt_mask);
+                row_to_pair[row] = (int32_t)p;
+                pair_to_row[p] = row;
+            }
+            __syncwarp();
+            if (e >= 0 && lane == __ffs(mask) - 1) mine[e] += __popc(mask);
+            __syncwarp();
+        }
     }
 }
 
