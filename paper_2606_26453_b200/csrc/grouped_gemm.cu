@@ -71,7 +71,15 @@ constexpr int FIX_WARP = 2 + NUM_EPI_WARPS;
 constexpr int TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
-enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3 };
+// The _T kinds compute the same products as FWD_PLAIN / DGRAD with the operand roles swapped: the weights are the
+// M side of the MMA (128 output features per tile) and the expert's packed rows the N side, so a row tile can have
+// any height that is a multiple of 16 (up to 256) instead of a fixed 128 / 256: an expert's rows are split into
+// equal tiles and almost no tensor work goes to padding.  The accumulator comes out transposed (lane = feature,
+// column = row); the epilogue transposes it back through its shared-memory staging blocks.
+enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3, FWD_PLAIN_T = 4, DGRAD_T = 5 };
+__host__ __device__ constexpr bool swapped(int kind) { return kind == FWD_PLAIN_T || kind == DGRAD_T; }
+constexpr int SWAP_ROWS = 256;   // most rows of a swapped tile
+constexpr int SWAP_FEATS = 128;  // output features of a swapped tile
 
 struct Params {
     const int32_t* offsets;
@@ -100,6 +108,7 @@ struct SharedCtl {
     unsigned long long drain;
     uint32_t tmem_base;
     int abort_flag;
+    int stage_n[MAX_STAGES];   // swapped kinds: MMA N (rows of the tile rounded up to 16) of the tile a stage belongs to
     int32_t offs[MAX_E + 1];
     int32_t tile_prefix[MAX_E + 1];
     int32_t sorted_rows[MAX_E];   // WGRAD: row count of the expert at each position of the largest-first order
@@ -335,6 +344,7 @@ struct Tile {
     int k_blocks; // contraction blocks of this tile
     int k_row0;   // WGRAD: first packed row of the contraction
     int k_rows;   // WGRAD: rows of the contraction
+    int rows;     // swapped kinds: rows of this tile (1..256)
 };
 
 // Order of an expert's m_tiles x n_tiles output tiles: bands of RASTER_BAND row tiles; inside a band
@@ -391,6 +401,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
         tl.k_rows = ctl->offs[tl.e + 1] - tl.k_row0;
         tl.k_blocks = (tl.k_rows + BK - 1) / BK;
         tl.row_end = 0;
+        tl.rows = 0;
     } else {
         // tile_prefix[e] = number of TILE_M-row tiles of experts < e
         int lo = 0, hi = p.E;                          // largest e with tile_prefix[e]*n_tiles <= t
@@ -403,9 +414,19 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
         const int local = (int)(t - (long long)ctl->tile_prefix[lo] * p.n_tiles);
         int mt, nt;
         raster(local, m_tiles_e, p.n_tiles, mt, nt);
-        tl.row0 = ctl->offs[lo] + mt * TILE_M;
         tl.row_end = ctl->offs[lo + 1];
-        tl.n0 = nt * BN;
+        tl.rows = 0;
+        if (swapped(KIND)) {
+            // the expert's rows in m_tiles_e equal tiles, each a multiple of 16 rows (the last one takes what is left)
+            const int n_e = tl.row_end - ctl->offs[lo];
+            const int per_tile = ((n_e + m_tiles_e - 1) / m_tiles_e + 15) & ~15;
+            tl.row0 = ctl->offs[lo] + mt * per_tile;
+            tl.rows = min(per_tile, tl.row_end - tl.row0);
+            tl.n0 = nt * TILE_M;   // output features per tile: 128, or 256 over a CTA pair
+        } else {
+            tl.row0 = ctl->offs[lo] + mt * TILE_M;
+            tl.n0 = nt * BN;
+        }
         tl.k_blocks = p.k_blocks;
         tl.k_row0 = 0;
         tl.k_rows = 0;
@@ -429,10 +450,38 @@ __device__ __forceinline__ void zero_k_rows(uint8_t* stage_ptr, int n_chunks, in
 // tried and cost 10-15 %: the L2 -> SM path, not DRAM latency, is what these kernels saturate.)
 template <int KIND, bool PAIR>
 __device__ __forceinline__ void stage_loads(const Tile& tl, int kb, const Params& p, const CUtensorMap* map_a,
+                                         const CUtensorMap* map_r2, const CUtensorMap* map_r1,
                                          const CUtensorMap* map_b0, const CUtensorMap* map_b1, uint32_t a_dst,
                                          uint32_t b_dst, uint32_t full, uint32_t rank, int my_rows) {
     const int n_local = tl.n0 + (PAIR ? my_rows : 0);   // first B column this CTA loads
-    if (KIND == WGRAD) {
+    if (swapped(KIND)) {
+        // M side (a_dst): the weight tile, 128 output features x 64 k.  N side (b_dst): the tile's rows in boxes of
+        // 64 rows (map_a is the activation map with a 64-row box), only as many boxes as the tile has rows.
+        // In pair mode each CTA loads its own 128 features and half of the tile's rows (N/2 of the MMA's N,
+        // N = rows rounded up to 16), in boxes of 32 rows; a single CTA loads all rows in boxes of 64.
+        const int feat0 = tl.n0 + (PAIR ? (int)rank * SWAP_FEATS : 0);
+        if (KIND == FWD_PLAIN_T) {
+            tma_load_3d(a_dst, map_b0, 0, tl.e * p.b_rows_per_e + kb * BK, feat0 >> 6, full);
+        } else {
+            const bool second = kb >= p.k_split;
+            const int kx = (second ? kb - p.k_split : kb) * BK;
+            tma_load_2d(a_dst, second ? map_b1 : map_b0, kx, tl.e * p.b_rows_per_e + feat0, full);
+        }
+        // at most two loads: boxes of 1, 2 or 4 times BOX rows (map_r1, map_r2, map_a), or 2 + 1
+        constexpr int BOX = PAIR ? 32 : 64;
+        const int my_n = PAIR ? (((tl.rows + 15) & ~15) >> 1) : tl.rows;           // rows this CTA provides
+        const int my_row0 = tl.row0 + (PAIR ? (int)rank * my_n : 0);
+        if (my_n <= BOX) {
+            tma_load_2d(b_dst, map_r1, kb * BK, my_row0, full);
+        } else if (my_n <= 2 * BOX) {
+            tma_load_2d(b_dst, map_r2, kb * BK, my_row0, full);
+        } else if (my_n <= 3 * BOX) {
+            tma_load_2d(b_dst, map_r2, kb * BK, my_row0, full);
+            tma_load_2d(b_dst + 2 * BOX * 128, map_r1, kb * BK, my_row0 + 2 * BOX, full);
+        } else {
+            tma_load_2d(b_dst, map_a, kb * BK, my_row0, full);
+        }
+    } else if (KIND == WGRAD) {
         const int krow = tl.k_row0 + kb * BK;
         // MN-major operands: one 3-D box = all 64-wide chunks, chunk-major in shared memory
         tma_load_3d(a_dst, map_a, 0, krow, (tl.row0 + my_rows) >> 6, full);
@@ -468,12 +517,16 @@ template <int KIND, bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b0,
                     const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_o0,
-                    const __grid_constant__ CUtensorMap map_o1, const Params p) {
+                    const __grid_constant__ CUtensorMap map_o1, const __grid_constant__ CUtensorMap map_x,
+                    const Params p) {
     using G = Geo<PAIR>;
     constexpr int STAGES = G::STAGES;
     constexpr int STAGE_BYTES = G::STAGE_BYTES;
-    constexpr bool A_MN = (KIND == WGRAD);
-    constexpr bool B_MN = (KIND != DGRAD);
+    constexpr bool SWAP = swapped(KIND);
+    constexpr int ROW_TILE = SWAP ? SWAP_ROWS : G::TILE_M;   // rows an expert's tile count is computed from
+    // operand major-ness of the MMA's M side (A) and N side (B); for the swapped kinds A is the weight tile
+    constexpr bool A_MN = (KIND == WGRAD || KIND == FWD_PLAIN_T);
+    constexpr bool B_MN = (KIND == FWD_SWIGLU || KIND == FWD_PLAIN || KIND == WGRAD);
     constexpr uint32_t IDESC = make_idesc(G::TILE_M, BN, A_MN, B_MN);
     constexpr uint32_t A_KSTEP = A_MN ? 2048 : 32;   // bytes per 16 k inside a stage
     constexpr uint32_t B_KSTEP = B_MN ? 2048 : 32;
@@ -515,6 +568,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         prefetch_tmap(&map_b1);
         prefetch_tmap(&map_o0);
         prefetch_tmap(&map_o1);
+        prefetch_tmap(&map_x);
     }
     __syncthreads();
     if (KIND == WGRAD) {
@@ -533,7 +587,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         int run = 0;
         for (int e = 0; e < p.E; ++e) {
             ctl->tile_prefix[e] = run;
-            run += (ctl->offs[e + 1] - ctl->offs[e] + G::TILE_M - 1) / G::TILE_M;
+            run += (ctl->offs[e + 1] - ctl->offs[e] + ROW_TILE - 1) / ROW_TILE;
         }
         ctl->tile_prefix[p.E] = run;
     }
@@ -570,9 +624,17 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 for (int kb = 0; kb < tl.k_blocks; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t land = smem_u32(local_fix ? &ctl->landed[stage] : &ctl->full[stage]);
-                    mbar_arrive_expect_tx(land, STAGE_BYTES);
+                    if (SWAP) {
+                        ctl->stage_n[stage] = (tl.rows + 15) & ~15;   // read by the MMA thread after its wait on full[stage]
+                        const int my_n = PAIR ? (((tl.rows + 15) & ~15) >> 1) : tl.rows;
+                        constexpr int BOX = PAIR ? 32 : 64;
+                        mbar_arrive_expect_tx(land, G::A_BYTES + min(4, (my_n + BOX - 1) / BOX) * (BOX * BK * 2));
+                    } else {
+                        mbar_arrive_expect_tx(land, STAGE_BYTES);
+                    }
                     const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
-                    stage_loads<KIND, PAIR>(tl, kb, p, &map_a, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES, land, rank, my_rows);
+                    stage_loads<KIND, PAIR>(tl, kb, p, &map_a, &map_o1, &map_x, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES, land,
+                                            rank, my_rows);
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -613,9 +675,12 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 return ctl->sorted_rows[e_pos];
             };
             // one K block: n_mma MMAs from ring stage `stage`, then the stage is released
+            uint32_t idesc = IDESC;
             auto issue_block = [&](uint32_t d_tmem, bool first_block, int n_mma, bool partial) -> bool {
                 if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) return false;
                 tc_fence_after();
+                // swapped kinds: the MMA's N is the tile's row count (rounded up to 16), published with each stage
+                if (SWAP && first_block) idesc = make_idesc(G::TILE_M, ctl->stage_n[stage], A_MN, B_MN);
                 const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
                 const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
                 const uint64_t b_desc = make_smem_desc<B_MN>(a_base + G::A_BYTES);
@@ -627,7 +692,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                                         b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, accumulate, kk < n_mma ? 1u : 0u);
                     else
                         tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
-                                     b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, accumulate);
+                                     b_desc + (uint64_t)((kk * B_KSTEP) >> 4), SWAP ? idesc : IDESC, accumulate);
                 }
                 tc_commit<PAIR>(smem_u32(&ctl->empty[stage]));
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -744,6 +809,31 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
             for (int j = 0; j < 4; ++j) d4[j] = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
         };
+        // swapped kinds: this lane holds one output feature for 32 consecutive rows; the block is transposed on its
+        // way into the staging buffer (row j of the block, feature `lane`: 2-byte stores, 64 contiguous bytes per
+        // warp instruction) and then stored like any other 32 x 32 block
+        auto stage_transposed_and_store = [&](const uint32_t (&v)[32], const CUtensorMap* map, int x, int y) {
+            uint8_t* blk = stage_ptr + (n_stores % G::STAGING_BLOCKS) * STAGING_BLOCK_BYTES;
+            if (n_stores >= (uint32_t)G::STAGING_BLOCKS) {
+                if (lane == 0) {
+                    if (G::STAGING_BLOCKS == 2 && !drain_first) bulk_wait_read1(); else bulk_wait_read0();
+                }
+                __syncwarp();
+                drain_first = false;
+            }
+            const int piece = lane >> 3, within = (lane & 7) * 2;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                *reinterpret_cast<__nv_bfloat16*>(blk + j * 64 + (((piece ^ ((j >> 1) & 3)) << 4) + within)) =
+                    __float2bfloat16_rn(__uint_as_float(v[j]));
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(map, x, y, smem_u32(blk));
+                bulk_commit();
+            }
+            ++n_stores;
+        };
         const uint32_t tmem_empty_remote0 = PAIR ? map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0) : 0u;
         const uint32_t tmem_empty_remote1 = PAIR ? map_to_cta(smem_u32(&ctl->tmem_empty[1]), 0) : 0u;
 
@@ -760,7 +850,29 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const int rows_valid = (KIND == WGRAD) ? (slab0 < p.m_rows ? 32 : 0) : max(0, min(32, tl.row_end - slab0));
             const int slab_y = (KIND == WGRAD) ? tl.e * p.m_rows + slab0 : slab0;
             const long long row = (long long)slab0 + lane;
-            if (KIND == FWD_SWIGLU) {
+            if (SWAP) {
+                // lane = output feature, tensor-memory column = row of the tile; the two warps of a lane quarter
+                // take the 32-row blocks alternately
+                const int feat0 = tl.n0 + (PAIR ? (int)rank * SWAP_FEATS : 0) + quarter * 32;
+                const int n_row_blocks = (tl.rows + 31) >> 5;
+#pragma unroll 1
+                for (int i = half; i < n_row_blocks; i += 2) {
+                    uint32_t v[32];
+                    tc_ld32(taddr + i * 32, v);
+                    tc_wait_ld();
+                    if (feat0 >= p.n_cols) continue;
+                    const int r0 = tl.row0 + i * 32;
+                    const int rv = min(32, tl.rows - i * 32);
+                    if (rv == 32) {
+                        stage_transposed_and_store(v, &map_o0, feat0, r0);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)   // rows past the tile belong to the expert's next tile, or to nobody
+                            if (j < rv)
+                                p.out0[(long long)(r0 + j) * p.ldo + feat0 + lane] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    }
+                }
+            } else if (KIND == FWD_SWIGLU) {
                 const int ng = tl.n0 >> 1;
 #pragma unroll 1
                 for (int c = 2 * half; c < 2 * half + 2; ++c) {
@@ -945,9 +1057,11 @@ bool make_out_map(CUtensorMap* map, const void* base, uint64_t cols, uint64_t ro
 // Grid of a launch: one CTA per SM (single), or as many CTA pairs as can be resident at once (pair).
 // A pair that could not be co-scheduled would run after the others and double the kernel's duration,
 // so the pair grid is sized from the occupancy query, per device and kernel.
+// Swapped kinds: `a`, `o1` and `x` are the row operand's maps with boxes of 4, 2 and 1 times the smallest box
+// (32 rows in pair mode, 64 otherwise); the other kinds pass `a` for `x`.
 template <int KIND, bool PAIR>
 int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const CUtensorMap& o0,
-           const CUtensorMap& o1, const Params& p, cudaStream_t s) {
+           const CUtensorMap& o1, const CUtensorMap& x, const Params& p, cudaStream_t s) {
     static int grid_of_device[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
@@ -983,15 +1097,20 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
         attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
     }
-    if (cudaLaunchKernelEx(&cfg, kernel, a, b0, b1, o0, o1, p) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kernel, a, b0, b1, o0, o1, x, p) != cudaSuccess) return MOE_ERR_CUDA;
     return check_launch();
 }
 
-// CTA pairs (256-row tiles) are used when experts hold at least 512 rows on average: below that the extra
-// padding of each expert's last tile (row-ragged kinds) and the pair's per-tile hand-shakes (short
-// contractions in the weight gradients) cost more than the halved operand traffic buys.  Measured: at 384
-// rows per expert single tiles are 8-25 % faster, from 1024 rows per expert on pairs are 5-15 % faster.
+// Fixed-height CTA-pair tiles (256 rows) are used when experts hold at least 512 rows on average: below that the
+// padding of each expert's last tile costs more than the halved operand traffic buys.  The SwiGLU forward then
+// runs single-CTA 128-row tiles, the plain row-ragged GEMMs the swapped kinds (next comment).
 bool use_pairs_for_rows(const moe_dims_t& d) { return (long long)d.T * d.K >= 512ll * d.E; }
+// The plain row-ragged GEMMs (down forward, down dgrad, gate/up dgrad) run with swapped operand roles -- always as
+// CTA pairs: 256 output features x up to 256 rows per tile -- when experts hold fewer than 512 rows on average:
+// there the fixed 128-row tiles lose 10-15 % of the tensor work to padding (measured: +2-5 % per kernel on the
+// 384- and 451-rows-per-expert workloads).  With larger experts the padding is small and the fixed-height tiles
+// are as fast or faster (the swapped kernels' issue thread, not the tensor pipe, bounds tiles of fewer than 256 rows).
+bool use_swapped(const moe_dims_t& d) { return (long long)d.T * d.K < 512ll * d.E; }
 // Weight gradients have no row padding to lose, so pairs already win from 256 rows per expert.
 bool use_pairs_for_wgrad(const moe_dims_t& d) { return (long long)d.T * d.K >= 256ll * d.E; }
 
@@ -1011,24 +1130,39 @@ int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gat
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
     p.n_tiles = (d.I + 127) / 128; p.n_cols = 2 * d.I; p.b_rows_per_e = d.H;
     p.out0 = h_act; p.gu = gu; p.I = d.I; p.ldo = d.I; p.n_split = 2 * d.I;
-    return use_pairs_for_rows(d) ? launch<FWD_SWIGLU, true>(a, b0, b1, o0, o1, p, s)
-                                 : launch<FWD_SWIGLU, false>(a, b0, b1, o0, o1, p, s);
+    return use_pairs_for_rows(d) ? launch<FWD_SWIGLU, true>(a, b0, b1, o0, o1, a, p, s)
+                                 : launch<FWD_SWIGLU, false>(a, b0, b1, o0, o1, a, p, s);
 }
 
 // Down forward: A = h_act [R,I]; B = w_down viewed as [E*I, H].
 int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, const int32_t* offsets,
                     bf16* y_perm, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    const bool pair = use_pairs_for_rows(d);
+    if (use_swapped(d)) {
+        // swapped roles: M side = w_down tile (128 features of H, MN-major), N side = rows of h_act (64-row boxes)
+        const int feats = 2 * SWAP_FEATS;   // a CTA pair's tile
+        const uint32_t box = 32;            // row boxes of 32 / 64 / 128 rows per CTA
+        CUtensorMap a, a2, a1, b0, o0;
+        if (!make_map(&a, h_act, d.I, R, BK, 4 * box) || !make_map(&a2, h_act, d.I, R, BK, 2 * box) ||
+            !make_map(&a1, h_act, d.I, R, BK, box) ||
+            !make_map_mn(&b0, w_down, d.H, (uint64_t)d.E * d.I, SWAP_FEATS / 64) || !make_out_map(&o0, y_perm, d.H, R))
+            return MOE_ERR_CUDA;
+        Params p = {};
+        p.offsets = offsets; p.E = d.E; p.k_blocks = d.I / BK; p.k_split = p.k_blocks;
+        p.n_tiles = (d.H + feats - 1) / feats; p.n_cols = d.H; p.b_rows_per_e = d.I;
+        p.out0 = y_perm; p.ldo = d.H; p.n_split = d.H;
+        return launch<FWD_PLAIN_T, true>(a, b0, b0, o0, a2, a1, p, s);
+    }
+    // larger experts: 256-row pair tiles (each CTA loads half of B's columns)
     CUtensorMap a, b0, o0;
-    if (!make_map(&a, h_act, d.I, R, BK, BM) ||
-        !make_map_mn(&b0, w_down, d.H, (uint64_t)d.E * d.I, pair ? BN / 128 : BN / 64) || !make_out_map(&o0, y_perm, d.H, R))
+    if (!make_map(&a, h_act, d.I, R, BK, BM) || !make_map_mn(&b0, w_down, d.H, (uint64_t)d.E * d.I, BN / 128) ||
+        !make_out_map(&o0, y_perm, d.H, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.I / BK; p.k_split = p.k_blocks;
     p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.b_rows_per_e = d.I;
     p.out0 = y_perm; p.ldo = d.H; p.n_split = d.H;
-    return pair ? launch<FWD_PLAIN, true>(a, b0, b0, o0, o0, p, s) : launch<FWD_PLAIN, false>(a, b0, b0, o0, o0, p, s);
+    return launch<FWD_PLAIN, true>(a, b0, b0, o0, o0, a, p, s);
 }
 
 // Down dgrad: dh_act = dy_perm . w_down[e]^T.  A = dy_perm [R,H]; B = w_down viewed as [E*I, H] (rows are
@@ -1036,16 +1170,30 @@ int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, 
 int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_down, const int32_t* offsets,
                       bf16* dh_act, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    const bool pair = use_pairs_for_rows(d);
+    if (use_swapped(d)) {
+        // swapped roles: M side = w_down tile (128 features of I, K-major), N side = rows of dy_perm
+        const int feats = 2 * SWAP_FEATS;   // a CTA pair's tile
+        const uint32_t box = 32;            // row boxes of 32 / 64 / 128 rows per CTA
+        CUtensorMap a, a2, a1, b0, o0;
+        if (!make_map(&a, dy_perm, d.H, R, BK, 4 * box) || !make_map(&a2, dy_perm, d.H, R, BK, 2 * box) ||
+            !make_map(&a1, dy_perm, d.H, R, BK, box) ||
+            !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, SWAP_FEATS) || !make_out_map(&o0, dh_act, d.I, R))
+            return MOE_ERR_CUDA;
+        Params p = {};
+        p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
+        p.n_tiles = (d.I + feats - 1) / feats; p.n_cols = d.I; p.b_rows_per_e = d.I;
+        p.out0 = dh_act; p.ldo = d.I; p.n_split = d.I;
+        return launch<DGRAD_T, true>(a, b0, b0, o0, a2, a1, p, s);
+    }
     CUtensorMap a, b0, o0;
-    if (!make_map(&a, dy_perm, d.H, R, BK, BM) ||
-        !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, pair ? BN / 2 : BN) || !make_out_map(&o0, dh_act, d.I, R))
+    if (!make_map(&a, dy_perm, d.H, R, BK, BM) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, BN / 2) ||
+        !make_out_map(&o0, dh_act, d.I, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
     p.n_tiles = (d.I + BN - 1) / BN; p.n_cols = d.I; p.b_rows_per_e = d.I;
     p.out0 = dh_act; p.ldo = d.I; p.n_split = d.I;
-    return pair ? launch<DGRAD, true>(a, b0, b0, o0, o0, p, s) : launch<DGRAD, false>(a, b0, b0, o0, o0, p, s);
+    return launch<DGRAD, true>(a, b0, b0, o0, o0, a, p, s);
 }
 
 // Gate/up dgrad: dx_perm = dg . w_gate[e]^T + du . w_up[e]^T.  A = dgu [R,2I]; the contraction runs over the
@@ -1053,8 +1201,22 @@ int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_do
 int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate, const bf16* w_up,
                         const int32_t* offsets, bf16* dx_perm, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    const bool pair = use_pairs_for_rows(d);
-    const uint32_t bn = pair ? BN / 2 : BN;
+    if (use_swapped(d)) {
+        const int feats = 2 * SWAP_FEATS;   // a CTA pair's tile
+        const uint32_t box = 32;            // row boxes of 32 / 64 / 128 rows per CTA
+        CUtensorMap a, a2, a1, b0, b1, o0;
+        if (!make_map(&a, dgu, 2ull * d.I, R, BK, 4 * box) || !make_map(&a2, dgu, 2ull * d.I, R, BK, 2 * box) ||
+            !make_map(&a1, dgu, 2ull * d.I, R, BK, box) ||
+            !make_map(&b0, w_gate, d.I, (uint64_t)d.E * d.H, BK, SWAP_FEATS) ||
+            !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, BK, SWAP_FEATS) || !make_out_map(&o0, dx_perm, d.H, R))
+            return MOE_ERR_CUDA;
+        Params p = {};
+        p.offsets = offsets; p.E = d.E; p.k_blocks = 2 * d.I / BK; p.k_split = d.I / BK;
+        p.n_tiles = (d.H + feats - 1) / feats; p.n_cols = d.H; p.b_rows_per_e = d.H;
+        p.out0 = dx_perm; p.ldo = d.H; p.n_split = d.H;
+        return launch<DGRAD_T, true>(a, b0, b1, o0, a2, a1, p, s);
+    }
+    const uint32_t bn = BN / 2;
     CUtensorMap a, b0, b1, o0;
     if (!make_map(&a, dgu, 2ull * d.I, R, BK, BM) || !make_map(&b0, w_gate, d.I, (uint64_t)d.E * d.H, BK, bn) ||
         !make_map(&b1, w_up, d.I, (uint64_t)d.E * d.H, BK, bn) || !make_out_map(&o0, dx_perm, d.H, R))
@@ -1063,7 +1225,7 @@ int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate
     p.offsets = offsets; p.E = d.E; p.k_blocks = 2 * d.I / BK; p.k_split = d.I / BK;
     p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.b_rows_per_e = d.H;
     p.out0 = dx_perm; p.ldo = d.H; p.n_split = d.H;
-    return pair ? launch<DGRAD, true>(a, b0, b1, o0, o0, p, s) : launch<DGRAD, false>(a, b0, b1, o0, o0, p, s);
+    return launch<DGRAD, true>(a, b0, b1, o0, o0, a, p, s);
 }
 
 // Weight gradients: the tile grid is static (M x N per expert).  Pairs (256 x 256 tiles) pay off once an
@@ -1083,7 +1245,7 @@ int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_per
     p.offsets = offsets; p.E = d.E; p.m_rows = d.I; p.m_tiles = (d.I + tile_m - 1) / tile_m;
     p.n_tiles = (d.H + BN - 1) / BN; p.n_cols = d.H; p.n_split = d.H; p.ldo = d.H;
     p.out0 = dw_down; p.out1 = nullptr;
-    return pair ? launch<WGRAD, true>(a, b0, b0, o0, o0, p, s) : launch<WGRAD, false>(a, b0, b0, o0, o0, p, s);
+    return pair ? launch<WGRAD, true>(a, b0, b0, o0, o0, a, p, s) : launch<WGRAD, false>(a, b0, b0, o0, o0, a, p, s);
 }
 
 // Gate/up wgrad (the paper's dW1): [dw_gate[e] | dw_up[e]] = x_perm_e^T . dgu_e.  A = x_perm [R,H] (M = H),
@@ -1101,7 +1263,7 @@ int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu
     p.offsets = offsets; p.E = d.E; p.m_rows = d.H; p.m_tiles = (d.H + tile_m - 1) / tile_m;
     p.n_tiles = (2 * d.I + BN - 1) / BN; p.n_cols = 2 * d.I; p.n_split = d.I; p.ldo = d.I;
     p.out0 = dw_gate; p.out1 = dw_up;
-    return pair ? launch<WGRAD, true>(a, b0, b0, o0, o1, p, s) : launch<WGRAD, false>(a, b0, b0, o0, o1, p, s);
+    return pair ? launch<WGRAD, true>(a, b0, b0, o0, o1, a, p, s) : launch<WGRAD, false>(a, b0, b0, o0, o1, a, p, s);
 }
 
 }  // namespace moe
