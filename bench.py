@@ -38,12 +38,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of each grouped-GEMM kernel, from the
 # ncu captures summarised in profiles/ncu_full_<workload>.md.  Workloads without a capture report null.
 NCU_TRAFFIC_BYTES = {
-    ("fine_grained", "gateup_swiglu"): 1023.6e6, ("fine_grained", "down"): 525.3e6,
-    ("fine_grained", "down_dgrad"): 527.4e6, ("fine_grained", "down_wgrad"): 498.4e6,
-    ("fine_grained", "gateup_dgrad"): 980.8e6, ("fine_grained", "gateup_wgrad"): 939.8e6,
-    ("many_small", "gateup_swiglu"): 1924.7e6, ("many_small", "down"): 1108.8e6,
-    ("many_small", "down_dgrad"): 1130.1e6, ("many_small", "down_wgrad"): 1121.1e6,
-    ("many_small", "gateup_dgrad"): 1725.6e6, ("many_small", "gateup_wgrad"): 1754.2e6,
+    ("fine_grained", "gateup_swiglu"): 1024.7e6, ("fine_grained", "down"): 523.5e6,
+    ("fine_grained", "down_dgrad"): 528.3e6, ("fine_grained", "down_wgrad"): 497.6e6,
+    ("fine_grained", "gateup_dgrad"): 972.5e6, ("fine_grained", "gateup_wgrad"): 939.7e6,
+    ("many_small", "gateup_swiglu"): 1922.2e6, ("many_small", "down"): 1109.4e6,
+    ("many_small", "down_dgrad"): 1130.6e6, ("many_small", "down_wgrad"): 1122.0e6,
+    ("many_small", "gateup_dgrad"): 1726.5e6, ("many_small", "gateup_wgrad"): 1759.7e6,
 }
 
 
