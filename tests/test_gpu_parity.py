@@ -91,8 +91,7 @@ def _check_permute(B, idx_np, E, X_np=None):
 
 @pytest.mark.parametrize("T,E,K,seed", [(1, 1, 1, 0), (5, 3, 2, 1), (256, 8, 2, 2), (1000, 64, 6, 3), (4099, 128, 8, 4),
                                         (300, 1024, 3, 5), (777, 5, 5, 6),
-                                        (4096, 256, 8, 7),      # largest problem of the one-block index kernel
-                                        (4097, 256, 8, 8), (1000, 257, 8, 9)])   # just past it: the two-launch path
+                                        (4096, 256, 8, 7), (4097, 256, 8, 8), (1000, 257, 8, 9)])   # 16+ block-chunks
 def test_permute_indices_random_with_duplicates(B, T, E, K, seed):
     rng = np.random.default_rng(seed)
     idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
