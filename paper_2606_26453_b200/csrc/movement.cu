@@ -38,9 +38,11 @@ __device__ __forceinline__ uint4 pack8(const float f[8]) {
 // ------------------------------------------------------------------------------------------------
 // a1, index part.  Two small kernels over the R = T*K pairs, split into block-chunks of `chunk`
 // consecutive pairs (a multiple of 256; one block per chunk, one eighth of it per warp):
-//   hist : per block-chunk, the number of pairs of each expert                  -> ws[block][e]
+//   hist : per block-chunk, the number of pairs of each expert (shared-memory atomics: counts are
+//          order-free)                                                          -> ws[block][e]
 //   rank : every block sums the histogram rows before it (its base) and all rows (the counts),
-//          turns the counts into offsets, ranks its warps' pairs with match/popc scans:
+//          turns the counts into offsets, ranks its warps' pairs (per-warp counts by atomics, then the
+//          same-expert lane mask of each 32 pairs from 32 broadcasts, and popc):
 //          row(p) = offsets[e] + base[e] + pairs of e in earlier warps of the block + earlier
 //          pairs of e in the same warp.
 // ------------------------------------------------------------------------------------------------
@@ -50,12 +52,11 @@ __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* _
                                                                 int chunk, int32_t* __restrict__ ws) {
     extern __shared__ int32_t smem_i[];
     int32_t* hist = smem_i;   // [E]
-    const int lane = threadIdx.x & 31;
     for (int e = threadIdx.x; e < E; e += kThreads) hist[e] = 0;
     __syncthreads();
     const long long p0 = (long long)blockIdx.x * chunk;
     // chunk is a multiple of kThreads: whole warps stay together.  The indices of kIdxGroup iterations are loaded
-    // first, so that their global-memory latencies overlap instead of adding up in front of every match.
+    // first, so that their global-memory latencies overlap instead of adding up one after the other.
     for (int i0 = threadIdx.x; i0 < chunk; i0 += kThreads * kIdxGroup) {
         int ev[kIdxGroup];
 #pragma unroll
@@ -68,9 +69,7 @@ __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* _
 #pragma unroll
         for (int g = 0; g < kIdxGroup; ++g) {
             if (i0 - (int)threadIdx.x + g * kThreads >= chunk) break;   // block-uniform
-            const int e = ev[g];
-            const unsigned mask = __match_any_sync(0xffffffffu, e);
-            if (e >= 0 && lane == __ffs(mask) - 1) atomicAdd(&hist[e], __popc(mask));   // counts only: order-free
+            if (ev[g] >= 0) atomicAdd(&hist[ev[g]], 1);   // counts only: order-free
         }
     }
     __syncthreads();
@@ -140,10 +139,7 @@ __global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* _
 #pragma unroll
         for (int g = 0; g < kIdxGroup; ++g) {
             if (i0 + g * 32 >= per_warp) break;   // warp-uniform
-            const int e = ev[g];
-            const unsigned mask = __match_any_sync(0xffffffffu, e);
-            if (e >= 0 && lane == __ffs(mask) - 1) mine[e] += __popc(mask);
-            __syncwarp();
+            if (ev[g] >= 0) atomicAdd(&mine[ev[g]], 1);   // counts only: order-free
         }
     }
     __syncthreads();
@@ -179,7 +175,11 @@ __global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* _
             if (i0 + g * 32 >= per_warp) break;   // warp-uniform
             const int e = ev[g];
             const long long p = p0 + i0 + g * 32 + lane;
-            const unsigned mask = __match_any_sync(0xffffffffu, e);
+            // lanes of the warp with the same expert: 32 broadcasts are several times faster than match.any here
+            // (whose time grows with the number of distinct values, and routing makes most of them distinct)
+            unsigned mask = 0;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) mask |= (__shfl_sync(0xffffffffu, e, j) == e ? 1u : 0u) << j;
             if (e >= 0) {
                 const int row = mine[e] + __popc(mask & lt_mask);
                 row_to_pair[row] = (int32_t)p;
