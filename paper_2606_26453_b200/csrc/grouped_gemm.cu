@@ -76,7 +76,10 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 // any height that is a multiple of 16 (up to 256) instead of a fixed 128 / 256: an expert's rows are split into
 // equal tiles and almost no tensor work goes to padding.  The accumulator comes out transposed (lane = feature,
 // column = row); the epilogue transposes it back through its shared-memory staging blocks.
-enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3, FWD_PLAIN_T = 4, DGRAD_T = 5 };
+// FWD_SWIGLU_H is FWD_SWIGLU in pair mode with half-height last tiles (small experts); a kind of its own so that the
+// kernel for large experts carries none of its bookkeeping.
+enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3, FWD_PLAIN_T = 4, DGRAD_T = 5, FWD_SWIGLU_H = 6 };
+__host__ __device__ constexpr bool swiglu(int kind) { return kind == FWD_SWIGLU || kind == FWD_SWIGLU_H; }
 __host__ __device__ constexpr bool swapped(int kind) { return kind == FWD_PLAIN_T || kind == DGRAD_T; }
 constexpr int SWAP_ROWS = 256;   // most rows of a swapped tile
 constexpr int SWAP_FEATS = 128;  // output features of a swapped tile
@@ -108,6 +111,7 @@ struct SharedCtl {
     unsigned long long drain;
     uint32_t tmem_base;
     int abort_flag;
+    int stage_half[MAX_STAGES];   // FWD_SWIGLU pair: the stage belongs to a half-height tile (published by the producer)
     int stage_n[MAX_STAGES];   // swapped kinds: MMA N (rows of the tile rounded up to 16) of the tile a stage belongs to
     int32_t offs[MAX_E + 1];
     int32_t tile_prefix[MAX_E + 1];
@@ -345,6 +349,7 @@ struct Tile {
     int k_row0;   // WGRAD: first packed row of the contraction
     int k_rows;   // WGRAD: rows of the contraction
     int rows;     // swapped kinds: rows of this tile (1..256)
+    int half;     // FWD_SWIGLU pair: the tile holds <= 128 rows and runs as a 128-row pair tile (64 rows per CTA)
 };
 
 // Order of an expert's m_tiles x n_tiles output tiles: bands of RASTER_BAND row tiles; inside a band
@@ -402,6 +407,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
         tl.k_blocks = (tl.k_rows + BK - 1) / BK;
         tl.row_end = 0;
         tl.rows = 0;
+        tl.half = 0;
     } else {
         // tile_prefix[e] = number of TILE_M-row tiles of experts < e
         int lo = 0, hi = p.E;                          // largest e with tile_prefix[e]*n_tiles <= t
@@ -427,6 +433,7 @@ __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ct
             tl.row0 = ctl->offs[lo] + mt * TILE_M;
             tl.n0 = nt * BN;
         }
+        tl.half = (KIND == FWD_SWIGLU_H && tl.row_end - tl.row0 <= BM) ? 1 : 0;
         tl.k_blocks = p.k_blocks;
         tl.k_row0 = 0;
         tl.k_rows = 0;
@@ -487,7 +494,10 @@ __device__ __forceinline__ void stage_loads(const Tile& tl, int kb, const Params
         tma_load_3d(a_dst, map_a, 0, krow, (tl.row0 + my_rows) >> 6, full);
         tma_load_3d(b_dst, map_b0, 0, krow, n_local >> 6, full);
     } else {
-        tma_load_2d(a_dst, map_a, kb * BK, tl.row0 + my_rows, full);
+        // half-height pair tile (FWD_SWIGLU): rows [row0, row0+64) in the first CTA, [row0+64, row0+128) in the second;
+        // map_r1 is the A map with a 64-row box there
+        if (KIND == FWD_SWIGLU_H && tl.half) tma_load_2d(a_dst, map_r1, kb * BK, tl.row0 + (int)rank * (BM / 2), full);
+        else tma_load_2d(a_dst, map_a, kb * BK, tl.row0 + my_rows, full);
         if (KIND == DGRAD) {
             const bool second = kb >= p.k_split;
             const int kx = (second ? kb - p.k_split : kb) * BK;
@@ -498,8 +508,22 @@ __device__ __forceinline__ void stage_loads(const Tile& tl, int kb, const Params
         } else {  // FWD_SWIGLU: 128 gate columns then 128 up columns
             const int ky = tl.e * p.b_rows_per_e + kb * BK;
             const int ng = tl.n0 >> 1;   // n0 counts fused (gate+up) columns
-            if (PAIR) {                  // first CTA holds the gate half of B, second the up half
-                tma_load_3d(b_dst, rank == 0 ? map_b0 : map_b1, 0, ky, ng >> 6, full);
+            if (PAIR) {
+                // pair mode with half-height tiles (small experts): the maps have one-chunk (64-column) boxes.  Full tile: the first CTA holds the 128 gate
+                // columns of B, the second the 128 up columns.  Half tile: the accumulator of an M = 128 pair MMA
+                // keeps columns 0..127 in lanes 0..63 and columns 128..255 in lanes 64..127, and gate and up of a
+                // feature must meet in one lane: each CTA holds [64 gate | 64 up] columns of the same 64 features.
+                const int c = ng >> 6;
+                const CUtensorMap* mb = rank == 0 ? map_b0 : map_b1;
+                if (KIND != FWD_SWIGLU_H) {   // large experts: two-chunk boxes, one load
+                    tma_load_3d(b_dst, mb, 0, ky, c, full);
+                } else if (tl.half) {
+                    tma_load_3d(b_dst, map_b0, 0, ky, c + (int)rank, full);
+                    tma_load_3d(b_dst + CHUNK_BYTES, map_b1, 0, ky, c + (int)rank, full);
+                } else {
+                    tma_load_3d(b_dst, mb, 0, ky, c, full);
+                    tma_load_3d(b_dst + CHUNK_BYTES, mb, 0, ky, c + 1, full);
+                }
             } else {
                 tma_load_3d(b_dst, map_b0, 0, ky, ng >> 6, full);
                 tma_load_3d(b_dst + 2 * CHUNK_BYTES, map_b1, 0, ky, ng >> 6, full);
@@ -523,11 +547,16 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     constexpr int STAGES = G::STAGES;
     constexpr int STAGE_BYTES = G::STAGE_BYTES;
     constexpr bool SWAP = swapped(KIND);
+    // SwiGLU forward in pair mode: an expert's last <= 128 rows run as a half-height tile (tcgen05.mma M = 128 over the
+    // pair, 64 rows per CTA, half the MMA time) instead of a padded 256-row tile
+    constexpr bool HALF_TILES = (KIND == FWD_SWIGLU_H);
+    static_assert(!HALF_TILES || PAIR, "half-height tiles exist in pair mode only");
     constexpr int ROW_TILE = SWAP ? SWAP_ROWS : G::TILE_M;   // rows an expert's tile count is computed from
     // operand major-ness of the MMA's M side (A) and N side (B); for the swapped kinds A is the weight tile
     constexpr bool A_MN = (KIND == WGRAD || KIND == FWD_PLAIN_T);
-    constexpr bool B_MN = (KIND == FWD_SWIGLU || KIND == FWD_PLAIN || KIND == WGRAD);
+    constexpr bool B_MN = (swiglu(KIND) || KIND == FWD_PLAIN || KIND == WGRAD);
     constexpr uint32_t IDESC = make_idesc(G::TILE_M, BN, A_MN, B_MN);
+    constexpr uint32_t IDESC_HALF = make_idesc(BM, BN, A_MN, B_MN);   // 128 x 256 over the CTA pair
     constexpr uint32_t A_KSTEP = A_MN ? 2048 : 32;   // bytes per 16 k inside a stage
     constexpr uint32_t B_KSTEP = B_MN ? 2048 : 32;
     constexpr int STAGE_CHUNKS = BM / 64 + G::BN_LOCAL / 64;   // 64-wide MN-major blocks per stage (WGRAD)
@@ -629,6 +658,9 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         const int my_n = PAIR ? (((tl.rows + 15) & ~15) >> 1) : tl.rows;
                         constexpr int BOX = PAIR ? 32 : 64;
                         mbar_arrive_expect_tx(land, G::A_BYTES + min(4, (my_n + BOX - 1) / BOX) * (BOX * BK * 2));
+                    } else if (HALF_TILES) {
+                        ctl->stage_half[stage] = tl.half;   // read by the MMA thread after its wait on full[stage]
+                        mbar_arrive_expect_tx(land, tl.half ? STAGE_BYTES - G::A_BYTES / 2 : STAGE_BYTES);
                     } else {
                         mbar_arrive_expect_tx(land, STAGE_BYTES);
                     }
@@ -681,6 +713,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 tc_fence_after();
                 // swapped kinds: the MMA's N is the tile's row count (rounded up to 16), published with each stage
                 if (SWAP && first_block) idesc = make_idesc(G::TILE_M, ctl->stage_n[stage], A_MN, B_MN);
+                if (HALF_TILES && first_block) idesc = ctl->stage_half[stage] ? IDESC_HALF : IDESC;
                 const uint32_t a_base = tiles_base + stage * STAGE_BYTES;
                 const uint64_t a_desc = make_smem_desc<A_MN>(a_base);
                 const uint64_t b_desc = make_smem_desc<B_MN>(a_base + G::A_BYTES);
@@ -692,7 +725,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                                         b_desc + (uint64_t)((kk * B_KSTEP) >> 4), IDESC, accumulate, kk < n_mma ? 1u : 0u);
                     else
                         tc_mma<PAIR>(d_tmem, a_desc + (uint64_t)((kk * A_KSTEP) >> 4),
-                                     b_desc + (uint64_t)((kk * B_KSTEP) >> 4), SWAP ? idesc : IDESC, accumulate);
+                                     b_desc + (uint64_t)((kk * B_KSTEP) >> 4), (SWAP || HALF_TILES) ? idesc : IDESC, accumulate);
                 }
                 tc_commit<PAIR>(smem_u32(&ctl->empty[stage]));
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -845,7 +878,11 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + acc * BN + ((uint32_t)(quarter * 32) << 16);
-            const int slab0 = tl.row0 + my_rows + quarter * 32;       // first row of this warp's slab
+            // first row of this warp's slab.  Half-height pair tile (FWD_SWIGLU, M = 128 over two CTAs): this CTA holds
+            // 64 rows; tensor-memory lanes 0..63 carry them for the MMA's columns 0..127, lanes 64..127 carry the same
+            // rows for columns 128..255 (128 tensor-memory columns per accumulator instead of 256).
+            const bool half_tile = HALF_TILES && tl.half;
+            const int slab0 = half_tile ? tl.row0 + (int)rank * (BM / 2) + (quarter & 1) * 32 : tl.row0 + my_rows + quarter * 32;
             // rows of the slab that are owed: inside the expert (row-ragged kinds) / inside M (WGRAD); 32 = whole slab
             const int rows_valid = (KIND == WGRAD) ? (slab0 < p.m_rows ? 32 : 0) : max(0, min(32, tl.row_end - slab0));
             const int slab_y = (KIND == WGRAD) ? tl.e * p.m_rows + slab0 : slab0;
@@ -872,15 +909,20 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                                 p.out0[(long long)(r0 + j) * p.ldo + feat0 + lane] = __float2bfloat16_rn(__uint_as_float(v[j]));
                     }
                 }
-            } else if (KIND == FWD_SWIGLU) {
+            } else if (swiglu(KIND)) {
                 const int ng = tl.n0 >> 1;
+                // full tile: gate in tensor-memory columns 0..127, up in 128..255, this warp takes two 32-column blocks.
+                // half tile: this lane group's 64 features: gate in columns 0..63, up in 64..127, one block per warp.
+                const int c_begin = half_tile ? half : 2 * half, c_end = half_tile ? half + 1 : 2 * half + 2;
+                const int u_off = half_tile ? 64 : 128;
+                const int x_base = ng + (half_tile ? (quarter >> 1) * 64 : 0);
 #pragma unroll 1
-                for (int c = 2 * half; c < 2 * half + 2; ++c) {
+                for (int c = c_begin; c < c_end; ++c) {
                     uint32_t g[32], u[32];
                     tc_ld32(taddr + c * 32, g);
-                    tc_ld32(taddr + 128 + c * 32, u);
+                    tc_ld32(taddr + u_off + c * 32, u);
                     tc_wait_ld();
-                    if (rows_valid == 0 || ng + c * 32 >= p.I) continue;   // past the expert's rows / past column I
+                    if (rows_valid == 0 || x_base + c * 32 >= p.I) continue;   // past the expert's rows / past column I
                     uint32_t hp[16], gp[16], up[16];
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
@@ -892,7 +934,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         gp[j] = pack_bf16(g0, g1);
                         up[j] = pack_bf16(u0, u1);
                     }
-                    const int x = ng + c * 32;
+                    const int x = x_base + c * 32;
                     if (rows_valid == 32) {
                         stage_and_store(hp, &map_o0, x, slab_y);
                         if (p.gu) {
@@ -1101,16 +1143,18 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
     return check_launch();
 }
 
-// Fixed-height CTA-pair tiles (256 rows) are used when experts hold at least 512 rows on average: below that the
-// padding of each expert's last tile costs more than the halved operand traffic buys.  The SwiGLU forward then
-// runs single-CTA 128-row tiles, the plain row-ragged GEMMs the swapped kinds (next comment).
-bool use_pairs_for_rows(const moe_dims_t& d) { return (long long)d.T * d.K >= 512ll * d.E; }
 // The plain row-ragged GEMMs (down forward, down dgrad, gate/up dgrad) run with swapped operand roles -- always as
 // CTA pairs: 256 output features x up to 256 rows per tile -- when experts hold fewer than 512 rows on average:
 // there the fixed 128-row tiles lose 10-15 % of the tensor work to padding (measured: +2-5 % per kernel on the
 // 384- and 451-rows-per-expert workloads).  With larger experts the padding is small and the fixed-height tiles
 // are as fast or faster (the swapped kernels' issue thread, not the tensor pipe, bounds tiles of fewer than 256 rows).
 bool use_swapped(const moe_dims_t& d) { return (long long)d.T * d.K < 512ll * d.E; }
+// The SwiGLU forward has no swapped form (measured slower: two accumulators per tile).  Its pair kernel runs an
+// expert's last <= 128 rows as a half-height tile, which makes pairs worthwhile from MOE_SWIGLU_PAIR_ROWS rows per expert.
+#ifndef MOE_SWIGLU_PAIR_ROWS
+#define MOE_SWIGLU_PAIR_ROWS 320
+#endif
+bool use_pairs_for_swiglu(const moe_dims_t& d) { return (long long)d.T * d.K >= (long long)MOE_SWIGLU_PAIR_ROWS * d.E; }
 // Weight gradients have no row padding to lose, so pairs already win from 256 rows per expert.
 bool use_pairs_for_wgrad(const moe_dims_t& d) { return (long long)d.T * d.K >= 256ll * d.E; }
 
@@ -1121,17 +1165,24 @@ bool use_pairs_for_wgrad(const moe_dims_t& d) { return (long long)d.T * d.K >= 2
 int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gate, const bf16* w_up,
                       const int32_t* offsets, bf16* h_act, bf16* gu, cudaStream_t s) {
     const uint64_t R = (uint64_t)d.T * d.K;
-    CUtensorMap a, b0, b1, o0, o1;
-    if (!make_map(&a, x_perm, d.H, R, BK, BM) || !make_map_mn(&b0, w_gate, d.I, (uint64_t)d.E * d.H, 2) ||
-        !make_map_mn(&b1, w_up, d.I, (uint64_t)d.E * d.H, 2) || !make_out_map(&o0, h_act, d.I, R) ||
+    const bool pair = use_pairs_for_swiglu(d);
+    // pair mode with small experts (fewer than 512 rows on average): an expert's last <= 128 rows run as a half-height
+    // tile; that takes one-chunk weight boxes (a half-height tile mixes gate and up chunks per CTA) and a second A map
+    // with a 64-row box.  With larger experts the padding is small and the two-chunk boxes (one load less per stage)
+    // are 2-4 % faster.
+    const bool half_tiles = pair && use_swapped(d);
+    CUtensorMap a, ah, b0, b1, o0, o1;
+    if (!make_map(&a, x_perm, d.H, R, BK, BM) || !make_map(&ah, x_perm, d.H, R, BK, BM / 2) ||
+        !make_map_mn(&b0, w_gate, d.I, (uint64_t)d.E * d.H, half_tiles ? 1 : 2) ||
+        !make_map_mn(&b1, w_up, d.I, (uint64_t)d.E * d.H, half_tiles ? 1 : 2) || !make_out_map(&o0, h_act, d.I, R) ||
         !make_out_map(&o1, gu ? gu : h_act, gu ? 2ull * d.I : d.I, R))
         return MOE_ERR_CUDA;
     Params p = {};
     p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
     p.n_tiles = (d.I + 127) / 128; p.n_cols = 2 * d.I; p.b_rows_per_e = d.H;
     p.out0 = h_act; p.gu = gu; p.I = d.I; p.ldo = d.I; p.n_split = 2 * d.I;
-    return use_pairs_for_rows(d) ? launch<FWD_SWIGLU, true>(a, b0, b1, o0, o1, a, p, s)
-                                 : launch<FWD_SWIGLU, false>(a, b0, b1, o0, o1, a, p, s);
+    if (half_tiles) return launch<FWD_SWIGLU_H, true>(a, b0, b1, o0, o1, ah, p, s);
+    return pair ? launch<FWD_SWIGLU, true>(a, b0, b1, o0, o1, a, p, s) : launch<FWD_SWIGLU, false>(a, b0, b1, o0, o1, a, p, s);
 }
 
 // Down forward: A = h_act [R,I]; B = w_down viewed as [E*I, H].
