@@ -38,12 +38,12 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of each grouped-GEMM kernel, from the
 # ncu captures summarised in profiles/ncu_full_<workload>.md.  Workloads without a capture report null.
 NCU_TRAFFIC_BYTES = {
-    ("fine_grained", "gateup_swiglu"): 1024.7e6, ("fine_grained", "down"): 523.5e6,
-    ("fine_grained", "down_dgrad"): 528.3e6, ("fine_grained", "down_wgrad"): 497.6e6,
-    ("fine_grained", "gateup_dgrad"): 972.5e6, ("fine_grained", "gateup_wgrad"): 939.7e6,
-    ("many_small", "gateup_swiglu"): 1922.2e6, ("many_small", "down"): 1109.4e6,
-    ("many_small", "down_dgrad"): 1130.6e6, ("many_small", "down_wgrad"): 1122.0e6,
-    ("many_small", "gateup_dgrad"): 1726.5e6, ("many_small", "gateup_wgrad"): 1759.7e6,
+    ("fine_grained", "gateup_swiglu"): 1025.5e6, ("fine_grained", "down"): 522.5e6,
+    ("fine_grained", "down_dgrad"): 528.9e6, ("fine_grained", "down_wgrad"): 496.4e6,
+    ("fine_grained", "gateup_dgrad"): 973.3e6, ("fine_grained", "gateup_wgrad"): 942.8e6,
+    ("many_small", "gateup_swiglu"): 1924.5e6, ("many_small", "down"): 1107.7e6,
+    ("many_small", "down_dgrad"): 1131.1e6, ("many_small", "down_wgrad"): 1120.7e6,
+    ("many_small", "gateup_dgrad"): 1725.9e6, ("many_small", "gateup_wgrad"): 1757.2e6,
 }
 
 
