@@ -458,7 +458,9 @@ def run_ours(args):
         "e2e": {"value": aggregate_tflops(world, cfg.flops_fwd_bwd, e2e_ms_max), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_max,
                 "note": "moe_layer_fwd_bwd_host: activations, routing and upstream gradient from pinned host "
-                        "memory each step; weights and weight gradients stay on the device"},
+                        "memory each step, results read back each step; weights and weight gradients stay on the "
+                        "device; the copies run on side streams and, with steps following one another, under the "
+                        "neighbouring steps' GEMMs"},
         "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline_object(cfg, res, peaks, peaks_kind),
         "pct_of_dense_bf16_peak_nominal": 100.0 * summary["gemm_frac_of_nominal_2250"],

@@ -203,14 +203,19 @@ int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const f
  * into the device arena, runs a1..a8, and copies y [T,H], dx [T,H] (bf16) and dtopk_w [T,K]
  * (fp32) back to HOST pointers.  Weights w_* and weight gradients dw_* are DEVICE pointers (the
  * parameters stay resident, as in training).  `arena` is device scratch of at least
- * moe_layer_arena_bytes(dims) bytes holding every intermediate of the step.  The kernels and
- * most copies are enqueued on `stream`; the upload of dy and the downloads of y, dx and dtopk_w run on
- * one internal copy stream per device (created on the first call, the only CUDA object the
- * library ever creates) so that they overlap the forward pass, the backward pass and the two
- * weight-gradient GEMMs (which run last: nothing downstream waits for them), and are tied to `stream` with
- * events in both directions: the call behaves as if everything were on `stream`, and the host
- * results are valid after the caller synchronises it.  Not safe to call from two host threads at
- * once on the same device. */
+ * moe_layer_arena_bytes(dims) bytes holding every intermediate of the step.  The kernels are
+ * enqueued on `stream`; the uploads and the downloads run on two internal copy streams per
+ * device (created on the first call, the only CUDA objects the library ever creates), tied to
+ * `stream` with events: y comes down under the backward pass, dx and dtopk_w under the two
+ * weight-gradient GEMMs (which run last: nothing downstream waits for them), and the uploads of a
+ * call start as soon as the PREVIOUS call's last reader of the arena's input blocks is done, so
+ * that back-to-back calls overlap the next step's uploads with this step's backward GEMMs.
+ * Consequences for the caller: (1) the host results are valid after `stream` is synchronised;
+ * (2) the host INPUT buffers are read from the moment of the call on, not in stream order: they
+ * must hold their final values when the function is called and stay untouched until `stream`
+ * has passed this call; (3) successive calls that share an arena must be made on the same stream;
+ * (4) the first call on a device orders its uploads after all work already on `stream`.
+ * Not safe to call from two host threads at once on the same device. */
 size_t moe_layer_arena_bytes(const moe_dims_t* dims);
 int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int32_t* topk_idx_host,
                            const float* topk_w_host, const void* dy_host, const void* w_gate,

@@ -228,12 +228,14 @@ int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const f
 
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).
 namespace {
-// One side stream and five events per device for moe_layer_fwd_bwd_host, created on first use and kept for
-// the life of the process (the one place where the library creates CUDA objects of its own).
+// Two side streams (uploads, downloads) and a few events per device for moe_layer_fwd_bwd_host, created on first
+// use and kept for the life of the process (the one place where the library creates CUDA objects of its own).
 struct HostCopyLane {
-    cudaStream_t stream;
-    cudaEvent_t begin, dy_up, y_ready, dx_ready, down_done;
+    cudaStream_t stream;      // downloads
+    cudaStream_t up_stream;   // uploads
+    cudaEvent_t begin, x_up, dy_up, y_ready, dx_ready, down_done, inputs_free;
     bool ready;
+    bool primed;              // inputs_free has been recorded by an earlier call
 };
 HostCopyLane* host_copy_lane() {
     static HostCopyLane lanes[64] = {};
@@ -242,7 +244,8 @@ HostCopyLane* host_copy_lane() {
     HostCopyLane& l = lanes[dev];
     if (!l.ready) {
         if (cudaStreamCreateWithFlags(&l.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-        cudaEvent_t* evs[5] = {&l.begin, &l.dy_up, &l.y_ready, &l.dx_ready, &l.down_done};
+        if (cudaStreamCreateWithFlags(&l.up_stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+        cudaEvent_t* evs[7] = {&l.begin, &l.x_up, &l.dy_up, &l.y_ready, &l.dx_ready, &l.down_done, &l.inputs_free};
         for (cudaEvent_t* e : evs)
             if (cudaEventCreateWithFlags(e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
         l.ready = true;
@@ -294,18 +297,27 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
     auto P = [&](size_t off) { return static_cast<void*>(base + off); };
     auto Pi = [&](size_t off) { return reinterpret_cast<int32_t*>(base + off); };
 
-    // Side stream for the copies that can overlap compute: dy goes up while the forward pass runs, y comes
-    // down while the backward pass runs, dx and dtopk_w come down under the last weight-gradient GEMM.  Everything is ordered against the caller's stream with events.
+    // Side streams for the copies, so that they overlap compute: y comes down while the backward pass runs, dx and
+    // dtopk_w come down under the two weight-gradient GEMMs, and the uploads of a call wait only until the PREVIOUS
+    // call's last reader of the input blocks of the arena (its combine-backward) is done -- when calls follow one
+    // another, the next call's x, routing and dy travel to the device under this call's backward GEMMs.  The first
+    // call on a device orders its uploads after everything already on the caller's stream.  Everything else is
+    // ordered against the caller's stream with events.
     HostCopyLane* lane = host_copy_lane();
     if (lane == nullptr) return MOE_ERR_CUDA;
-    cudaStream_t c = lane->stream;
-    if (cudaEventRecord(lane->begin, s) != cudaSuccess || cudaStreamWaitEvent(c, lane->begin, 0) != cudaSuccess ||
-        cudaMemcpyAsync(P(a.dy), dy_host, T * H * 2, cudaMemcpyHostToDevice, c) != cudaSuccess ||
-        cudaEventRecord(lane->dy_up, c) != cudaSuccess)
-        return MOE_ERR_CUDA;
-    if (cudaMemcpyAsync(P(a.x), x_host, T * H * 2, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(P(a.idx), topk_idx_host, R * 4, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(P(a.w), topk_w_host, R * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    cudaStream_t c = lane->stream, u = lane->up_stream;
+    if (lane->primed) {
+        if (cudaStreamWaitEvent(u, lane->inputs_free, 0) != cudaSuccess) return MOE_ERR_CUDA;
+    } else {
+        if (cudaEventRecord(lane->begin, s) != cudaSuccess || cudaStreamWaitEvent(u, lane->begin, 0) != cudaSuccess)
+            return MOE_ERR_CUDA;
+    }
+    if (cudaMemcpyAsync(P(a.x), x_host, T * H * 2, cudaMemcpyHostToDevice, u) != cudaSuccess ||
+        cudaMemcpyAsync(P(a.idx), topk_idx_host, R * 4, cudaMemcpyHostToDevice, u) != cudaSuccess ||
+        cudaMemcpyAsync(P(a.w), topk_w_host, R * 4, cudaMemcpyHostToDevice, u) != cudaSuccess ||
+        cudaEventRecord(lane->x_up, u) != cudaSuccess ||
+        cudaMemcpyAsync(P(a.dy), dy_host, T * H * 2, cudaMemcpyHostToDevice, u) != cudaSuccess ||
+        cudaEventRecord(lane->dy_up, u) != cudaSuccess || cudaStreamWaitEvent(s, lane->x_up, 0) != cudaSuccess)
         return MOE_ERR_CUDA;
 
     int rc;
@@ -321,6 +333,9 @@ int moe_layer_fwd_bwd_host(const moe_dims_t* dims, const void* x_host, const int
         return MOE_ERR_CUDA;
     MOE_STEP(moe_unpermute_combine_bwd(dims, P(a.dy), P(a.yp), reinterpret_cast<float*>(base + a.w), Pi(a.p2r),
                                        P(a.dyp), reinterpret_cast<float*>(base + a.dw), stream));
+    // x, routing and dy have been read for the last time: a following call may overwrite them from here on
+    if (cudaEventRecord(lane->inputs_free, s) != cudaSuccess) return MOE_ERR_CUDA;
+    lane->primed = true;
     // backward in pieces: the whole data-gradient chain first, so that dx can travel to the host while the two
     // weight-gradient GEMMs (which nothing downstream waits for) are still running
     MOE_STEP(moe_grouped_gemm_down_dgrad(dims, P(a.dyp), w_down, Pi(a.offsets), P(a.dhact), stream));

@@ -336,6 +336,41 @@ def test_host_entry_point_matches_device_chain(B):
     assert torch.equal(dwg, b2.dw_gate) and torch.equal(dwd, b2.dw_down)
 
 
+def test_host_entry_point_pipelines_different_steps(B):
+    """Four calls in a row, each with its own host inputs, routing and host outputs, no synchronisation in between:
+    the uploads of a call run under the previous call's backward pass, and every call must still give exactly
+    the device chain's results for ITS inputs (a stress of the event ordering around the shared arena)."""
+    cfg, base = Hh.ragged_workload([600, 540, 0, 700], K=2, H=320, I=192, seed=11)   # large enough to overlap for real
+    d = _dims(B, cfg)
+    arena = torch.empty(B.moe_layer_arena_bytes(d), dtype=torch.uint8, device="cuda")
+    dev0 = Hh.device_workload(base)
+    pin = lambda t: t.cpu().pin_memory()
+    rng = np.random.default_rng(3)
+    steps = []
+    for i in range(4):
+        scale = float(2.0 ** (i - 1))
+        x = (dev0["X"].float() * scale).to(torch.bfloat16)
+        dy = (dev0["dY"].float() / scale).to(torch.bfloat16)
+        idx = dev0["topk_idx"].cpu().numpy().copy()
+        if i % 2:                                        # another routing on odd steps: expert ids mirrored
+            idx = (cfg.E - 1 - idx).astype(np.int32)
+        dev = dict(dev0, X=x, dY=dy, topk_idx=torch.from_numpy(idx).cuda())
+        out = dict(y=torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16).pin_memory(),
+                   dx=torch.empty((cfg.T, cfg.H), dtype=torch.bfloat16).pin_memory(),
+                   dw=torch.empty((cfg.T, cfg.K), dtype=torch.float32).pin_memory(),
+                   dwg=torch.empty_like(dev0["W_gate"]), dwu=torch.empty_like(dev0["W_up"]),
+                   dwd=torch.empty_like(dev0["W_down"]))
+        steps.append((dev, dict(x=pin(x), idx=pin(dev["topk_idx"]), w=pin(dev["topk_w"]), dy=pin(dy)), out))
+    for dev, h, o in steps:
+        B.moe_layer_fwd_bwd_host(d, h["x"], h["idx"], h["w"], h["dy"], dev["W_gate"], dev["W_up"], dev["W_down"],
+                                 o["y"], o["dx"], o["dw"], o["dwg"], o["dwu"], o["dwd"], arena)
+    torch.cuda.synchronize()
+    for dev, h, o in steps:
+        b = Hh.run_cuda_layer(dev, cfg.E)
+        assert torch.equal(o["y"], b.y.cpu()) and torch.equal(o["dx"], b.dx.cpu()) and torch.equal(o["dw"], b.dtopk_w.cpu())
+        assert torch.equal(o["dwg"], b.dw_gate) and torch.equal(o["dwu"], b.dw_up) and torch.equal(o["dwd"], b.dw_down)
+
+
 # ------------------------------------------------------------------------------------------------
 # degenerate shapes: a single expert, top-1, fewer rows than one tile, one token, many experts
 # ------------------------------------------------------------------------------------------------
