@@ -231,6 +231,27 @@ def time_router(B, cfg, device, reps=30):
     return out
 
 
+def time_sustained(B, cfg, res, device, seconds=2.0):
+    """The same step run back to back for at least `seconds` (the way the measured cuBLAS sustained peak was
+    taken), so that the power and thermal state of a long run shows: steps in batches of 20 between two events."""
+    step = make_step(B, res["buffers"], res["wl"])
+    sampler = ClockSampler(device.index if device.index is not None else 0)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    done, ms = 0, 0.0
+    while ms < seconds * 1e3 and done < 200000:
+        e0.record()
+        for _ in range(20):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms += e0.elapsed_time(e1)
+        done += 20
+    clocks = sampler.stop()
+    return {"seconds": ms * 1e-3, "steps": done, "ms_per_step": ms / done,
+            "value": cfg.flops_fwd_bwd / (ms / done * 1e-3) / 1e12, "unit": UNIT, "clocks": clocks}
+
+
 def summarize(cfg, res, steps, peaks):
     ms_step = res["total_ms"] / steps
     pc = res["per_call_ms"]
@@ -472,6 +493,7 @@ def run_ours(args):
     if rank == 0 and world == 1:
         extra = []
         wl_host = host_copy(res["wl"]) if not args.no_cpu_baseline else None
+        line["sustained"] = time_sustained(B, cfg, res, device)
         del res
         torch.cuda.empty_cache()
         for name in args.also:
