@@ -376,7 +376,8 @@ def test_host_entry_point_pipelines_different_steps(B):
 # ------------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("T,H,I,E,K", [(1, 128, 128, 1, 1), (3, 128, 128, 4, 2), (130, 256, 128, 1, 1),
                                        (64, 128, 256, 300, 4), (40, 384, 128, 33, 32), (513, 128, 128, 2, 1),
-                                       (70, 64, 64, 3, 2), (700, 64, 192, 2, 2), (1200, 192, 64, 2, 1)])   # smallest H, I
+                                       (70, 64, 64, 3, 2), (700, 64, 192, 2, 2), (1200, 192, 64, 2, 1),    # smallest H, I
+                                       (1500, 128, 128, 1024, 2)])                                         # most experts
 def test_degenerate_shapes_end_to_end(B, T, H, I, E, K):
     cfg = W.MoeConfig("deg", T=T, H=H, I=I, E=E, K=K, routing="softmax", cfg_id=70 + T % 7)
     host = W.make_workload(cfg)
