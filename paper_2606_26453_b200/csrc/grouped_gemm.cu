@@ -31,6 +31,10 @@
 // Two ragged shapes occur:
 //   row-ragged (forward, dgrad): output rows are the packed rows of an expert.  A tile starts at
 //     offsets[e] + TILE_M*i; loading past the expert's last row is harmless, stores are clipped.
+//     With small experts the padding of the fixed-height tiles is a sizeable share of the tensor
+//     work; two pair variants avoid it: the swapped kinds (FWD_PLAIN_T, DGRAD_T: weights on the M
+//     side of the MMA, the expert's rows on the N side, any tile height that is a multiple of 16)
+//     and, for the SwiGLU forward, half-height last tiles (FWD_SWIGLU_H: M = 128 over the pair).
 //   contraction-ragged (wgrad; the paper's dW1_e = X_e^T G_e): the expert's rows are the
 //     contraction.  The last K block issues only ceil(rem/16) MMAs (guard predicates) and the < 16
 //     surplus rows are zeroed in shared memory first, by the tail-fix warp (first CTA) and the relay
