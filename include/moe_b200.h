@@ -213,7 +213,9 @@ int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const f
  * Consequences for the caller: (1) the host results are valid after `stream` is synchronised;
  * (2) the host INPUT buffers are read from the moment of the call on, not in stream order: they
  * must hold their final values when the function is called and stay untouched until `stream`
- * has passed this call; (3) successive calls that share an arena must be made on the same stream;
+ * has passed this call; (3) successive calls that share an arena must be made on the same stream,
+ * and nothing else may write to the arena between them (the uploads of a call do not wait for
+ * other work on `stream`);
  * (4) the first call on a device orders its uploads after all work already on `stream`.
  * Not safe to call from two host threads at once on the same device. */
 size_t moe_layer_arena_bytes(const moe_dims_t* dims);
