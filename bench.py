@@ -5,10 +5,14 @@
 
 A step is one pass of the whole hot path (route-permute, gate/up GEMM + SwiGLU, down GEMM,
 unpermute-combine, and the four backward calls) over one batch of seeded synthetic input.  The
-metric is whole-layer throughput in TFLOP/s on the algorithmic work 18*R*H*I; the JSON line also
-carries the grouped-GEMM-only throughput, the permute bandwidth, a roofline object for the
-dominant kernel, an end-to-end number through the host-buffer entry point and the fp64 oracle
-timed on the host cores.  With N > 1 (torchrun) every rank runs an independent replica of the
+headline workload is the largest of the five configurations ("imbalanced"); it is timed for at
+least one second (the number of timed steps is raised above --steps when needed, and the line says
+how many were timed).  The metric is whole-layer throughput in TFLOP/s on the algorithmic work
+18*R*H*I; the JSON line also carries the grouped-GEMM-only throughput, the permute bandwidth, a
+roofline object for the dominant kernel, an end-to-end number through the host-buffer entry point,
+the same step run back to back for two seconds, and the fp64 oracle timed on the host cores -- all
+on that workload.  The other workloads follow in `other_configs`, each timed for at least half a
+second with its own roofline object.  With N > 1 (torchrun) every rank runs an independent replica of the
 same workload: the layer is single-GPU by design, there is no collective on the data path.
 `--impl reference` times the CPU oracle alone on a bounded sample of the same workload.
 """
@@ -35,16 +39,14 @@ UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of each grouped-GEMM kernel, from the
-# ncu captures summarised in profiles/ncu_full_<workload>.md.  Workloads without a capture report null.
-NCU_TRAFFIC_BYTES = {
-    ("fine_grained", "gateup_swiglu"): 1025.5e6, ("fine_grained", "down"): 522.5e6,
-    ("fine_grained", "down_dgrad"): 528.9e6, ("fine_grained", "down_wgrad"): 496.4e6,
-    ("fine_grained", "gateup_dgrad"): 973.3e6, ("fine_grained", "gateup_wgrad"): 942.8e6,
-    ("many_small", "gateup_swiglu"): 1924.5e6, ("many_small", "down"): 1107.7e6,
-    ("many_small", "down_dgrad"): 1131.1e6, ("many_small", "down_wgrad"): 1120.7e6,
-    ("many_small", "gateup_dgrad"): 1725.9e6, ("many_small", "gateup_wgrad"): 1757.2e6,
-}
+# Tensor-pipe rate of one SM per clock (a 128x256x16 bf16 tcgen05.mma retires in 128 cycles: measured with a bare
+# issue loop), used for the clock-normalised fractions.
+PIPE_FLOP_PER_CLK_PER_SM = 8192.0
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a workload's dominant grouped-GEMM
+# kernel, from one ncu capture on a SCALED copy of the workload (tokens and experts divided by `scale`, same H, I,
+# top-k, routing law and rows per expert), multiplied by `scale`: every operand and result of these kernels grows in
+# proportion.  (workload, call) -> (bytes per full launch, how it was obtained); absent -> null.
+NCU_TRAFFIC = {}
 
 
 def load_peaks():
@@ -167,7 +169,10 @@ def make_step(B, b, wl):
     return step
 
 
-def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True):
+def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True, min_seconds=0.0):
+    """Warm-up, then `steps` timed steps between two events (CUDA events around every call inside).  With
+    min_seconds > 0 the step count is raised until the timed region lasts at least that long (estimated from three
+    untimed steps after the warm-up; the maximum over ranks, so that every rank times the same count)."""
     wl = W.make_workload_device(cfg, device)
     b = B.alloc_layer_buffers(cfg.T, cfg.H, cfg.I, cfg.E, cfg.K, device=device)
     step = make_step(B, b, wl)
@@ -176,6 +181,15 @@ def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True):
     torch.cuda.synchronize()
     if B.moe_device_status() != 0:
         raise RuntimeError("device status word is set after warm-up")
+    if min_seconds > 0.0:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(3):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        est_ms = max_over_ranks([e0.elapsed_time(e1) / 3.0], dist, device)[0]
+        steps = max(steps, int(min_seconds * 1e3 / est_ms * 0.98) + 1)   # a step in a long run is a little slower than est
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(steps)]
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(device.index if device.index is not None else 0) if sample_clocks else None
@@ -198,7 +212,7 @@ def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True):
         per_call[name] = sum(evs[s][i].elapsed_time(evs[s][i + 1]) for s in range(steps)) / steps
     if B.moe_device_status() != 0:
         raise RuntimeError("device status word is set after the timed region")
-    return dict(wl=wl, buffers=b, total_ms=total_ms, per_call_ms=per_call, clocks=clocks)
+    return dict(wl=wl, buffers=b, total_ms=total_ms, per_call_ms=per_call, clocks=clocks, steps=steps)
 
 
 def time_router(B, cfg, device, reps=30):
@@ -252,46 +266,77 @@ def time_sustained(B, cfg, res, device, seconds=2.0):
             "value": cfg.flops_fwd_bwd / (ms / done * 1e-3) / 1e12, "unit": UNIT, "clocks": clocks}
 
 
-def summarize(cfg, res, steps, peaks):
+def fractions(tflops, peaks):
+    """A tensor-bound rate against the three ceilings in use: nominal dense bf16, measured cuBLAS burst, measured
+    cuBLAS sustained."""
+    return {"of_nominal_2250": tflops / NOMINAL_BF16_TFLOPS, "of_measured_burst": tflops / peaks["bf16_tflops"],
+            "of_measured_sustained": tflops / peaks["bf16_tflops_sustained"]}
+
+
+def summarize(cfg, res, peaks, peaks_kind, sms):
+    steps = res["steps"]
     ms_step = res["total_ms"] / steps
     pc = res["per_call_ms"]
     flops = call_flops(cfg)
     nbytes = call_bytes(cfg)
     gemm_ms = sum(pc[c] for c in GEMM_CALLS)
+    gemm_tflops = cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12
+    mhz = (res["clocks"] or {}).get("sm_mhz")
     out = {
-        "workload": cfg.name, "ms_per_step": ms_step,
+        "workload": cfg.name, "steps": steps, "timed_seconds": res["total_ms"] * 1e-3, "ms_per_step": ms_step,
         "layer_tflops": cfg.flops_fwd_bwd / (ms_step * 1e-3) / 1e12,
-        "gemm_tflops": cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12,
-        "gemm_frac_of_nominal_2250": cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS,
-        "gemm_frac_of_measured_burst": cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
-        "gemm_frac_of_measured_sustained": cfg.flops_fwd_bwd / (gemm_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+        "gemm_tflops": gemm_tflops,
+        "gemm_frac": fractions(gemm_tflops, peaks),
         "per_call_ms": {k: round(v, 5) for k, v in pc.items()},
         "per_call_tflops": {c: round(flops[c] / (pc[c] * 1e-3) / 1e12, 1) for c in GEMM_CALLS},
         "per_call_gbs": {c: round(nbytes[c] / (pc[c] * 1e-3) / 1e9, 1) for c in nbytes},
+        "per_call_gbs_frac_of_measured_copy": {c: round(nbytes[c] / (pc[c] * 1e-3) / 1e9 / peaks["hbm_gbs"], 3) for c in nbytes},
         "permute_gbs": nbytes["permute"] / (pc["permute"] * 1e-3) / 1e9,
         "permute_frac_of_nominal_8000": nbytes["permute"] / (pc["permute"] * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
         "permute_frac_of_measured": nbytes["permute"] / (pc["permute"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "roofline": roofline_object(cfg, res, peaks, peaks_kind),
+        "clocks": res["clocks"],
     }
+    if mhz:
+        # clock-normalised: per-call time x the median SM clock sampled over these steps (millions of SM cycles), and
+        # for the GEMMs the share of the tensor pipe's rate at that clock -- comparable across differently
+        # power-capped boxes
+        out["clock_normalised"] = {
+            "sm_mhz_median": mhz,
+            "per_call_mcycles": {k: round(v * 1e-3 * mhz, 3) for k, v in pc.items()},
+            "per_call_pipe_frac_at_sampled_clock": {
+                c: round(flops[c] / (pc[c] * 1e-3 * mhz * 1e6 * sms * PIPE_FLOP_PER_CLK_PER_SM), 3) for c in GEMM_CALLS},
+            "gemm_pipe_frac_at_sampled_clock": cfg.flops_fwd_bwd / (gemm_ms * 1e-3 * mhz * 1e6 * sms * PIPE_FLOP_PER_CLK_PER_SM),
+        }
     return out
 
 
 def roofline_object(cfg, res, peaks, peaks_kind):
+    """The grouped-GEMM call with the largest share of the step: algorithmic flops per launch / its average
+    CUDA-event duration inside the timed steps, against the measured cuBLAS bf16 rates and the nominal peak."""
     pc = res["per_call_ms"]
     flops = call_flops(cfg)
     dom = max(GEMM_CALLS, key=lambda c: pc[c])
     achieved = flops[dom] / (pc[dom] * 1e-3) / 1e12
-    peak = peaks["bf16_tflops"]
+    # a run of a second or more sits under the power cap: the sustained cuBLAS rate is the like-for-like ceiling
+    long_run = res["total_ms"] >= 1000.0
+    peak = peaks["bf16_tflops_sustained"] if long_run else peaks["bf16_tflops"]
+    traffic = NCU_TRAFFIC.get((cfg.name, dom))
     return {"bound": "tensor", "kernel": "grouped_gemm_kernel[" + dom + "]", "achieved": achieved, "peak": peak,
-            "peak_kind": "bf16 cuBLAS burst, of " + peaks_kind, "unit": "TFLOP/s", "frac": achieved / peak,
-            "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+            "peak_kind": ("bf16 cuBLAS sustained (timed region >= 1 s), of " if long_run else "bf16 cuBLAS burst, of ") + peaks_kind,
+            "unit": "TFLOP/s", "frac": achieved / peak,
+            "frac_of_burst": achieved / peaks["bf16_tflops"], "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+            "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
             "flops_per_launch": flops[dom], "avg_launch_ms": pc[dom],
-            "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, dom))}
+            "traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None}
 
 
 # --------------------------------------------------------------------------------------------
 # end to end through the host-buffer entry point
 # --------------------------------------------------------------------------------------------
 def time_e2e(B, cfg, wl, b, device, steps, warmup, dist=None):
+    """`steps` calls of moe_layer_fwd_bwd_host back to back: every call copies that step's activations, routing and
+    upstream gradient from pinned host memory and copies y, dx and dtopk_w back to pinned host memory."""
     d = b.d
     arena = torch.empty(B.moe_layer_arena_bytes(d), dtype=torch.uint8, device=device)
     pin = lambda t: t.cpu().pin_memory()
@@ -316,10 +361,12 @@ def time_e2e(B, cfg, wl, b, device, steps, warmup, dist=None):
     e1.record()
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
+    # the results that came back are the device-resident step's (same inputs, same kernels): bit for bit
+    same = bool(torch.equal(yh, b.y.cpu()) and torch.equal(dxh, b.dx.cpu()))
     h2d = xh.numel() * 2 + ih.numel() * 4 + wh.numel() * 4 + dyh.numel() * 2
     d2h = yh.numel() * 2 + dxh.numel() * 2 + dwh.numel() * 4
     del arena
-    return ms, h2d, d2h
+    return ms, h2d, d2h, same
 
 
 # --------------------------------------------------------------------------------------------
@@ -424,6 +471,38 @@ def stream_calibration(device):
     return out
 
 
+def stream_calibration_in_step(B, cfg, res, device, steps=12):
+    """The same three library stream kernels (512 MiB buffers), each timed with events right after a whole layer
+    step, i.e. in the power-capped state the step's own data-movement kernels run in.  On this part the write-heavy
+    rates drop well below their idle-chip values in that state while the read rate does not: context for the
+    per-call GB/s of the write-heavy calls (permute, combine backward, SwiGLU backward)."""
+    step = make_step(B, res["buffers"], res["wl"])
+    n = 1 << 28
+    a = torch.empty(n, dtype=torch.bfloat16, device=device)
+    b = torch.empty(n, dtype=torch.bfloat16, device=device)
+    a.zero_()
+    kinds = {"copy_gbs": (lambda: b.copy_(a), 4 * n), "write_only_gbs": (lambda: a.fill_(1.0), 2 * n),
+             "read_only_gbs": (lambda: a.sum(), 2 * n)}
+    for _ in range(3):
+        step()
+    out = {}
+    for name, (fn, nbytes) in kinds.items():
+        evs = []
+        for _ in range(steps):
+            step()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        out[name] = nbytes / (statistics.median(x.elapsed_time(y) for x, y in evs) * 1e-3) / 1e9
+    out["note"] = "torch copy_/fill_/sum on 512 MiB, each timed directly after a whole step of '" + cfg.name + "' (median)"
+    del a, b
+    torch.cuda.empty_cache()
+    return out
+
+
 def max_over_ranks(values, dist, device):
     """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
     if dist is None:
@@ -455,59 +534,72 @@ def run_ours(args):
         dist = dist_mod
     peaks, peaks_kind = load_peaks()
     cfg = W.CONFIGS[args.config]
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
 
-    res = time_config(B, cfg, device, args.steps, args.warmup, dist)
+    res = time_config(B, cfg, device, args.steps, args.warmup, dist, min_seconds=args.min_seconds)
+    steps = res["steps"]
     if args.no_e2e:
-        e2e_ms, h2d, d2h = float("nan"), 0, 0
+        e2e_ms, h2d, d2h, e2e_same = float("nan"), 0, 0, None
     else:
-        e2e_ms, h2d, d2h = time_e2e(B, cfg, res["wl"], res["buffers"], device, args.steps, args.warmup, dist)
+        e2e_ms, h2d, d2h, e2e_same = time_e2e(B, cfg, res["wl"], res["buffers"], device, steps, args.warmup, dist)
 
     total_ms, e2e_ms_max = max_over_ranks([res["total_ms"], e2e_ms], dist, device)
-    ms_step = total_ms / args.steps
+    ms_step = total_ms / steps
     value = aggregate_tflops(world, cfg.flops_fwd_bwd, ms_step)
-    summary = summarize(cfg, res, args.steps, peaks)
+    summary = summarize(cfg, res, peaks, peaks_kind, sms)
     launches_per_step = sum(LAUNCHES_PER_CALL.get(c, 1) for c in CALLS)
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "steps_requested": args.steps,
+        "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E": cfg.E, "K": cfg.K,
                    "routing": cfg.routing, "parallelism": "replicas only (single-GPU layer)" if world > 1 else "1 GPU",
+                   "timed_seconds": total_ms * 1e-3,
                    "l2": "no flush: the step's working set (weights + activations) exceeds the 126 MB L2 many times"},
         "clocks": res["clocks"],
         "e2e": {"value": aggregate_tflops(world, cfg.flops_fwd_bwd, e2e_ms_max), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms_max,
+                "results_equal_device_resident_step": e2e_same,
                 "note": "moe_layer_fwd_bwd_host: activations, routing and upstream gradient from pinned host "
                         "memory each step, results read back each step; weights and weight gradients stay on the "
                         "device; the copies run on side streams and, with steps following one another, under the "
                         "neighbouring steps' GEMMs"},
-        "gpu_launches": launches_per_step * args.steps,
-        "roofline": roofline_object(cfg, res, peaks, peaks_kind),
-        "pct_of_dense_bf16_peak_nominal": 100.0 * summary["gemm_frac_of_nominal_2250"],
+        "gpu_launches": launches_per_step * steps,
+        "roofline": summary["roofline"],
+        "pct_of_dense_bf16_peak_nominal": 100.0 * summary["gemm_frac"]["of_nominal_2250"],
         "gemm_tflops": summary["gemm_tflops"], "permute_gbs": summary["permute_gbs"],
         "detail": summary, "peaks": {"kind": peaks_kind, "hbm_gbs": peaks["hbm_gbs"], "bf16_tflops": peaks["bf16_tflops"],
-                                     "bf16_tflops_sustained": peaks["bf16_tflops_sustained"]},
+                                     "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
+                                     "nominal_bf16_tflops": NOMINAL_BF16_TFLOPS, "nominal_hbm_gbs": NOMINAL_HBM_GBS},
     }
 
     if rank == 0 and world == 1:
         extra = []
-        wl_host = host_copy(res["wl"]) if not args.no_cpu_baseline else None
+        wl_host = None
+        if not args.no_cpu_baseline:
+            n_tok = min(args.ref_tokens, cfg.T)
+            wl_host = host_copy({k: (v[:n_tok] if k in ("X", "dY", "topk_idx", "topk_w") else v) for k, v in res["wl"].items()})
         line["sustained"] = time_sustained(B, cfg, res, device)
+        line["sustained"]["frac"] = fractions(line["sustained"]["value"], peaks)
+        line["stream_calibration_in_step"] = stream_calibration_in_step(B, cfg, res, device)
         del res
         torch.cuda.empty_cache()
         for name in args.also:
+            if name == cfg.name:
+                continue
             c2 = W.CONFIGS[name]
-            r2 = time_config(B, c2, device, max(3, args.steps // 4), 3, None, sample_clocks=True)
-            s2 = summarize(c2, r2, max(3, args.steps // 4), peaks)
-            s2["clocks"] = r2["clocks"]
-            extra.append(s2)
+            r2 = time_config(B, c2, device, 3, 3, None, sample_clocks=True, min_seconds=args.other_min_seconds)
+            extra.append(summarize(c2, r2, peaks, peaks_kind, sms))
             del r2
             torch.cuda.empty_cache()
         if extra:
             line["other_configs"] = extra
-        router = time_router(B, cfg, device)
+        router_cfg = cfg if cfg.routing in ("softmax", "skew") else W.CONFIGS["many_small"]
+        router = time_router(B, router_cfg, device)
         if router is not None:
+            router["workload"] = router_cfg.name
             line["router"] = router
         line["stream_calibration"] = stream_calibration(device)
         if wl_host is not None:
@@ -525,11 +617,14 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--config", default="fine_grained", choices=list(W.CONFIGS))
+    ap.add_argument("--config", default="imbalanced", choices=list(W.CONFIGS))
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="the headline workload's timed region lasts at least this long (steps are added to --steps)")
+    ap.add_argument("--other-min-seconds", type=float, default=0.5, help="the same floor for each of the --also workloads")
     ap.add_argument("--custom", default="", help="T,H,I,E,K of an ad-hoc softmax-routed workload (profiling aid)")
-    ap.add_argument("--also", default="many_small,few_large,imbalanced,paper_dw1",
+    ap.add_argument("--also", default="fine_grained,many_small,few_large,paper_dw1",
                     help="comma-separated other configurations to time briefly at N=1 ('' for none)")
-    ap.add_argument("--ref-tokens", type=int, default=512, help="tokens in the oracle's timed sample")
+    ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens in the oracle's timed sample")
     ap.add_argument("--host-inputs", default="device", choices=["device", "numpy"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (profiling runs)")

@@ -61,6 +61,7 @@ typedef enum {
     MOE_ERR_ALIGNMENT = 4,         /* a pointer is not 16-byte aligned */
     MOE_ERR_WORKSPACE = 5,         /* workspace / arena too small */
     MOE_ERR_CUDA = 6,              /* a CUDA runtime or driver call failed */
+    MOE_ERR_BAD_INDEX = 7,         /* device status only: moe_permute met an expert id outside [0, E) */
     MOE_ERR_TIMEOUT = 8            /* device status only: a bounded wait inside a kernel ran out */
 } moe_status_t;
 

@@ -69,6 +69,7 @@ const char* moe_status_string(int status) {
         case MOE_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
         case MOE_ERR_WORKSPACE: return "workspace or arena too small";
         case MOE_ERR_CUDA: return "CUDA call failed";
+        case MOE_ERR_BAD_INDEX: return "an expert id outside [0, E) was met (the pair was dropped)";
         case MOE_ERR_TIMEOUT: return "a bounded device-side wait ran out";
         default: return "unknown status";
     }

@@ -36,23 +36,33 @@ __device__ __forceinline__ uint4 pack8(const float f[8]) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// a1, index part.  Two small kernels over the R = T*K pairs, split into block-chunks of `chunk`
-// consecutive pairs (a multiple of 256; one block per chunk, one eighth of it per warp):
-//   hist : per block-chunk, the number of pairs of each expert (shared-memory atomics: counts are
-//          order-free)                                                          -> ws[block][e]
-//   rank : every block sums the histogram rows before it (its base) and all rows (the counts),
-//          turns the counts into offsets, ranks its warps' pairs (per-warp counts by atomics, then the
-//          same-expert lane mask of each 32 pairs from 32 broadcasts, and popc):
-//          row(p) = offsets[e] + base[e] + pairs of e in earlier warps of the block + earlier
-//          pairs of e in the same warp.
+// a1 in two launches.
+//   hist      : one block per `chunk` consecutive pairs (a multiple of 256): the number of pairs of each
+//               expert in the chunk (shared-memory atomics: counts are order-free)          -> ws[chunk][e]
+//   rank_rows : one block per kTokPerBlock consecutive tokens.  The block
+//               (1) starts bulk loads of its first token rows and counts, from the routing indices alone,
+//                   the pairs between the start of its histogram chunk and its own first pair, and its own
+//                   pairs per warp -- all before the histogram kernel's output is needed;
+//               (2) sums the histogram rows: all of them (the counts), those before its chunk (its base);
+//                   counts -> offsets by a warp scan;
+//               (3) ranks its own pairs: row(p) = offsets[e] + base[e] + pairs of e in earlier warps of
+//                   the block + earlier pairs of e in the same warp (same-expert lane mask of each 32
+//                   pairs from 32 broadcasts, and popc): the unique stable sort, no atomic decides an index;
+//               (4) pushes its tokens' rows to their K destination rows with the bulk-copy engine: a ring
+//                   of shared-memory buffers, one cp.async.bulk load per row (or <= 16 KB segment), K
+//                   cp.async.bulk stores (lane k issues store k).  Each row is read from HBM once, no data
+//                   passes through registers, and a block copies as soon as ITS pairs are ranked: nothing
+//                   waits for the whole index to exist.
+// A pair whose expert id lies outside [0, E) is dropped (it gets no row; the rows past offsets[E] stay
+// unwritten) and MOE_ERR_BAD_INDEX is recorded in the device status word.
 // ------------------------------------------------------------------------------------------------
-// Programmatic dependent launch: the three permute kernels are launched so that a later one may start (and run its
-// set-up) while the earlier one is still finishing; grid_dependency_wait() then blocks until everything the earlier
-// kernel wrote is visible.  Saves the launch gaps of the two small index kernels.
+// Programmatic dependent launch: rank_rows may start (and run step 1) while hist is still finishing;
+// grid_dependency_wait() then blocks until everything hist wrote is visible.
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 constexpr int kIdxGroup = 8;   // index loads in flight per thread in the permute index kernels
+__device__ int g_movement_status = 0;
 
 __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* __restrict__ topk_idx, int R, int E,
                                                                 int chunk, int32_t* __restrict__ ws) {
@@ -84,55 +94,141 @@ __global__ void __launch_bounds__(kThreads) permute_hist_kernel(const int32_t* _
     for (int e = threadIdx.x; e < E; e += kThreads) out[e] = hist[e];
 }
 
-__global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* __restrict__ topk_idx, int R, int E,
-                                                                int chunk, int n_blocks,
-                                                                const int32_t* __restrict__ ws,
-                                                                int32_t* __restrict__ counts,
-                                                                int32_t* __restrict__ offsets,
-                                                                int32_t* __restrict__ row_to_pair,
-                                                                int32_t* __restrict__ pair_to_row) {
-    extern __shared__ int32_t smem_i[];
-    int32_t* offs = smem_i;                       // [E+1] exclusive prefix of the counts
-    int32_t* total = smem_i + (E + 1);            // [E]   counts
-    int32_t* base = total + E;                    // [E]   pairs of e in earlier blocks
-    int32_t* whist = base + E;                    // [warps][E] per-warp counts, then running row cursors
+// Geometry of rank_rows, from sweeps on B200 over the benchmark workloads (whole call, L2 flushed): 8 warps, 4
+// tokens per block and a ring of 3 buffers with loads 2 units ahead were best everywhere.  Blocks this small keep
+// eight of them resident per SM, each in a different phase (counting, ranking, copying); larger blocks, deeper rings
+// or 4-warp blocks (more but slower blocks per SM) all lost 5-20 % on the large workloads.
+constexpr int kPermWarps = 8, kPermThreads = 32 * kPermWarps;
+constexpr int kTokPerBlock = 4;
+constexpr int kRowBufs = 3, kRowLookahead = 2, kRowMaxSeg = 16384;
+constexpr int kMaxOwnPairs = kTokPerBlock * 32;   // K <= 32
+static_assert(kMaxOwnPairs <= 32 * kPermWarps, "each warp ranks at most one group of 32 own pairs");
+constexpr unsigned long long kRowWaitLimitNs = 2000000000ull;
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long movement_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait for a bulk load (2 s on %globaltimer).  False when the wait ran out.
+__device__ __forceinline__ bool row_bar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns) {
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 0;; ++spin) {
+        uint32_t done;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(done)
+                     : "r"(bar), "r"(parity)
+                     : "memory");
+        if (done) return true;
+        if ((spin & 0xFF) == 0xFF) {
+            const unsigned long long now = movement_timer_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > limit_ns) return false;
+        }
+    }
+}
+
+// Shared memory of rank_rows: the row ring first (128-byte aligned), then the index tables.
+struct RankRowsSmem {
+    int ring_bytes;     // kRowBufs * seg_bytes, 0 without a row copy
+    int total_bytes;
+    __host__ __device__ RankRowsSmem(int E, int seg_bytes, bool rows) {
+        ring_bytes = rows ? kRowBufs * seg_bytes : 0;
+        total_bytes = ring_bytes + ((kPermWarps + 3) * E + 1 + kMaxOwnPairs) * (int)sizeof(int32_t);
+    }
+};
+
+__global__ void __launch_bounds__(kPermThreads) permute_rank_rows_kernel(
+    const int32_t* __restrict__ topk_idx, int R, int E, int K, int T, int chunk, int n_chunks,
+    const int32_t* __restrict__ ws, int32_t* __restrict__ counts, int32_t* __restrict__ offsets,
+    int32_t* __restrict__ row_to_pair, int32_t* __restrict__ pair_to_row, const uint8_t* __restrict__ x,
+    uint8_t* __restrict__ x_perm, int row_bytes, int seg_bytes, int n_seg) {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
+    __shared__ unsigned long long bars[kRowBufs];
+    const bool rows = x_perm != nullptr;
+    const RankRowsSmem lay(E, seg_bytes, rows);
+    uint8_t* bufs = smem_raw;                                        // [kRowBufs][seg_bytes]
+    int32_t* offs = reinterpret_cast<int32_t*>(smem_raw + lay.ring_bytes);   // [E+1] exclusive prefix of the counts
+    int32_t* total = offs + (E + 1);                                 // [E]   counts
+    int32_t* base = total + E;                                       // [E]   pairs of e before this block's first pair
+    int32_t* whist = base + E;                                       // [warps][E] per-warp counts, then running row cursors
+    int32_t* dest = whist + kPermWarps * E;                      // [own pairs] destination row of each own pair (-1: dropped)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // Before the histogram kernel's output is needed: this warp's own counts over its eighth of the chunk (pass 1,
-    // from the routing indices alone).
-    grid_launch_dependents();
-    for (int i = threadIdx.x; i < kWarpsPerBlock * E; i += kThreads) whist[i] = 0;
+    const int t0 = blockIdx.x * kTokPerBlock, t1 = min(T, t0 + kTokPerBlock);
+    const long long p_begin = (long long)t0 * K, p_end = (long long)t1 * K;
+    const int n_own = (int)(p_end - p_begin);
+    const int my_chunk = (int)(p_begin / chunk);                     // histogram rows wholly before this block: a < my_chunk
+    const long long chunk_begin = (long long)my_chunk * chunk;
+    const int n_units = rows ? (t1 - t0) * n_seg : 0;                // row segments this block copies
+    const int n_pre = min(kRowLookahead, n_units);
+
+    // ---- (1) nothing here needs the histogram kernel's output ----
+    auto issue_load = [&](int u) {   // lane 0 of warp 0
+        const int s = u % kRowBufs;
+        const int t = t0 + u / n_seg, seg = u % n_seg;
+        const int bytes = min(seg_bytes, row_bytes - seg * seg_bytes);
+        const uint32_t bar = smem_addr(&bars[s]);
+        asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         smem_addr(bufs + (size_t)s * seg_bytes)),
+                     "l"(x + (long long)t * row_bytes + (long long)seg * seg_bytes), "r"(bytes), "r"(bar)
+                     : "memory");
+    };
+    if (threadIdx.x == 0 && rows) {
+        for (int s = 0; s < kRowBufs; ++s)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[s])) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        for (int u = 0; u < n_pre; ++u) issue_load(u);
+    }
+    // this warp's contiguous share of the block's own pairs (at most 32: one per lane); the expert id stays in a
+    // register from here to the ranking pass.  -1: no pair here; -2: a pair with an invalid expert id
+    const int per_warp = (n_own + kPermWarps - 1) / kPermWarps;
+    const long long my_p = p_begin + (long long)warp * per_warp + lane;
+    int own = -1;
+    bool bad = false;
+    if (lane < per_warp && my_p < p_end) {
+        own = topk_idx[my_p];
+        if (own < 0 || own >= E) { bad = true; own = -2; }
+    }
+    // pairs between the start of the histogram chunk and this block's first pair (fewer than `chunk`): the first
+    // batch of their ids is requested before anything waits
+    const int n_before = (int)(p_begin - chunk_begin);
+    int before0[kIdxGroup];
+#pragma unroll
+    for (int g = 0; g < kIdxGroup; ++g) {
+        const int i = (int)threadIdx.x + g * kPermThreads;
+        before0[g] = i < n_before ? topk_idx[chunk_begin + i] : -1;
+    }
+    for (int i = threadIdx.x; i < (kPermWarps + 2) * E; i += kPermThreads) total[i] = 0;   // total, base, whist
     __syncthreads();
-    // pass 1: this warp's histogram over its eighth of the chunk
-    const int per_warp = chunk / kWarpsPerBlock;
-    const long long p0 = (long long)blockIdx.x * chunk + (long long)warp * per_warp;
-    int32_t* mine = whist + warp * E;
-#pragma unroll 1
-    for (int i0 = 0; i0 < per_warp; i0 += 32 * kIdxGroup) {   // indices of kIdxGroup iterations loaded up front
+#pragma unroll
+    for (int g = 0; g < kIdxGroup; ++g)
+        if (before0[g] >= 0 && before0[g] < E) atomicAdd(&base[before0[g]], 1);   // counts only: order-free
+    for (int i0 = threadIdx.x + kPermThreads * kIdxGroup; i0 < n_before; i0 += kPermThreads * kIdxGroup) {
         int ev[kIdxGroup];
 #pragma unroll
         for (int g = 0; g < kIdxGroup; ++g) {
-            const int i = i0 + g * 32 + lane;
-            const long long p = p0 + i;
-            int e = (i < per_warp && p < R) ? topk_idx[p] : -1;
-            ev[g] = e >= E ? -1 : e;
+            const int i = i0 + g * kPermThreads;
+            ev[g] = i < n_before ? topk_idx[chunk_begin + i] : -1;
         }
 #pragma unroll
-        for (int g = 0; g < kIdxGroup; ++g) {
-            if (i0 + g * 32 >= per_warp) break;   // warp-uniform
-            if (ev[g] >= 0) atomicAdd(&mine[ev[g]], 1);   // counts only: order-free
-        }
+        for (int g = 0; g < kIdxGroup; ++g)
+            if (ev[g] >= 0 && ev[g] < E) atomicAdd(&base[ev[g]], 1);
     }
-    grid_dependency_wait();   // the per-block histograms of the first kernel are complete and visible from here on
-    for (int e = threadIdx.x; e < E; e += kThreads) {
-        int before = 0, all = 0;
-        for (int b = 0; b < n_blocks; ++b) {
-            const int v = ws[(size_t)b * E + e];
-            all += v;
-            if (b < (int)blockIdx.x) before += v;
+    // pass 1: this warp's histogram over its own pairs
+    int32_t* mine = whist + warp * E;
+    if (own >= 0) atomicAdd(&mine[own], 1);   // counts only: order-free
+    // ---- (2) the chunk histograms are complete and visible from here on ----
+    grid_dependency_wait();
+    for (int i = threadIdx.x; i < n_chunks * E; i += kPermThreads) {
+        const int v = ws[i];
+        if (v != 0) {
+            const int a = i / E, e = i - a * E;
+            atomicAdd(&total[e], v);
+            if (a < my_chunk) atomicAdd(&base[e], v);
         }
-        total[e] = all;
-        base[e] = before;
     }
     __syncthreads();
     // offsets = exclusive prefix of counts, by warp 0 (each lane owns a contiguous run of experts)
@@ -156,129 +252,68 @@ __global__ void __launch_bounds__(kThreads) permute_rank_kernel(const int32_t* _
     }
     __syncthreads();
     if (blockIdx.x == 0) {
-        for (int e = threadIdx.x; e <= E; e += kThreads) offsets[e] = offs[e];
-        for (int e = threadIdx.x; e < E; e += kThreads) counts[e] = total[e];
+        for (int e = threadIdx.x; e <= E; e += kPermThreads) offsets[e] = offs[e];
+        for (int e = threadIdx.x; e < E; e += kPermThreads) counts[e] = total[e];
     }
     // per-warp counts -> first row of each (warp, expert)
-    for (int e = threadIdx.x; e < E; e += kThreads) {
+    for (int e = threadIdx.x; e < E; e += kPermThreads) {
         int run = offs[e] + base[e];
 #pragma unroll
-        for (int w = 0; w < kWarpsPerBlock; ++w) {
+        for (int w = 0; w < kPermWarps; ++w) {
             const int v = whist[w * E + e];
             whist[w * E + e] = run;
             run += v;
         }
     }
     __syncthreads();
-    // pass 2: stable ranks
-    const unsigned lt_mask = (1u << lane) - 1u;
-#pragma unroll 1
-    for (int i0 = 0; i0 < per_warp; i0 += 32 * kIdxGroup) {
-        int ev[kIdxGroup];
+    // ---- (3) stable ranks of the own pairs ----
+    {
+        // lanes of the warp with the same expert: 32 broadcasts are several times faster than match.any here
+        // (whose time grows with the number of distinct values, and routing makes most of them distinct)
+        unsigned mask = 0;
 #pragma unroll
-        for (int g = 0; g < kIdxGroup; ++g) {
-            const int i = i0 + g * 32 + lane;
-            const long long p = p0 + i;
-            int e = (i < per_warp && p < R) ? topk_idx[p] : -1;
-            ev[g] = e >= E ? -1 : e;
-        }
-#pragma unroll
-        for (int g = 0; g < kIdxGroup; ++g) {
-            if (i0 + g * 32 >= per_warp) break;   // warp-uniform
-            const int e = ev[g];
-            const long long p = p0 + i0 + g * 32 + lane;
-            // lanes of the warp with the same expert: 32 broadcasts are several times faster than match.any here
-            // (whose time grows with the number of distinct values, and routing makes most of them distinct)
-            unsigned mask = 0;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) mask |= (__shfl_sync(0xffffffffu, e, j) == e ? 1u : 0u) << j;
-            if (e >= 0) {
-                const int row = mine[e] + __popc(mask & lt_mask);
-                row_to_pair[row] = (int32_t)p;
-                pair_to_row[p] = row;
-            }
-            __syncwarp();
-            if (e >= 0 && lane == __ffs(mask) - 1) mine[e] += __popc(mask);
-            __syncwarp();
+        for (int j = 0; j < 32; ++j) mask |= (__shfl_sync(0xffffffffu, own, j) == own ? 1u : 0u) << j;
+        if (own >= 0) {
+            const int row = mine[own] + __popc(mask & ((1u << lane) - 1u));
+            row_to_pair[row] = (int32_t)my_p;
+            pair_to_row[my_p] = row;
+            dest[my_p - p_begin] = row;
+        } else if (own == -2) {
+            dest[my_p - p_begin] = -1;
         }
     }
-}
-
-// ------------------------------------------------------------------------------------------------
-// a1, row part: x_perm[pair_to_row[t*K+k], :] = x[t, :] with the bulk-copy engine.  One warp per CTA
-// runs a ring of NBUF shared-memory buffers: a token row (or a <= 16 KB segment of it) is pulled in
-// with one cp.async.bulk load and pushed to its K destination rows with K cp.async.bulk stores
-// (lane k issues store k), so the row is read from HBM once and no data passes through registers.
-// Loads run kRowLookahead units ahead of the stores.
-// ------------------------------------------------------------------------------------------------
-constexpr int kRowBufs = 4, kRowLookahead = 2, kRowMaxSeg = 16384;
-__device__ int g_movement_status = 0;
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__global__ void __launch_bounds__(32) permute_rows_bulk_kernel(const uint8_t* __restrict__ x,
-                                                               const int32_t* __restrict__ pair_to_row,
-                                                               uint8_t* __restrict__ x_perm, int T, int K,
-                                                               int row_bytes, int seg_bytes, int n_seg) {
-    extern __shared__ __align__(128) uint8_t bufs[];   // [kRowBufs][seg_bytes]
-    __shared__ unsigned long long bars[kRowBufs];
-    __shared__ int32_t dest[kRowBufs][32];
-    const int lane = threadIdx.x;
-    if (lane == 0) {
-        for (int s = 0; s < kRowBufs; ++s)
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_addr(&bars[s])) : "memory");
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncwarp();
-    grid_dependency_wait();   // pair_to_row comes from the rank kernel, which may still be finishing
-    const long long n_units_all = (long long)T * n_seg;
-    const long long first = blockIdx.x, stride = gridDim.x;
-    const long long n_mine = first < n_units_all ? (n_units_all - first + stride - 1) / stride : 0;
+    if (bad) atomicExch(&g_movement_status, (int)MOE_ERR_BAD_INDEX);
+    __syncthreads();
+    // ---- (4) rows: warp 0 runs the ring, loads kRowLookahead units ahead of the stores ----
+    if (warp != 0 || n_units == 0) return;
     bool ok = true;
-    for (long long it = 0; ok && it < n_mine + kRowLookahead; ++it) {
-        if (it < n_mine) {
-            const int s = (int)(it % kRowBufs);
-            const long long u = first + it * stride;
-            const int t = (int)(u / n_seg), seg = (int)(u - (long long)t * n_seg);
-            const int bytes = min(seg_bytes, row_bytes - seg * seg_bytes);
-            // the stores that last read this buffer were committed kRowLookahead iterations ago
-            if (it >= kRowBufs) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kRowLookahead - 1) : "memory");
-            if (lane < K) dest[s][lane] = __ldg(pair_to_row + (long long)t * K + lane);
+    int loads_issued = n_pre;
+    for (int it = 0; it < n_units + kRowLookahead; ++it) {
+        if (it >= n_pre && it < n_units) {
+            // the stores that last read this buffer were committed kRowBufs - kRowLookahead iterations ago
+            if (it >= kRowBufs) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kRowBufs - kRowLookahead - 1) : "memory");
             __syncwarp();
-            if (lane == 0) {
-                const uint32_t bar = smem_addr(&bars[s]);
-                asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes)
-                             : "memory");
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                                 smem_addr(bufs + (size_t)s * seg_bytes)),
-                             "l"(x + (long long)t * row_bytes + (long long)seg * seg_bytes), "r"(bytes), "r"(bar)
-                             : "memory");
-            }
+            if (lane == 0) issue_load(it);
+            loads_issued = it + 1;
         }
-        const long long j = it - kRowLookahead;
+        const int j = it - kRowLookahead;
         if (j >= 0) {
-            const int s = (int)(j % kRowBufs);
+            const int s = j % kRowBufs;
             const uint32_t parity = (uint32_t)((j / kRowBufs) & 1);
-            const long long u = first + j * stride;
-            const int t = (int)(u / n_seg), seg = (int)(u - (long long)t * n_seg);
+            const int t = t0 + j / n_seg, seg = j % n_seg;
             const int bytes = min(seg_bytes, row_bytes - seg * seg_bytes);
-            const uint32_t bar = smem_addr(&bars[s]);
-            uint32_t done = 0;
-            for (uint32_t spin = 0; !done; ++spin) {
-                asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                             : "=r"(done)
-                             : "r"(bar), "r"(parity)
-                             : "memory");
-                if (!done && spin > (1u << 24)) {   // bounded: give up, report, leave
-                    atomicExch(&g_movement_status, (int)MOE_ERR_TIMEOUT);
-                    ok = false;
-                    break;
-                }
-            }
+            ok = row_bar_wait(smem_addr(&bars[s]), parity, kRowWaitLimitNs);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            if (lane < K) {
-                uint8_t* dst = x_perm + (long long)dest[s][lane] * row_bytes + (long long)seg * seg_bytes;
+            if (!ok) {
+                // give up: report, and leave no load in flight (bounded wait for each load issued after this one)
+                if (lane == 0) atomicExch(&g_movement_status, (int)MOE_ERR_TIMEOUT);
+                for (int u = j + 1; u < loads_issued; ++u)
+                    row_bar_wait(smem_addr(&bars[u % kRowBufs]), (uint32_t)((u / kRowBufs) & 1), kRowWaitLimitNs / 8);
+                break;
+            }
+            const int row = lane < K ? dest[(t - t0) * K + lane] : -1;
+            if (row >= 0) {
+                uint8_t* dst = x_perm + (long long)row * row_bytes + (long long)seg * seg_bytes;
                 asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
                              "r"(smem_addr(bufs + (size_t)s * seg_bytes)), "r"(bytes)
                              : "memory");
@@ -449,8 +484,8 @@ size_t permute_workspace_bytes(const moe_dims_t& d) {
     return (size_t)(n_chunks * d.E) * sizeof(int32_t);
 }
 
-// pairs per block-chunk: 2048, or more (a multiple of 256) when R is so large that the rank kernel's
-// per-block sum over all histogram rows would otherwise grow past 512 rows
+// pairs per histogram chunk: 2048, or more (a multiple of 256) when R is so large that the sum over all
+// histogram rows in every rank_rows block would otherwise grow past 512 rows
 static int permute_chunk(long long R) {
     long long chunk = 2048;
     const long long need = (R + 511) / 512;
@@ -471,52 +506,40 @@ int launch_permute(const moe_dims_t& d, const bf16* x, const int32_t* topk_idx, 
                    cudaStream_t s) {
     const int R = d.T * d.K, E = d.E;
     const int chunk = permute_chunk(R);
-    const int n_blocks = (R + chunk - 1) / chunk;
+    const int n_chunks = (R + chunk - 1) / chunk;
     int32_t* ws = static_cast<int32_t*>(workspace);
-    permute_hist_kernel<<<n_blocks, kThreads, E * sizeof(int32_t), s>>>(topk_idx, R, E, chunk, ws);
-    // the two following kernels may start before their predecessor has finished (see grid_dependency_wait) -- for
-    // small problems only, where the launch gaps are a third of the call; measured on the large ones (>= 131072
-    // pairs) the early-started row kernel made the call 4-15 % slower
+    permute_hist_kernel<<<n_chunks, kThreads, E * sizeof(int32_t), s>>>(topk_idx, R, E, chunk, ws);
+
+    const bool rows = x_perm != nullptr;
+    const int row_bytes = d.H * 2;
+    const int n_seg = (row_bytes + kRowMaxSeg - 1) / kRowMaxSeg;
+    const int seg_bytes = ((row_bytes + n_seg - 1) / n_seg + 15) / 16 * 16;
+    const RankRowsSmem lay(E, seg_bytes, rows);
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
+    if (!attr_set[dev]) {
+        const RankRowsSmem largest(1024, kRowMaxSeg, true);
+        if (cudaFuncSetAttribute(permute_rank_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 largest.total_bytes) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        attr_set[dev] = true;
+    }
+    const unsigned grid = (unsigned)((d.T + kTokPerBlock - 1) / kTokPerBlock);
+    // launched as a programmatic dependent of the histogram kernel: its blocks start, prefetch rows and count from
+    // the routing indices while the histogram kernel is still running
     cudaLaunchAttribute pdl[1];
     pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     pdl[0].val.programmaticStreamSerializationAllowed = 1;
-    const unsigned n_pdl = R <= 65536 ? 1u : 0u;
-    {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(n_blocks); cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = ((kWarpsPerBlock + 3) * E + 1) * sizeof(int32_t); cfg.stream = s;
-        cfg.attrs = pdl; cfg.numAttrs = n_pdl;
-        const int32_t* ws_c = ws;
-        if (cudaLaunchKernelEx(&cfg, permute_rank_kernel, topk_idx, R, E, chunk, n_blocks, ws_c, counts, offsets,
-                               row_to_pair, pair_to_row) != cudaSuccess)
-            return MOE_ERR_CUDA;
-    }
-    if (x_perm != nullptr) {
-        const int row_bytes = d.H * 2;
-        const int n_seg = (row_bytes + kRowMaxSeg - 1) / kRowMaxSeg;
-        const int seg_bytes = ((row_bytes + n_seg - 1) / n_seg + 15) / 16 * 16;
-        const size_t smem = (size_t)kRowBufs * seg_bytes;
-        static bool attr_set[64] = {};
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
-        if (!attr_set[dev]) {
-            if (cudaFuncSetAttribute(permute_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     kRowBufs * kRowMaxSeg) != cudaSuccess)
-                return MOE_ERR_CUDA;
-            attr_set[dev] = true;
-        }
-        const long long units = (long long)d.T * n_seg;
-        const int per_sm = (int)(196608 / (smem + 1024) < 8 ? 196608 / (smem + 1024) : 8);
-        long long grid = (long long)sm_count() * (per_sm < 1 ? 1 : per_sm);
-        if (grid > units) grid = units;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3(32); cfg.dynamicSmemBytes = smem; cfg.stream = s;
-        cfg.attrs = pdl; cfg.numAttrs = n_pdl;
-        const int32_t* p2r_c = pair_to_row;
-        if (cudaLaunchKernelEx(&cfg, permute_rows_bulk_kernel, reinterpret_cast<const uint8_t*>(x), p2r_c,
-                               reinterpret_cast<uint8_t*>(x_perm), d.T, d.K, row_bytes, seg_bytes, n_seg) != cudaSuccess)
-            return MOE_ERR_CUDA;
-    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid); cfg.blockDim = dim3(kPermThreads); cfg.dynamicSmemBytes = lay.total_bytes; cfg.stream = s;
+    cfg.attrs = pdl; cfg.numAttrs = 1;
+    const int32_t* ws_c = ws;
+    if (cudaLaunchKernelEx(&cfg, permute_rank_rows_kernel, topk_idx, R, E, (int)d.K, (int)d.T, chunk,
+                           n_chunks, ws_c, counts, offsets, row_to_pair, pair_to_row,
+                           reinterpret_cast<const uint8_t*>(x), reinterpret_cast<uint8_t*>(x_perm), row_bytes,
+                           seg_bytes, n_seg) != cudaSuccess)
+        return MOE_ERR_CUDA;
     return check_launch();
 }
 
@@ -584,8 +607,8 @@ int launch_combine_bwd(const moe_dims_t& d, const bf16* dy, const bf16* y_perm, 
 // file-scope device array instead, so that a caller who may not allocate device memory (see the
 // header) can still run the call.  The array's name is only a host-side handle in host code; the
 // device address is looked up once per device with cudaGetSymbolAddress and handed to the
-// ordinary permute launch.  Every entry the rank kernel reads is written by the histogram and
-// scan kernels of the same call first, so nothing has to be cleared between calls.
+// ordinary permute launch.  Every entry the second kernel reads is written by the histogram kernel of
+// the same call first, so nothing has to be cleared between calls.
 // ------------------------------------------------------------------------------------------------
 static __device__ __align__(256) unsigned char g_permute_static_scratch[MOE_PERMUTE_STATIC_SCRATCH_BYTES];
 

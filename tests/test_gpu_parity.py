@@ -105,6 +105,69 @@ def test_permute_rows_and_indices(B, case):
     _check_permute(B, host["topk_idx"], cfg.E, host["X"])
 
 
+@pytest.mark.parametrize("T,H,E,K,seed", [(3, 64, 4, 2, 0),            # fewer tokens than one block takes
+                                          (37, 8256, 40, 32, 1),       # rows longer than one bulk-copy segment, K = 32
+                                          (1027, 8192, 9, 3, 2),       # 16 KB rows, a ragged last block
+                                          (6001, 192, 130, 7, 3)])     # several histogram chunks, odd K
+def test_permute_rows_odd_shapes(B, T, H, E, K, seed):
+    rng = np.random.default_rng(seed)
+    idx = np.stack([rng.permutation(E)[:K] for _ in range(T)]).astype(np.int32)
+    X = W.round_to_bf16(rng.standard_normal((T, H), dtype=np.float32))
+    _check_permute(B, idx, E, X)
+
+
+def test_permute_drops_invalid_expert_ids_and_reports_them(B):
+    """Expert ids outside [0, E) are a precondition violation: the pairs are dropped (no row, no fault, nothing
+    written outside the outputs) and MOE_ERR_BAD_INDEX lands in the device status word; the valid pairs are
+    ranked as the stable sort of the valid pairs alone."""
+    T, H, E, K = 700, 128, 12, 4
+    rng = np.random.default_rng(11)
+    idx_np = rng.integers(0, E, size=(T, K)).astype(np.int32)
+    flat = idx_np.reshape(-1)
+    bad_at = rng.choice(flat.size, size=25, replace=False)
+    flat[bad_at] = rng.choice(np.array([-1, -7, E, E + 1, 2 ** 30, -2 ** 31], dtype=np.int64), size=25).astype(np.int32)
+    flat[0] = E                      # the very first and the very last pair too
+    flat[-1] = -1
+    valid = (flat >= 0) & (flat < E)
+    R, n_valid = flat.size, int(valid.sum())
+    X = W.round_to_bf16(rng.standard_normal((T, H), dtype=np.float32))
+    d = B.dims(T, H, 128, E, K)
+    guard = 64
+    counts = torch.full((E + 2 * guard,), -7, dtype=torch.int32, device="cuda")
+    offsets = torch.full((E + 1 + 2 * guard,), -7, dtype=torch.int32, device="cuda")
+    r2p = torch.full((R + 2 * guard,), -7, dtype=torch.int32, device="cuda")
+    p2r = torch.full((R + 2 * guard,), -7, dtype=torch.int32, device="cuda")
+    xp = torch.full((R + 2 * guard, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    ws = torch.empty(max(B.moe_permute_workspace_bytes(d), 16), dtype=torch.uint8, device="cuda")
+    assert B.moe_device_status() == 0
+    B.moe_permute(d, Hh.to_dev_bf16(X), _i32(idx_np), xp[guard:guard + R], counts[guard:guard + E],
+                  offsets[guard:guard + E + 1], r2p[guard:guard + R], p2r[guard:guard + R], ws)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 7                 # MOE_ERR_BAD_INDEX, read once ...
+    assert B.moe_device_status() == 0                 # ... and cleared by the read
+    # expected: the stable sort of the valid pairs (written out here: the oracle refuses invalid ids)
+    vp = np.flatnonzero(valid)
+    order = vp[np.argsort(flat[vp], kind="stable")]
+    exp_counts = np.bincount(flat[vp], minlength=E)
+    exp_p2r = np.full(R, -7, dtype=np.int64)
+    exp_p2r[order] = np.arange(n_valid)
+    assert np.array_equal(counts[guard:guard + E].cpu().numpy(), exp_counts)
+    assert np.array_equal(offsets[guard:guard + E + 1].cpu().numpy(), np.concatenate([[0], np.cumsum(exp_counts)]))
+    got_r2p = r2p[guard:guard + R].cpu().numpy()
+    assert np.array_equal(got_r2p[:n_valid], order)
+    assert np.all(got_r2p[n_valid:] == -7)            # rows past offsets[E] stay unwritten
+    assert np.array_equal(p2r[guard:guard + R].cpu().numpy(), exp_p2r)   # dropped pairs keep the sentinel
+    rows = Hh.to_np64(xp[guard:guard + R])
+    assert np.array_equal(rows[:n_valid], X[order // K].astype(np.float64))
+    assert np.all(np.isnan(rows[n_valid:]))
+    for t in (counts, offsets, r2p, p2r):              # guard bands untouched
+        assert torch.all(t[:guard] == -7) and torch.all(t[-guard:] == -7)
+    assert torch.isnan(xp[:guard]).all() and torch.isnan(xp[-guard:]).all()
+    # the next ordinary call is unaffected
+    _check_permute(B, rng.integers(0, E, size=(T, K)).astype(np.int32), E, X)
+    assert B.moe_device_status() == 0
+
+
 @pytest.mark.parametrize("name", ["fine_grained", "many_small", "few_large", "imbalanced"])
 def test_permute_indices_full_size(B, name):
     cfg = W.CONFIGS[name]

@@ -1,12 +1,15 @@
 """moe_permute_static_scratch: the route-permute variant for callers that cannot allocate device
 memory (its scratch is a fixed array inside the library).  It must give exactly what moe_permute
-gives, call after call, although all calls share that one array.  This file sorts last so that a
-run stopping at the first failure has already run everything else."""
+gives -- and what the CPU oracle gives -- call after call, although all calls share that one array,
+and a call must leave the amount of free device memory as it found it.  This file sorts last so that
+a run stopping at the first failure has already run everything else."""
 import ctypes
 
 import numpy as np
 import pytest
 import torch
+
+from oracle import moe_oracle as O
 
 
 def _routing(T, E, K, seed):
@@ -47,6 +50,20 @@ def test_static_scratch_permute_matches_moe_permute_on_consecutive_calls():
                                                                  o["r2p"], o["p2r"]), d, x, idx, H)
             for k in ref:                                   # integers and row copies: bit-exact
                 assert torch.equal(got[k], ref[k]), (k, T, E, K)
+        # and against the oracle: the stable sort itself, and bit copies of the token rows
+        oc, oo, or2p, op2r = O.permute_indices(idx.cpu().numpy(), E)
+        assert np.array_equal(got["counts"].cpu().numpy(), oc) and np.array_equal(got["offsets"].cpu().numpy(), oo)
+        assert np.array_equal(got["r2p"].cpu().numpy(), or2p) and np.array_equal(got["p2r"].cpu().numpy(), op2r)
+        assert torch.equal(got["xp"], x[torch.from_numpy(or2p.astype(np.int64) // K).cuda()])
+        # what the entry point exists for: a call (after the first one on this device, which resolved the
+        # array's address) allocates nothing -- the free device memory is the same before and after
+        out = dict(got)
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        B.moe_permute_static_scratch(d, x, idx, out["xp"], out["counts"], out["offsets"], out["r2p"], out["p2r"])
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before
     assert B.moe_device_status() == 0
 
 
