@@ -169,6 +169,13 @@ int moe_grouped_gemm_down_bwd(const moe_dims_t* dims, const void* dy_perm, const
  * scratch that also returns dGU. */
 int moe_swiglu_bwd(const moe_dims_t* dims, const void* dh_act, const void* gu_saved, void* dgu,
                    moe_stream_t stream);
+/* Fused form of the down dgrad and moe_swiglu_bwd (an additional entry point; the two-call form stays):
+ * dgu[r,:] = [dg | du] computed from dh = dy_perm[r,:] . w_down[e]^T held in fp32 -- dh_act is never
+ * written, and the chain to dx loses one bf16 rounding -- and from g, u read from gu_saved [R,2I].
+ * dy_perm [R,H], w_down [E,I,H], dgu [R,2I].  Replaces moe_grouped_gemm_down_dgrad + moe_swiglu_bwd. */
+int moe_grouped_gemm_down_dgrad_swiglu_bwd(const moe_dims_t* dims, const void* dy_perm,
+                                           const void* w_down, const void* gu_saved,
+                                           const int32_t* offsets, void* dgu, moe_stream_t stream);
 int moe_grouped_gemm_gateup_dgrad(const moe_dims_t* dims, const void* dgu, const void* w_gate,
                                   const void* w_up, const int32_t* offsets, void* dx_perm,
                                   moe_stream_t stream);

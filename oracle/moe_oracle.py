@@ -182,6 +182,19 @@ def swiglu_bwd(dH_act, GU):
     return np.concatenate([dg, du], axis=1)
 
 
+def down_dgrad_swiglu_bwd(dY_perm, W_down, GU, offsets):
+    """The fused call's result: dGU = swiglu_bwd(dHact, GU) with dHact[r,:] = dYp[r,:] @ Wd[e]^T, the two
+    definitions above applied one after the other with nothing rounded in between."""
+    dYp = _f64(dY_perm)
+    E, I, H = W_down.shape
+    dHact = np.zeros((dYp.shape[0], I), F64)
+    for e in range(E):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        if r1 > r0:
+            dHact[r0:r1] = dYp[r0:r1] @ _f64(W_down[e]).T
+    return swiglu_bwd(dHact, GU)
+
+
 def gateup_bwd_from_dgu(dGU, X_perm, W_gate, W_up, offsets):
     """dXp[r,:] = dg[r,:] @ Wg[e]^T + du[r,:] @ Wu[e]^T;  dWg[e] = Xp_e^T @ dg_e;  dWu likewise."""
     dGU = _f64(dGU)

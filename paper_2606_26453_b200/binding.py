@@ -20,7 +20,7 @@ EXPORTS = [
     "moe_permute_bwd",
     "moe_grouped_gemm_gateup_swiglu", "moe_grouped_gemm_down", "moe_unpermute_combine",
     "moe_unpermute_combine_bwd", "moe_grouped_gemm_down_dgrad", "moe_grouped_gemm_down_wgrad",
-    "moe_grouped_gemm_down_bwd", "moe_swiglu_bwd", "moe_grouped_gemm_gateup_dgrad",
+    "moe_grouped_gemm_down_bwd", "moe_swiglu_bwd", "moe_grouped_gemm_down_dgrad_swiglu_bwd", "moe_grouped_gemm_gateup_dgrad",
     "moe_grouped_gemm_gateup_wgrad", "moe_grouped_gemm_gateup_swiglu_bwd", "moe_layer_arena_bytes",
     "moe_layer_fwd_bwd_host", "moe_router_topk", "moe_router_topk_bwd",
 ]
@@ -69,6 +69,7 @@ def load_library() -> ctypes.CDLL:
             "moe_grouped_gemm_down_wgrad": [dp, p, p, p, p, p],
             "moe_grouped_gemm_down_bwd": [dp, p, p, p, p, p, p, p],
             "moe_swiglu_bwd": [dp, p, p, p, p],
+            "moe_grouped_gemm_down_dgrad_swiglu_bwd": [dp, p, p, p, p, p, p],
             "moe_router_topk": [dp, p, p, p, p],
             "moe_router_topk_bwd": [dp, p, p, p, p, p],
             "moe_grouped_gemm_gateup_dgrad": [dp, p, p, p, p, p, p],
@@ -190,6 +191,11 @@ def moe_swiglu_bwd(d, dh_act, gu_saved, dgu):
     _call("moe_swiglu_bwd", ctypes.byref(d), _ptr(dh_act), _ptr(gu_saved), _ptr(dgu), _stream())
 
 
+def moe_grouped_gemm_down_dgrad_swiglu_bwd(d, dy_perm, w_down, gu_saved, offsets, dgu):
+    _call("moe_grouped_gemm_down_dgrad_swiglu_bwd", ctypes.byref(d), _ptr(dy_perm), _ptr(w_down), _ptr(gu_saved),
+          _ptr(offsets), _ptr(dgu), _stream())
+
+
 def moe_grouped_gemm_gateup_dgrad(d, dgu, w_gate, w_up, offsets, dx_perm):
     _call("moe_grouped_gemm_gateup_dgrad", ctypes.byref(d), _ptr(dgu), _ptr(w_gate), _ptr(w_up), _ptr(offsets),
           _ptr(dx_perm), _stream())
@@ -267,10 +273,17 @@ def layer_forward(b: LayerBuffers, x, topk_idx, topk_w, w_gate, w_up, w_down):
     moe_unpermute_combine(b.d, b.y_perm, topk_w, b.pair_to_row, b.y)
 
 
-def layer_backward(b: LayerBuffers, dy, topk_w, w_gate, w_up, w_down):
-    """a5..a8 in order on the current stream (after layer_forward)."""
+def layer_backward(b: LayerBuffers, dy, topk_w, w_gate, w_up, w_down, fused_swiglu_bwd: bool = False):
+    """a5..a8 in order on the current stream (after layer_forward).  With fused_swiglu_bwd the down dgrad and the
+    SwiGLU backward run as the one fused call (dh_act is then not written)."""
     moe_unpermute_combine_bwd(b.d, dy, b.y_perm, topk_w, b.pair_to_row, b.dy_perm, b.dtopk_w)
-    moe_grouped_gemm_down_bwd(b.d, b.dy_perm, b.h_act, w_down, b.offsets, b.dh_act, b.dw_down)
-    moe_grouped_gemm_gateup_swiglu_bwd(b.d, b.dh_act, b.gu, b.x_perm, w_gate, w_up, b.offsets, b.dgu, b.dx_perm,
-                                       b.dw_gate, b.dw_up)
+    if fused_swiglu_bwd:
+        moe_grouped_gemm_down_dgrad_swiglu_bwd(b.d, b.dy_perm, w_down, b.gu, b.offsets, b.dgu)
+        moe_grouped_gemm_down_wgrad(b.d, b.h_act, b.dy_perm, b.offsets, b.dw_down)
+        moe_grouped_gemm_gateup_dgrad(b.d, b.dgu, w_gate, w_up, b.offsets, b.dx_perm)
+        moe_grouped_gemm_gateup_wgrad(b.d, b.x_perm, b.dgu, b.offsets, b.dw_gate, b.dw_up)
+    else:
+        moe_grouped_gemm_down_bwd(b.d, b.dy_perm, b.h_act, w_down, b.offsets, b.dh_act, b.dw_down)
+        moe_grouped_gemm_gateup_swiglu_bwd(b.d, b.dh_act, b.gu, b.x_perm, w_gate, w_up, b.offsets, b.dgu, b.dx_perm,
+                                           b.dw_gate, b.dw_up)
     moe_permute_bwd(b.d, b.dx_perm, b.pair_to_row, b.dx)

@@ -161,6 +161,15 @@ int moe_grouped_gemm_down_dgrad(const moe_dims_t* dims, const void* dy_perm, con
     return launch_down_dgrad(*dims, cb(dy_perm), cb(w_down), offsets, mb(dh_act), st(stream));
 }
 
+int moe_grouped_gemm_down_dgrad_swiglu_bwd(const moe_dims_t* dims, const void* dy_perm, const void* w_down,
+                                           const void* gu_saved, const int32_t* offsets, void* dgu,
+                                           moe_stream_t stream) {
+    const void* const req[] = {dy_perm, w_down, gu_saved, offsets, dgu};
+    const void* const opt[] = {nullptr};
+    MOE_VALIDATE(dims, req, opt);
+    return launch_down_dgrad_swiglu_bwd(*dims, cb(dy_perm), cb(w_down), cb(gu_saved), offsets, mb(dgu), st(stream));
+}
+
 int moe_grouped_gemm_down_wgrad(const moe_dims_t* dims, const void* h_act, const void* dy_perm,
                                 const int32_t* offsets, void* dw_down, moe_stream_t stream) {
     const void* const req[] = {h_act, dy_perm, offsets, dw_down};

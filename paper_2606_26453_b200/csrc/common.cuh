@@ -49,6 +49,8 @@ int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_do
                       bf16* dh_act, cudaStream_t s);
 int launch_down_wgrad(const moe_dims_t& d, const bf16* h_act, const bf16* dy_perm, const int32_t* offsets,
                       bf16* dw_down, cudaStream_t s);
+int launch_down_dgrad_swiglu_bwd(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_down, const bf16* gu,
+                                 const int32_t* offsets, bf16* dgu, cudaStream_t s);
 int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate, const bf16* w_up,
                         const int32_t* offsets, bf16* dx_perm, cudaStream_t s);
 int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu, const int32_t* offsets,

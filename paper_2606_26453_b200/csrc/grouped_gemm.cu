@@ -82,9 +82,16 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 // column = row); the epilogue transposes it back through its shared-memory staging blocks.
 // FWD_SWIGLU_H is FWD_SWIGLU in pair mode with half-height last tiles (small experts); a kind of its own so that the
 // kernel for large experts carries none of its bookkeeping.
-enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3, FWD_PLAIN_T = 4, DGRAD_T = 5, FWD_SWIGLU_H = 6 };
+// DGRAD_SB / DGRAD_T_SB are DGRAD / DGRAD_T of the down projection with the SwiGLU backward fused into the epilogue:
+// the accumulator (dHact, fp32, never rounded) meets the saved pre-activations [g | u], which the epilogue warps fetch
+// as 32 x 32 blocks with bulk tensor loads, and the kernel writes dGU = [dg | du] instead of dHact.
+enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3, FWD_PLAIN_T = 4, DGRAD_T = 5, FWD_SWIGLU_H = 6,
+            DGRAD_SB = 7, DGRAD_T_SB = 8 };
 __host__ __device__ constexpr bool swiglu(int kind) { return kind == FWD_SWIGLU || kind == FWD_SWIGLU_H; }
-__host__ __device__ constexpr bool swapped(int kind) { return kind == FWD_PLAIN_T || kind == DGRAD_T; }
+__host__ __device__ constexpr bool swapped(int kind) { return kind == FWD_PLAIN_T || kind == DGRAD_T || kind == DGRAD_T_SB; }
+__host__ __device__ constexpr bool fused_sb(int kind) { return kind == DGRAD_SB || kind == DGRAD_T_SB; }
+// the kind whose operand loads and MMAs a kind shares
+__host__ __device__ constexpr int load_kind(int kind) { return kind == DGRAD_SB ? DGRAD : (kind == DGRAD_T_SB ? DGRAD_T : kind); }
 constexpr int SWAP_ROWS = 256;   // most rows of a swapped tile
 constexpr int SWAP_FEATS = 128;  // output features of a swapped tile
 
@@ -115,6 +122,7 @@ struct SharedCtl {
     unsigned long long drain;
     uint32_t tmem_base;
     int abort_flag;
+    unsigned long long gu_full[NUM_EPI_WARPS];   // fused SwiGLU backward: an epilogue warp's [g | u] blocks have landed
     int stage_half[MAX_STAGES];   // FWD_SWIGLU pair: the stage belongs to a half-height tile (published by the producer)
     int stage_n[MAX_STAGES];   // swapped kinds: MMA N (rows of the tile rounded up to 16) of the tile a stage belongs to
     int32_t offs[MAX_E + 1];
@@ -122,24 +130,19 @@ struct SharedCtl {
     int32_t sorted_rows[MAX_E];   // WGRAD: row count of the expert at each position of the largest-first order
 };
 
-// Ring geometry of the two launch shapes.
-template <bool PAIR>
+// Ring geometry of the two launch shapes.  WIDE: the epilogue warps also hold two 32 x 32 input blocks each (fused
+// SwiGLU backward), paid for with one ring stage.
+template <bool PAIR, bool WIDE = false>
 struct Geo {
-#ifndef MOE_PAIR_STAGES
-#define MOE_PAIR_STAGES 6
-#endif
-#ifndef MOE_PAIR_STAGING
-#define MOE_PAIR_STAGING 1
-#endif
-    static constexpr int STAGES = PAIR ? MOE_PAIR_STAGES : 4;
-    static constexpr int STAGING_BLOCKS = PAIR ? MOE_PAIR_STAGING : 1;   // staging blocks per epilogue warp (2 = ping-pong)
+    static constexpr int STAGES = PAIR ? (WIDE ? 5 : 6) : 4;
+    static constexpr int STAGING_BLOCKS = WIDE ? 3 : 1;   // per epilogue warp: the staging block (+ the g and u input blocks)
     static constexpr int TILE_M = PAIR ? 2 * BM : BM;        // output rows per tile (whole pair)
     static constexpr int BN_LOCAL = PAIR ? BN / 2 : BN;      // B columns this CTA keeps in shared memory
     static constexpr int A_BYTES = BM * BK * 2;              // 16 KB
     static constexpr int B_BYTES = BN_LOCAL * BK * 2;        // 16 / 32 KB
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;    // 32 / 48 KB
     static constexpr int RING_BYTES = STAGES * STAGE_BYTES;  // 160 / 192 KB
-    static constexpr int STAGING_BYTES = NUM_EPI_WARPS * STAGING_BLOCKS * STAGING_BLOCK_BYTES;   // 32 / 16 KB
+    static constexpr int STAGING_BYTES = NUM_EPI_WARPS * STAGING_BLOCKS * STAGING_BLOCK_BYTES;   // 16 KB (48 KB wide)
     static constexpr int SMEM_BYTES = RING_BYTES + STAGING_BYTES + 1024 + (int)sizeof(SharedCtl);
 };
 
@@ -502,7 +505,7 @@ __device__ __forceinline__ void stage_loads(const Tile& tl, int kb, const Params
         // map_r1 is the A map with a 64-row box there
         if (KIND == FWD_SWIGLU_H && tl.half) tma_load_2d(a_dst, map_r1, kb * BK, tl.row0 + (int)rank * (BM / 2), full);
         else tma_load_2d(a_dst, map_a, kb * BK, tl.row0 + my_rows, full);
-        if (KIND == DGRAD) {
+        if (load_kind(KIND) == DGRAD) {
             const bool second = kb >= p.k_split;
             const int kx = (second ? kb - p.k_split : kb) * BK;
             tma_load_2d(b_dst, second ? map_b1 : map_b0, kx, tl.e * p.b_rows_per_e + n_local, full);
@@ -547,7 +550,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const __grid_constant__ CUtensorMap map_b1, const __grid_constant__ CUtensorMap map_o0,
                     const __grid_constant__ CUtensorMap map_o1, const __grid_constant__ CUtensorMap map_x,
                     const Params p) {
-    using G = Geo<PAIR>;
+    using G = Geo<PAIR, fused_sb(KIND)>;
     constexpr int STAGES = G::STAGES;
     constexpr int STAGE_BYTES = G::STAGE_BYTES;
     constexpr bool SWAP = swapped(KIND);
@@ -594,6 +597,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             mbar_init(smem_u32(&ctl->tmem_empty[a]), PAIR ? 2 * NUM_EPI_WARPS : NUM_EPI_WARPS);
         }
         mbar_init(smem_u32(&ctl->drain), 1);
+        for (int w = 0; w < NUM_EPI_WARPS; ++w) mbar_init(smem_u32(&ctl->gu_full[w]), 1);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tmap(&map_a);
@@ -816,30 +820,31 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         uint8_t* stage_ptr = tiles_ptr + G::RING_BYTES + (warp - 2) * (G::STAGING_BLOCKS * STAGING_BLOCK_BYTES);
         const int sw = (lane >> 1) & 3;             // 64-byte swizzle: 16-byte piece j of row r sits at j ^ ((r>>1)&3)
         uint32_t n_stores = 0;                      // bulk stores issued so far by this warp
-        bool drain_first = false;                   // the next staging write must wait for ALL earlier stores
 
-        // stage one 32x32 bf16 block (this thread: 16 packed words of its row) and issue its bulk store;
-        // with two staging blocks the warp only waits for the store issued two blocks ago
-        auto stage_and_store = [&](const uint32_t (&w)[16], const CUtensorMap* map, int x, int y) {
-            uint8_t* blk = stage_ptr + (n_stores % G::STAGING_BLOCKS) * STAGING_BLOCK_BYTES;
-            if (n_stores >= (uint32_t)G::STAGING_BLOCKS) {
-                if (lane == 0) {
-                    if (G::STAGING_BLOCKS == 2 && !drain_first) bulk_wait_read1(); else bulk_wait_read0();
-                }
+        // before the staging block is written again: all earlier stores of this warp must have read it
+        auto staging_free = [&]() {
+            if (n_stores != 0) {
+                if (lane == 0) bulk_wait_read0();
                 __syncwarp();
-                drain_first = false;
             }
-            uint8_t* my_row = blk + lane * 64;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                *reinterpret_cast<uint4*>(my_row + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+        };
+        auto send_block = [&](const CUtensorMap* map, int x, int y) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
-                tma_store_2d(map, x, y, smem_u32(blk));
+                tma_store_2d(map, x, y, smem_u32(stage_ptr));
                 bulk_commit();
             }
             ++n_stores;
+        };
+        // stage one 32x32 bf16 block (this thread: 16 packed words of its row) and issue its bulk store
+        auto stage_and_store = [&](const uint32_t (&w)[16], const CUtensorMap* map, int x, int y) {
+            staging_free();
+            uint8_t* my_row = stage_ptr + lane * 64;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                *reinterpret_cast<uint4*>(my_row + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+            send_block(map, x, y);
         };
         auto direct_store = [&](const uint32_t (&w)[16], bf16* dst) {
             uint4* d4 = reinterpret_cast<uint4*>(dst);
@@ -849,27 +854,43 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // swapped kinds: this lane holds one output feature for 32 consecutive rows; the block is transposed on its
         // way into the staging buffer (row j of the block, feature `lane`: 2-byte stores, 64 contiguous bytes per
         // warp instruction) and then stored like any other 32 x 32 block
-        auto stage_transposed_and_store = [&](const uint32_t (&v)[32], const CUtensorMap* map, int x, int y) {
-            uint8_t* blk = stage_ptr + (n_stores % G::STAGING_BLOCKS) * STAGING_BLOCK_BYTES;
-            if (n_stores >= (uint32_t)G::STAGING_BLOCKS) {
-                if (lane == 0) {
-                    if (G::STAGING_BLOCKS == 2 && !drain_first) bulk_wait_read1(); else bulk_wait_read0();
-                }
-                __syncwarp();
-                drain_first = false;
-            }
+        auto stage_transposed_and_store = [&](const float (&v)[32], const CUtensorMap* map, int x, int y) {
+            staging_free();
             const int piece = lane >> 3, within = (lane & 7) * 2;
 #pragma unroll
             for (int j = 0; j < 32; ++j)
-                *reinterpret_cast<__nv_bfloat16*>(blk + j * 64 + (((piece ^ ((j >> 1) & 3)) << 4) + within)) =
-                    __float2bfloat16_rn(__uint_as_float(v[j]));
+                *reinterpret_cast<__nv_bfloat16*>(stage_ptr + j * 64 + (((piece ^ ((j >> 1) & 3)) << 4) + within)) =
+                    __float2bfloat16_rn(v[j]);
+            send_block(map, x, y);
+        };
+        // fused SwiGLU backward: the warp's g and u input blocks (behind its staging block), fetched with two bulk
+        // tensor loads from the saved pre-activations [R, 2I] (map_b1: 32 x 32 boxes, 64-byte swizzle)
+        uint8_t* g_blk = stage_ptr + STAGING_BLOCK_BYTES;
+        uint8_t* u_blk = stage_ptr + 2 * STAGING_BLOCK_BYTES;
+        const uint32_t gu_bar = smem_u32(&ctl->gu_full[warp - 2]);
+        uint32_t gu_phase = 0;
+        auto fetch_gu = [&](int x, int y) {   // x: column inside [0, I), y: first row of the block
+            if (lane == 0) {
+                mbar_arrive_expect_tx(gu_bar, 2 * STAGING_BLOCK_BYTES);
+                tma_load_2d(smem_u32(g_blk), &map_b1, x, y, gu_bar);
+                tma_load_2d(smem_u32(u_blk), &map_b1, p.I + x, y, gu_bar);
+            }
+        };
+        // Called by every lane with a value derived from ALL of its reads of the input blocks, before the next fetch
+        // into them is issued: the empty asm cannot run before those reads have delivered their data, and the warp
+        // barrier then holds lane 0's fetch back until every lane got here.  (A warp barrier alone only orders the
+        // ISSUE of the reads; under the operand traffic of the main loop a read can sit in the shared-memory queue long
+        // enough for a bulk load that hits in L2 to overwrite its word first: seen as a few wrong elements per 10^8.)
+        auto inputs_consumed = [&](uint32_t seen) {
+            asm volatile("" ::"r"(seen) : "memory");
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
-            if (lane == 0) {
-                tma_store_2d(map, x, y, smem_u32(blk));
-                bulk_commit();
-            }
-            ++n_stores;
+        };
+        // dg = dh*u*s*(1+g*(1-s)), du = dh*g*s with s = 1/(1+exp(-g))
+        auto swiglu_grad = [](float dh, float g, float u, float& dg, float& du) {
+            const float sg = 1.f / (1.f + __expf(-g));
+            dg = dh * u * sg * (1.f + g * (1.f - sg));
+            du = dh * g * sg;
         };
         const uint32_t tmem_empty_remote0 = PAIR ? map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0) : 0u;
         const uint32_t tmem_empty_remote1 = PAIR ? map_to_cta(smem_u32(&ctl->tmem_empty[1]), 0) : 0u;
@@ -897,20 +918,54 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 const int feat0 = tl.n0 + (PAIR ? (int)rank * SWAP_FEATS : 0) + quarter * 32;
                 const int n_row_blocks = (tl.rows + 31) >> 5;
 #pragma unroll 1
+                const bool feats_owed = feat0 < p.n_cols;
+                if (fused_sb(KIND) && feats_owed && half < n_row_blocks) fetch_gu(feat0, tl.row0 + half * 32);
                 for (int i = half; i < n_row_blocks; i += 2) {
-                    uint32_t v[32];
-                    tc_ld32(taddr + i * 32, v);
+                    uint32_t vr[32];
+                    tc_ld32(taddr + i * 32, vr);
                     tc_wait_ld();
-                    if (feat0 >= p.n_cols) continue;
+                    if (!feats_owed) continue;
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(vr[j]);
                     const int r0 = tl.row0 + i * 32;
                     const int rv = min(32, tl.rows - i * 32);
-                    if (rv == 32) {
+                    if (fused_sb(KIND)) {
+                        // element (row j, feature `lane`) of the g and u blocks; then the next block's fetch may start
+                        if (!mbar_wait(gu_bar, gu_phase, abort_flag)) break;
+                        gu_phase ^= 1u;
+                        const int piece = lane >> 3, within = (lane & 7) * 2;
+                        float du[32];
+                        uint32_t seen = 0;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int off = j * 64 + (((piece ^ ((j >> 1) & 3)) << 4) + within);
+                            const uint32_t gr = *reinterpret_cast<const uint16_t*>(g_blk + off);
+                            const uint32_t ur = *reinterpret_cast<const uint16_t*>(u_blk + off);
+                            seen ^= gr ^ (ur << 16);
+                            swiglu_grad(v[j], __uint_as_float(gr << 16), __uint_as_float(ur << 16), v[j], du[j]);
+                        }
+                        if (i + 2 < n_row_blocks) {
+                            inputs_consumed(seen);   // all reads of the two input blocks have returned
+                            fetch_gu(feat0, tl.row0 + (i + 2) * 32);
+                        }
+                        if (rv == 32) {
+                            stage_transposed_and_store(v, &map_o0, feat0, r0);
+                            stage_transposed_and_store(du, &map_o0, p.I + feat0, r0);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < rv) {
+                                    p.out0[(long long)(r0 + j) * p.ldo + feat0 + lane] = __float2bfloat16_rn(v[j]);
+                                    p.out0[(long long)(r0 + j) * p.ldo + p.I + feat0 + lane] = __float2bfloat16_rn(du[j]);
+                                }
+                        }
+                    } else if (rv == 32) {
                         stage_transposed_and_store(v, &map_o0, feat0, r0);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)   // rows past the tile belong to the expert's next tile, or to nobody
-                            if (j < rv)
-                                p.out0[(long long)(r0 + j) * p.ldo + feat0 + lane] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                            if (j < rv) p.out0[(long long)(r0 + j) * p.ldo + feat0 + lane] = __float2bfloat16_rn(v[j]);
                     }
                 }
             } else if (swiglu(KIND)) {
@@ -959,10 +1014,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     // expert without rows (WGRAD): a zero tile.  Clear the staging block once and send it to
                     // all of this warp's 32 x 32 output blocks back to back.
                     uint8_t* blk = stage_ptr;
-                    if (n_stores != 0) {
-                        if (lane == 0) bulk_wait_read0();
-                        __syncwarp();
-                    }
+                    staging_free();
 #pragma unroll
                     for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(blk + lane * 64 + j * 16) = make_uint4(0, 0, 0, 0);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -976,10 +1028,61 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         }
                         bulk_commit();
                     }
-                    n_stores += G::STAGING_BLOCKS;   // keeps the block rotation; the next staging write drains first
-                    drain_first = true;
-                } else
-                {
+                    ++n_stores;
+                } else if (fused_sb(KIND)) {
+                    // row-major tile with the SwiGLU backward fused: per 32-column block, the accumulator (dHact, fp32)
+                    // meets this row's g and u values (16-byte pieces of the lane's row of the two input blocks)
+                    constexpr int NC = BN / 64;
+                    const int c0 = half * NC;
+                    int n_owed = 0;                      // blocks of this warp inside the I columns
+                    for (int c = c0; c < c0 + NC; ++c) n_owed += (rows_valid != 0 && tl.n0 + c * 32 < p.n_cols) ? 1 : 0;
+                    if (n_owed != 0) fetch_gu(tl.n0 + c0 * 32, slab0);
+#pragma unroll 1
+                    for (int i = 0; i < NC; ++i) {
+                        uint32_t vr[32];
+                        tc_ld32(taddr + (c0 + i) * 32, vr);
+                        tc_wait_ld();
+                        if (i >= n_owed) continue;
+                        const int x = tl.n0 + (c0 + i) * 32;
+                        if (!mbar_wait(gu_bar, gu_phase, abort_flag)) break;
+                        gu_phase ^= 1u;
+                        uint4 gq[4], uq[4];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            gq[j] = *reinterpret_cast<const uint4*>(g_blk + lane * 64 + ((j ^ sw) << 4));
+                            uq[j] = *reinterpret_cast<const uint4*>(u_blk + lane * 64 + ((j ^ sw) << 4));
+                        }
+                        if (i + 1 < n_owed) {
+                            // the next fetch overwrites the two input blocks: every lane's reads must have RETURNED
+                            // (not merely been issued) before it starts
+                            uint32_t seen = 0;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) seen ^= gq[j].x ^ gq[j].y ^ gq[j].z ^ gq[j].w ^ uq[j].x ^ uq[j].y ^ uq[j].z ^ uq[j].w;
+                            inputs_consumed(seen);
+                            fetch_gu(x + 32, slab0);
+                        }
+                        uint32_t dgp[16], dup[16];
+                        const uint32_t* gw = reinterpret_cast<const uint32_t*>(gq);
+                        const uint32_t* uw = reinterpret_cast<const uint32_t*>(uq);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float2 g2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw[j]));
+                            const float2 u2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&uw[j]));
+                            float dg0, du0, dg1, du1;
+                            swiglu_grad(__uint_as_float(vr[2 * j]), g2.x, u2.x, dg0, du0);
+                            swiglu_grad(__uint_as_float(vr[2 * j + 1]), g2.y, u2.y, dg1, du1);
+                            dgp[j] = pack_bf16(dg0, dg1);
+                            dup[j] = pack_bf16(du0, du1);
+                        }
+                        if (rows_valid == 32) {
+                            stage_and_store(dgp, &map_o0, x, slab_y);
+                            stage_and_store(dup, &map_o0, p.I + x, slab_y);
+                        } else if (lane < rows_valid) {
+                            direct_store(dgp, p.out0 + row * p.ldo + x);
+                            direct_store(dup, p.out0 + row * p.ldo + p.I + x);
+                        }
+                    }
+                } else {
                     // software pipeline over the warp's four 32-column blocks: the TMEM load of the next block
                     // is in flight while the current one is converted, staged and stored
                     constexpr int NC = BN / 64;
@@ -1050,7 +1153,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     }
 }
 
-static_assert(Geo<false>::SMEM_BYTES <= 232448 && Geo<true>::SMEM_BYTES <= 232448,
+static_assert(Geo<false>::SMEM_BYTES <= 232448 && Geo<true>::SMEM_BYTES <= 232448 && Geo<true, true>::SMEM_BYTES <= 232448,
               "exceeds the 227 KB of shared memory a CTA can opt in to");
 
 // ---- host side ------------------------------------------------------------------------------------
@@ -1113,7 +1216,7 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
     auto kernel = grouped_gemm_kernel<KIND, PAIR>;
     if (grid_of_device[dev] == 0) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<PAIR>::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Geo<PAIR, fused_sb(KIND)>::SMEM_BYTES) != cudaSuccess)
             return MOE_ERR_CUDA;
         const int sms = sm_count();
         if (sms <= 0) return MOE_ERR_CUDA;
@@ -1122,7 +1225,7 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
             cudaLaunchAttribute qa[1];
             qa[0].id = cudaLaunchAttributeClusterDimension;
             qa[0].val.clusterDim.x = 2; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
-            qc.gridDim = dim3(2 * (sms / 2)); qc.blockDim = dim3(NUM_THREADS); qc.dynamicSmemBytes = Geo<PAIR>::SMEM_BYTES;
+            qc.gridDim = dim3(2 * (sms / 2)); qc.blockDim = dim3(NUM_THREADS); qc.dynamicSmemBytes = Geo<PAIR, fused_sb(KIND)>::SMEM_BYTES;
             qc.attrs = qa; qc.numAttrs = 1;
             int clusters = 0;
             if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &qc) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
@@ -1136,7 +1239,7 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
     cudaLaunchAttribute attr[1];
     cfg.gridDim = dim3(grid_of_device[dev]);
     cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = Geo<PAIR>::SMEM_BYTES;
+    cfg.dynamicSmemBytes = Geo<PAIR, fused_sb(KIND)>::SMEM_BYTES;
     cfg.stream = s;
     if (PAIR) {
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1249,6 +1352,34 @@ int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_do
     p.n_tiles = (d.I + BN - 1) / BN; p.n_cols = d.I; p.b_rows_per_e = d.I;
     p.out0 = dh_act; p.ldo = d.I; p.n_split = d.I;
     return launch<DGRAD, true>(a, b0, b0, o0, o0, a, p, s);
+}
+
+// Down dgrad with the SwiGLU backward in its epilogue: dgu = [dg | du] from dh = dy_perm . w_down[e]^T (kept in fp32)
+// and the saved pre-activations gu [R, 2I].  Same operands and tile schedules as launch_down_dgrad; the epilogue
+// warps fetch the [g | u] blocks through `g` (32 x 32 boxes of gu) and write two blocks of dgu per accumulator block.
+int launch_down_dgrad_swiglu_bwd(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_down, const bf16* gu,
+                                 const int32_t* offsets, bf16* dgu, cudaStream_t s) {
+    const uint64_t R = (uint64_t)d.T * d.K;
+    CUtensorMap g, o0;
+    if (!make_out_map(&g, gu, 2ull * d.I, R) || !make_out_map(&o0, dgu, 2ull * d.I, R)) return MOE_ERR_CUDA;
+    Params p = {};
+    p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
+    p.n_cols = d.I; p.b_rows_per_e = d.I; p.out0 = dgu; p.ldo = 2ll * d.I; p.n_split = d.I; p.I = d.I;
+    if (use_swapped(d)) {
+        const int feats = 2 * SWAP_FEATS;   // a CTA pair's tile
+        const uint32_t box = 32;            // row boxes of 32 / 64 / 128 rows per CTA
+        CUtensorMap a, a2, a1, b0;
+        if (!make_map(&a, dy_perm, d.H, R, BK, 4 * box) || !make_map(&a2, dy_perm, d.H, R, BK, 2 * box) ||
+            !make_map(&a1, dy_perm, d.H, R, BK, box) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, SWAP_FEATS))
+            return MOE_ERR_CUDA;
+        p.n_tiles = (d.I + feats - 1) / feats;
+        return launch<DGRAD_T_SB, true>(a, b0, g, o0, a2, a1, p, s);
+    }
+    CUtensorMap a, b0;
+    if (!make_map(&a, dy_perm, d.H, R, BK, BM) || !make_map(&b0, w_down, d.H, (uint64_t)d.E * d.I, BK, BN / 2))
+        return MOE_ERR_CUDA;
+    p.n_tiles = (d.I + BN - 1) / BN;
+    return launch<DGRAD_SB, true>(a, b0, g, o0, o0, a, p, s);
 }
 
 // Gate/up dgrad: dx_perm = dg . w_gate[e]^T + du . w_up[e]^T.  A = dgu [R,2I]; the contraction runs over the

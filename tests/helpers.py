@@ -65,7 +65,7 @@ def host_view(dev: dict) -> dict:
     return out
 
 
-def run_cuda_layer(dev: dict, E: int):
+def run_cuda_layer(dev: dict, E: int, fused_swiglu_bwd: bool = False):
     """Forward + backward through the C ABI; returns the buffer bundle."""
     from paper_2606_26453_b200 import binding as B
     T, H = dev["X"].shape
@@ -73,7 +73,8 @@ def run_cuda_layer(dev: dict, E: int):
     I = dev["W_gate"].shape[2]
     b = B.alloc_layer_buffers(T, H, I, E, K, device=dev["X"].device)
     B.layer_forward(b, dev["X"], dev["topk_idx"], dev["topk_w"], dev["W_gate"], dev["W_up"], dev["W_down"])
-    B.layer_backward(b, dev["dY"], dev["topk_w"], dev["W_gate"], dev["W_up"], dev["W_down"])
+    B.layer_backward(b, dev["dY"], dev["topk_w"], dev["W_gate"], dev["W_up"], dev["W_down"],
+                     fused_swiglu_bwd=fused_swiglu_bwd)
     torch.cuda.synchronize()
     assert B.moe_device_status() == 0
     return b

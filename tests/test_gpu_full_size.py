@@ -53,11 +53,16 @@ def test_indices_bit_exact(full):
     assert torch.equal(b.x_perm[rows], dev["X"][src])
 
 
+PACKED = [("x_perm", "X_perm"), ("h_act", "H_act"), ("gu", "GU"), ("y_perm", "Y_perm"), ("dy_perm", "dY_perm"),
+          ("dh_act", "dH_act"), ("dgu", "dGU"), ("dx_perm", "dX_perm")]
+
+
 def test_sampled_tokens_against_exact_chain(full):
+    """64 tokens (the first and the last among them) through the exact chain with all of their experts' weights:
+    Y, dX, dtopk_w of those tokens, and every packed intermediate row that belongs to one of their pairs."""
     cfg, dev, b = full
-    n_tok = {"few_large": 12, "paper_dw1": 8}.get(cfg.name, 24)
     rng = np.random.default_rng(cfg.cfg_id)
-    toks = np.sort(rng.choice(cfg.T, size=n_tok, replace=False))
+    toks = np.sort(rng.choice(cfg.T, size=64, replace=False))
     toks[0], toks[-1] = 0, cfg.T - 1
     idx = dev["topk_idx"].cpu().numpy()[toks]
     touched = np.unique(idx)
@@ -71,6 +76,23 @@ def test_sampled_tokens_against_exact_chain(full):
     Hh.assert_close(Hh.to_np64(b.y[tsel]), ref["Y"], "Y[sample]")
     Hh.assert_close(Hh.to_np64(b.dx[tsel]), ref["dX"], "dX[sample]")
     Hh.assert_close(b.dtopk_w[tsel].cpu().numpy().astype(np.float64), ref["dtopk_w"], "dtopk_w[sample]")
+    # row r' of the reduced layer is pair (t', k): the full layer keeps that pair in row pair_to_row[toks[t'] * K + k]
+    K = cfg.K
+    small_pairs = ref["row_to_pair"].astype(np.int64)
+    full_pairs = toks[small_pairs // K] * K + small_pairs % K
+    rows = b.pair_to_row[torch.from_numpy(full_pairs).cuda()].long()
+    for attr, key in PACKED:
+        Hh.assert_close(Hh.to_np64(getattr(b, attr)[rows]), ref[key], key + "[rows of the sampled tokens]")
+    # the same tokens through the chain that uses the fused down-dgrad + SwiGLU-backward call
+    from paper_2606_26453_b200 import binding as B
+    B.layer_backward(b, dev["dY"], dev["topk_w"], dev["W_gate"], dev["W_up"], dev["W_down"], fused_swiglu_bwd=True)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    Hh.assert_close(Hh.to_np64(b.dgu[rows]), ref["dGU"], "fused chain dGU[rows]")
+    Hh.assert_close(Hh.to_np64(b.dx_perm[rows]), ref["dX_perm"], "fused chain dX_perm[rows]")
+    Hh.assert_close(Hh.to_np64(b.dx[tsel]), ref["dX"], "fused chain dX[sample]")
+    B.layer_backward(b, dev["dY"], dev["topk_w"], dev["W_gate"], dev["W_up"], dev["W_down"])   # back to the two-call chain
+    torch.cuda.synchronize()
 
 
 def test_sampled_weight_gradient_blocks_against_exact_chain(full):
@@ -78,10 +100,12 @@ def test_sampled_weight_gradient_blocks_against_exact_chain(full):
     counts = b.counts.cpu().numpy()
     offsets = b.offsets.cpu().numpy()
     nonempty = np.flatnonzero(counts > 0)
+    rng = np.random.default_rng(100 + cfg.cfg_id)
+    # the largest expert, the smallest one with rows, a random one (an expert without rows is checked for exact zeros)
     chosen = {int(nonempty[np.argmax(counts[nonempty])]), int(nonempty[np.argmin(counts[nonempty])]),
-              int(nonempty[len(nonempty) // 2])}
+              int(rng.choice(nonempty)), int(nonempty[len(nonempty) // 2])}
     if cfg.name == "few_large":
-        chosen = {int(nonempty[0])}
+        chosen = {int(nonempty[0]), int(nonempty[-1])}        # 2k rows x 14336 columns each: two are enough
     chosen = sorted(chosen)
     I = cfg.I
     S = np.concatenate([np.arange(96, 160), np.arange(I - 64, I)])          # straddles a tile edge; last columns
@@ -108,3 +132,38 @@ def test_sampled_weight_gradient_blocks_against_exact_chain(full):
     # experts without rows: exact zeros everywhere
     for e in np.flatnonzero(counts == 0):
         assert not bool(b.dw_gate[e].any()) and not bool(b.dw_up[e].any()) and not bool(b.dw_down[e].any())
+
+
+# ------------------------------------------------------------------------------------------------
+# every element of every output, where the oracle can afford the whole layer (about 15 s and 45 s of host time)
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["fine_grained", "many_small"])
+def test_every_element_against_exact_chain(name):
+    from paper_2606_26453_b200 import binding as B
+    B.load_library()
+    cfg = W.CONFIGS[name]
+    dev = W.make_workload_device(cfg, torch.device("cuda", 0))
+    b = Hh.run_cuda_layer(dev, cfg.E)
+    host = Hh.host_view(dev)
+    ref = O.layer_fwd_bwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"], host["W_down"],
+                          host["dY"])
+    del host
+    for k in ("counts", "offsets", "row_to_pair", "pair_to_row"):
+        assert np.array_equal(getattr(b, k).cpu().numpy(), ref[k]), k
+    outputs = [("y", "Y"), ("dx", "dX"), ("dw_gate", "dW_gate"), ("dw_up", "dW_up"), ("dw_down", "dW_down")] + PACKED
+    for attr, key in outputs:
+        Hh.assert_close(getattr(b, attr).to(torch.float32).cpu().numpy(), ref[key], f"{name} {key} (every element)")
+    Hh.assert_close(b.dtopk_w.cpu().numpy(), ref["dtopk_w"], f"{name} dtopk_w (every element)")
+    # and the chain with the fused down-dgrad + SwiGLU-backward call
+    B.layer_backward(b, dev["dY"], dev["topk_w"], dev["W_gate"], dev["W_up"], dev["W_down"], fused_swiglu_bwd=True)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    for attr, key in (("dgu", "dGU"), ("dx_perm", "dX_perm"), ("dx", "dX"), ("dw_gate", "dW_gate"), ("dw_up", "dW_up")):
+        Hh.assert_close(getattr(b, attr).to(torch.float32).cpu().numpy(), ref[key], f"{name} fused chain {key} (every element)")
+    # run to run the fused call gives the same bits (a race on its shared-memory input blocks would show here)
+    first = b.dgu.clone()
+    for _ in range(4):
+        b.dgu.fill_(float("nan"))
+        B.moe_grouped_gemm_down_dgrad_swiglu_bwd(b.d, b.dy_perm, dev["W_down"], b.gu, b.offsets, b.dgu)
+        torch.cuda.synchronize()
+        assert torch.equal(b.dgu, first)

@@ -59,3 +59,29 @@ def test_random_layer_against_oracle(seed):
     for attr, key in FLOAT_OUTPUTS:
         Hh.assert_close(Hh.to_np64(getattr(b, attr)), ref[key], f"{key} counts={list(counts)} K={K} H={H} I={I}")
     Hh.assert_close(b.dtopk_w.cpu().numpy().astype(np.float64), ref["dtopk_w"], "dtopk_w")
+    # the same layer with the down dgrad and the SwiGLU backward as the one fused call
+    bf = Hh.run_cuda_layer(Hh.device_workload(host), cfg.E, fused_swiglu_bwd=True)
+    for attr, key in FLOAT_OUTPUTS:
+        if attr != "dh_act":                                  # never written by the fused chain
+            Hh.assert_close(Hh.to_np64(getattr(bf, attr)), ref[key], f"fused chain {key} counts={list(counts)} K={K} H={H} I={I}")
+
+
+@pytest.mark.parametrize("H,I,counts,K", [
+    (1408, 2880, [300, 1, 129, 430, 0], 2),          # the real widths: 1408 = 5.5 x 256, 2880 = 45 x 64 (partial column tiles)
+    (2880, 1408, [40, 700, 1, 0, 259], 1),
+    (2880, 2880, [520, 528, 8], 2),               # rows per expert above the pair / fixed-tile thresholds
+    (1408, 1408, [255, 257, 0, 600, 88], 2),
+])
+def test_real_widths_at_small_row_counts(H, I, counts, K):
+    from paper_2606_26453_b200 import binding as B
+    B.load_library()
+    cfg, host = Hh.ragged_workload(counts, K=K, H=H, I=I, seed=7)
+    ref = O.layer_fwd_bwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"], host["W_down"],
+                          host["dY"])
+    for fused in (False, True):
+        b = Hh.run_cuda_layer(Hh.device_workload(host), cfg.E, fused_swiglu_bwd=fused)
+        for name in ("counts", "offsets", "row_to_pair", "pair_to_row"):
+            assert np.array_equal(getattr(b, name).cpu().numpy(), ref[name]), name
+        for attr, key in FLOAT_OUTPUTS:
+            if not (fused and attr == "dh_act"):
+                Hh.assert_close(Hh.to_np64(getattr(b, attr)), ref[key], f"{key} H={H} I={I} fused={fused}")

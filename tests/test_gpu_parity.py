@@ -268,6 +268,28 @@ def test_gateup_swiglu_bwd(B, case):
         assert not Hh.to_np64(dwg[e]).any() and not Hh.to_np64(dwu[e]).any()
 
 
+def test_fused_down_dgrad_swiglu_bwd(B, case):
+    """The fused entry point against its oracle (inputs from the oracle chain, rounded to bf16), and against the
+    two-call form it replaces: the fused result may differ from it only by the rounding of dH_act it avoids."""
+    cfg, host, ref = case
+    d, R = _dims(B, cfg), cfg.R
+    dyp, gu = _r(ref["dY_perm"]), _r(ref["GU"])
+    off = _i32(ref["offsets"])
+    dgu = _nan((R, 2 * cfg.I))
+    B.moe_grouped_gemm_down_dgrad_swiglu_bwd(d, _bf(dyp), _bf(host["W_down"]), _bf(gu), off, dgu)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    o_dgu = O.down_dgrad_swiglu_bwd(dyp, host["W_down"], gu, ref["offsets"])
+    Hh.assert_close(Hh.to_np64(dgu), o_dgu, "dGU (fused)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    dh, dgu2 = _nan((R, cfg.I)), _nan((R, 2 * cfg.I))
+    B.moe_grouped_gemm_down_dgrad(d, _bf(dyp), _bf(host["W_down"]), off, dh)
+    B.moe_swiglu_bwd(d, dh, _bf(gu), dgu2)
+    torch.cuda.synchronize()
+    two = Hh.error_stats(Hh.to_np64(dgu2), o_dgu)
+    one = Hh.error_stats(Hh.to_np64(dgu), o_dgu)
+    assert one["rel_fro"] <= two["rel_fro"] * 1.02, (one, two)      # one rounding fewer: never worse
+
+
 def test_gateup_pieces_from_given_dgu(B, case):
     """dgrad and wgrad alone, fed the oracle's dGU: isolates the two GEMMs from the elementwise kernel."""
     cfg, host, ref = case

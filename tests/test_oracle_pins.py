@@ -267,6 +267,33 @@ def test_packed_intermediate_gradients_match_autograd():
     np.testing.assert_allclose(f["Y"], Y.detach().numpy(), rtol=1e-12, atol=1e-12)
 
 
+def test_fused_down_dgrad_swiglu_bwd_is_the_gradient_of_the_loss_wrt_the_pre_activations():
+    """The fused call's oracle: dGU from dY_perm, W_down and the saved pre-activations alone.  Pinned by torch
+    autograd of sum(dY_perm * (silu(g) * u) @ Wd[e]) with respect to [g | u] (an expert without rows included), and
+    by a central difference along a random direction."""
+    Xn, idx, wn, Wgn, Wun, Wdn, dYn = small_problem(T=15, H=6, I=10, E=5, K=2, seed=41, empty=(3,))
+    f = O.layer_fwd_bwd(Xn, idx, wn, Wgn, Wun, Wdn, dYn)
+    off, I = f["offsets"], Wgn.shape[2]
+    assert off[4] == off[3]                                   # the expert without rows is really there
+    got = O.down_dgrad_swiglu_bwd(f["dY_perm"], Wdn, f["GU"], off)
+    GU = torch.tensor(f["GU"]).requires_grad_(True)
+    Wd, dYp = torch.tensor(Wdn), torch.tensor(f["dY_perm"])
+
+    def loss(gu):
+        h = torch.nn.functional.silu(gu[:, :I]) * gu[:, I:]
+        return sum(((h[off[e]:off[e + 1]] @ Wd[e]) * dYp[off[e]:off[e + 1]]).sum() for e in range(Wd.shape[0]))
+
+    loss(GU).backward()
+    np.testing.assert_allclose(got, GU.grad.numpy(), rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(got, f["dGU"], rtol=1e-12, atol=1e-13)      # and it is the chain's dGU
+    rng = np.random.default_rng(5)
+    D = rng.standard_normal(f["GU"].shape)
+    eps = 1e-6
+    with torch.no_grad():
+        fd = (loss(torch.tensor(f["GU"] + eps * D)) - loss(torch.tensor(f["GU"] - eps * D))).item() / (2 * eps)
+    assert abs(fd - float((got * D).sum())) <= 1e-7 * max(1.0, abs(fd))
+
+
 def test_backward_central_differences():
     X, idx, w, Wg, Wu, Wd, dY = small_problem(T=10, H=7, I=9, E=4, K=2, seed=41)
     f = O.layer_fwd_bwd(X, idx, w, Wg, Wu, Wd, dY)
