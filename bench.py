@@ -138,23 +138,31 @@ def call_bytes(cfg):
             "permute_bwd": R * H * 2 + T * H * 2 + R * 4}
 
 
-def make_step(B, b, wl):
+CALLS_FUSED = ["permute", "gateup_swiglu", "down", "combine", "combine_bwd", "down_dgrad_swiglu_bwd", "down_wgrad",
+               "gateup_dgrad", "gateup_wgrad", "permute_bwd"]
+
+
+def make_step(B, b, wl, fused=False):
+    """One layer step as a list of C-ABI calls: CALLS, or CALLS_FUSED (the down dgrad and the SwiGLU backward as the
+    one fused call)."""
     x, idx, w, dy = wl["X"], wl["topk_idx"], wl["topk_w"], wl["dY"]
     wg, wu, wd = wl["W_gate"], wl["W_up"], wl["W_down"]
     d = b.d
-    fns = [
-        lambda: B.moe_permute(d, x, idx, b.x_perm, b.counts, b.offsets, b.row_to_pair, b.pair_to_row, b.workspace),
-        lambda: B.moe_grouped_gemm_gateup_swiglu(d, b.x_perm, wg, wu, b.offsets, b.h_act, b.gu),
-        lambda: B.moe_grouped_gemm_down(d, b.h_act, wd, b.offsets, b.y_perm),
-        lambda: B.moe_unpermute_combine(d, b.y_perm, w, b.pair_to_row, b.y),
-        lambda: B.moe_unpermute_combine_bwd(d, dy, b.y_perm, w, b.pair_to_row, b.dy_perm, b.dtopk_w),
-        lambda: B.moe_grouped_gemm_down_dgrad(d, b.dy_perm, wd, b.offsets, b.dh_act),
-        lambda: B.moe_grouped_gemm_down_wgrad(d, b.h_act, b.dy_perm, b.offsets, b.dw_down),
-        lambda: B.moe_swiglu_bwd(d, b.dh_act, b.gu, b.dgu),
-        lambda: B.moe_grouped_gemm_gateup_dgrad(d, b.dgu, wg, wu, b.offsets, b.dx_perm),
-        lambda: B.moe_grouped_gemm_gateup_wgrad(d, b.x_perm, b.dgu, b.offsets, b.dw_gate, b.dw_up),
-        lambda: B.moe_permute_bwd(d, b.dx_perm, b.pair_to_row, b.dx),
-    ]
+    table = {
+        "permute": lambda: B.moe_permute(d, x, idx, b.x_perm, b.counts, b.offsets, b.row_to_pair, b.pair_to_row, b.workspace),
+        "gateup_swiglu": lambda: B.moe_grouped_gemm_gateup_swiglu(d, b.x_perm, wg, wu, b.offsets, b.h_act, b.gu),
+        "down": lambda: B.moe_grouped_gemm_down(d, b.h_act, wd, b.offsets, b.y_perm),
+        "combine": lambda: B.moe_unpermute_combine(d, b.y_perm, w, b.pair_to_row, b.y),
+        "combine_bwd": lambda: B.moe_unpermute_combine_bwd(d, dy, b.y_perm, w, b.pair_to_row, b.dy_perm, b.dtopk_w),
+        "down_dgrad": lambda: B.moe_grouped_gemm_down_dgrad(d, b.dy_perm, wd, b.offsets, b.dh_act),
+        "down_wgrad": lambda: B.moe_grouped_gemm_down_wgrad(d, b.h_act, b.dy_perm, b.offsets, b.dw_down),
+        "swiglu_bwd": lambda: B.moe_swiglu_bwd(d, b.dh_act, b.gu, b.dgu),
+        "down_dgrad_swiglu_bwd": lambda: B.moe_grouped_gemm_down_dgrad_swiglu_bwd(d, b.dy_perm, wd, b.gu, b.offsets, b.dgu),
+        "gateup_dgrad": lambda: B.moe_grouped_gemm_gateup_dgrad(d, b.dgu, wg, wu, b.offsets, b.dx_perm),
+        "gateup_wgrad": lambda: B.moe_grouped_gemm_gateup_wgrad(d, b.x_perm, b.dgu, b.offsets, b.dw_gate, b.dw_up),
+        "permute_bwd": lambda: B.moe_permute_bwd(d, b.dx_perm, b.pair_to_row, b.dx),
+    }
+    fns = [table[c] for c in (CALLS_FUSED if fused else CALLS)]
 
     def step(events=None):
         if events is None:
@@ -167,6 +175,39 @@ def make_step(B, b, wl):
             events[i + 1].record()
 
     return step
+
+
+def time_fused_variant(B, cfg, res, device, seconds=0.8, rounds=4):
+    """The step with moe_grouped_gemm_down_dgrad_swiglu_bwd in place of moe_grouped_gemm_down_dgrad + moe_swiglu_bwd,
+    timed beside the two-call step: blocks of steps of the two forms alternate (so that both see the same power and
+    clock state), events around every call."""
+    b, wl = res["buffers"], res["wl"]
+    forms = {"two_call": (make_step(B, b, wl), CALLS), "fused": (make_step(B, b, wl, fused=True), CALLS_FUSED)}
+    ms_est = res["total_ms"] / res["steps"]
+    n = max(2, int(seconds * 1e3 / ms_est / (2 * rounds)))
+    tot = {k: 0.0 for k in forms}
+    per = {k: {c: 0.0 for c in names} for k, (_, names) in forms.items()}
+    for _ in range(2):
+        forms["fused"][0]()
+    for _ in range(rounds):
+        for k, (step, names) in forms.items():
+            evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(n)]
+            for s in range(n):
+                step(evs[s])
+            torch.cuda.synchronize()
+            tot[k] += evs[0][0].elapsed_time(evs[-1][-1])
+            for i, c in enumerate(names):
+                per[k][c] += sum(e[i].elapsed_time(e[i + 1]) for e in evs)
+    steps = n * rounds
+    if B.moe_device_status() != 0:
+        raise RuntimeError("device status word is set after the fused-variant steps")
+    two, fus = tot["two_call"] / steps, tot["fused"] / steps
+    return {"steps_each": steps, "two_call_ms_per_step": two, "fused_ms_per_step": fus, "step_time_ratio": fus / two,
+            "fused_layer_tflops": cfg.flops_fwd_bwd / (fus * 1e-3) / 1e12,
+            "down_dgrad_ms": per["two_call"]["down_dgrad"] / steps, "swiglu_bwd_ms": per["two_call"]["swiglu_bwd"] / steps,
+            "down_dgrad_swiglu_bwd_ms": per["fused"]["down_dgrad_swiglu_bwd"] / steps,
+            "note": "alternating blocks of the two step forms; the fused call writes dGU straight from the fp32 "
+                    "accumulator (dH_act is never materialised)"}
 
 
 def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True, min_seconds=0.0):
@@ -584,6 +625,7 @@ def run_ours(args):
         line["sustained"] = time_sustained(B, cfg, res, device)
         line["sustained"]["frac"] = fractions(line["sustained"]["value"], peaks)
         line["stream_calibration_in_step"] = stream_calibration_in_step(B, cfg, res, device)
+        line["fused_dgrad_swiglu_bwd"] = time_fused_variant(B, cfg, res, device)
         del res
         torch.cuda.empty_cache()
         for name in args.also:
@@ -592,6 +634,7 @@ def run_ours(args):
             c2 = W.CONFIGS[name]
             r2 = time_config(B, c2, device, 3, 3, None, sample_clocks=True, min_seconds=args.other_min_seconds)
             extra.append(summarize(c2, r2, peaks, peaks_kind, sms))
+            extra[-1]["fused_dgrad_swiglu_bwd"] = time_fused_variant(B, c2, r2, device, seconds=0.5)
             del r2
             torch.cuda.empty_cache()
         if extra:

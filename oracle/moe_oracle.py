@@ -28,7 +28,11 @@ Pins (tests/test_oracle_*.py): brute-force counting sort, stable-sort library ro
 SwiGLU MLP special cases evaluated with an independent library (torch, fp64), per-token loop,
 torch.autograd on a per-token formulation, central finite differences, identities of
 permute/unpermute, empty-expert zeros; for the router: a per-row selection loop, a library softmax,
-shift invariance, the all-ties closed form, finite differences.  No function here is "parity unpinned".
+shift invariance, the all-ties closed form, finite differences; for the fused down-dgrad + SwiGLU backward:
+autograd with respect to the saved pre-activations; for the block-scaled FP8 quantiser: the round trip of all 254
+finite codes, a library FP8 cast inside the range, hand-built blocks for the scale choice, ties and saturation,
+the half-ulp error bound, idempotence, and per-element products written out by hand.  No function here is
+"parity unpinned".
 """
 from __future__ import annotations
 
@@ -292,3 +296,77 @@ def router_topk_bwd(topk_idx, topk_w, dtopk_w, E):
     dz = np.zeros((T, E), dtype=F64)
     np.put_along_axis(dz, idx, w * (dw - inner), axis=1)
     return dz
+
+
+# ---- block-scaled FP8 (MXFP8) operands for the grouped GEMMs --------------------------------------
+# Format (the OCP Microscaling "MXFP8" format the Blackwell tensor cores consume with kind::mxf8f6f4):
+#   * elements: FP8 E4M3 -- 1 sign, 4 exponent (bias 7), 3 mantissa bits; no infinities, S.1111.111 is NaN,
+#     largest finite value 448 = 1.75 * 2^8, subnormals m * 2^-9;
+#   * one shared scale per block of 32 consecutive elements ALONG THE CONTRACTION AXIS: E8M0, i.e. the power of
+#     two 2^(s - 127) stored as the byte s in [0, 254];
+#   * the scale of a block with largest magnitude a > 0 is 2^(floor(log2 a) - 8) (8 = exponent of the largest E4M3
+#     power of two), clamped to the E8M0 range; the elements are v / scale rounded to nearest even onto the E4M3
+#     grid, magnitudes above 448 saturating to 448; an all-zero block takes the smallest scale and zero codes.
+# The paper itself only names FP8 tensor-core paths among its micro-profiling tools; this is the Blackwell follow-up
+# of the bf16 GEMMs and is held to its own tolerance (a 3-bit mantissa cannot meet the bf16 bounds).
+E4M3_MAX = 448.0
+MX_BLOCK = 32
+
+
+def e4m3_decode(codes):
+    """uint8 E4M3 codes -> float64 values (NaN for the two NaN codes)."""
+    c = np.asarray(codes).astype(np.int64)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = (c & 0x7).astype(F64)
+    val = np.where(e == 0, m * 2.0 ** -9, (1.0 + m / 8.0) * np.exp2((e - 7).astype(F64)))
+    val = np.where((e == 15) & ((c & 0x7) == 7), np.nan, val)
+    return sign * val
+
+
+def e4m3_encode(y):
+    """float64 -> uint8 E4M3 codes: round to nearest, ties to even, magnitudes above 448 saturate to 448."""
+    y = _f64(y)
+    a = np.minimum(np.abs(y), 1e30)
+    # spacing of the E4M3 grid around a: 2^-9 below the smallest normal 2^-6, else 2^(floor(log2 a) - 3)
+    ex = np.floor(np.log2(np.maximum(a, 2.0 ** -6)))
+    step = np.exp2(ex - 3.0)
+    q = np.rint(a / step) * step            # numpy rint = round half to even; a/step is exact (step a power of two)
+    q = np.minimum(q, E4M3_MAX)
+    # q back to fields
+    qe = np.floor(np.log2(np.maximum(q, 2.0 ** -6)))
+    is_sub = q < 2.0 ** -6
+    e_field = np.where(is_sub, 0, qe + 7).astype(np.int64)
+    m_field = np.where(is_sub, np.rint(q * 2.0 ** 9), np.rint((q / np.exp2(qe) - 1.0) * 8.0)).astype(np.int64)
+    code = (e_field << 3) | m_field
+    code = np.where(np.signbit(y), code | 0x80, code)
+    return code.astype(np.uint8)
+
+
+def mxfp8_quantize(x):
+    """Block-scaled FP8 quantisation along the LAST axis (length a multiple of 32).
+
+    Returns (codes uint8 same shape, scales uint8 [..., n/32], dequantised float64 same shape)."""
+    x = _f64(x)
+    n = x.shape[-1]
+    assert n % MX_BLOCK == 0
+    blocks = x.reshape(x.shape[:-1] + (n // MX_BLOCK, MX_BLOCK))
+    amax = np.max(np.abs(blocks), axis=-1)
+    safe = np.where(amax > 0, amax, 1.0)
+    s_exp = np.where(amax > 0, np.floor(np.log2(safe)) - 8.0, -127.0)
+    s_exp = np.clip(s_exp, -127.0, 127.0)
+    scale = np.exp2(s_exp)
+    codes = e4m3_encode(blocks / scale[..., None])
+    deq = e4m3_decode(codes) * scale[..., None]
+    return codes.reshape(x.shape), (s_exp + 127.0).astype(np.uint8), deq.reshape(x.shape)
+
+
+def down_mxfp8(H_act, W_down, offsets):
+    """The down projection with both operands block-scaled FP8 along the contraction (I):
+    Yp[r,:] = Q(Hact[r,:]) @ Q(Wd[e]) where Q quantises Hact row-wise in blocks of 32 along I and Wd[e] column-wise
+    in blocks of 32 along I (each output feature h has its own scales), and the product of the dequantised
+    operands is taken exactly.  Returns Yp [R,H] float64."""
+    _, _, a_deq = mxfp8_quantize(H_act)
+    Wt = np.swapaxes(_f64(W_down), 1, 2)                 # [E, H, I]: contraction last
+    _, _, b_deq = mxfp8_quantize(Wt)
+    return down(a_deq, np.swapaxes(b_deq, 1, 2), offsets)

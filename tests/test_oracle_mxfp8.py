@@ -1,0 +1,106 @@
+"""Pins of the oracle's block-scaled FP8 (MXFP8: E4M3 elements, E8M0 scale per 32 elements) quantiser and of the
+quantised down projection, against what the format definition and the mathematics fix."""
+import numpy as np
+import torch
+
+from oracle import moe_oracle as O
+
+
+def test_all_e4m3_codes_round_trip_and_match_the_library_type():
+    codes = np.arange(256, dtype=np.uint8)
+    vals = O.e4m3_decode(codes)
+    finite = ~np.isnan(vals)
+    assert (~finite).sum() == 2 and np.isnan(vals[0x7F]) and np.isnan(vals[0xFF])
+    assert vals[0x7E] == 448.0 and vals[0x01] == 2.0 ** -9 and vals[0x08] == 2.0 ** -6 and vals[0x38] == 1.0
+    # decode agrees with torch's float8_e4m3fn bit pattern interpretation
+    lib = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(vals[finite], lib[finite])
+    # every representable value encodes to its own code (negative zero keeps its sign bit)
+    back = O.e4m3_encode(vals[finite])
+    assert np.array_equal(back, codes[finite])
+
+
+def test_e4m3_encode_rounds_to_nearest_even_and_saturates():
+    # halfway between 1.0 (mantissa 000, even) and 1.125 (001): ties to 1.0; between 1.125 and 1.25 (010): to 1.25
+    assert O.e4m3_decode(O.e4m3_encode([1.0625, 1.1875, -1.0625]))[...].tolist() == [1.0, 1.25, -1.0]
+    # just above / below a halfway point
+    assert O.e4m3_decode(O.e4m3_encode([1.0625 + 1e-9, 1.1875 - 1e-9])).tolist() == [1.125, 1.125]
+    # subnormal grid 2^-9: 1.5 * 2^-9 ties to even (2 * 2^-9), 0.5 * 2^-9 ties to zero
+    assert O.e4m3_decode(O.e4m3_encode([1.5 * 2.0 ** -9, 0.5 * 2.0 ** -9, 0.75 * 2.0 ** -9])).tolist() == [2.0 ** -8, 0.0, 2.0 ** -9]
+    # saturation instead of NaN/inf; 464 is halfway between 448 and the (non-existent) 480
+    assert O.e4m3_decode(O.e4m3_encode([449.0, 464.0, 500.0, 1e9, -1e9])).tolist() == [448.0, 448.0, 448.0, 448.0, -448.0]
+    # in range, the library cast (round to nearest even) gives the same codes
+    rng = np.random.default_rng(0)
+    y = np.concatenate([rng.uniform(-440, 440, 4000), rng.standard_normal(4000) * 0.01, rng.standard_normal(4000)])
+    lib = torch.from_numpy(y).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = O.e4m3_encode(y)
+    nz = O.e4m3_decode(got) != 0          # the sign of a value that rounds to zero is the one place conventions may differ
+    assert np.array_equal(got[nz], lib[nz])
+
+
+def test_scale_selection_on_hand_built_blocks():
+    blk = np.zeros((5, 32))
+    blk[0, 3] = 1.0            # amax 1 = 2^0        -> scale 2^-8, code of 256 = 1.0 * 2^8
+    blk[1, 7] = -447.9         # amax in [256, 512)  -> scale 2^0
+    blk[2, :] = 3.0e-5         # amax 3e-5 ~ 1.97 * 2^-16 -> floor(log2) = -16 -> scale 2^-24
+    blk[3, 0] = 500.0          # amax 500 -> floor(log2) = 8 -> scale 2^0: 500 saturates to 448
+    # row 4 stays all zero
+    codes, scales, deq = O.mxfp8_quantize(blk)
+    assert scales[:, 0].tolist() == [127 - 8, 127, 127 - 24, 127, 0]
+    assert deq[0, 3] == 1.0 and codes[0, 3] == O.e4m3_encode([256.0])[0]
+    assert deq[1, 7] == -448.0
+    assert deq[3, 0] == 448.0
+    assert not codes[4].any() and not deq[4].any()
+    # the largest element of a block always lands in [256, 512) before rounding: top binade, never a subnormal
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((64, 96)) * np.exp2(rng.integers(-20, 20, size=(64, 1)))
+    codes, scales, deq = O.mxfp8_quantize(x)
+    top = np.max(np.abs(O.e4m3_decode(codes)).reshape(64, 3, 32), axis=-1)
+    assert np.all((top >= 256.0) & (top <= 448.0))
+    # scales are per block of 32 along the last axis and nothing else
+    assert scales.shape == (64, 3)
+    c2, s2, d2 = O.mxfp8_quantize(x[:, 32:64])
+    assert np.array_equal(c2, codes[:, 32:64]) and np.array_equal(s2[:, 0], scales[:, 1])
+
+
+def test_quantisation_error_bound_and_idempotence():
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((200, 128))
+    codes, scales, deq = O.mxfp8_quantize(x)
+    scale = np.exp2(scales.astype(np.float64) - 127.0).repeat(32, axis=1)
+    # elements that stay normal after scaling (|v| >= 2^-6 * scale): relative error at most half an ulp = 2^-4;
+    # the rest: absolute error at most half the subnormal spacing; saturated top elements: below 512 -> 448, 12.5 %
+    normal = np.abs(x) >= 2.0 ** -6 * scale
+    sat = np.abs(x) / scale > 448.0
+    assert np.all(np.abs(deq - x)[normal & ~sat] <= 2.0 ** -4 * np.abs(x)[normal & ~sat] * (1 + 1e-12))
+    assert np.all(np.abs(deq - x)[~normal] <= 2.0 ** -10 * scale[~normal] * (1 + 1e-12))
+    assert np.all(np.abs(deq - x)[sat] <= 0.125 * np.abs(x)[sat])
+    # quantising the dequantised values changes nothing (they are representable with the same scales)
+    c2, s2, d2 = O.mxfp8_quantize(deq)
+    assert np.array_equal(c2, codes) and np.array_equal(s2, scales) and np.array_equal(d2, deq)
+    # typical size of the error of a Gaussian block: a few per cent, far above bf16's 2^-9
+    rel = np.linalg.norm(deq - x) / np.linalg.norm(x)
+    assert 0.015 < rel < 0.04
+
+
+def test_down_mxfp8_is_the_exact_product_of_the_dequantised_operands():
+    rng = np.random.default_rng(3)
+    E, I, H = 3, 64, 24
+    counts = [5, 0, 9]
+    offsets = np.concatenate([[0], np.cumsum(counts)])
+    Hact = rng.standard_normal((14, I))
+    Wd = rng.standard_normal((E, I, H)) * 0.05
+    got = O.down_mxfp8(Hact, Wd, offsets)
+    # written out per element with the quantiser applied by hand to each operand vector
+    for r, e in ((0, 0), (4, 0), (5, 2), (13, 2)):
+        a = O.mxfp8_quantize(Hact[r])[2]
+        for h in (0, 7, 23):
+            b = O.mxfp8_quantize(Wd[e, :, h])[2]          # the weight column's own scales along I
+            assert abs(got[r, h] - float(a @ b)) <= 1e-12
+    # against the unquantised product: a few per cent, and exactly equal when the operands are representable
+    ref = O.down(Hact, Wd, offsets)
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert 0.01 < rel < 0.06
+    Hq = O.mxfp8_quantize(Hact)[2]
+    Wq = np.swapaxes(O.mxfp8_quantize(np.swapaxes(Wd, 1, 2))[2], 1, 2)
+    assert np.array_equal(O.down_mxfp8(Hq, Wq, offsets), O.down(Hq, Wq, offsets))
