@@ -205,6 +205,34 @@ int moe_router_topk(const moe_dims_t* dims, const float* logits, int32_t* topk_i
 int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const float* topk_w,
                         const float* dtopk_w, float* dlogits, moe_stream_t stream);
 
+/* ---- block-scaled FP8 (MXFP8) down projection -------------------------------------------------
+ * A lower-precision twin of moe_grouped_gemm_down on the block-scaled tensor-core path (the paper only names FP8
+ * tensor-core paths among its micro-profiling tools; the format is the OCP Microscaling MXFP8 one): both operands
+ * as FP8 E4M3 codes with one E8M0 scale byte s (value 2^(s-127)) per 32 consecutive elements ALONG THE CONTRACTION
+ * (I).  Scale of a block with largest magnitude a > 0: 2^(floor(log2 a) - 8), clamped to the E8M0 range; elements:
+ * value / scale rounded to nearest even onto the E4M3 grid, magnitudes above 448 saturating; an all-zero block has
+ * s = 0 and zero codes.  Products of the dequantised operands accumulate in fp32; y_perm is bf16.  The result is
+ * that of the quantised operands, NOT within the bf16 tolerances of the unquantised layer (a 3-bit mantissa: a few
+ * per cent relative error per tensor).  Requires H and I to be multiples of 128 (MOE_ERR_UNSUPPORTED_SHAPE otherwise).
+ *   moe_mxfp8_quantize_h_act   h_act [R,I] bf16 -> codes [R,I] bytes; scales: moe_mxfp8_act_scale_bytes(dims) bytes
+ *                              laid out [I/128][R][4]: the scale bytes of the 4 blocks of 32 inside the 128-wide
+ *                              slice kt of row r are bytes scales[(kt*R + r)*4 + 0..3].
+ *   moe_mxfp8_quantize_w_down  w_down [E,I,H] bf16 -> codes_t [E,H,I] bytes (transposed: contraction contiguous);
+ *                              scales: moe_mxfp8_w_down_scale_bytes(dims) bytes laid out [E][H/128][I/128][512]:
+ *                              the scale of feature h, block b of 32 along I, is byte
+ *                              (h%32)*16 + ((h%128)/32)*4 + b%4 of the 512-byte group (e, h/128, b/4).
+ *   moe_grouped_gemm_down_mxfp8  y_perm[r,:] = dequant(h row r) . dequant(w_down[e]) for rows r of expert e.
+ * All pointers device, 16-byte aligned; codes and scales are caller-owned buffers. */
+size_t moe_mxfp8_act_scale_bytes(const moe_dims_t* dims);
+size_t moe_mxfp8_w_down_scale_bytes(const moe_dims_t* dims);
+int moe_mxfp8_quantize_h_act(const moe_dims_t* dims, const void* h_act, void* codes, void* scales,
+                             moe_stream_t stream);
+int moe_mxfp8_quantize_w_down(const moe_dims_t* dims, const void* w_down, void* codes_t, void* scales,
+                              moe_stream_t stream);
+int moe_grouped_gemm_down_mxfp8(const moe_dims_t* dims, const void* h_codes, const void* h_scales,
+                                const void* w_codes_t, const void* w_scales, const int32_t* offsets,
+                                void* y_perm, moe_stream_t stream);
+
 /* ---- whole layer from HOST activations ------------------------------------------------------
  * One training step of the layer for a caller whose per-step tensors live in host memory:
  * copies x, topk_idx, topk_w, dy (HOST pointers; pinned memory makes the copies asynchronous)

@@ -23,6 +23,8 @@ EXPORTS = [
     "moe_grouped_gemm_down_bwd", "moe_swiglu_bwd", "moe_grouped_gemm_down_dgrad_swiglu_bwd", "moe_grouped_gemm_gateup_dgrad",
     "moe_grouped_gemm_gateup_wgrad", "moe_grouped_gemm_gateup_swiglu_bwd", "moe_layer_arena_bytes",
     "moe_layer_fwd_bwd_host", "moe_router_topk", "moe_router_topk_bwd",
+    "moe_mxfp8_act_scale_bytes", "moe_mxfp8_w_down_scale_bytes", "moe_mxfp8_quantize_h_act", "moe_mxfp8_quantize_w_down",
+    "moe_grouped_gemm_down_mxfp8",
 ]
 
 
@@ -53,6 +55,9 @@ def load_library() -> ctypes.CDLL:
         lib.moe_permute_workspace_bytes.argtypes = [ctypes.POINTER(MoeDims)]
         lib.moe_layer_arena_bytes.restype = ctypes.c_size_t
         lib.moe_layer_arena_bytes.argtypes = [ctypes.POINTER(MoeDims)]
+        for name in ("moe_mxfp8_act_scale_bytes", "moe_mxfp8_w_down_scale_bytes"):
+            getattr(lib, name).restype = ctypes.c_size_t
+            getattr(lib, name).argtypes = [ctypes.POINTER(MoeDims)]
         lib.moe_device_status.restype = ctypes.c_int
         lib.moe_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
         p = ctypes.c_void_p
@@ -76,6 +81,9 @@ def load_library() -> ctypes.CDLL:
             "moe_grouped_gemm_gateup_wgrad": [dp, p, p, p, p, p, p],
             "moe_grouped_gemm_gateup_swiglu_bwd": [dp, p, p, p, p, p, p, p, p, p, p, p],
             "moe_layer_fwd_bwd_host": [dp] + [p] * 14 + [ctypes.c_size_t, p],
+            "moe_mxfp8_quantize_h_act": [dp, p, p, p, p],
+            "moe_mxfp8_quantize_w_down": [dp, p, p, p, p],
+            "moe_grouped_gemm_down_mxfp8": [dp, p, p, p, p, p, p, p],
         }
         for name, argtypes in sigs.items():
             fn = getattr(lib, name)
@@ -209,6 +217,27 @@ def moe_grouped_gemm_gateup_wgrad(d, x_perm, dgu, offsets, dw_gate, dw_up):
 def moe_grouped_gemm_gateup_swiglu_bwd(d, dh_act, gu_saved, x_perm, w_gate, w_up, offsets, dgu, dx_perm, dw_gate, dw_up):
     _call("moe_grouped_gemm_gateup_swiglu_bwd", ctypes.byref(d), _ptr(dh_act), _ptr(gu_saved), _ptr(x_perm),
           _ptr(w_gate), _ptr(w_up), _ptr(offsets), _ptr(dgu), _ptr(dx_perm), _ptr(dw_gate), _ptr(dw_up), _stream())
+
+
+def moe_mxfp8_act_scale_bytes(d: MoeDims) -> int:
+    return int(load_library().moe_mxfp8_act_scale_bytes(ctypes.byref(d)))
+
+
+def moe_mxfp8_w_down_scale_bytes(d: MoeDims) -> int:
+    return int(load_library().moe_mxfp8_w_down_scale_bytes(ctypes.byref(d)))
+
+
+def moe_mxfp8_quantize_h_act(d, h_act, codes, scales):
+    _call("moe_mxfp8_quantize_h_act", ctypes.byref(d), _ptr(h_act), _ptr(codes), _ptr(scales), _stream())
+
+
+def moe_mxfp8_quantize_w_down(d, w_down, codes_t, scales):
+    _call("moe_mxfp8_quantize_w_down", ctypes.byref(d), _ptr(w_down), _ptr(codes_t), _ptr(scales), _stream())
+
+
+def moe_grouped_gemm_down_mxfp8(d, h_codes, h_scales, w_codes_t, w_scales, offsets, y_perm):
+    _call("moe_grouped_gemm_down_mxfp8", ctypes.byref(d), _ptr(h_codes), _ptr(h_scales), _ptr(w_codes_t), _ptr(w_scales),
+          _ptr(offsets), _ptr(y_perm), _stream())
 
 
 def moe_layer_fwd_bwd_host(d, x_host, topk_idx_host, topk_w_host, dy_host, w_gate, w_up, w_down, y_host, dx_host,

@@ -8,8 +8,8 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libmoe_b200.so")
-SOURCES = ["api.cu", "movement.cu", "router.cu", "grouped_gemm.cu"]
-HEADERS = ["common.cuh", os.path.join("..", "..", "include", "moe_b200.h")]
+SOURCES = ["api.cu", "movement.cu", "router.cu", "grouped_gemm.cu", "mxfp8.cu"]
+HEADERS = ["common.cuh", "tc_ptx.cuh", os.path.join("..", "..", "include", "moe_b200.h")]
 
 
 def _nvcc() -> str:

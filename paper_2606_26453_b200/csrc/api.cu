@@ -236,6 +236,57 @@ int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const f
     return launch_router_topk_bwd(*dims, topk_idx, topk_w, dtopk_w, dlogits, st(stream));
 }
 
+// ---- block-scaled FP8 down projection ----
+static int check_mx_dims(const moe_dims_t* d) {
+    const int st_ = check_dims(d);
+    if (st_ != MOE_OK) return st_;
+    return (d->H % 128 != 0 || d->I % 128 != 0) ? MOE_ERR_UNSUPPORTED_SHAPE : MOE_OK;
+}
+
+size_t moe_mxfp8_act_scale_bytes(const moe_dims_t* dims) {
+    if (check_mx_dims(dims) != MOE_OK) return 0;
+    return (size_t)(dims->I / 128) * (size_t)dims->T * dims->K * 4;
+}
+
+size_t moe_mxfp8_w_down_scale_bytes(const moe_dims_t* dims) {
+    if (check_mx_dims(dims) != MOE_OK) return 0;
+    return (size_t)dims->E * (dims->H / 128) * (dims->I / 128) * 512;
+}
+
+int moe_mxfp8_quantize_h_act(const moe_dims_t* dims, const void* h_act, void* codes, void* scales, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {h_act, codes, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_rows((long long)dims->T * dims->K, dims->I, cb(h_act), static_cast<uint8_t*>(codes),
+                                   static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_mxfp8_quantize_w_down(const moe_dims_t* dims, const void* w_down, void* codes_t, void* scales, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {w_down, codes_t, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_w_down(*dims, cb(w_down), static_cast<uint8_t*>(codes_t), static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_grouped_gemm_down_mxfp8(const moe_dims_t* dims, const void* h_codes, const void* h_scales, const void* w_codes_t,
+                                const void* w_scales, const int32_t* offsets, void* y_perm, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {h_codes, h_scales, w_codes_t, w_scales, offsets, y_perm};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_down_fwd_mxfp8(*dims, static_cast<const uint8_t*>(h_codes), static_cast<const uint8_t*>(h_scales),
+                                 static_cast<const uint8_t*>(w_codes_t), static_cast<const uint8_t*>(w_scales), offsets,
+                                 mb(y_perm), st(stream));
+}
+
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).
 namespace {
 // Two side streams (uploads, downloads) and a few events per device for moe_layer_fwd_bwd_host, created on first

@@ -15,6 +15,7 @@ typedef __nv_bfloat16 bf16;
 // record MOE_ERR_TIMEOUT there when a bounded wait runs out.  Synchronises the device.
 int read_and_clear_device_status(int* status_out);
 int movement_read_and_clear_status(int* status_out);   // the data-movement kernels' word (movement.cu)
+int mx_read_and_clear_status(int* status_out);         // the block-scaled FP8 kernels' word (mxfp8.cu)
 
 // Number of SMs of the current device (cached per device ordinal).
 int sm_count();
@@ -55,5 +56,11 @@ int launch_gateup_dgrad(const moe_dims_t& d, const bf16* dgu, const bf16* w_gate
                         const int32_t* offsets, bf16* dx_perm, cudaStream_t s);
 int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu, const int32_t* offsets,
                         bf16* dw_gate, bf16* dw_up, cudaStream_t s);
+
+// ---- block-scaled FP8 down projection (mxfp8.cu) -------------------------------------------------
+int launch_mx_quantize_rows(long long rows, int n, const bf16* x, uint8_t* codes, uint8_t* scales, cudaStream_t s);
+int launch_mx_quantize_w_down(const moe_dims_t& d, const bf16* w_down, uint8_t* codes_t, uint8_t* scales, cudaStream_t s);
+int launch_down_fwd_mxfp8(const moe_dims_t& d, const uint8_t* h_codes, const uint8_t* h_scales, const uint8_t* w_codes_t,
+                          const uint8_t* w_scales, const int32_t* offsets, bf16* y_perm, cudaStream_t s);
 
 }  // namespace moe

@@ -1,0 +1,95 @@
+"""Block-scaled FP8 (MXFP8) down projection through the C ABI against the oracle's quantiser and quantised product.
+
+Integer results (element codes, scale bytes) are compared bit for bit: both sides decide them on exact values.  The GEMM
+is held to the per-call bound of the bf16 kernels against the EXACT product of the dequantised operands (products of
+two E4M3 values and their power-of-two scales are exact in fp32; what remains is fp32 accumulation and the one rounding
+of the output to bf16).  Against the unquantised layer the result is a few per cent off by construction: stated, not
+tested against the bf16 tolerances."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_2606_26453_b200 import workloads as W
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2606_26453_b200 import binding
+    binding.load_library()
+    return binding
+
+
+def _act_scales_from_layout(raw, R, I):
+    """[I/128][R][4] bytes -> [R, I/32]"""
+    return raw.reshape(I // 128, R, 4).transpose(1, 0, 2).reshape(R, I // 32)
+
+
+def _w_scales_from_layout(raw, E, H, I):
+    """[E][H/128][I/128][512] bytes with byte (h%32)*16 + ((h%128)/32)*4 + b%4 -> [E, H, I/32]"""
+    g = raw.reshape(E, H // 128, I // 128, 32, 4, 4)          # [..., h%32, (h%128)/32, b%4]
+    return g.transpose(0, 1, 4, 3, 2, 5).reshape(E, H, I // 32)
+
+
+CASES = {
+    "one_tile": ([128], 1, 128, 128),
+    "ragged": ([0, 1, 127, 0, 129, 128, 300, 15, 0], 2, 256, 384),
+    "wide": ([200, 0, 31, 290, 1], 2, 384, 1408),              # 11 slices of the contraction, 3 column tiles
+    "many_tiles": ([700, 513, 64], 1, 128, 256),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_quantisers_and_gemm_against_the_oracle(B, name):
+    counts, K, H, I = CASES[name]
+    cfg, host = Hh.ragged_workload(counts, K=K, H=H, I=I, seed=21)
+    ref = O.layer_fwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"], host["W_down"])
+    R, E = cfg.R, cfg.E
+    d = B.dims(cfg.T, H, I, E, K)
+    # the activation as the CUDA side sees it: the oracle's H_act rounded to bf16, with a few awkward values put in
+    h = W.round_to_bf16(ref["H_act"].astype(np.float32))
+    h[0, :32] = 0.0                                  # an all-zero block
+    h[min(3, R - 1), 32:64] = 2.0 ** -100            # tiny block
+    h[R - 1, I - 32:] = np.linspace(-500.0, 500.0, 32, dtype=np.float32)   # includes values that saturate after scaling
+    h = W.round_to_bf16(h)
+    w = host["W_down"].copy()
+    w[0, :32, 0] = 0.0
+    h_dev, w_dev = Hh.to_dev_bf16(h), Hh.to_dev_bf16(w)
+    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    hc, hs = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    wc, ws = u8(E * H * I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
+    assert hs.numel() == (I // 128) * R * 4 and ws.numel() == E * (H // 128) * (I // 128) * 512
+    B.moe_mxfp8_quantize_h_act(d, h_dev, hc, hs)
+    B.moe_mxfp8_quantize_w_down(d, w_dev, wc, ws)
+    torch.cuda.synchronize()
+    o_hc, o_hs, h_deq = O.mxfp8_quantize(h)
+    wt = np.swapaxes(w, 1, 2)                        # [E, H, I]
+    o_wc, o_ws, _ = O.mxfp8_quantize(wt)
+    assert np.array_equal(_act_scales_from_layout(hs.cpu().numpy(), R, I), o_hs)
+    assert np.array_equal(hc.cpu().numpy().reshape(R, I), o_hc)
+    assert np.array_equal(_w_scales_from_layout(ws.cpu().numpy(), E, H, I), o_ws)
+    assert np.array_equal(wc.cpu().numpy().reshape(E, H, I), o_wc)
+    # the GEMM on the quantised operands
+    yp = torch.full((R, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    off = torch.from_numpy(ref["offsets"]).cuda()
+    B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, off, yp)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    o_y = O.down_mxfp8(h, w, ref["offsets"])
+    Hh.assert_close(Hh.to_np64(yp), o_y, f"{name}: Y_perm (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    # for orientation: distance to the unquantised product (a few per cent: the format, not the kernel)
+    exact = O.down(h, w, ref["offsets"])
+    rel = np.linalg.norm(Hh.to_np64(yp) - exact) / np.linalg.norm(exact)
+    assert rel < 0.08
+
+
+def test_shapes_the_block_scaled_path_does_not_take_are_refused(B):
+    d = B.dims(64, 192, 128, 2, 1)                   # H not a multiple of 128
+    assert B.moe_mxfp8_act_scale_bytes(d) == 0
+    t = torch.zeros(64 * 192, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_mxfp8_quantize_h_act(d, t, t, t)
+    assert ei.value.status == 3
