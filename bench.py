@@ -177,6 +177,43 @@ def make_step(B, b, wl, fused=False):
     return step
 
 
+def time_mxfp8_down(B, cfg, res, device, reps=20):
+    """The block-scaled FP8 twin of the down projection on this workload's own H_act, weights and offsets: the two
+    quantisers and the GEMM, each timed alone (back to back, events), beside the bf16 call timed the same way."""
+    if cfg.H % 128 or cfg.I % 128:
+        return None
+    b, wl = res["buffers"], res["wl"]
+    d = b.d
+    u8 = lambda n: torch.empty(n, dtype=torch.uint8, device=device)
+    hc, hs = u8(cfg.R * cfg.I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    wc, ws = u8(cfg.E * cfg.H * cfg.I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
+    yq = torch.empty_like(b.y_perm)
+    fns = {"bf16_down_ms": lambda: B.moe_grouped_gemm_down(d, b.h_act, wl["W_down"], b.offsets, b.y_perm),
+           "quantize_h_act_ms": lambda: B.moe_mxfp8_quantize_h_act(d, b.h_act, hc, hs),
+           "quantize_w_down_ms": lambda: B.moe_mxfp8_quantize_w_down(d, wl["W_down"], wc, ws),
+           "mxfp8_down_ms": lambda: B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, b.offsets, yq)}
+    out = {}
+    for name, fn in fns.items():
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = e0.elapsed_time(e1) / reps
+    fl = 2.0 * cfg.R * cfg.H * cfg.I
+    out["bf16_down_tflops"] = fl / (out["bf16_down_ms"] * 1e-3) / 1e12
+    out["mxfp8_down_tflops"] = fl / (out["mxfp8_down_ms"] * 1e-3) / 1e12
+    out["rel_frobenius_to_bf16_result"] = float((yq.float() - b.y_perm.float()).norm() / b.y_perm.float().norm())
+    out["note"] = ("E4M3 elements, E8M0 scale per 32 along the contraction; 128 x 128 single-CTA tiles on "
+                   "tcgen05.mma kind::mxf8f6f4.block_scale; the bf16 twin runs 256 x 256 CTA-pair tiles")
+    if B.moe_device_status() != 0:
+        raise RuntimeError("device status word is set after the MXFP8 calls")
+    return out
+
+
 def time_fused_variant(B, cfg, res, device, seconds=0.8, rounds=4):
     """The step with moe_grouped_gemm_down_dgrad_swiglu_bwd in place of moe_grouped_gemm_down_dgrad + moe_swiglu_bwd,
     timed beside the two-call step: blocks of steps of the two forms alternate (so that both see the same power and
@@ -626,6 +663,7 @@ def run_ours(args):
         line["sustained"]["frac"] = fractions(line["sustained"]["value"], peaks)
         line["stream_calibration_in_step"] = stream_calibration_in_step(B, cfg, res, device)
         line["fused_dgrad_swiglu_bwd"] = time_fused_variant(B, cfg, res, device)
+        line["mxfp8_down"] = time_mxfp8_down(B, cfg, res, device)
         del res
         torch.cuda.empty_cache()
         for name in args.also:
@@ -635,6 +673,7 @@ def run_ours(args):
             r2 = time_config(B, c2, device, 3, 3, None, sample_clocks=True, min_seconds=args.other_min_seconds)
             extra.append(summarize(c2, r2, peaks, peaks_kind, sms))
             extra[-1]["fused_dgrad_swiglu_bwd"] = time_fused_variant(B, c2, r2, device, seconds=0.5)
+            extra[-1]["mxfp8_down"] = time_mxfp8_down(B, c2, r2, device)
             del r2
             torch.cuda.empty_cache()
         if extra:
