@@ -10,9 +10,9 @@
 //   warps 2..9  epilogue: tcgen05.ld the accumulator (32-lane quarter x half of the columns), apply
 //               the epilogue (plain / SwiGLU), round to bf16, stage 32x32 blocks in swizzled shared
 //               memory and write them with bulk tensor stores
-//   warp 10     (WGRAD only) tail-fix warp: clears the surplus rows of an expert's last K block once its
-//               loads have landed and only then signals the stage as full, so that the MMA warp's issue
-//               loop carries no tail handling
+//   warp 10     (WGRAD only) tail-fix warp: clears the surplus rows of an expert's ragged last K block once its
+//               loads have landed and only then signals that stage as full, so that the MMA warp's issue
+//               loop carries no tail handling (all other stages go from the loads straight to the MMA warp)
 // The accumulator is double buffered (2 x 256 of the 512 TMEM columns) so the epilogue of one tile
 // overlaps the main loop of the next.
 //
@@ -22,11 +22,12 @@
 //           loads its 128 rows of A and HALF of B (6 stages of 32 KB), the tensor cores of both SMs
 //           read both halves.  That cuts the bytes each SM must pull from L2 per flop by a third
 //           and deepens the ring, which is what the L2 -> SM path needs at full MMA rate.  Every
-//           TMA load has a single destination CTA: each CTA's loads complete on its own
-//           barrier, a relay warp in the second CTA forwards "my half has landed" to the first
-//           CTA's barrier with a remote mbarrier arrive, and the first CTA's MMA warp releases
-//           stages / publishes accumulators in both CTAs with one tcgen05.commit that arrives on
-//           the barriers of both CTAs.
+//           TMA load has a single destination CTA (no multicast), but both CTAs' loads of a stage
+//           report their bytes to the SAME barrier, the one of the first CTA whose MMA warp waits on
+//           it (cp.async.bulk.tensor with .cta_group::2 may complete on the peer's barrier), so a
+//           stage goes from the two producers to the MMA warp without a relay in between; the MMA
+//           warp releases stages / publishes accumulators in both CTAs with one tcgen05.commit
+//           that arrives on the barriers of both CTAs.
 //
 // Two ragged shapes occur:
 //   row-ragged (forward, dgrad): output rows are the packed rows of an expert.  A tile starts at
@@ -37,8 +38,8 @@
 //     and, for the SwiGLU forward, half-height last tiles (FWD_SWIGLU_H: M = 128 over the pair).
 //   contraction-ragged (wgrad; the paper's dW1_e = X_e^T G_e): the expert's rows are the
 //     contraction.  The last K block issues only ceil(rem/16) MMAs (guard predicates) and the < 16
-//     surplus rows are zeroed in shared memory first, by the tail-fix warp (first CTA) and the relay
-//     warp (second CTA); an expert without rows gets a zero tile.
+//     surplus rows are zeroed in shared memory first, by the tail-fix warp of each CTA (warp 10 in the
+//     first, warp 1 in the second); an expert without rows gets a zero tile.
 //
 // All waits are bounded: a wait that runs out records MOE_ERR_TIMEOUT in the device status word,
 // raises a CTA-wide abort flag and every role leaves through the common teardown.
@@ -83,6 +84,7 @@ constexpr int TMEM_COLS = 512;
 // as 32 x 32 blocks with bulk tensor loads, and the kernel writes dGU = [dg | du] instead of dHact.
 enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3, FWD_PLAIN_T = 4, DGRAD_T = 5, FWD_SWIGLU_H = 6,
             DGRAD_SB = 7, DGRAD_T_SB = 8 };
+__host__ __device__ constexpr bool wgrad(int kind) { return kind == WGRAD; }
 __host__ __device__ constexpr bool swiglu(int kind) { return kind == FWD_SWIGLU || kind == FWD_SWIGLU_H; }
 __host__ __device__ constexpr bool swapped(int kind) { return kind == FWD_PLAIN_T || kind == DGRAD_T || kind == DGRAD_T_SB; }
 __host__ __device__ constexpr bool fused_sb(int kind) { return kind == DGRAD_SB || kind == DGRAD_T_SB; }
@@ -137,7 +139,7 @@ struct Geo {
     static constexpr int A_BYTES = BM * BK * 2;              // 16 KB
     static constexpr int B_BYTES = BN_LOCAL * BK * 2;        // 16 / 32 KB
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;    // 32 / 48 KB
-    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;  // 160 / 192 KB
+    static constexpr int RING_BYTES = STAGES * STAGE_BYTES;  // 160 ... 192 KB
     static constexpr int STAGING_BYTES = NUM_EPI_WARPS * STAGING_BLOCKS * STAGING_BLOCK_BYTES;   // 16 KB (48 KB wide)
     static constexpr int SMEM_BYTES = RING_BYTES + STAGING_BYTES + 1024 + (int)sizeof(SharedCtl);
 };
@@ -199,7 +201,7 @@ __device__ __forceinline__ void raster(int local, int m_tiles, int n_tiles, int&
 template <int KIND>
 __device__ __forceinline__ long long tile_of(long long it, long long who, long long n_who, long long total) {
     long long t;
-    if (KIND == WGRAD) {
+    if (wgrad(KIND)) {
         if (it * n_who >= total) return -1;
         t = it * n_who + ((it & 1) ? n_who - 1 - who : who);
     } else {
@@ -210,14 +212,14 @@ __device__ __forceinline__ long long tile_of(long long it, long long who, long l
 
 template <int KIND>
 __device__ __forceinline__ long long total_tiles(const Params& p, const SharedCtl* ctl) {
-    if (KIND == WGRAD) return (long long)p.E * p.m_tiles * p.n_tiles;
+    if (wgrad(KIND)) return (long long)p.E * p.m_tiles * p.n_tiles;
     return (long long)ctl->tile_prefix[p.E] * p.n_tiles;
 }
 
 template <int KIND, int TILE_M>
 __device__ __forceinline__ Tile decode_tile(const Params& p, const SharedCtl* ctl, long long t) {
     Tile tl;
-    if (KIND == WGRAD) {
+    if (wgrad(KIND)) {
         const int per_e = p.m_tiles * p.n_tiles;
         const int e_rank = (int)(t / per_e);
         tl.e = ctl->tile_prefix[e_rank];   // WGRAD: this array holds the experts ordered by row count, largest first
@@ -279,11 +281,19 @@ __device__ __forceinline__ void zero_k_rows(uint8_t* stage_ptr, int n_chunks, in
 // The TMA loads of one ring stage: k-block `kb` of tile `tl`, for the CTA with row offset `my_rows` inside
 // the tile (and, in pair mode, its half of B).  (Prefetching the same boxes into L2 a few k-blocks ahead was
 // tried and cost 10-15 %: the L2 -> SM path, not DRAM latency, is what these kernels saturate.)
-template <int KIND, bool PAIR>
+// `full` is the barrier the loads report to: a shared::cta address, or (REMOTE_BAR, pair mode) a shared::cluster address
+// of a barrier of the MMA-issuing CTA.
+template <int KIND, bool PAIR, bool REMOTE_BAR>
 __device__ __forceinline__ void stage_loads(const Tile& tl, int kb, const Params& p, const CUtensorMap* map_a,
                                          const CUtensorMap* map_r2, const CUtensorMap* map_r1,
                                          const CUtensorMap* map_b0, const CUtensorMap* map_b1, uint32_t a_dst,
                                          uint32_t b_dst, uint32_t full, uint32_t rank, int my_rows) {
+    auto tma_load_2d = [](uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+        if (REMOTE_BAR) tma_load_2d_pair(dst, map, x, y, bar); else moe::tma_load_2d(dst, map, x, y, bar);
+    };
+    auto tma_load_3d = [](uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+        if (REMOTE_BAR) tma_load_3d_pair(dst, map, x, y, z, bar); else moe::tma_load_3d(dst, map, x, y, z, bar);
+    };
     const int n_local = tl.n0 + (PAIR ? my_rows : 0);   // first B column this CTA loads
     if (swapped(KIND)) {
         // M side (a_dst): the weight tile, 128 output features x 64 k.  N side (b_dst): the tile's rows in boxes of
@@ -312,7 +322,7 @@ __device__ __forceinline__ void stage_loads(const Tile& tl, int kb, const Params
         } else {
             tma_load_2d(b_dst, map_a, kb * BK, my_row0, full);
         }
-    } else if (KIND == WGRAD) {
+    } else if (wgrad(KIND)) {
         const int krow = tl.k_row0 + kb * BK;
         // MN-major operands: one 3-D box = all 64-wide chunks, chunk-major in shared memory
         tma_load_3d(a_dst, map_a, 0, krow, (tl.row0 + my_rows) >> 6, full);
@@ -377,8 +387,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     static_assert(!HALF_TILES || PAIR, "half-height tiles exist in pair mode only");
     constexpr int ROW_TILE = SWAP ? SWAP_ROWS : G::TILE_M;   // rows an expert's tile count is computed from
     // operand major-ness of the MMA's M side (A) and N side (B); for the swapped kinds A is the weight tile
-    constexpr bool A_MN = (KIND == WGRAD || KIND == FWD_PLAIN_T);
-    constexpr bool B_MN = (swiglu(KIND) || KIND == FWD_PLAIN || KIND == WGRAD);
+    constexpr bool A_MN = (wgrad(KIND) || KIND == FWD_PLAIN_T);
+    constexpr bool B_MN = (swiglu(KIND) || KIND == FWD_PLAIN || wgrad(KIND));
     constexpr uint32_t IDESC = make_idesc(G::TILE_M, BN, A_MN, B_MN);
     constexpr uint32_t IDESC_HALF = make_idesc(BM, BN, A_MN, B_MN);   // 128 x 256 over the CTA pair
     constexpr uint32_t A_KSTEP = A_MN ? 2048 : 32;   // bytes per 16 k inside a stage
@@ -396,9 +406,6 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const long long first_tile = PAIR ? (long long)(blockIdx.x >> 1) : (long long)blockIdx.x;
     const long long tile_stride = PAIR ? (long long)(gridDim.x >> 1) : (long long)gridDim.x;
     const int my_rows = rank * BM;                                 // this CTA's row offset inside the tile
-    // WGRAD, MMA-issuing CTA: loads complete on landed[]; the tail-fix warp clears surplus contraction rows
-    // and only then arrives on full[], so the MMA warp's loop has no tail branch at all
-    const bool local_fix = (KIND == WGRAD) && rank == 0;
 
     // ---- set-up: barriers, schedule tables, TMEM ----
     for (int e = threadIdx.x; e <= p.E; e += NUM_THREADS) ctl->offs[e] = p.offsets[e];
@@ -425,7 +432,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         prefetch_tmap(&map_x);
     }
     __syncthreads();
-    if (KIND == WGRAD) {
+    if (wgrad(KIND)) {
         // experts by row count, largest first (ties: lower id first): rank by counting, O(E^2 / threads)
         for (int e = threadIdx.x; e < p.E; e += NUM_THREADS) {
             const int n_e = ctl->offs[e + 1] - ctl->offs[e];
@@ -467,46 +474,54 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
     if (warp == 0) {
         // ================= TMA producer (both CTAs of a pair; each fills its own ring) =================
+        // Where a stage's loads report: normally straight to full[stage] of the MMA-issuing CTA -- in pair mode both
+        // CTAs' loads complete on that one barrier (two arrivals, one per producer, each announcing its own bytes), so
+        // a stage travels producer -> loads -> MMA with no relay hop.  Only a weight-gradient stage whose ragged last
+        // K block needs surplus rows cleared reports to this CTA's landed[stage]; the tail-fix / relay warp clears the
+        // rows and makes the arrival on full[stage] in the producer's place.
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0;
             bool ok = true;
+            const uint32_t full0 = PAIR ? map_to_cta(smem_u32(&ctl->full[0]), 0) : smem_u32(&ctl->full[0]);
             for (long long it = 0; ok; ++it) {
                 const long long t = tile_of<KIND>(it, first_tile, tile_stride, n_tiles_total);
                 if (t < 0) break;
                 const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
                 for (int kb = 0; kb < tl.k_blocks; ++kb) {
                     if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t land = smem_u32(local_fix ? &ctl->landed[stage] : &ctl->full[stage]);
+                    const bool fix = wgrad(KIND) && kb == tl.k_blocks - 1 && (tl.k_rows & 15) != 0;
+                    uint32_t bytes = STAGE_BYTES;
                     if (SWAP) {
                         ctl->stage_n[stage] = (tl.rows + 15) & ~15;   // read by the MMA thread after its wait on full[stage]
                         const int my_n = PAIR ? (((tl.rows + 15) & ~15) >> 1) : tl.rows;
                         constexpr int BOX = PAIR ? 32 : 64;
-                        mbar_arrive_expect_tx(land, G::A_BYTES + min(4, (my_n + BOX - 1) / BOX) * (BOX * BK * 2));
+                        bytes = G::A_BYTES + min(4, (my_n + BOX - 1) / BOX) * (BOX * BK * 2);
                     } else if (HALF_TILES) {
                         ctl->stage_half[stage] = tl.half;   // read by the MMA thread after its wait on full[stage]
-                        mbar_arrive_expect_tx(land, tl.half ? STAGE_BYTES - G::A_BYTES / 2 : STAGE_BYTES);
-                    } else {
-                        mbar_arrive_expect_tx(land, STAGE_BYTES);
+                        if (tl.half) bytes = STAGE_BYTES - G::A_BYTES / 2;
                     }
                     const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
-                    stage_loads<KIND, PAIR>(tl, kb, p, &map_a, &map_o1, &map_x, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES, land,
-                                            rank, my_rows);
+                    if (fix) {
+                        const uint32_t land = smem_u32(&ctl->landed[stage]);
+                        mbar_arrive_expect_tx(land, bytes);
+                        stage_loads<KIND, PAIR, false>(tl, kb, p, &map_a, &map_o1, &map_x, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES,
+                                                       land, rank, my_rows);
+                    } else {
+                        const uint32_t land = full0 + stage * (uint32_t)sizeof(unsigned long long);
+                        if (PAIR) mbar_arrive_expect_tx_cluster(land, bytes); else mbar_arrive_expect_tx(land, bytes);
+                        stage_loads<KIND, PAIR, PAIR>(tl, kb, p, &map_a, &map_o1, &map_x, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES,
+                                                      land, rank, my_rows);
+                    }
                     ++issued;
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) {
-                // leave no bulk copy in flight: wait (bounded) for the copies issued into each stage
-                const uint32_t n_wait = issued < (uint32_t)STAGES ? issued : (uint32_t)STAGES;
-                uint32_t s = stage, ph = phase;
-                for (uint32_t i = 0; i < n_wait; ++i) {
-                    if (s == 0) { s = STAGES - 1; ph ^= 1u; } else { --s; }
-                    if (PAIR && rank == 0 && !local_fix) continue;   // completion there also needs the relay; the copies were bounded by it
-                    const unsigned long long t0 = global_timer_ns();
-                    const uint32_t land = smem_u32(local_fix ? &ctl->landed[s] : &ctl->full[s]);
-                    while (!mbar_try_wait(land, ph) && global_timer_ns() - t0 < WAIT_LIMIT_NS / 4) {}
-                }
+            if (!ok && issued != 0) {
+                // leave no bulk copy in flight.  The copies report to barriers this thread cannot always poll (the other
+                // CTA's), so simply outwait them: a copy that was issued completes within microseconds.
+                const unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 2000000ull) {}
             }
         }
     } else if (warp == 1 && rank == 0) {
@@ -595,37 +610,36 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
         }
         __syncwarp();
-    } else if (warp == 1 || (warp == FIX_WARP && local_fix)) {
-        // ================= relay (second CTA of a pair) / tail-fix warp (WGRAD, MMA-issuing CTA) =================
-        // Waits until this CTA's loads of a stage have landed, clears the surplus contraction rows
-        // (WGRAD) and then tells the first CTA's full[] barrier that this CTA's part of the stage is ready:
-        // with a remote arrive from the second CTA, with a local one in the first.
+    } else if (wgrad(KIND) && ((warp == 1 && rank != 0) || (warp == FIX_WARP && rank == 0))) {
+        // ================= tail-fix warp (weight gradients): warp 10 of the MMA-issuing CTA, warp 1 of the second =======
+        // Only the ragged last K block of a tile whose row count is not a multiple of 16 comes this way: its loads
+        // complete on landed[stage]; this warp clears the surplus contraction rows of its CTA's half of the stage and
+        // then makes this CTA's arrival on full[stage] of the MMA-issuing CTA (locally, or with a remote arrive).  All
+        // other stages are skipped: it only keeps count of them.
         const bool remote = rank != 0;
-        uint32_t stage = 0, phase = 0;
+        uint32_t stage = 0;
+        uint32_t landed_parity = 0;   // bit s: parity of the next use of landed[s]
         bool ok = true;
         for (long long it = 0; ok; ++it) {
             const long long t = tile_of<KIND>(it, first_tile, tile_stride, n_tiles_total);
             if (t < 0) break;
             const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
-            for (int kb = 0; kb < tl.k_blocks; ++kb) {
-                const uint32_t land = smem_u32(remote ? &ctl->full[stage] : &ctl->landed[stage]);
-                if (!mbar_wait(land, phase, abort_flag)) { ok = false; break; }
-                if (KIND == WGRAD) {
-                    const int rem = tl.k_rows - kb * BK;
-                    if (rem < BK) {
-                        const int z1 = ((rem + 15) >> 4) * 16;
-                        if (z1 > rem) zero_k_rows(tiles_ptr + stage * STAGE_BYTES, STAGE_CHUNKS, rem, z1, lane);
-                    }
-                }
+            if (tl.k_blocks == 0) continue;
+            const uint32_t last = (stage + (uint32_t)tl.k_blocks - 1u) % (uint32_t)STAGES;
+            if ((tl.k_rows & 15) != 0) {
+                if (!mbar_wait(smem_u32(&ctl->landed[last]), (landed_parity >> last) & 1u, abort_flag)) { ok = false; break; }
+                landed_parity ^= 1u << last;
+                const int rem = tl.k_rows - (tl.k_blocks - 1) * BK;
+                zero_k_rows(tiles_ptr + last * STAGE_BYTES, STAGE_CHUNKS, rem, ((rem + 15) >> 4) * 16, lane);
                 __syncwarp();
                 if (lane == 0) {
-                    if (remote) mbar_arrive_remote(map_to_cta(smem_u32(&ctl->full[stage]), 0));
-                    else mbar_arrive(smem_u32(&ctl->full[stage]));
+                    if (remote) mbar_arrive_remote(map_to_cta(smem_u32(&ctl->full[last]), 0));
+                    else mbar_arrive(smem_u32(&ctl->full[last]));
                 }
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
+            stage = (last + 1u) % (uint32_t)STAGES;
         }
-    } else if (warp < FIX_WARP) {
+    } else if (warp >= 2 && warp < FIX_WARP) {
         // ================= epilogue (warps 2..9) =================
         // Each warp owns a 32-row slab (its TMEM lane quarter) and half of the tile's columns.  A
         // 32 x 32 block is rounded to bf16, written to the warp's 2 KB staging buffer in the 64-byte
@@ -709,6 +723,66 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             dg = dh * u * sg * (1.f + g * (1.f - sg));
             du = dh * g * sg;
         };
+        // a zero tile (expert without rows, weight gradients): clear the staging block once and send it to the four
+        // 32 x 32 output blocks of this warp that start at column n_first, back to back
+        auto zero_blocks = [&](int n_first, int y) {
+            staging_free();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(stage_ptr + lane * 64 + j * 16) = make_uint4(0, 0, 0, 0);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                for (int c = 0; c < BN / 64; ++c) {
+                    const int n = n_first + c * 32;
+                    if (n >= p.n_cols) continue;
+                    const bool first = n < p.n_split;
+                    tma_store_2d(first ? &map_o0 : &map_o1, first ? n : n - p.n_split, y, smem_u32(stage_ptr));
+                }
+                bulk_commit();
+            }
+            ++n_stores;
+        };
+        // the warp's four 32-column blocks of one accumulator (tensor-memory address t_acc, first output column n_base):
+        // software pipeline, the tensor-memory load of the next block is in flight while the current one is converted,
+        // staged and stored
+        auto drain_plain = [&](uint32_t t_acc, int n_base, bool have_acc, int rows_valid, int y, long long row) {
+            constexpr int NC = BN / 64;
+            const int c0 = half * NC;
+            auto emit = [&](const uint32_t (&v)[32], int c) {
+                const int n = n_base + c * 32;
+                if (rows_valid == 0 || n >= p.n_cols) return;
+                uint32_t w[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                const bool first = n < p.n_split;
+                const int x = first ? n : n - p.n_split;
+                if (rows_valid == 32) {
+                    stage_and_store(w, first ? &map_o0 : &map_o1, x, y);
+                } else if (lane < rows_valid) {
+                    direct_store(w, p.out0 + row * p.ldo + x);     // row-ragged kinds have a single output
+                }
+            };
+            uint32_t va[32], vb[32];
+            if (have_acc) {
+                tc_ld32(t_acc + c0 * 32, va);
+            } else {   // only reached for a partial zero slab, which cannot occur; kept total
+#pragma unroll
+                for (int j = 0; j < 32; ++j) va[j] = vb[j] = 0u;
+            }
+#pragma unroll
+            for (int i = 0; i < NC; i += 2) {
+                if (have_acc) {
+                    tc_wait_ld();
+                    tc_ld32(t_acc + (c0 + i + 1) * 32, vb);
+                }
+                emit(va, c0 + i);
+                if (have_acc) {
+                    tc_wait_ld();
+                    if (i + 2 < NC) tc_ld32(t_acc + (c0 + i + 2) * 32, va);
+                }
+                emit(vb, c0 + i + 1);
+            }
+        };
         const uint32_t tmem_empty_remote0 = PAIR ? map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0) : 0u;
         const uint32_t tmem_empty_remote1 = PAIR ? map_to_cta(smem_u32(&ctl->tmem_empty[1]), 0) : 0u;
 
@@ -726,17 +800,17 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const bool half_tile = HALF_TILES && tl.half;
             const int slab0 = half_tile ? tl.row0 + (int)rank * (BM / 2) + (quarter & 1) * 32 : tl.row0 + my_rows + quarter * 32;
             // rows of the slab that are owed: inside the expert (row-ragged kinds) / inside M (WGRAD); 32 = whole slab
-            const int rows_valid = (KIND == WGRAD) ? (slab0 < p.m_rows ? 32 : 0) : max(0, min(32, tl.row_end - slab0));
-            const int slab_y = (KIND == WGRAD) ? tl.e * p.m_rows + slab0 : slab0;
+            const int rows_valid = wgrad(KIND) ? (slab0 < p.m_rows ? 32 : 0) : max(0, min(32, tl.row_end - slab0));
+            const int slab_y = wgrad(KIND) ? tl.e * p.m_rows + slab0 : slab0;
             const long long row = (long long)slab0 + lane;
             if (SWAP) {
                 // lane = output feature, tensor-memory column = row of the tile; the two warps of a lane quarter
                 // take the 32-row blocks alternately
                 const int feat0 = tl.n0 + (PAIR ? (int)rank * SWAP_FEATS : 0) + quarter * 32;
                 const int n_row_blocks = (tl.rows + 31) >> 5;
-#pragma unroll 1
                 const bool feats_owed = feat0 < p.n_cols;
                 if (fused_sb(KIND) && feats_owed && half < n_row_blocks) fetch_gu(feat0, tl.row0 + half * 32);
+#pragma unroll 1
                 for (int i = half; i < n_row_blocks; i += 2) {
                     uint32_t vr[32];
                     tc_ld32(taddr + i * 32, vr);
@@ -828,24 +902,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             } else {
                 const bool have_acc = tl.k_blocks > 0;
                 if (!have_acc && rows_valid == 32) {
-                    // expert without rows (WGRAD): a zero tile.  Clear the staging block once and send it to
-                    // all of this warp's 32 x 32 output blocks back to back.
-                    uint8_t* blk = stage_ptr;
-                    staging_free();
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) *reinterpret_cast<uint4*>(blk + lane * 64 + j * 16) = make_uint4(0, 0, 0, 0);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) {
-                        for (int c = half * (BN / 64); c < (half + 1) * (BN / 64); ++c) {
-                            const int n = tl.n0 + c * 32;
-                            if (n >= p.n_cols) continue;
-                            const bool first = n < p.n_split;
-                            tma_store_2d(first ? &map_o0 : &map_o1, first ? n : n - p.n_split, slab_y, smem_u32(blk));
-                        }
-                        bulk_commit();
-                    }
-                    ++n_stores;
+                    zero_blocks(tl.n0 + half * (BN / 2), slab_y);
                 } else if (fused_sb(KIND)) {
                     // row-major tile with the SwiGLU backward fused: per 32-column block, the accumulator (dHact, fp32)
                     // meets this row's g and u values (16-byte pieces of the lane's row of the two input blocks)
@@ -900,44 +957,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         }
                     }
                 } else {
-                    // software pipeline over the warp's four 32-column blocks: the TMEM load of the next block
-                    // is in flight while the current one is converted, staged and stored
-                    constexpr int NC = BN / 64;
-                    const int c0 = half * NC;
-                    auto emit = [&](const uint32_t (&v)[32], int c) {
-                        const int n = tl.n0 + c * 32;
-                        if (rows_valid == 0 || n >= p.n_cols) return;
-                        uint32_t w[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-                        const bool first = n < p.n_split;
-                        const int x = first ? n : n - p.n_split;
-                        if (rows_valid == 32) {
-                            stage_and_store(w, first ? &map_o0 : &map_o1, x, slab_y);
-                        } else if (lane < rows_valid) {
-                            direct_store(w, p.out0 + row * p.ldo + x);     // row-ragged kinds have a single output
-                        }
-                    };
-                    uint32_t va[32], vb[32];
-                    if (have_acc) {
-                        tc_ld32(taddr + c0 * 32, va);
-                    } else {   // only reached for a partial zero slab, which cannot occur; kept total
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) va[j] = vb[j] = 0u;
-                    }
-#pragma unroll
-                    for (int i = 0; i < NC; i += 2) {
-                        if (have_acc) {
-                            tc_wait_ld();
-                            tc_ld32(taddr + (c0 + i + 1) * 32, vb);
-                        }
-                        emit(va, c0 + i);
-                        if (have_acc) {
-                            tc_wait_ld();
-                            if (i + 2 < NC) tc_ld32(taddr + (c0 + i + 2) * 32, va);
-                        }
-                        emit(vb, c0 + i + 1);
-                    }
+                    drain_plain(taddr, tl.n0, have_acc, rows_valid, slab_y, row);
                 }
             }
             tc_fence_before();
