@@ -17,23 +17,33 @@
  * dW1_e = X_e^T G_e over a ragged number of rows per expert, is the kernel of the paper's section
  * "Production Validation: VeOmni MoE".
  *
+ * Where the calls come from: the paper covers the packed layout and one kernel, the weight gradient of the first
+ * projection (moe_grouped_gemm_gateup_wgrad).  The other calls -- route-permute, the two forward GEMMs, combine, and
+ * every other backward call -- are the standard expert-FFN algebra and its chain rule as this library's task
+ * statement lists them; the paper is silent on them, so their comments below state the operation itself.
+ *
  * Conventions for every call
  *   - Notation: R = T*K routed rows; pair id p = t*K + k (token-major).
  *   - All tensors are row-major with the last index contiguous.  `void*` tensors hold bf16
  *     (bfloat16 as 16-bit words); all results are rounded once, to nearest even, from fp32.
  *   - Unless a parameter says "host", every pointer is a DEVICE pointer to memory owned by the
- *     caller, 16-byte aligned.  The library allocates nothing, keeps no pointer after a call
+ *     caller, 16-byte aligned.  The library allocates no memory, keeps no pointer after a call
  *     returns, and never synchronises: all work is enqueued on `stream` (a cudaStream_t) in
- *     order.  Outputs are overwritten.  Inputs and outputs must not overlap.  Nothing a call does depends
+ *     order.  (One exception to "creates nothing": moe_layer_fwd_bwd_host creates two copy streams and a few
+ *     events per device on its first call; see there.)  Outputs are overwritten.  Inputs and outputs must not
+ *     overlap.  Nothing a call does depends
  *     on data that must first travel to the host, so a sequence of calls can be captured in a CUDA
  *     graph and replayed; run each kind of call once on the device before capturing (the first call of a
  *     kernel sets its launch attributes and queries occupancy).
  *   - H and I must be multiples of 64; 1 <= K <= E <= 1024; K <= 32; T*K < 2^31.
  *   - Return value: MOE_OK or an error code.  Argument errors are detected on the host before
- *     anything is launched.  A kernel that gives up waiting (bounded waits, never a trap) records
- *     MOE_ERR_TIMEOUT in a device status word readable with moe_device_status().
+ *     anything is launched.  Problems only the device can see are recorded in a per-device status word
+ *     that moe_device_status() reads and clears: a kernel that gives up waiting (every device-side wait is
+ *     bounded; there is never a trap) records MOE_ERR_TIMEOUT, and moe_permute records MOE_ERR_BAD_INDEX
+ *     when it meets an expert id outside [0, E).
  *   - `offsets` passed to a GEMM call must be the array moe_permute produced (non-decreasing,
- *     offsets[0] = 0, offsets[E] = R).  Expert ids in topk_idx must lie in [0, E).
+ *     offsets[0] = 0, offsets[E] = R).  Expert ids in topk_idx must lie in [0, E); a pair that violates this
+ *     is dropped (it gets no row, offsets[E] < R then) and reported as above.
  */
 #ifndef MOE_B200_H
 #define MOE_B200_H
@@ -85,7 +95,9 @@ int moe_device_status(int* status_out);
  * x_perm[r,:]  = x[row_to_pair[r] / K, :]                                        bf16  [R,H]
  * x [T,H] bf16, topk_idx [T,K] int32.  workspace: moe_permute_workspace_bytes(dims) bytes,
  * contents undefined before and after.  x_perm may be NULL (indices only).
- * Layout follows the paper's packed-by-expert buffer (appendix, "What the kernel computes"). */
+ * Layout follows the paper's packed-by-expert buffer (appendix, "What the kernel computes").
+ * A pair whose expert id is outside [0, E) is left out: it gets no row, its pair_to_row entry and the
+ * rows from offsets[E] on are not written, and the device status word reads MOE_ERR_BAD_INDEX. */
 int moe_permute(const moe_dims_t* dims, const void* x, const int32_t* topk_idx, void* x_perm,
                 int32_t* counts, int32_t* offsets, int32_t* row_to_pair, int32_t* pair_to_row,
                 void* workspace, size_t workspace_bytes, moe_stream_t stream);
@@ -115,7 +127,8 @@ int moe_permute_static_scratch(const moe_dims_t* dims, const void* x, const int3
                                void* x_perm, int32_t* counts, int32_t* offsets,
                                int32_t* row_to_pair, int32_t* pair_to_row, moe_stream_t stream);
 
-/* ---- a8: dx[t,:] = sum_k dx_perm[pair_to_row[t*K+k], :]   (fp32 sum in slot order) ---------- */
+/* ---- a8: dx[t,:] = sum_k dx_perm[pair_to_row[t*K+k], :]   (fp32 sum in slot order) ----------
+ * The gradient of a1's row copy (chain rule; the paper has no counterpart). */
 int moe_permute_bwd(const moe_dims_t* dims, const void* dx_perm, const int32_t* pair_to_row,
                     void* dx, moe_stream_t stream);
 
@@ -129,18 +142,20 @@ int moe_grouped_gemm_gateup_swiglu(const moe_dims_t* dims, const void* x_perm, c
                                    const void* w_up, const int32_t* offsets, void* h_act,
                                    void* gu_saved, moe_stream_t stream);
 
-/* ---- a3: y_perm[r,:] = h_act[r,:] . w_down[e]      w_down [E,I,H], y_perm [R,H] -------------- */
+/* ---- a3: y_perm[r,:] = h_act[r,:] . w_down[e]      w_down [E,I,H], y_perm [R,H] --------------
+ * The expert's second projection (standard expert-FFN algebra; the paper has no counterpart). */
 int moe_grouped_gemm_down(const moe_dims_t* dims, const void* h_act, const void* w_down,
                           const int32_t* offsets, void* y_perm, moe_stream_t stream);
 
 /* ---- a4: y[t,:] = sum_k topk_w[t,k] * y_perm[pair_to_row[t*K+k], :] -------------------------
- * topk_w [T,K] fp32; fp32 sum in slot order, one rounding.  y [T,H]. */
+ * topk_w [T,K] fp32; fp32 sum in slot order, one rounding.  y [T,H].  The routing weights enter the layer
+ * here and nowhere else (standard top-k combine; the paper has no counterpart). */
 int moe_unpermute_combine(const moe_dims_t* dims, const void* y_perm, const float* topk_w,
                           const int32_t* pair_to_row, void* y, moe_stream_t stream);
 
 /* ---- a5: dy_perm[pair_to_row[p],:] = topk_w[p] * dy[t(p),:];
  *          dtopk_w[t,k] = <dy[t,:], y_perm[pair_to_row[t*K+k],:]>   (fp32 [T,K]; may be NULL,
- *          and then y_perm may be NULL too) */
+ *          and then y_perm may be NULL too).  The chain rule applied to a4 (the paper has no counterpart). */
 int moe_unpermute_combine_bwd(const moe_dims_t* dims, const void* dy, const void* y_perm,
                               const float* topk_w, const int32_t* pair_to_row, void* dy_perm,
                               float* dtopk_w, moe_stream_t stream);
@@ -149,7 +164,8 @@ int moe_unpermute_combine_bwd(const moe_dims_t* dims, const void* dy, const void
  * dgrad  dh_act[r,:] = dy_perm[r,:] . w_down[e]^T                      dh_act [R,I]
  * wgrad  dw_down[e]  = sum over rows r of expert e of h_act[r,:]^T dy_perm[r,:]   [E,I,H]
  *        (all zeros for an expert without rows; written for every expert).
- * moe_grouped_gemm_down_bwd runs the dgrad then the wgrad. */
+ * moe_grouped_gemm_down_bwd runs the dgrad then the wgrad.  The chain rule applied to a3; the weight gradient has
+ * the shape of the paper's kernel (contraction over the expert's ragged rows), the paper itself treats only a7's. */
 int moe_grouped_gemm_down_dgrad(const moe_dims_t* dims, const void* dy_perm, const void* w_down,
                                 const int32_t* offsets, void* dh_act, moe_stream_t stream);
 int moe_grouped_gemm_down_wgrad(const moe_dims_t* dims, const void* h_act, const void* dy_perm,
@@ -189,9 +205,9 @@ int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_ac
                                        void* dw_gate, void* dw_up, moe_stream_t stream);
 
 /* ---- router in front of a1 ---------------------------------------------------------------------
- * The step that produces a1's routing inputs; the north-star workloads describe it as "softmax
+ * The step that produces a1's routing inputs; the benchmark workloads describe it as "softmax
  * over router logits, top-k renormalised" (the paper itself has no counterpart: its kernel starts
- * from the packed buffer).  Uses dims->T, E, K.
+ * from the packed buffer).  Uses dims->T, E, K only (1 <= K <= E <= 1024, K <= 32, T >= 1; H and I are not looked at).
  * moe_router_topk      logits [T,E] fp32 (device, no NaN).  Per token the K largest logits, slots in
  *                      descending order, equal values ordered by lower expert id, decided on the
  *                      fp32 values as given -> topk_idx [T,K] int32.  topk_w [T,K] fp32 =

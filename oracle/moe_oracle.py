@@ -266,7 +266,7 @@ def layer_fwd_bwd(X, topk_idx, topk_w, W_gate, W_up, W_down, dY):
 
 # ---- router in front of the layer (the step before route-permute) ------------------------------
 def router_topk(logits, K):
-    """Top-k routing as the spec workloads describe it: softmax over the router logits, the K
+    """Top-k routing as the benchmark workloads describe it: softmax over the router logits, the K
     largest per token kept and renormalised to sum 1.
 
     logits [T,E] float32.  Selection is decided on the float32 values as given: the K largest per

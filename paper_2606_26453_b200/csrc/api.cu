@@ -220,11 +220,23 @@ int moe_grouped_gemm_gateup_swiglu_bwd(const moe_dims_t* dims, const void* dh_ac
     return moe_grouped_gemm_gateup_wgrad(dims, x_perm, dgu, offsets, dw_gate, dw_up, stream);
 }
 
+// The router looks at T, E and K only.
+static int check_router_dims(const moe_dims_t* d) {
+    if (d == nullptr) return MOE_ERR_NULL;
+    if (d->T <= 0 || d->E <= 0 || d->K <= 0 || d->K > d->E) return MOE_ERR_DIMS;
+    if ((long long)d->T * d->K >= (1ll << 31)) return MOE_ERR_DIMS;
+    if (d->E > 1024 || d->K > 32) return MOE_ERR_UNSUPPORTED_SHAPE;
+    return MOE_OK;
+}
+
 int moe_router_topk(const moe_dims_t* dims, const float* logits, int32_t* topk_idx, float* topk_w,
                     moe_stream_t stream) {
     const void* const req[] = {logits, topk_idx, topk_w};
     const void* const opt[] = {nullptr};
-    MOE_VALIDATE(dims, req, opt);
+    int st_ = check_router_dims(dims);
+    if (st_ != MOE_OK) return st_;
+    st_ = check_ptrs(req, opt);
+    if (st_ != MOE_OK) return st_;
     return launch_router_topk(*dims, logits, topk_idx, topk_w, st(stream));
 }
 
@@ -232,7 +244,10 @@ int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const f
                         float* dlogits, moe_stream_t stream) {
     const void* const req[] = {topk_idx, topk_w, dtopk_w, dlogits};
     const void* const opt[] = {nullptr};
-    MOE_VALIDATE(dims, req, opt);
+    int st_ = check_router_dims(dims);
+    if (st_ != MOE_OK) return st_;
+    st_ = check_ptrs(req, opt);
+    if (st_ != MOE_OK) return st_;
     return launch_router_topk_bwd(*dims, topk_idx, topk_w, dtopk_w, dlogits, st(stream));
 }
 

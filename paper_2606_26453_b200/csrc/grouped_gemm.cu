@@ -49,6 +49,16 @@ namespace moe {
 
 __device__ int g_device_status = 0;
 
+#ifdef MOE_TEST_HOOKS
+// Test-only build: when set, every producer leaves out the loads AND the barrier arrival of its first ring stage, so
+// that the MMA warp's bounded wait on that stage runs out -- the one way to exercise the give-up path (status word,
+// abort flag, teardown) without a fault, a trap or an endless loop.
+__device__ int g_test_withhold_first_stage = 0;
+extern "C" int moe_test_withhold_first_stage(int on) {
+    return cudaMemcpyToSymbol(g_test_withhold_first_stage, &on, sizeof(int)) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+#endif
+
 int read_and_clear_device_status(int* status_out) {
     int v = 0, zero = 0;
     if (cudaDeviceSynchronize() != cudaSuccess) return MOE_ERR_CUDA;
@@ -502,6 +512,13 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                         if (tl.half) bytes = STAGE_BYTES - G::A_BYTES / 2;
                     }
                     const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
+#ifdef MOE_TEST_HOOKS
+                    if (g_test_withhold_first_stage != 0 && issued == 0) {
+                        ++issued;
+                        if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
+#endif
                     if (fix) {
                         const uint32_t land = smem_u32(&ctl->landed[stage]);
                         mbar_arrive_expect_tx(land, bytes);

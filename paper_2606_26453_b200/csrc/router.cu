@@ -1,6 +1,6 @@
 // Router in front of the layer: per token, the K largest of E logits (descending, equal values to the lower
 // expert id) and the softmax over the kept logits (= the full softmax renormalised over the kept experts),
-// plus the backward from the weight gradients to the logits.  The spec workloads describe this step as
+// plus the backward from the weight gradients to the logits.  The benchmark workloads describe this step as
 // how their routing inputs are made; the paper has no counterpart.
 //
 // One warp per token.  The E <= 1024 logits of a row sit in registers, element e = j*32 + lane (coalesced

@@ -10,7 +10,11 @@
 namespace moe {
 namespace {
 
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+// Every device-side wait gives up after this long (2 s; a test-only build of the library shortens it).
+#ifndef MOE_WAIT_LIMIT_NS
+#define MOE_WAIT_LIMIT_NS 2000000000ull
+#endif
+constexpr unsigned long long WAIT_LIMIT_NS = MOE_WAIT_LIMIT_NS;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
