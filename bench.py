@@ -45,8 +45,31 @@ PIPE_FLOP_PER_CLK_PER_SM = 8192.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a workload's dominant grouped-GEMM
 # kernel, from one ncu capture on a SCALED copy of the workload (tokens and experts divided by `scale`, same H, I,
 # top-k, routing law and rows per expert), multiplied by `scale`: every operand and result of these kernels grows in
-# proportion.  (workload, call) -> (bytes per full launch, how it was obtained); absent -> null.
-NCU_TRAFFIC = {}
+# proportion.  (workload, call) -> (bytes per full launch, which capture it comes from); absent -> null.
+NCU_TRAFFIC = {
+    ("imbalanced", "gateup_swiglu"): (9193.2e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("imbalanced", "down"): (3608.0e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("imbalanced", "down_dgrad"): (4548.4e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("imbalanced", "down_wgrad"): (4209.6e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("imbalanced", "gateup_dgrad"): (6412.4e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("imbalanced", "gateup_wgrad"): (8502.4e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("fine_grained", "gateup_swiglu"): (1029.0e6, "ncu capture of the full-size workload"),
+    ("fine_grained", "down"): (525.0e6, "ncu capture of the full-size workload"),
+    ("fine_grained", "down_wgrad"): (497.6e6, "ncu capture of the full-size workload"),
+    ("fine_grained", "gateup_dgrad"): (982.3e6, "ncu capture of the full-size workload"),
+    ("fine_grained", "gateup_wgrad"): (939.5e6, "ncu capture of the full-size workload"),
+    ("many_small", "gateup_swiglu"): (1953.2e6, "ncu capture of the full-size workload"),
+    ("many_small", "down"): (1110.1e6, "ncu capture of the full-size workload"),
+    ("many_small", "down_wgrad"): (1152.4e6, "ncu capture of the full-size workload"),
+    ("many_small", "gateup_dgrad"): (1727.9e6, "ncu capture of the full-size workload"),
+    ("many_small", "gateup_wgrad"): (1883.8e6, "ncu capture of the full-size workload"),
+    ("paper_dw1", "gateup_swiglu"): (5112.0e6, "ncu on a 1/8 copy (tokens and experts divided by 8), scaled x 8"),
+    ("paper_dw1", "down"): (2520.8e6, "ncu on a 1/8 copy (tokens and experts divided by 8), scaled x 8"),
+    ("paper_dw1", "down_dgrad"): (2548.8e6, "ncu on a 1/8 copy (tokens and experts divided by 8), scaled x 8"),
+    ("paper_dw1", "down_wgrad"): (2372.8e6, "ncu on a 1/8 copy (tokens and experts divided by 8), scaled x 8"),
+    ("paper_dw1", "gateup_dgrad"): (5536.8e6, "ncu on a 1/8 copy (tokens and experts divided by 8), scaled x 8"),
+    ("paper_dw1", "gateup_wgrad"): (4871.2e6, "ncu on a 1/8 copy (tokens and experts divided by 8), scaled x 8"),
+}
 
 
 def load_peaks():
@@ -247,13 +270,14 @@ def time_fused_variant(B, cfg, res, device, seconds=0.8, rounds=4):
                     "accumulator (dH_act is never materialised)"}
 
 
-def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True, min_seconds=0.0):
+def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True, min_seconds=0.0, fused=False):
     """Warm-up, then `steps` timed steps between two events (CUDA events around every call inside).  With
     min_seconds > 0 the step count is raised until the timed region lasts at least that long (estimated from three
     untimed steps after the warm-up; the maximum over ranks, so that every rank times the same count)."""
     wl = W.make_workload_device(cfg, device)
     b = B.alloc_layer_buffers(cfg.T, cfg.H, cfg.I, cfg.E, cfg.K, device=device)
-    step = make_step(B, b, wl)
+    step = make_step(B, b, wl, fused=fused)
+    calls = CALLS_FUSED if fused else CALLS
     for _ in range(warmup):
         step()
     torch.cuda.synchronize()
@@ -268,7 +292,7 @@ def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True, mi
         torch.cuda.synchronize()
         est_ms = max_over_ranks([e0.elapsed_time(e1) / 3.0], dist, device)[0]
         steps = max(steps, int(min_seconds * 1e3 / est_ms * 0.98) + 1)   # a step in a long run is a little slower than est
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(CALLS) + 1)] for _ in range(steps)]
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(steps)]
     t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(device.index if device.index is not None else 0) if sample_clocks else None
     if dist is not None:
@@ -286,7 +310,7 @@ def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True, mi
         dist.barrier()
     total_ms = t_start.elapsed_time(t_end)
     per_call = {}
-    for i, name in enumerate(CALLS):
+    for i, name in enumerate(calls):
         per_call[name] = sum(evs[s][i].elapsed_time(evs[s][i + 1]) for s in range(steps)) / steps
     if B.moe_device_status() != 0:
         raise RuntimeError("device status word is set after the timed region")
@@ -614,6 +638,16 @@ def run_ours(args):
     cfg = W.CONFIGS[args.config]
     sms = torch.cuda.get_device_properties(device).multi_processor_count
 
+    if args.only_steps:
+        # profiling runs: the warm-up and the timed steps and nothing else (optionally the fused step form and the
+        # block-scaled FP8 calls), one short line
+        res = time_config(B, cfg, device, args.steps, args.warmup, dist, min_seconds=0.0, fused=args.fused)
+        out = {"workload": cfg.name, "steps": res["steps"], "ms_per_step": res["total_ms"] / res["steps"],
+               "per_call_ms": {k: round(v, 5) for k, v in res["per_call_ms"].items()}}
+        if args.with_mxfp8:
+            out["mxfp8_down"] = time_mxfp8_down(B, cfg, res, device, reps=2)
+        print(json.dumps(out), flush=True)
+        return
     res = time_config(B, cfg, device, args.steps, args.warmup, dist, min_seconds=args.min_seconds)
     steps = res["steps"]
     if args.no_e2e:
@@ -704,12 +738,18 @@ def main():
                     help="the headline workload's timed region lasts at least this long (steps are added to --steps)")
     ap.add_argument("--other-min-seconds", type=float, default=0.5, help="the same floor for each of the --also workloads")
     ap.add_argument("--custom", default="", help="T,H,I,E,K of an ad-hoc softmax-routed workload (profiling aid)")
+    ap.add_argument("--scale", type=int, default=1,
+                    help="profiling aid: run a 1/SCALE copy of --config (tokens and experts divided by SCALE; same H, I, "
+                         "top-k, routing law and rows per expert) so that a multi-pass ncu capture stays small")
     ap.add_argument("--also", default="fine_grained,many_small,few_large,paper_dw1",
                     help="comma-separated other configurations to time briefly at N=1 ('' for none)")
     ap.add_argument("--ref-tokens", type=int, default=1024, help="tokens in the oracle's timed sample")
     ap.add_argument("--host-inputs", default="device", choices=["device", "numpy"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer pass (profiling runs)")
+    ap.add_argument("--only-steps", action="store_true", help="profiling runs: warm-up and timed steps only")
+    ap.add_argument("--fused", action="store_true", help="with --only-steps: the step form with the fused down-dgrad + SwiGLU-backward call")
+    ap.add_argument("--with-mxfp8", action="store_true", help="with --only-steps: also run the block-scaled FP8 calls")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     args.also = [s for s in args.also.split(",") if s]
@@ -717,6 +757,12 @@ def main():
         T, H, I, E, K = (int(v) for v in args.custom.split(","))
         W.CONFIGS["custom"] = W.MoeConfig("custom", T=T, H=H, I=I, E=E, K=K, routing="softmax", cfg_id=9)
         args.config = "custom"
+    if args.scale > 1:
+        c = W.CONFIGS[args.config]
+        name = f"{c.name}_scaled{args.scale}"
+        W.CONFIGS[name] = W.MoeConfig(name, T=c.T // args.scale, H=c.H, I=c.I, E=c.E // args.scale, K=c.K, routing=c.routing,
+                                      n_empty=max(1, c.n_empty // args.scale) if c.n_empty else 0, cfg_id=c.cfg_id)
+        args.config = name
     if args.impl == "reference":
         run_reference(args)
     else:
