@@ -142,16 +142,6 @@ int moe_grouped_gemm_gateup_swiglu(const moe_dims_t* dims, const void* x_perm, c
                                    const void* w_up, const int32_t* offsets, void* h_act,
                                    void* gu_saved, moe_stream_t stream);
 
-/* Gathering form of a2 (an additional entry point; a2 itself stays): the same h_act and gu_saved, bit for bit, but the
- * A operand is read straight from the token-major x [T,H] through row_to_pair (packed row r uses token
- * row_to_pair[r] / K), four rows per bulk tensor gather, so the forward needs the INDEX part of moe_permute only
- * (x_perm = NULL there) and does not wait for the packed copy.  The weight gradient still wants x_perm; it can be
- * produced off the forward's critical path. */
-int moe_grouped_gemm_gateup_swiglu_gather(const moe_dims_t* dims, const void* x,
-                                          const int32_t* row_to_pair, const void* w_gate,
-                                          const void* w_up, const int32_t* offsets, void* h_act,
-                                          void* gu_saved, moe_stream_t stream);
-
 /* ---- a3: y_perm[r,:] = h_act[r,:] . w_down[e]      w_down [E,I,H], y_perm [R,H] --------------
  * The expert's second projection (standard expert-FFN algebra; the paper has no counterpart). */
 int moe_grouped_gemm_down(const moe_dims_t* dims, const void* h_act, const void* w_down,

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_PKG_DIR, "libmoe_b200.so")
 EXPORTS = [
     "moe_status_string", "moe_permute_workspace_bytes", "moe_device_status", "moe_permute", "moe_permute_static_scratch",
     "moe_permute_bwd",
-    "moe_grouped_gemm_gateup_swiglu", "moe_grouped_gemm_gateup_swiglu_gather", "moe_grouped_gemm_down", "moe_unpermute_combine",
+    "moe_grouped_gemm_gateup_swiglu", "moe_grouped_gemm_down", "moe_unpermute_combine",
     "moe_unpermute_combine_bwd", "moe_grouped_gemm_down_dgrad", "moe_grouped_gemm_down_wgrad",
     "moe_grouped_gemm_down_bwd", "moe_swiglu_bwd", "moe_grouped_gemm_down_dgrad_swiglu_bwd", "moe_grouped_gemm_gateup_dgrad",
     "moe_grouped_gemm_gateup_wgrad", "moe_grouped_gemm_gateup_swiglu_bwd", "moe_layer_arena_bytes",
@@ -67,7 +67,6 @@ def load_library() -> ctypes.CDLL:
             "moe_permute_static_scratch": [dp, p, p, p, p, p, p, p, p],
             "moe_permute_bwd": [dp, p, p, p, p],
             "moe_grouped_gemm_gateup_swiglu": [dp, p, p, p, p, p, p, p],
-            "moe_grouped_gemm_gateup_swiglu_gather": [dp, p, p, p, p, p, p, p, p],
             "moe_grouped_gemm_down": [dp, p, p, p, p, p],
             "moe_unpermute_combine": [dp, p, p, p, p, p],
             "moe_unpermute_combine_bwd": [dp, p, p, p, p, p, p, p],
@@ -158,11 +157,6 @@ def moe_permute_bwd(d, dx_perm, pair_to_row, dx):
 def moe_grouped_gemm_gateup_swiglu(d, x_perm, w_gate, w_up, offsets, h_act, gu_saved):
     _call("moe_grouped_gemm_gateup_swiglu", ctypes.byref(d), _ptr(x_perm), _ptr(w_gate), _ptr(w_up), _ptr(offsets),
           _ptr(h_act), _ptr(gu_saved), _stream())
-
-
-def moe_grouped_gemm_gateup_swiglu_gather(d, x, row_to_pair, w_gate, w_up, offsets, h_act, gu_saved):
-    _call("moe_grouped_gemm_gateup_swiglu_gather", ctypes.byref(d), _ptr(x), _ptr(row_to_pair), _ptr(w_gate), _ptr(w_up),
-          _ptr(offsets), _ptr(h_act), _ptr(gu_saved), _stream())
 
 
 def moe_grouped_gemm_down(d, h_act, w_down, offsets, y_perm):

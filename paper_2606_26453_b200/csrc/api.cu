@@ -128,16 +128,6 @@ int moe_grouped_gemm_gateup_swiglu(const moe_dims_t* dims, const void* x_perm, c
     return launch_gateup_fwd(*dims, cb(x_perm), cb(w_gate), cb(w_up), offsets, mb(h_act), mb(gu_saved), st(stream));
 }
 
-int moe_grouped_gemm_gateup_swiglu_gather(const moe_dims_t* dims, const void* x, const int32_t* row_to_pair,
-                                          const void* w_gate, const void* w_up, const int32_t* offsets, void* h_act,
-                                          void* gu_saved, moe_stream_t stream) {
-    const void* const req[] = {x, row_to_pair, w_gate, w_up, offsets, h_act};
-    const void* const opt[] = {gu_saved};
-    MOE_VALIDATE(dims, req, opt);
-    return launch_gateup_fwd_gather(*dims, cb(x), row_to_pair, cb(w_gate), cb(w_up), offsets, mb(h_act), mb(gu_saved),
-                                    st(stream));
-}
-
 int moe_grouped_gemm_down(const moe_dims_t* dims, const void* h_act, const void* w_down, const int32_t* offsets,
                           void* y_perm, moe_stream_t stream) {
     const void* const req[] = {h_act, w_down, offsets, y_perm};

@@ -44,8 +44,6 @@ int launch_router_topk_bwd(const moe_dims_t& d, const int32_t* topk_idx, const f
 // ---- grouped GEMMs (grouped_gemm.cu) -----------------------------------------------------------
 int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gate, const bf16* w_up,
                       const int32_t* offsets, bf16* h_act, bf16* gu, cudaStream_t s);
-int launch_gateup_fwd_gather(const moe_dims_t& d, const bf16* x, const int32_t* row_to_pair, const bf16* w_gate,
-                             const bf16* w_up, const int32_t* offsets, bf16* h_act, bf16* gu, cudaStream_t s);
 int launch_down_fwd(const moe_dims_t& d, const bf16* h_act, const bf16* w_down, const int32_t* offsets,
                     bf16* y_perm, cudaStream_t s);
 int launch_down_dgrad(const moe_dims_t& d, const bf16* dy_perm, const bf16* w_down, const int32_t* offsets,

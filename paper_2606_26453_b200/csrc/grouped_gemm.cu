@@ -92,13 +92,10 @@ constexpr int TMEM_COLS = 512;
 // DGRAD_SB / DGRAD_T_SB are DGRAD / DGRAD_T of the down projection with the SwiGLU backward fused into the epilogue:
 // the accumulator (dHact, fp32, never rounded) meets the saved pre-activations [g | u], which the epilogue warps fetch
 // as 32 x 32 blocks with bulk tensor loads, and the kernel writes dGU = [dg | du] instead of dHact.
-// FWD_SWIGLU_G is FWD_SWIGLU reading its A operand straight from the token-major x [T,H] through the row list
-// row_to_pair (tile::gather4 loads: the whole producer warp, four rows per lane), so that the forward does not wait
-// for the packed copy x_perm.
 enum Kind { FWD_SWIGLU = 0, FWD_PLAIN = 1, DGRAD = 2, WGRAD = 3, FWD_PLAIN_T = 4, DGRAD_T = 5, FWD_SWIGLU_H = 6,
-            DGRAD_SB = 7, DGRAD_T_SB = 8, FWD_SWIGLU_G = 9 };
+            DGRAD_SB = 7, DGRAD_T_SB = 8 };
 __host__ __device__ constexpr bool wgrad(int kind) { return kind == WGRAD; }
-__host__ __device__ constexpr bool swiglu(int kind) { return kind == FWD_SWIGLU || kind == FWD_SWIGLU_H || kind == FWD_SWIGLU_G; }
+__host__ __device__ constexpr bool swiglu(int kind) { return kind == FWD_SWIGLU || kind == FWD_SWIGLU_H; }
 __host__ __device__ constexpr bool swapped(int kind) { return kind == FWD_PLAIN_T || kind == DGRAD_T || kind == DGRAD_T_SB; }
 __host__ __device__ constexpr bool fused_sb(int kind) { return kind == DGRAD_SB || kind == DGRAD_T_SB; }
 // the kind whose operand loads and MMAs a kind shares
@@ -122,9 +119,6 @@ struct Params {
     bf16* out1;
     bf16* gu;            // FWD_SWIGLU: [R, 2I] or null
     int I;               // FWD_SWIGLU
-    const int32_t* row_to_pair;   // FWD_SWIGLU_G: packed row -> pair id
-    int K;                        // FWD_SWIGLU_G: pairs per token
-    long long R;                  // FWD_SWIGLU_G: packed rows in total
 };
 
 struct SharedCtl {
@@ -347,7 +341,7 @@ __device__ __forceinline__ void stage_loads(const Tile& tl, int kb, const Params
         // half-height pair tile (FWD_SWIGLU): rows [row0, row0+64) in the first CTA, [row0+64, row0+128) in the second;
         // map_r1 is the A map with a 64-row box there
         if (KIND == FWD_SWIGLU_H && tl.half) tma_load_2d(a_dst, map_r1, kb * BK, tl.row0 + (int)rank * (BM / 2), full);
-        else if (KIND != FWD_SWIGLU_G) tma_load_2d(a_dst, map_a, kb * BK, tl.row0 + my_rows, full);   // _G: gathered by the whole warp
+        else tma_load_2d(a_dst, map_a, kb * BK, tl.row0 + my_rows, full);
         if (load_kind(KIND) == DGRAD) {
             const bool second = kb >= p.k_split;
             const int kx = (second ? kb - p.k_split : kb) * BK;
@@ -495,44 +489,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // a stage travels producer -> loads -> MMA with no relay hop.  Only a weight-gradient stage whose ragged last
         // K block needs surplus rows cleared reports to this CTA's landed[stage]; the tail-fix / relay warp clears the
         // rows and makes the arrival on full[stage] in the producer's place.
-        if (KIND == FWD_SWIGLU_G) {
-            // The whole warp: lane l owns rows 4l .. 4l+3 of this CTA's 128 rows of the tile and fetches them from x with
-            // one gather4 per K block (source row = pair / K); lane 0 also makes the barrier arrival and loads B.
-            uint32_t stage = 0, phase = 0;
-            uint32_t issued = 0;
-            bool ok = true;
-            const uint32_t full0 = PAIR ? map_to_cta(smem_u32(&ctl->full[0]), 0) : smem_u32(&ctl->full[0]);
-            for (long long it = 0; ok; ++it) {
-                const long long t = tile_of<KIND>(it, first_tile, tile_stride, n_tiles_total);
-                if (t < 0) break;
-                const Tile tl = decode_tile<KIND, G::TILE_M>(p, ctl, t);
-                int src[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const long long r = (long long)tl.row0 + my_rows + 4 * lane + i;
-                    // rows past the expert's end are never stored: any valid row of x will do for them
-                    src[i] = r < p.R ? __ldg(p.row_to_pair + r) / p.K : 0;
-                }
-                for (int kb = 0; kb < tl.k_blocks; ++kb) {
-                    if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t a_dst = tiles_base + stage * STAGE_BYTES;
-                    const uint32_t land = full0 + stage * (uint32_t)sizeof(unsigned long long);
-                    if (lane == 0) {
-                        if (PAIR) mbar_arrive_expect_tx_cluster(land, STAGE_BYTES); else mbar_arrive_expect_tx(land, STAGE_BYTES);
-                        stage_loads<KIND, PAIR, PAIR>(tl, kb, p, &map_a, &map_o1, &map_x, &map_b0, &map_b1, a_dst, a_dst + G::A_BYTES,
-                                                      land, rank, my_rows);
-                    }
-                    __syncwarp();
-                    tma_gather4<PAIR>(a_dst + lane * 512, &map_x, kb * BK, src[0], src[1], src[2], src[3], land);
-                    ++issued;
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
-            }
-            if (!ok && issued != 0) {
-                const unsigned long long t0 = global_timer_ns();
-                while (global_timer_ns() - t0 < 2000000ull) {}
-            }
-        } else if (lane == 0) {
+        if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             uint32_t issued = 0;
             bool ok = true;
@@ -1156,25 +1113,6 @@ int launch_gateup_fwd(const moe_dims_t& d, const bf16* x_perm, const bf16* w_gat
     p.out0 = h_act; p.gu = gu; p.I = d.I; p.ldo = d.I; p.n_split = 2 * d.I;
     if (half_tiles) return launch<FWD_SWIGLU_H, true>(a, b0, b1, o0, o1, ah, p, s);
     return pair ? launch<FWD_SWIGLU, true>(a, b0, b1, o0, o1, a, p, s) : launch<FWD_SWIGLU, false>(a, b0, b1, o0, o1, a, p, s);
-}
-
-// Gate/up forward from the token-major x: same tiles as launch_gateup_fwd without half-height tiles; `g` is x [T,H] with
-// a {64 columns, 1 row} box for the gather loads.
-int launch_gateup_fwd_gather(const moe_dims_t& d, const bf16* x, const int32_t* row_to_pair, const bf16* w_gate,
-                             const bf16* w_up, const int32_t* offsets, bf16* h_act, bf16* gu, cudaStream_t s) {
-    const uint64_t R = (uint64_t)d.T * d.K;
-    const bool pair = use_pairs_for_swiglu(d);
-    CUtensorMap g, b0, b1, o0, o1;
-    if (!make_map(&g, x, d.H, d.T, BK, 1) || !make_map_mn(&b0, w_gate, d.I, (uint64_t)d.E * d.H, 2) ||
-        !make_map_mn(&b1, w_up, d.I, (uint64_t)d.E * d.H, 2) || !make_out_map(&o0, h_act, d.I, R) ||
-        !make_out_map(&o1, gu ? gu : h_act, gu ? 2ull * d.I : d.I, R))
-        return MOE_ERR_CUDA;
-    Params p = {};
-    p.offsets = offsets; p.E = d.E; p.k_blocks = d.H / BK; p.k_split = p.k_blocks;
-    p.n_tiles = (d.I + 127) / 128; p.n_cols = 2 * d.I; p.b_rows_per_e = d.H;
-    p.out0 = h_act; p.gu = gu; p.I = d.I; p.ldo = d.I; p.n_split = 2 * d.I;
-    p.row_to_pair = row_to_pair; p.K = d.K; p.R = (long long)R;
-    return pair ? launch<FWD_SWIGLU_G, true>(g, b0, b1, o0, o1, g, p, s) : launch<FWD_SWIGLU_G, false>(g, b0, b1, o0, o1, g, p, s);
 }
 
 // Down forward: A = h_act [R,I]; B = w_down viewed as [E*I, H].

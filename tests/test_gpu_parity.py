@@ -203,26 +203,6 @@ def test_gateup_swiglu(B, case):
     assert torch.equal(hact, hact2)
 
 
-def test_gateup_swiglu_gather_equals_the_packed_form(B, case):
-    """The gathering form reads x through row_to_pair instead of x_perm: same operands, same MMA order, so the same
-    bits as the packed form -- and both within the per-call bound of the oracle."""
-    cfg, host, ref = case
-    d, R = _dims(B, cfg), cfg.R
-    x = _bf(host["X"])
-    xp = x[torch.from_numpy(ref["row_to_pair"].astype(np.int64) // cfg.K).cuda()].contiguous()
-    wg, wu, off = _bf(host["W_gate"]), _bf(host["W_up"]), _i32(ref["offsets"])
-    hact, gu = _nan((R, cfg.I)), _nan((R, 2 * cfg.I))
-    B.moe_grouped_gemm_gateup_swiglu(d, xp, wg, wu, off, hact, gu)
-    hact_g, gu_g = _nan((R, cfg.I)), _nan((R, 2 * cfg.I))
-    B.moe_grouped_gemm_gateup_swiglu_gather(d, x, _i32(ref["row_to_pair"]), wg, wu, off, hact_g, gu_g)
-    torch.cuda.synchronize()
-    assert B.moe_device_status() == 0
-    o_h, o_gu = O.gateup_swiglu(ref["X_perm"], host["W_gate"], host["W_up"], ref["offsets"])
-    Hh.assert_close(Hh.to_np64(gu_g), o_gu, "GU (gather)", rel_fro=Hh.PER_CALL_FROBENIUS)
-    Hh.assert_close(Hh.to_np64(hact_g), o_h, "H_act (gather)", rel_fro=Hh.PER_CALL_FROBENIUS)
-    assert torch.equal(hact_g, hact) and torch.equal(gu_g, gu)
-
-
 def test_down(B, case):
     cfg, host, ref = case
     d, R = _dims(B, cfg), cfg.R
