@@ -605,6 +605,47 @@ def stream_calibration_in_step(B, cfg, res, device, steps=12):
     return out
 
 
+def gemm_calibration(device, seconds=1.5):
+    """The library bf16 GEMM (torch.matmul, 8192^3) on THIS box, the way the measured peaks were taken: best of 10 single
+    calls (burst) and back to back for `seconds` with the SM clock sampled (sustained).  Boxes of the pool differ in how
+    hard the power cap bites; this puts the layer's numbers and the library's on the same chip and in the same minute."""
+    n = 8192
+    a = torch.randn(n, n, device=device, dtype=torch.bfloat16)
+    b = torch.randn(n, n, device=device, dtype=torch.bfloat16)
+    c = torch.empty(n, n, device=device, dtype=torch.bfloat16)
+    fl = 2.0 * n ** 3
+    for _ in range(3):
+        torch.matmul(a, b, out=c)
+    best = float("inf")
+    for _ in range(10):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        torch.matmul(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1))
+    sampler = ClockSampler(device.index if device.index is not None else 0)
+    sampler.start()
+    done, ms = 0, 0.0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    while ms < seconds * 1e3:
+        e0.record()
+        for _ in range(50):
+            torch.matmul(a, b, out=c)
+        e1.record()
+        torch.cuda.synchronize()
+        ms += e0.elapsed_time(e1)
+        done += 50
+    clocks = sampler.stop()
+    del a, b, c
+    torch.cuda.empty_cache()
+    sustained = fl * done / (ms * 1e-3) / 1e12
+    out = {"burst_tflops": fl / (best * 1e-3) / 1e12, "sustained_tflops": sustained, "clocks": clocks}
+    if clocks.get("sm_mhz"):
+        out["sustained_pipe_frac_at_sampled_clock"] = sustained * 1e12 / (clocks["sm_mhz"] * 1e6 * torch.cuda.get_device_properties(device).multi_processor_count * PIPE_FLOP_PER_CLK_PER_SM)
+    return out
+
+
 def max_over_ranks(values, dist, device):
     """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
     if dist is None:
@@ -718,6 +759,7 @@ def run_ours(args):
             router["workload"] = router_cfg.name
             line["router"] = router
         line["stream_calibration"] = stream_calibration(device)
+        line["gemm_calibration"] = gemm_calibration(device)
         if wl_host is not None:
             line["cpu_baseline"] = cpu_baseline(cfg, wl_host, min(args.ref_tokens, cfg.T))
     if rank == 0:

@@ -736,7 +736,7 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         };
         // dg = dh*u*s*(1+g*(1-s)), du = dh*g*s with s = 1/(1+exp(-g))
         auto swiglu_grad = [](float dh, float g, float u, float& dg, float& du) {
-            const float sg = 1.f / (1.f + __expf(-g));
+            const float sg = __fdividef(1.f, 1.f + __expf(-g));
             dg = dh * u * sg * (1.f + g * (1.f - sg));
             du = dh * g * sg;
         };
@@ -895,8 +895,8 @@ grouped_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     for (int j = 0; j < 16; ++j) {
                         const float g0 = __uint_as_float(g[2 * j]), g1 = __uint_as_float(g[2 * j + 1]);
                         const float u0 = __uint_as_float(u[2 * j]), u1 = __uint_as_float(u[2 * j + 1]);
-                        const float h0 = g0 / (1.f + __expf(-g0)) * u0;
-                        const float h1 = g1 / (1.f + __expf(-g1)) * u1;
+                        const float h0 = __fdividef(g0, 1.f + __expf(-g0)) * u0;
+                        const float h1 = __fdividef(g1, 1.f + __expf(-g1)) * u1;
                         hp[j] = pack_bf16(h0, h1);
                         gp[j] = pack_bf16(g0, g1);
                         up[j] = pack_bf16(u0, u1);

@@ -375,10 +375,11 @@ __global__ void __launch_bounds__(kThreads) gather_sum_kernel(const uint4* __res
 // a5: one block per token, one thread per 16-byte piece of the row.
 // dy_perm[row_k, :] = w_k * dy[t, :]; dtopk_w[t,k] = <dy[t,:], y_perm[row_k,:]> (warp shuffles, then a
 // fixed-order sum over the block's warps: deterministic).  y_perm pieces are fetched four slots at a time
-// to keep the register count low enough for five blocks per SM.
+// (three blocks per SM: with the 80 registers that allows nothing spills; at five blocks per SM the K = 8 kernel
+// spilled and ran 16 % slower inside a step).
 // ------------------------------------------------------------------------------------------------
 template <int KT, bool WITH_DW>
-__global__ void __launch_bounds__(kThreads, 5) combine_bwd_kernel(const uint4* __restrict__ dy,
+__global__ void __launch_bounds__(kThreads, 3) combine_bwd_kernel(const uint4* __restrict__ dy,
                                                                   const uint4* __restrict__ y_perm,
                                                                   const float* __restrict__ topk_w,
                                                                   const int32_t* __restrict__ pair_to_row,
@@ -466,7 +467,9 @@ __global__ void __launch_bounds__(kThreads) swiglu_bwd_kernel(const uint4* __res
     unpack8(uv, u);
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const float s = 1.f / (1.f + __expf(-g[j]));
+        // approximate division (2 ulp): inside a power-capped step this kernel is bound by instruction issue at the
+        // low clock, not by HBM -- the exact division cost 18 % of its time there
+        const float s = __fdividef(1.f, 1.f + __expf(-g[j]));
         dg[j] = dh[j] * u[j] * s * (1.f + g[j] * (1.f - s));
         du[j] = dh[j] * g[j] * s;
     }
