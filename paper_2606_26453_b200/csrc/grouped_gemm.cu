@@ -1080,11 +1080,9 @@ int launch(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, c
 // are as fast or faster (the swapped kernels' issue thread, not the tensor pipe, bounds tiles of fewer than 256 rows).
 bool use_swapped(const moe_dims_t& d) { return (long long)d.T * d.K < 512ll * d.E; }
 // The SwiGLU forward has no swapped form (measured slower: two accumulators per tile).  Its pair kernel runs an
-// expert's last <= 128 rows as a half-height tile, which makes pairs worthwhile from MOE_SWIGLU_PAIR_ROWS rows per expert.
-#ifndef MOE_SWIGLU_PAIR_ROWS
-#define MOE_SWIGLU_PAIR_ROWS 320
-#endif
-bool use_pairs_for_swiglu(const moe_dims_t& d) { return (long long)d.T * d.K >= (long long)MOE_SWIGLU_PAIR_ROWS * d.E; }
+// expert's last <= 128 rows as a half-height tile, which makes pairs worthwhile from 320 rows per expert on average.
+constexpr long long kSwigluPairRows = 320;
+bool use_pairs_for_swiglu(const moe_dims_t& d) { return (long long)d.T * d.K >= kSwigluPairRows * d.E; }
 // Weight gradients have no row padding to lose, so pairs already win from 256 rows per expert.
 bool use_pairs_for_wgrad(const moe_dims_t& d) { return (long long)d.T * d.K >= 256ll * d.E; }
 
