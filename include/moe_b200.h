@@ -234,9 +234,14 @@ int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const f
  *                              laid out [I/128][R][4]: the scale bytes of the 4 blocks of 32 inside the 128-wide
  *                              slice kt of row r are bytes scales[(kt*R + r)*4 + 0..3].
  *   moe_mxfp8_quantize_w_down  w_down [E,I,H] bf16 -> codes_t [E,H,I] bytes (transposed: contraction contiguous);
- *                              scales: moe_mxfp8_w_down_scale_bytes(dims) bytes laid out [E][H/128][I/128][512]:
- *                              the scale of feature h, block b of 32 along I, is byte
- *                              (h%32)*16 + ((h%128)/32)*4 + b%4 of the 512-byte group (e, h/128, b/4).
+ *                              scales: moe_mxfp8_w_down_scale_bytes(dims) bytes holding every scale twice, once
+ *                              per tiling of the two GEMM kernels (128-feature tiles on one CTA; 208-feature tiles
+ *                              on a CTA pair, used from 256 rows per expert on average):
+ *                              first [E][H/128][I/128][512]: the scale of feature h, block b of 32 along I, is
+ *                              byte (h%32)*16 + ((h%128)/32)*4 + b%4 of the 512-byte group (e, h/128, b/4);
+ *                              then [E][ceil(H/208)][I/128][1024]: with h' = h%208 the same scale is byte
+ *                              (h'/128)*512 + (h'%32)*16 + ((h'%128)/32)*4 + b%4 of the 1024-byte group
+ *                              (e, h/208, b/4); bytes of a group that no feature owns are left unwritten.
  *   moe_grouped_gemm_down_mxfp8  y_perm[r,:] = dequant(h row r) . dequant(w_down[e]) for rows r of expert e.
  * All pointers device, 16-byte aligned; codes and scales are caller-owned buffers. */
 size_t moe_mxfp8_act_scale_bytes(const moe_dims_t* dims);

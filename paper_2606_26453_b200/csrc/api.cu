@@ -265,7 +265,7 @@ size_t moe_mxfp8_act_scale_bytes(const moe_dims_t* dims) {
 
 size_t moe_mxfp8_w_down_scale_bytes(const moe_dims_t* dims) {
     if (check_mx_dims(dims) != MOE_OK) return 0;
-    return (size_t)dims->E * (dims->H / 128) * (dims->I / 128) * 512;
+    return mx_w_scale_bytes(*dims);
 }
 
 int moe_mxfp8_quantize_h_act(const moe_dims_t* dims, const void* h_act, void* codes, void* scales, moe_stream_t stream) {

@@ -54,6 +54,7 @@ constexpr int MX_THREADS = 32 * (3 + MX_EPI_WARPS);
 constexpr int MX_STAGING_BYTES = MX_EPI_WARPS * 2048;
 constexpr int MX_MAX_E = 1024;
 constexpr int MX_TMEM_COLS = 512;
+constexpr int MX_SCALE_AHEAD = 4;   // K slices whose activation-scale words the scale warp keeps in flight
 constexpr int MX_SF_COL0 = 2 * MX_BN;   // first tensor-memory column of the scale slots (after the two accumulators)
 
 struct MxCtl {
@@ -260,20 +261,29 @@ mx_down_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const long long r = (long long)tl.row0 + 32 * i + lane;
                 rows[i] = r < p.R ? r : p.R - 1;   // rows past the end are never stored; any valid address will do
             }
-            uint4 next;
-            next.x = __ldg(p.sa + rows[0]); next.y = __ldg(p.sa + rows[1]); next.z = __ldg(p.sa + rows[2]); next.w = __ldg(p.sa + rows[3]);
-            for (int kt = 0; kt < p.k_tiles; ++kt) {
-                const uint4 cur = next;
-                if (kt + 1 < p.k_tiles) {   // the next slice's words travel while this one waits for its stage
-                    const uint32_t* s = p.sa + (long long)(kt + 1) * p.R;
-                    next.x = __ldg(s + rows[0]); next.y = __ldg(s + rows[1]); next.z = __ldg(s + rows[2]); next.w = __ldg(s + rows[3]);
+            // the words of MX_SCALE_AHEAD slices are in flight at any time: one slice per global-load round trip would
+            // bound the whole pipeline (the loads wait behind the operand traffic)
+            auto load_slice = [&](int kt) {
+                const uint32_t* s = p.sa + (long long)kt * p.R;
+                return make_uint4(__ldg(s + rows[0]), __ldg(s + rows[1]), __ldg(s + rows[2]), __ldg(s + rows[3]));
+            };
+            uint4 q[MX_SCALE_AHEAD];
+#pragma unroll
+            for (int i = 0; i < MX_SCALE_AHEAD; ++i) q[i] = load_slice(min(i, p.k_tiles - 1));
+            for (int kt0 = 0; ok && kt0 < p.k_tiles; kt0 += MX_SCALE_AHEAD) {
+#pragma unroll
+                for (int i = 0; i < MX_SCALE_AHEAD; ++i) {
+                    const int kt = kt0 + i;
+                    if (kt >= p.k_tiles) break;
+                    const uint4 cur = q[i];
+                    if (kt + MX_SCALE_AHEAD < p.k_tiles) q[i] = load_slice(kt + MX_SCALE_AHEAD);
+                    if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    *reinterpret_cast<uint4*>(tiles_ptr + stage * MX_STAGE_BYTES + MX_A_BYTES + MX_B_BYTES + lane * 16) = cur;
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl->full[stage]));
+                    if (++stage == MX_STAGES) { stage = 0; phase ^= 1u; }
                 }
-                if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-                *reinterpret_cast<uint4*>(tiles_ptr + stage * MX_STAGE_BYTES + MX_A_BYTES + MX_B_BYTES + lane * 16) = cur;
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->full[stage]));
-                if (++stage == MX_STAGES) { stage = 0; phase ^= 1u; }
             }
         }
     } else {
@@ -337,6 +347,393 @@ mx_down_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     }
 }
 
+// ---- the CTA-pair form ----------------------------------------------------------------------------------
+// Two CTAs of a cluster share one 256-row x 208-column tile (tcgen05.mma.cta_group::2, M = 256): each keeps its own 128
+// rows of A and 104 of the tile's weight rows in shared memory, so a K slice of 128 costs each SM 29 KB of operand
+// loads against 58 KB per two 128 x 128 tiles of the single-CTA form, which the L2 -> SM path bounds.  208 columns, not
+// 256: the two accumulators (tensor-memory columns 0 and 256) leave 48 columns behind each for three 16-column scale
+// slots, one slot per ring stage.  A tile at the right edge is narrower (a multiple of 16 columns; the MMA's N is set
+// per tile).
+//   scale factors: each CTA holds the scales of its own 128 rows of A (4 columns) and of ALL the tile's weight rows (two
+//   128-row blocks, 8 columns) in its own tensor memory; tcgen05.cp.cta_group::2, issued once, copies in both CTAs from
+//   the same shared-memory offsets.  The weight-scale blocks of a (tile, K slice) are 1024 contiguous bytes in global
+//   memory (a second copy of the scales in this tiling, written by the weight quantiser) and arrive by one tensor copy.
+//   warp 0      TMA producer (both CTAs; all loads complete on the first CTA's full[stage], as in the bf16 pair kernels)
+//   warp 1      first CTA: issues the MMAs and the commits for the pair
+//   warp 2      activation scales of this CTA's 128 rows
+//   warps 3..10 epilogue: 32-row slab x every other 32-column block (a 16-column remainder: plain stores)
+//   warp 11     first CTA: issues the scale copies (smem -> tensor memory) of each stage
+// What bounds it (cycle counters, throw-away builds): every tcgen05 instruction costs its issuing thread 60-85 cycles
+// whatever its size, so a K slice (wait, four MMAs, commit) takes the MMA warp ~470 cycles -- more than the ~420 the
+// tensor pipe needs for four N = 208 MMAs.  With the three scale copies in the same thread it was ~770; with two or four
+// scale slots the chain MMA -> stage released -> copies -> MMA set the pace instead (~510).
+constexpr int MXP_NT = 208;                 // tile columns over the pair
+constexpr int MXP_ROWS = 2 * MX_BM;         // tile rows over the pair
+constexpr int MXP_STAGES = 6;
+constexpr int MXP_A_BYTES = MX_BM * MX_BK;              // 16 KB
+constexpr int MXP_B_BYTES = (MXP_NT / 2) * MX_BK;       // 13 KB
+constexpr int MXP_SFA_OFF = MXP_A_BYTES + MXP_B_BYTES;  // 512 bytes: this CTA's activation scales
+constexpr int MXP_SFB_OFF = MXP_SFA_OFF + 512;          // 1024 bytes: the tile's weight scales
+constexpr int MXP_STAGE_BYTES = 31 * 1024;              // 30.5 KB used; stages stay 1024-byte aligned
+constexpr int MXP_TX_BYTES = MXP_A_BYTES + MXP_B_BYTES + 1024;   // bytes one CTA's loads deliver per stage
+constexpr int MXP_EPI_WARPS = 8;
+constexpr int MXP_COPY_WARP = 3 + MXP_EPI_WARPS;   // the scale-copy warp comes after the epilogue warps
+constexpr int MXP_THREADS = 32 * (4 + MXP_EPI_WARPS);
+constexpr int MXP_STAGING_BYTES = MXP_EPI_WARPS * 2048;
+constexpr int MXP_ACC_STRIDE = 256;         // tensor-memory columns between the two accumulators
+// one scale slot (16 columns) per ring stage, three behind each accumulator: a stage's slot is free when the stage is
+__device__ __forceinline__ uint32_t mxp_slot_col(uint32_t stage) { return MXP_NT + (stage / 3u) * MXP_ACC_STRIDE + (stage % 3u) * 16; }
+static_assert(MXP_STAGES == 6 && MXP_NT + 3 * 16 <= MXP_ACC_STRIDE, "scale slots");
+static_assert(MXP_SFB_OFF + 1024 <= MXP_STAGE_BYTES, "stage layout");
+
+struct MxPairCtl {
+    unsigned long long full[MXP_STAGES];
+    unsigned long long sf_full[MXP_STAGES];   // first CTA: the stage's scales are in tensor memory (and its operands landed)
+    unsigned long long empty[MXP_STAGES];
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    unsigned long long drain;
+    unsigned long long drain_copy;
+    uint32_t tmem_base;
+    int abort_flag;
+    int stage_n[MXP_STAGES];   // columns of the tile a stage belongs to (published by the first CTA's producer)
+    int32_t offs[MX_MAX_E + 1];
+    int32_t tile_prefix[MX_MAX_E + 1];
+};
+constexpr int MXP_SMEM_BYTES = MXP_STAGES * MXP_STAGE_BYTES + MXP_STAGING_BYTES + 1024 + (int)sizeof(MxPairCtl);
+static_assert(MXP_SMEM_BYTES <= 232448, "exceeds the shared memory a CTA can opt in to");
+
+struct MxPairParams {
+    const int32_t* offsets;
+    int E, k_tiles, n_tiles, n_cols;
+    long long R;
+    const uint32_t* sa;   // activation scale words [k_tiles][R]
+    bf16* out;
+    long long ldo;
+};
+
+__device__ __forceinline__ uint32_t mxp_idesc(uint32_t n, uint32_t sf) {
+    return (sf << 4) | ((n >> 3) << 17) | (1u << 23) | ((uint32_t)(MXP_ROWS >> 4) << 24) | (sf << 29);
+}
+__device__ __forceinline__ void mxp_copy_scales(uint32_t taddr, uint64_t sdesc) {
+    asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void mxp_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t sfa,
+                                        uint32_t sfb, uint32_t accumulate) {
+    asm volatile(
+        "{ .reg .pred p; setp.ne.u32 p, %4, 0;"
+        " tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale [%0], %1, %2, %3, [%5], [%6], p; }" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa), "r"(sfb)
+        : "memory");
+}
+// one lane of the (converged) warp
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred = 0;
+    asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; @p mov.u32 %0, 1; }" : "+r"(pred));
+    return pred != 0;
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t v[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+struct MxPairTile {
+    int e, row0, row_end, n0, nt, width;
+};
+__device__ __forceinline__ MxPairTile mxp_decode(const MxPairParams& p, const MxPairCtl* ctl, long long t) {
+    int lo = 0, hi = p.E;   // largest e with tile_prefix[e] * n_tiles <= t
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if ((long long)ctl->tile_prefix[mid] * p.n_tiles <= t) lo = mid; else hi = mid;
+    }
+    const int local = (int)(t - (long long)ctl->tile_prefix[lo] * p.n_tiles);
+    const int m_tiles_e = ctl->tile_prefix[lo + 1] - ctl->tile_prefix[lo];
+    MxPairTile tl;
+    tl.e = lo;
+    tl.nt = local / m_tiles_e;   // column tile major inside an expert (the pairs running together share weight tiles in L2)
+    const int mt = local - tl.nt * m_tiles_e;
+    tl.row0 = ctl->offs[lo] + mt * MXP_ROWS;
+    tl.row_end = ctl->offs[lo + 1];
+    tl.n0 = tl.nt * MXP_NT;
+    tl.width = min(MXP_NT, p.n_cols - tl.n0);
+    return tl;
+}
+
+__global__ void __launch_bounds__(MXP_THREADS, 1)
+mx_down_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_sfb, const __grid_constant__ CUtensorMap map_o,
+                    const MxPairParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
+    MxPairCtl* ctl = reinterpret_cast<MxPairCtl*>(tiles_ptr + MXP_STAGES * MXP_STAGE_BYTES + MXP_STAGING_BYTES);
+    volatile int* abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();   // 0 = the CTA that issues the MMAs
+    const long long first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;
+
+    for (int e = threadIdx.x; e <= p.E; e += MXP_THREADS) ctl->offs[e] = p.offsets[e];
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MXP_STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 4);   // per CTA: the producer's arrive (with its byte count) + the scale warp's
+            mbar_init(smem_u32(&ctl->sf_full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[a]), 2 * MXP_EPI_WARPS);
+        }
+        mbar_init(smem_u32(&ctl->drain), 1);
+        mbar_init(smem_u32(&ctl->drain_copy), 1);
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tmap(&map_a);
+        prefetch_tmap(&map_b);
+        prefetch_tmap(&map_sfb);
+        prefetch_tmap(&map_o);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int e = 0; e < p.E; ++e) {
+            ctl->tile_prefix[e] = run;
+            run += (ctl->offs[e + 1] - ctl->offs[e] + MXP_ROWS - 1) / MXP_ROWS;
+        }
+        ctl->tile_prefix[p.E] = run;
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                     "r"((uint32_t)MX_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();   // the other CTA's barriers and tensor memory exist from here on
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const long long n_tiles_total = (long long)ctl->tile_prefix[p.E] * p.n_tiles;
+    const uint32_t full0 = map_to_cta(smem_u32(&ctl->full[0]), 0);   // full[] of the MMA-issuing CTA
+
+    if (warp == 0) {
+        // ================= producer (both CTAs; each fills its own ring) =================
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, issued = 0;
+            bool ok = true;
+            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+                const MxPairTile tl = mxp_decode(p, ctl, t);
+                const int sfb_row0 = (tl.e * p.n_tiles + tl.nt) * p.k_tiles;
+                const int b_row = tl.e * p.n_cols + tl.n0 + (int)rank * (tl.width >> 1);
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (rank == 0) ctl->stage_n[stage] = tl.width;   // read by the MMA thread after its wait on full[stage]
+                    const uint32_t bar = full0 + stage * (uint32_t)sizeof(unsigned long long);
+                    const uint32_t dst = tiles_base + stage * MXP_STAGE_BYTES;
+                    mbar_arrive_expect_tx_cluster(bar, MXP_TX_BYTES);
+                    tma_load_2d_pair(dst, &map_a, kt * MX_BK, tl.row0 + (int)rank * MX_BM, bar);
+                    tma_load_2d_pair(dst + MXP_A_BYTES, &map_b, kt * MX_BK, b_row, bar);
+                    tma_load_2d_pair(dst + MXP_SFB_OFF, &map_sfb, 0, sfb_row0 + kt, bar);
+                    ++issued;
+                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok && issued != 0) {
+                // leave no bulk copy in flight: the copies report to a barrier this thread cannot always poll (the other
+                // CTA's), so outwait them -- a copy that was issued completes within microseconds
+                const unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 2000000ull) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer: the first CTA's warp 1 =================
+        // The whole warp runs the loop and waits; one elected lane issues the tcgen05 instructions.  With the loop
+        // under `if (lane == 0)` every operand of a tcgen05 instruction (descriptors, addresses: uniform registers) is
+        // computed in the per-thread datapath and moved over, and the thread needed ~600 cycles per K slice against
+        // 448 of the tensor pipe; in converged code the values live in uniform registers from the start.
+        if (rank == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, n = MXP_NT;
+            bool ok = true;
+            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+                if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * MXP_ACC_STRIDE;
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->sf_full[stage]), phase, abort_flag))) { ok = false; break; }
+                    tc_fence_after();
+                    if (kt == 0) n = (uint32_t)ctl->stage_n[stage];
+                    const uint32_t s_base = tiles_base + stage * MXP_STAGE_BYTES;
+                    const uint32_t sfa_t = tmem_base + mxp_slot_col(stage), sfb_t = sfa_t + 4;
+                    const uint64_t a_desc = mx_operand_desc(s_base), b_desc = mx_operand_desc(s_base + MXP_A_BYTES);
+                    if (elect_one()) {
+#pragma unroll
+                        for (int k = 0; k < MX_BK / 32; ++k)
+                            mxp_mma(d_tmem, a_desc + (uint64_t)((k * 32) >> 4), b_desc + (uint64_t)((k * 32) >> 4), mxp_idesc(n, k),
+                                    sfa_t, sfb_t, (kt != 0 || k != 0) ? 1u : 0u);
+                        tc_commit<true>(smem_u32(&ctl->empty[stage]));
+                    }
+                    __syncwarp();
+                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (elect_one()) tc_commit<true>(smem_u32(&ctl->tmem_full[acc]));
+                __syncwarp();
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            // all issued MMAs must have retired before tensor memory is released
+            if (lane == 0) {
+                tc_commit_local<true>(smem_u32(&ctl->drain));
+                const unsigned long long t0 = global_timer_ns();
+                while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
+            }
+        }
+        __syncwarp();
+    } else if (warp == 2) {
+        // ================= activation scales of this CTA's 128 rows =================
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+            const MxPairTile tl = mxp_decode(p, ctl, t);
+            long long rows[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const long long r = (long long)tl.row0 + (int)rank * MX_BM + 32 * i + lane;
+                rows[i] = r < p.R ? r : p.R - 1;   // rows past the end are never stored; any valid address will do
+            }
+            // the words of MX_SCALE_AHEAD slices are in flight at any time: one slice per global-load round trip would
+            // bound the whole pipeline (the loads wait behind the operand traffic)
+            auto load_slice = [&](int kt) {
+                const uint32_t* s = p.sa + (long long)kt * p.R;
+                return make_uint4(__ldg(s + rows[0]), __ldg(s + rows[1]), __ldg(s + rows[2]), __ldg(s + rows[3]));
+            };
+            uint4 q[MX_SCALE_AHEAD];
+#pragma unroll
+            for (int i = 0; i < MX_SCALE_AHEAD; ++i) q[i] = load_slice(min(i, p.k_tiles - 1));
+            for (int kt0 = 0; ok && kt0 < p.k_tiles; kt0 += MX_SCALE_AHEAD) {
+#pragma unroll
+                for (int i = 0; i < MX_SCALE_AHEAD; ++i) {
+                    const int kt = kt0 + i;
+                    if (kt >= p.k_tiles) break;
+                    const uint4 cur = q[i];
+                    if (kt + MX_SCALE_AHEAD < p.k_tiles) q[i] = load_slice(kt + MX_SCALE_AHEAD);
+                    if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    *reinterpret_cast<uint4*>(tiles_ptr + stage * MXP_STAGE_BYTES + MXP_SFA_OFF + lane * 16) = cur;
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(full0 + stage * (uint32_t)sizeof(unsigned long long));
+                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == MXP_COPY_WARP) {
+        // ================= scale copies: one thread of the first CTA =================
+        // Takes the three tcgen05.cp per K slice off the MMA thread (each tcgen05 instruction costs the issuing thread
+        // 60-85 cycles; with them the MMA thread needed ~770 cycles per slice).  Every ring stage has its own scale slot in
+        // tensor memory: full[stage] can only complete after the stage was released, i.e. after the MMAs that read the
+        // slot's previous contents have completed.
+        if (rank == 0 && lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+                for (int kt = 0; kt < p.k_tiles; ++kt) {
+                    if (!mx_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t s_base = tiles_base + stage * MXP_STAGE_BYTES;
+                    const uint32_t sfa_t = tmem_base + mxp_slot_col(stage), sfb_t = sfa_t + 4;
+                    mxp_copy_scales(sfa_t, mx_scale_desc(s_base + MXP_SFA_OFF));
+                    mxp_copy_scales(sfb_t, mx_scale_desc(s_base + MXP_SFB_OFF));
+                    mxp_copy_scales(sfb_t + 4, mx_scale_desc(s_base + MXP_SFB_OFF + 512));
+                    tc_commit_local<true>(smem_u32(&ctl->sf_full[stage]));
+                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            // all issued copies must have retired before tensor memory is released
+            tc_commit_local<true>(smem_u32(&ctl->drain_copy));
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(smem_u32(&ctl->drain_copy), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
+        }
+        __syncwarp();
+    } else {
+        // ================= epilogue (warps 3..10, both CTAs) =================
+        const int quarter = warp & 3;          // tensor-memory lanes [32 * quarter, 32 * quarter + 32)
+        const int half = (warp - 3) >> 2;      // 32-column blocks 0, 2, 4, 6 or 1, 3, 5 (+ the 16-column tail)
+        uint8_t* stage_ptr = tiles_ptr + MXP_STAGES * MXP_STAGE_BYTES + (warp - 3) * 2048;
+        const int sw = (lane >> 1) & 3;
+        const uint32_t empty0 = map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0);
+        uint32_t n_stores = 0, acc = 0, acc_phase = 0;
+        for (long long t = first_tile; t < n_tiles_total; t += tile_stride) {
+            const MxPairTile tl = mxp_decode(p, ctl, t);
+            if (!mx_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + acc * MXP_ACC_STRIDE + ((uint32_t)(quarter * 32) << 16);
+            const int slab0 = tl.row0 + (int)rank * MX_BM + quarter * 32;
+            const int rows_valid = max(0, min(32, tl.row_end - slab0));
+#pragma unroll 1
+            for (int c = half; c < 8; c += 2) {
+                const int left = tl.width - 32 * c;   // columns of the tile from this block on (warp-uniform)
+                if (left <= 0) break;
+                const int n = tl.n0 + c * 32;
+                uint32_t w[16];
+                if (left >= 32) {
+                    uint32_t v[32];
+                    tc_ld32(taddr + c * 32, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                } else {
+                    uint32_t v[16];
+                    tc_ld16(taddr + c * 32, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                }
+                if (rows_valid == 0) continue;
+                if (left >= 32 && rows_valid == 32) {
+                    if (n_stores != 0) {
+                        if (lane == 0) bulk_wait_read0();
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4*>(stage_ptr + lane * 64 + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&map_o, n, slab0, smem_u32(stage_ptr));
+                        bulk_commit();
+                    }
+                    ++n_stores;
+                } else if (lane < rows_valid) {
+                    uint4* d4 = reinterpret_cast<uint4*>(p.out + ((long long)slab0 + lane) * p.ldo + n);
+                    d4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                    d4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    if (left >= 32) {
+                        d4[2] = make_uint4(w[8], w[9], w[10], w[11]);
+                        d4[3] = make_uint4(w[12], w[13], w[14], w[15]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(empty0 + acc * (uint32_t)sizeof(unsigned long long));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (n_stores != 0 && lane == 0) bulk_wait_all0();
+        __syncwarp();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();   // neither CTA's shared memory / barriers may go away while the other still uses them
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)MX_TMEM_COLS) : "memory");
+    }
+}
+
 // ---- quantisers ---------------------------------------------------------------------------------------
 // scale exponent of a block with largest magnitude amax: floor(log2 amax) - 8, clamped to the E8M0 range; -127 for zero
 __device__ __forceinline__ int mx_scale_exp(float amax) {
@@ -384,7 +781,8 @@ __global__ void __launch_bounds__(256) mx_quantize_rows_kernel(const uint2* __re
 // consecutive lanes take consecutive h, so the 32 loads of a thread are coalesced across the warp; the thread keeps the
 // 32 values, picks the scale and writes 32 contiguous code bytes.
 __global__ void __launch_bounds__(256) mx_quantize_w_down_kernel(const bf16* __restrict__ w, int E, int I, int H,
-                                                                 uint8_t* __restrict__ codes, uint8_t* __restrict__ scales) {
+                                                                 uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
+                                                                 uint8_t* __restrict__ scales_pair) {
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int blocks_i = I / 32;
     const long long total = (long long)E * blocks_i * H;
@@ -413,9 +811,20 @@ __global__ void __launch_bounds__(256) mx_quantize_w_down_kernel(const bf16* __r
     const int k_tiles = I / 128;
     scales[(((long long)e * (H / 128) + h / 128) * k_tiles + ib / 4) * 512 + (h % 32) * 16 + ((h % 128) / 32) * 4 + (ib % 4)] =
         (uint8_t)(se + 127);
+    // the same byte in the tiling of the CTA-pair kernel: per (240-column tile, K slice) two 512-byte blocks
+    const int nt = h / MXP_NT, c = h % MXP_NT;
+    const int n_tiles_p = (H + MXP_NT - 1) / MXP_NT;
+    scales_pair[(((long long)e * n_tiles_p + nt) * k_tiles + ib / 4) * 1024 + (c >> 7) * 512 + (c % 32) * 16 + ((c % 128) / 32) * 4 +
+                (ib % 4)] = (uint8_t)(se + 127);
 }
 
 }  // namespace
+
+// The weight scales are stored twice: in the tiling of the single-CTA kernel, then in that of the CTA-pair kernel.
+size_t mx_w_scale_single_bytes(const moe_dims_t& d) { return (size_t)d.E * (d.H / 128) * (d.I / 128) * 512; }
+size_t mx_w_scale_bytes(const moe_dims_t& d) {
+    return mx_w_scale_single_bytes(d) + (size_t)d.E * ((d.H + MXP_NT - 1) / MXP_NT) * (d.I / 128) * 1024;
+}
 
 int launch_mx_quantize_rows(long long rows, int n, const bf16* x, uint8_t* codes, uint8_t* scales, cudaStream_t s) {
     const long long units = rows * (n / 128);
@@ -430,7 +839,54 @@ int launch_mx_quantize_rows(long long rows, int n, const bf16* x, uint8_t* codes
 
 int launch_mx_quantize_w_down(const moe_dims_t& d, const bf16* w_down, uint8_t* codes_t, uint8_t* scales, cudaStream_t s) {
     const long long total = (long long)d.E * (d.I / 32) * d.H;
-    mx_quantize_w_down_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(w_down, d.E, d.I, d.H, codes_t, scales);
+    mx_quantize_w_down_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(w_down, d.E, d.I, d.H, codes_t, scales,
+                                                                              scales + mx_w_scale_single_bytes(d));
+    return check_launch();
+}
+
+// CTA pairs from this many rows per expert on average (below it the 256-row tiles are mostly padding)
+constexpr long long kMxPairRows = 256;
+
+static int launch_down_fwd_mxfp8_pair(const moe_dims_t& d, const uint8_t* h_codes, const uint8_t* h_scales, const uint8_t* w_codes_t,
+                                      const uint8_t* w_scales_pair, const int32_t* offsets, bf16* y_perm, cudaStream_t s) {
+    const uint64_t R = (uint64_t)d.T * d.K;
+    const int n_tiles = (d.H + MXP_NT - 1) / MXP_NT, k_tiles = d.I / MX_BK;
+    CUtensorMap a, b, sfb, o;
+    if (!make_map_typed(&a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h_codes, d.I, R, MX_BK, MX_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_typed(&b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w_codes_t, d.I, (uint64_t)d.E * d.H, MX_BK, MXP_NT / 2,
+                        CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_typed(&sfb, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, w_scales_pair, 256, (uint64_t)d.E * n_tiles * k_tiles, 256, 1,
+                        CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_out_map(&o, y_perm, d.H, R))
+        return MOE_ERR_CUDA;
+    MxPairParams p = {};
+    p.offsets = offsets; p.E = d.E; p.k_tiles = k_tiles; p.n_tiles = n_tiles; p.n_cols = d.H; p.R = (long long)R;
+    p.sa = reinterpret_cast<const uint32_t*>(h_scales); p.out = y_perm; p.ldo = d.H;
+    static int grid_of_device[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(MXP_THREADS);
+    cfg.dynamicSmemBytes = MXP_SMEM_BYTES;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (grid_of_device[dev] == 0) {
+        if (cudaFuncSetAttribute(mx_down_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MXP_SMEM_BYTES) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        const int sms = sm_count();
+        if (sms <= 0) return MOE_ERR_CUDA;
+        // as many pairs as can be resident at once: a pair that had to wait for a free SM pair would double the duration
+        cfg.gridDim = dim3(2 * (sms / 2));
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, mx_down_pair_kernel, &cfg) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
+        if (clusters > sms / 2) clusters = sms / 2;
+        grid_of_device[dev] = 2 * clusters;
+    }
+    cfg.gridDim = dim3(grid_of_device[dev]);
+    cfg.stream = s;
+    if (cudaLaunchKernelEx(&cfg, mx_down_pair_kernel, a, b, sfb, o, p) != cudaSuccess) return MOE_ERR_CUDA;
     return check_launch();
 }
 
@@ -446,6 +902,8 @@ int launch_down_fwd_mxfp8(const moe_dims_t& d, const uint8_t* h_codes, const uin
     MxParams p = {};
     p.offsets = offsets; p.E = d.E; p.k_tiles = d.I / MX_BK; p.n_tiles = d.H / MX_BN; p.n_cols = d.H; p.R = (long long)R;
     p.sa = reinterpret_cast<const uint32_t*>(h_scales); p.sb = w_scales; p.out = y_perm; p.ldo = d.H;
+    if ((long long)R >= kMxPairRows * d.E)
+        return launch_down_fwd_mxfp8_pair(d, h_codes, h_scales, w_codes_t, w_scales + mx_w_scale_single_bytes(d), offsets, y_perm, s);
     static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;

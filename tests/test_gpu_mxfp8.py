@@ -34,11 +34,28 @@ def _w_scales_from_layout(raw, E, H, I):
     return g.transpose(0, 1, 4, 3, 2, 5).reshape(E, H, I // 32)
 
 
+def _w_scales_pair_layout(scales, E, H, I):
+    """[E, H, I/32] -> the second copy of the weight scales, in the tiling of the CTA-pair kernel:
+    [E][ceil(H/208)][I/128][2 blocks][h' % 32][(h' % 128) / 32][b % 4] with h' = h % 208; also the mask of written bytes"""
+    n_tiles = (H + 207) // 208
+    out = np.zeros((E, n_tiles, I // 128, 2, 32, 4, 4), dtype=np.uint8)
+    written = np.zeros(out.shape, dtype=bool)
+    h = np.arange(H)
+    c = h % 208
+    for b in range(I // 32):
+        out[:, h // 208, b // 4, c >> 7, c % 32, (c % 128) // 32, b % 4] = scales[:, :, b]
+        written[:, h // 208, b // 4, c >> 7, c % 32, (c % 128) // 32, b % 4] = True
+    return out.reshape(-1), written.reshape(-1)
+
+
 CASES = {
     "one_tile": ([128], 1, 128, 128),
     "ragged": ([0, 1, 127, 0, 129, 128, 300, 15, 0], 2, 256, 384),
     "wide": ([200, 0, 31, 290, 1], 2, 384, 1408),              # 11 slices of the contraction, 3 column tiles
-    "many_tiles": ([700, 513, 64], 1, 128, 256),
+    "many_tiles": ([700, 513, 64], 1, 128, 256),                # >= 256 rows per expert on average: CTA pairs from here on
+    "pair_narrow_edge": ([300, 256, 511, 1], 2, 256, 256),      # column tiles of 208 and 48
+    "pair_wide": ([700, 0, 514, 300, 1000], 2, 640, 384),       # column tiles 208, 208, 208, 16; an empty expert
+    "pair_one_row_tiles": ([257, 1, 769], 1, 384, 128),         # second CTA's rows empty / one row into the next tile
 }
 
 
@@ -61,7 +78,8 @@ def test_quantisers_and_gemm_against_the_oracle(B, name):
     u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
     hc, hs = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
     wc, ws = u8(E * H * I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
-    assert hs.numel() == (I // 128) * R * 4 and ws.numel() == E * (H // 128) * (I // 128) * 512
+    n_single = E * (H // 128) * (I // 128) * 512
+    assert hs.numel() == (I // 128) * R * 4 and ws.numel() == n_single + E * ((H + 207) // 208) * (I // 128) * 1024
     B.moe_mxfp8_quantize_h_act(d, h_dev, hc, hs)
     B.moe_mxfp8_quantize_w_down(d, w_dev, wc, ws)
     torch.cuda.synchronize()
@@ -70,7 +88,11 @@ def test_quantisers_and_gemm_against_the_oracle(B, name):
     o_wc, o_ws, _ = O.mxfp8_quantize(wt)
     assert np.array_equal(_act_scales_from_layout(hs.cpu().numpy(), R, I), o_hs)
     assert np.array_equal(hc.cpu().numpy().reshape(R, I), o_hc)
-    assert np.array_equal(_w_scales_from_layout(ws.cpu().numpy(), E, H, I), o_ws)
+    ws_host = ws.cpu().numpy()
+    assert np.array_equal(_w_scales_from_layout(ws_host[:n_single], E, H, I), o_ws)
+    want_pair, written = _w_scales_pair_layout(o_ws, E, H, I)
+    assert np.array_equal(ws_host[n_single:][written], want_pair[written])
+    assert np.all(ws_host[n_single:][~written] == 0xAB)          # bytes no column owns are left alone
     assert np.array_equal(wc.cpu().numpy().reshape(E, H, I), o_wc)
     # the GEMM on the quantised operands
     yp = torch.full((R, H), float("nan"), dtype=torch.bfloat16, device="cuda")
