@@ -134,6 +134,58 @@ def test_sampled_weight_gradient_blocks_against_exact_chain(full):
         assert not bool(b.dw_gate[e].any()) and not bool(b.dw_up[e].any()) and not bool(b.dw_down[e].any())
 
 
+def test_mxfp8_down_sampled_rows(full):
+    """The block-scaled FP8 down projection at full size (the CTA-pair kernel on the four workloads it takes): codes
+    and scale bytes of 48 sampled rows bit for bit, and those rows of Y_perm against the exact product of the
+    dequantised operands -- the oracle quantises the sampled rows and their experts' weights only.  The row of every
+    expert boundary is among the samples.  Run to run the result is the same bits."""
+    cfg, dev, b = full
+    if cfg.H % 128 or cfg.I % 128:
+        pytest.skip("the block-scaled path takes widths that are multiples of 128")
+    from paper_2606_26453_b200 import binding as B
+    d = b.d
+    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    hc, hs = u8(cfg.R * cfg.I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    wc, ws = u8(cfg.E * cfg.H * cfg.I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
+    B.moe_mxfp8_quantize_h_act(d, b.h_act, hc, hs)
+    B.moe_mxfp8_quantize_w_down(d, dev["W_down"], wc, ws)
+    yq = torch.full((cfg.R, cfg.H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, b.offsets, yq)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    assert not bool(torch.isnan(yq).any())                       # every row of every expert was written
+    offsets = b.offsets.cpu().numpy()
+    rng = np.random.default_rng(cfg.cfg_id + 7)
+    nonempty = np.flatnonzero(np.diff(offsets) > 0)
+    experts = rng.choice(nonempty, size=min(6, nonempty.size), replace=False)
+    rows = []
+    for e in experts:
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        rows += [lo, hi - 1] + list(rng.integers(lo, hi, size=6))    # first and last row of the expert + 6 inside
+    rows = np.array(sorted(set(rows)))
+    expert_of = np.searchsorted(offsets, rows, side="right") - 1
+    rsel = torch.from_numpy(rows).cuda()
+    h_rows = f32(b.h_act[rsel])
+    o_codes, o_scales, h_deq = O.mxfp8_quantize(h_rows)
+    assert np.array_equal(hc.view(cfg.R, cfg.I)[rsel].cpu().numpy(), o_codes)
+    got_scales = hs.view(cfg.I // 128, cfg.R, 4)[:, rsel].cpu().numpy().transpose(1, 0, 2).reshape(rows.size, cfg.I // 32)
+    assert np.array_equal(got_scales, o_scales)
+    got = Hh.to_np64(yq[rsel])
+    want = np.empty_like(got)
+    for e in experts:
+        wt = np.swapaxes(f32(dev["W_down"][int(e)]), 0, 1)       # [H, I]: contraction last
+        w_codes, _, w_deq = O.mxfp8_quantize(wt)
+        assert np.array_equal(wc.view(cfg.E, cfg.H, cfg.I)[int(e)].cpu().numpy(), w_codes)
+        sel = expert_of == e
+        want[sel] = h_deq[sel] @ w_deq.T
+    Hh.assert_close(got, want, f"{cfg.name}: Y_perm rows (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    first = yq.clone()
+    yq.fill_(float("nan"))
+    B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, b.offsets, yq)
+    torch.cuda.synchronize()
+    assert torch.equal(yq, first)
+
+
 # ------------------------------------------------------------------------------------------------
 # every element of every output, where the oracle can afford the whole layer (about 15 s and 45 s of host time)
 # ------------------------------------------------------------------------------------------------
