@@ -370,3 +370,19 @@ def down_mxfp8(H_act, W_down, offsets):
     Wt = np.swapaxes(_f64(W_down), 1, 2)                 # [E, H, I]: contraction last
     _, _, b_deq = mxfp8_quantize(Wt)
     return down(a_deq, np.swapaxes(b_deq, 1, 2), offsets)
+
+
+def down_dgrad_mxfp8(dY_perm, W_down, offsets):
+    """The data gradient of the down projection with both operands block-scaled FP8 along ITS contraction (H):
+    dHact[r,:] = Q(dYp[r,:]) @ Q(Wd[e])^T where Q quantises dYp row-wise in blocks of 32 along H and Wd[e] [I,H]
+    row-wise in blocks of 32 along H (each intermediate feature i has its own scales), and the product of the
+    dequantised operands is taken exactly.  Returns dHact [R,I] float64."""
+    _, _, a_deq = mxfp8_quantize(dY_perm)
+    _, _, b_deq = mxfp8_quantize(_f64(W_down))           # [E, I, H]: contraction last as it lies
+    E = b_deq.shape[0]
+    out = np.zeros((a_deq.shape[0], b_deq.shape[1]), dtype=F64)
+    for e in range(E):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        if hi > lo:
+            out[lo:hi] = a_deq[lo:hi] @ b_deq[e].T
+    return out

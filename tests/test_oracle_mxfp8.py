@@ -104,3 +104,33 @@ def test_down_mxfp8_is_the_exact_product_of_the_dequantised_operands():
     Hq = O.mxfp8_quantize(Hact)[2]
     Wq = np.swapaxes(O.mxfp8_quantize(np.swapaxes(Wd, 1, 2))[2], 1, 2)
     assert np.array_equal(O.down_mxfp8(Hq, Wq, offsets), O.down(Hq, Wq, offsets))
+
+
+def test_down_dgrad_mxfp8_is_the_exact_product_of_the_dequantised_operands():
+    rng = np.random.default_rng(4)
+    E, I, H = 3, 64, 96
+    counts = [0, 6, 7]
+    offsets = np.concatenate([[0], np.cumsum(counts)])
+    dYp = rng.standard_normal((13, H))
+    Wd = rng.standard_normal((E, I, H)) * 0.05
+    got = O.down_dgrad_mxfp8(dYp, Wd, offsets)
+    assert got.shape == (13, I)
+    # written out per element with the quantiser applied by hand to each operand vector (both along H)
+    for r, e in ((0, 1), (5, 1), (6, 2), (12, 2)):
+        a = O.mxfp8_quantize(dYp[r])[2]
+        for i in (0, 9, 19):
+            b = O.mxfp8_quantize(Wd[e, i, :])[2]
+            assert abs(got[r, i] - float(a @ b)) <= 1e-12
+    # against the unquantised data gradient: a few per cent; exactly equal when the operands are representable
+    ref = O.down_bwd(dYp, rng.standard_normal((13, I)), Wd, offsets)[0]
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert 0.01 < rel < 0.06
+    dq, wq = O.mxfp8_quantize(dYp)[2], O.mxfp8_quantize(Wd)[2]
+    assert np.array_equal(O.down_dgrad_mxfp8(dq, wq, offsets), O.down_bwd(dq, np.zeros((13, I)), wq, offsets)[0])
+    # a transposed weight operand (scales taken along I instead of H) is a different, detectably different, result
+    wrong = np.zeros_like(got)
+    w_alt = np.swapaxes(O.mxfp8_quantize(np.swapaxes(Wd, 1, 2))[2], 1, 2)
+    for e in range(E):
+        lo, hi = offsets[e], offsets[e + 1]
+        wrong[lo:hi] = O.mxfp8_quantize(dYp)[2][lo:hi] @ w_alt[e].T
+    assert np.abs(wrong - got).max() > 1e-6
