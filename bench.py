@@ -213,10 +213,18 @@ def time_mxfp8_down(B, cfg, res, device, reps=20, min_seconds=0.3):
     hc, hs = u8(cfg.R * cfg.I), u8(B.moe_mxfp8_act_scale_bytes(d))
     wc, ws = u8(cfg.E * cfg.H * cfg.I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
     yq = torch.empty_like(b.y_perm)
+    dc, ds = u8(cfg.R * cfg.H), u8(B.moe_mxfp8_dy_scale_bytes(d))
+    vc, vs = u8(cfg.E * cfg.I * cfg.H), u8(B.moe_mxfp8_w_down_dgrad_scale_bytes(d))
+    dhq = torch.empty_like(b.dh_act)
+    dh_ref = b.dh_act.clone()
     fns = {"bf16_down_ms": lambda: B.moe_grouped_gemm_down(d, b.h_act, wl["W_down"], b.offsets, b.y_perm),
            "quantize_h_act_ms": lambda: B.moe_mxfp8_quantize_h_act(d, b.h_act, hc, hs),
            "quantize_w_down_ms": lambda: B.moe_mxfp8_quantize_w_down(d, wl["W_down"], wc, ws),
-           "mxfp8_down_ms": lambda: B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, b.offsets, yq)}
+           "mxfp8_down_ms": lambda: B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, b.offsets, yq),
+           "bf16_down_dgrad_ms": lambda: B.moe_grouped_gemm_down_dgrad(d, b.dy_perm, wl["W_down"], b.offsets, dh_ref),
+           "quantize_dy_perm_ms": lambda: B.moe_mxfp8_quantize_dy_perm(d, b.dy_perm, dc, ds),
+           "quantize_w_down_dgrad_ms": lambda: B.moe_mxfp8_quantize_w_down_dgrad(d, wl["W_down"], vc, vs),
+           "mxfp8_down_dgrad_ms": lambda: B.moe_grouped_gemm_down_dgrad_mxfp8(d, dc, ds, vc, vs, b.offsets, dhq)}
     out = {}
     for name, fn in fns.items():
         for _ in range(3):
@@ -236,7 +244,10 @@ def time_mxfp8_down(B, cfg, res, device, reps=20, min_seconds=0.3):
     fl = 2.0 * cfg.R * cfg.H * cfg.I
     out["bf16_down_tflops"] = fl / (out["bf16_down_ms"] * 1e-3) / 1e12
     out["mxfp8_down_tflops"] = fl / (out["mxfp8_down_ms"] * 1e-3) / 1e12
+    out["bf16_down_dgrad_tflops"] = fl / (out["bf16_down_dgrad_ms"] * 1e-3) / 1e12
+    out["mxfp8_down_dgrad_tflops"] = fl / (out["mxfp8_down_dgrad_ms"] * 1e-3) / 1e12
     out["rel_frobenius_to_bf16_result"] = float((yq.float() - b.y_perm.float()).norm() / b.y_perm.float().norm())
+    out["dgrad_rel_frobenius_to_bf16_result"] = float((dhq.float() - dh_ref.float()).norm() / dh_ref.float().norm())
     out["note"] = ("E4M3 elements, E8M0 scale per 32 along the contraction; tcgen05.mma kind::mxf8f6f4.block_scale on "
                    "256 x 208 CTA-pair tiles from 256 rows per expert on average, 128 x 128 single-CTA tiles below; "
                    "the bf16 twin runs 256 x 256 CTA-pair tiles")

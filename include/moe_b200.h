@@ -254,6 +254,26 @@ int moe_grouped_gemm_down_mxfp8(const moe_dims_t* dims, const void* h_codes, con
                                 const void* w_codes_t, const void* w_scales, const int32_t* offsets,
                                 void* y_perm, moe_stream_t stream);
 
+/* The data gradient of the down projection on the same kernels: dh_act[r,:] = dequant(dy row r) . dequant(w_down[e])^T
+ * with both operands block-scaled along ITS contraction, H (defined by the benchmark spec's backward counterparts
+ * and the format above; the paper has no FP8 path of its own).  w_down [E,I,H] is already contraction-contiguous:
+ *   moe_mxfp8_quantize_dy_perm       dy_perm [R,H] bf16 -> codes [R,H] bytes; scales: moe_mxfp8_dy_scale_bytes(dims)
+ *                                    bytes laid out [H/128][R][4] (as the activation scales above, slices along H).
+ *   moe_mxfp8_quantize_w_down_dgrad  w_down [E,I,H] bf16 -> codes [E,I,H] bytes (same layout); scales:
+ *                                    moe_mxfp8_w_down_dgrad_scale_bytes(dims) bytes, the two tilings described above
+ *                                    with the roles of the axes exchanged (feature = i, 128-wide slices along H).
+ *   moe_grouped_gemm_down_dgrad_mxfp8  dh_act [R,I] bf16, overwritten.
+ * Same requirements, status codes and tolerance statement as the forward call. */
+size_t moe_mxfp8_dy_scale_bytes(const moe_dims_t* dims);
+size_t moe_mxfp8_w_down_dgrad_scale_bytes(const moe_dims_t* dims);
+int moe_mxfp8_quantize_dy_perm(const moe_dims_t* dims, const void* dy_perm, void* codes, void* scales,
+                               moe_stream_t stream);
+int moe_mxfp8_quantize_w_down_dgrad(const moe_dims_t* dims, const void* w_down, void* codes, void* scales,
+                                    moe_stream_t stream);
+int moe_grouped_gemm_down_dgrad_mxfp8(const moe_dims_t* dims, const void* dy_codes, const void* dy_scales,
+                                      const void* w_codes, const void* w_scales, const int32_t* offsets,
+                                      void* dh_act, moe_stream_t stream);
+
 /* ---- whole layer from HOST activations ------------------------------------------------------
  * One training step of the layer for a caller whose per-step tensors live in host memory:
  * copies x, topk_idx, topk_w, dy (HOST pointers; pinned memory makes the copies asynchronous)

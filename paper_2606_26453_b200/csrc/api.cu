@@ -265,7 +265,7 @@ size_t moe_mxfp8_act_scale_bytes(const moe_dims_t* dims) {
 
 size_t moe_mxfp8_w_down_scale_bytes(const moe_dims_t* dims) {
     if (check_mx_dims(dims) != MOE_OK) return 0;
-    return mx_w_scale_bytes(*dims);
+    return mx_w_scale_bytes(dims->E, dims->H, dims->I);
 }
 
 int moe_mxfp8_quantize_h_act(const moe_dims_t* dims, const void* h_act, void* codes, void* scales, moe_stream_t stream) {
@@ -297,9 +297,55 @@ int moe_grouped_gemm_down_mxfp8(const moe_dims_t* dims, const void* h_codes, con
     const void* const opt[] = {nullptr};
     s = check_ptrs(req, opt);
     if (s != MOE_OK) return s;
-    return launch_down_fwd_mxfp8(*dims, static_cast<const uint8_t*>(h_codes), static_cast<const uint8_t*>(h_scales),
-                                 static_cast<const uint8_t*>(w_codes_t), static_cast<const uint8_t*>(w_scales), offsets,
-                                 mb(y_perm), st(stream));
+    return launch_mx_gemm((long long)dims->T * dims->K, dims->E, dims->H, dims->I, static_cast<const uint8_t*>(h_codes),
+                          static_cast<const uint8_t*>(h_scales), static_cast<const uint8_t*>(w_codes_t),
+                          static_cast<const uint8_t*>(w_scales), offsets, mb(y_perm), st(stream));
+}
+
+// ---- block-scaled FP8 data gradient of the down projection (contraction over H) ----
+size_t moe_mxfp8_dy_scale_bytes(const moe_dims_t* dims) {
+    if (check_mx_dims(dims) != MOE_OK) return 0;
+    return (size_t)(dims->H / 128) * (size_t)dims->T * dims->K * 4;
+}
+
+size_t moe_mxfp8_w_down_dgrad_scale_bytes(const moe_dims_t* dims) {
+    if (check_mx_dims(dims) != MOE_OK) return 0;
+    return mx_w_scale_bytes(dims->E, dims->I, dims->H);
+}
+
+int moe_mxfp8_quantize_dy_perm(const moe_dims_t* dims, const void* dy_perm, void* codes, void* scales, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {dy_perm, codes, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_rows((long long)dims->T * dims->K, dims->H, cb(dy_perm), static_cast<uint8_t*>(codes),
+                                   static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_mxfp8_quantize_w_down_dgrad(const moe_dims_t* dims, const void* w_down, void* codes, void* scales, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {w_down, codes, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_w_rows(dims->E, dims->I, dims->H, cb(w_down), static_cast<uint8_t*>(codes),
+                                     static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_grouped_gemm_down_dgrad_mxfp8(const moe_dims_t* dims, const void* dy_codes, const void* dy_scales, const void* w_codes,
+                                      const void* w_scales, const int32_t* offsets, void* dh_act, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {dy_codes, dy_scales, w_codes, w_scales, offsets, dh_act};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_gemm((long long)dims->T * dims->K, dims->E, dims->I, dims->H, static_cast<const uint8_t*>(dy_codes),
+                          static_cast<const uint8_t*>(dy_scales), static_cast<const uint8_t*>(w_codes),
+                          static_cast<const uint8_t*>(w_scales), offsets, mb(dh_act), st(stream));
 }
 
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).

@@ -745,35 +745,79 @@ __device__ __forceinline__ int mx_scale_exp(float amax) {
 __device__ __forceinline__ float mx_inv_scale(int s) {
     return s == 127 ? __int_as_float(0x00400000) : __int_as_float((127 - s) << 23);
 }
+// two values -> two codes (the first in the low byte), one conversion instruction
+__device__ __forceinline__ uint32_t mx_e4m3x2(float lo, float hi) {
+    return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
+}
 __device__ __forceinline__ uint32_t mx_e4m3(float v) {
     return (uint32_t)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
 }
 
-// rows x n bf16 -> codes and scale words.  One warp per (row, 128-wide slice): lane l holds elements 4l..4l+3, the 8
-// lanes of a block of 32 agree on its scale through three shuffles.
-__global__ void __launch_bounds__(256) mx_quantize_rows_kernel(const uint2* __restrict__ x, long long rows, int n,
-                                                               uint32_t* __restrict__ codes, uint32_t* __restrict__ scales) {
+// rows x n bf16 -> codes (same layout) and scales.  A warp takes two (row, 128-wide slice) units per load: lane l holds
+// the 8 elements 8l..8l+7 of the 256 contiguous ones (one 16-byte load), the 4 lanes of a block of 32 agree on its scale
+// through two shuffles; two such loads are in flight per lane.  The 4 scale bytes of a (row, slice) are one 32-bit word:
+//   WEIGHTS = false (activations): word [slice][row];
+//   WEIGHTS = true  (weights whose contraction axis is contiguous, rows = E * n_feat, e.g. W_down read as [I, H] for the
+//                    data gradient): the word's place in each of the two weight-scale tilings.
+template <bool WEIGHTS>
+__global__ void __launch_bounds__(256) mx_quantize_rows_kernel(const uint4* __restrict__ x, long long rows, int n, int n_feat,
+                                                               uint2* __restrict__ codes, uint8_t* __restrict__ scales,
+                                                               uint8_t* __restrict__ scales_pair) {
+    constexpr int U = 2;
     const int lane = threadIdx.x & 31;
     const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
     const int k_tiles = n / 128;
-    for (long long u = warp; u < rows * k_tiles; u += n_warps) {
-        const long long r = u / k_tiles;
-        const int kt = (int)(u - r * k_tiles);
-        const uint2 raw = __ldg(x + (r * n + kt * 128) / 4 + lane);
-        const float2 v01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
-        const float2 v23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
-        float amax = fmaxf(fmaxf(fabsf(v01.x), fabsf(v01.y)), fmaxf(fabsf(v23.x), fabsf(v23.y)));
+    const long long total = rows * k_tiles;            // units of 128 elements, contiguous in memory
+    const long long pairs = (total + 1) / 2;
+    const int n_tiles_p = WEIGHTS ? (n_feat + MXP_NT - 1) / MXP_NT : 0;
+    for (long long p0 = warp * U; p0 < pairs; p0 += n_warps * U) {
+        uint4 raw[U];
 #pragma unroll
-        for (int s = 1; s < 8; s <<= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, s));
-        const int se = mx_scale_exp(amax);
-        const float inv = mx_inv_scale(se);
-        codes[(r * n + kt * 128) / 4 + lane] = mx_e4m3(v01.x * inv) | (mx_e4m3(v01.y * inv) << 8) | (mx_e4m3(v23.x * inv) << 16) |
-                                               (mx_e4m3(v23.y * inv) << 24);
-        const uint32_t sbyte = (uint32_t)(se + 127);
-        const uint32_t word = __shfl_sync(0xffffffffu, sbyte, 0) | (__shfl_sync(0xffffffffu, sbyte, 8) << 8) |
-                              (__shfl_sync(0xffffffffu, sbyte, 16) << 16) | (__shfl_sync(0xffffffffu, sbyte, 24) << 24);
-        if (lane == 0) scales[(long long)kt * rows + r] = word;
+        for (int i = 0; i < U; ++i) {
+            const long long u = 2 * (p0 + i) + (lane >> 4);
+            raw[i] = (u < total) ? __ldg(x + (p0 + i) * 32 + lane) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int i = 0; i < U; ++i) {
+            if (p0 + i >= pairs) break;
+            const long long u = 2 * (p0 + i) + (lane >> 4);   // this half-warp's unit
+            const uint32_t* rw = reinterpret_cast<const uint32_t*>(&raw[i]);
+            float v[8];
+            float amax = 0.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&rw[j]));
+                v[2 * j] = f.x; v[2 * j + 1] = f.y;
+                amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
+            }
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+            const int se = mx_scale_exp(amax);
+            const float inv = mx_inv_scale(se);
+            uint2 out;
+            out.x = mx_e4m3x2(v[0] * inv, v[1] * inv) | (mx_e4m3x2(v[2] * inv, v[3] * inv) << 16);
+            out.y = mx_e4m3x2(v[4] * inv, v[5] * inv) | (mx_e4m3x2(v[6] * inv, v[7] * inv) << 16);
+            if (u < total) codes[(p0 + i) * 32 + lane] = out;
+            const uint32_t sbyte = (uint32_t)(se + 127);
+            const int base = lane & 16;                       // first lane of this half-warp
+            const uint32_t word = __shfl_sync(0xffffffffu, sbyte, base) | (__shfl_sync(0xffffffffu, sbyte, base + 4) << 8) |
+                                  (__shfl_sync(0xffffffffu, sbyte, base + 8) << 16) | (__shfl_sync(0xffffffffu, sbyte, base + 12) << 24);
+            if ((lane & 15) == 0 && u < total) {
+                const long long r = u / k_tiles;
+                const int kt = (int)(u - r * k_tiles);
+                if (!WEIGHTS) {
+                    reinterpret_cast<uint32_t*>(scales)[(long long)kt * rows + r] = word;
+                } else {
+                    const int e = (int)(r / n_feat), f = (int)(r - (long long)e * n_feat);
+                    *reinterpret_cast<uint32_t*>(scales + (((long long)e * (n_feat / 128) + f / 128) * k_tiles + kt) * 512 +
+                                                 (f % 32) * 16 + ((f % 128) / 32) * 4) = word;
+                    const int nt = f / MXP_NT, c = f % MXP_NT;
+                    *reinterpret_cast<uint32_t*>(scales_pair + (((long long)e * n_tiles_p + nt) * k_tiles + kt) * 1024 +
+                                                 (c >> 7) * 512 + (c % 32) * 16 + ((c % 128) / 32) * 4) = word;
+                }
+            }
+        }
     }
 }
 
@@ -820,48 +864,59 @@ __global__ void __launch_bounds__(256) mx_quantize_w_down_kernel(const bf16* __r
 
 }  // namespace
 
-// The weight scales are stored twice: in the tiling of the single-CTA kernel, then in that of the CTA-pair kernel.
-size_t mx_w_scale_single_bytes(const moe_dims_t& d) { return (size_t)d.E * (d.H / 128) * (d.I / 128) * 512; }
-size_t mx_w_scale_bytes(const moe_dims_t& d) {
-    return mx_w_scale_single_bytes(d) + (size_t)d.E * ((d.H + MXP_NT - 1) / MXP_NT) * (d.I / 128) * 1024;
+// Weight scales of a GEMM with E experts, n_feat output features and a contraction of k: stored twice, in the tiling of
+// the single-CTA kernel, then in that of the CTA-pair kernel.
+size_t mx_w_scale_single_bytes(int E, int n_feat, int k) { return (size_t)E * (n_feat / 128) * (k / 128) * 512; }
+size_t mx_w_scale_bytes(int E, int n_feat, int k) {
+    return mx_w_scale_single_bytes(E, n_feat, k) + (size_t)E * ((n_feat + MXP_NT - 1) / MXP_NT) * (k / 128) * 1024;
+}
+
+static unsigned mx_row_quantiser_blocks(long long units) {
+    long long blocks = (units + 31) / 32;   // 8 warps x 4 units per block and pass
+    const long long cap = (long long)sm_count() * 16;
+    if (blocks > cap) blocks = cap;
+    return (unsigned)(blocks < 1 ? 1 : blocks);
 }
 
 int launch_mx_quantize_rows(long long rows, int n, const bf16* x, uint8_t* codes, uint8_t* scales, cudaStream_t s) {
-    const long long units = rows * (n / 128);
-    long long blocks = (units + 7) / 8;
-    const long long cap = (long long)sm_count() * 16;
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
-    mx_quantize_rows_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const uint2*>(x), rows, n,
-                                                           reinterpret_cast<uint32_t*>(codes), reinterpret_cast<uint32_t*>(scales));
+    mx_quantize_rows_kernel<false><<<mx_row_quantiser_blocks(rows * (n / 128)), 256, 0, s>>>(
+        reinterpret_cast<const uint4*>(x), rows, n, 0, reinterpret_cast<uint2*>(codes), scales, nullptr);
     return check_launch();
 }
 
 int launch_mx_quantize_w_down(const moe_dims_t& d, const bf16* w_down, uint8_t* codes_t, uint8_t* scales, cudaStream_t s) {
     const long long total = (long long)d.E * (d.I / 32) * d.H;
     mx_quantize_w_down_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(w_down, d.E, d.I, d.H, codes_t, scales,
-                                                                              scales + mx_w_scale_single_bytes(d));
+                                                                              scales + mx_w_scale_single_bytes(d.E, d.H, d.I));
+    return check_launch();
+}
+
+int launch_mx_quantize_w_rows(int E, int n_feat, int k, const bf16* w, uint8_t* codes, uint8_t* scales, cudaStream_t s) {
+    const long long rows = (long long)E * n_feat;
+    mx_quantize_rows_kernel<true><<<mx_row_quantiser_blocks(rows * (k / 128)), 256, 0, s>>>(
+        reinterpret_cast<const uint4*>(w), rows, k, n_feat, reinterpret_cast<uint2*>(codes), scales,
+        scales + mx_w_scale_single_bytes(E, n_feat, k));
     return check_launch();
 }
 
 // CTA pairs from this many rows per expert on average (below it the 256-row tiles are mostly padding)
 constexpr long long kMxPairRows = 256;
 
-static int launch_down_fwd_mxfp8_pair(const moe_dims_t& d, const uint8_t* h_codes, const uint8_t* h_scales, const uint8_t* w_codes_t,
-                                      const uint8_t* w_scales_pair, const int32_t* offsets, bf16* y_perm, cudaStream_t s) {
-    const uint64_t R = (uint64_t)d.T * d.K;
-    const int n_tiles = (d.H + MXP_NT - 1) / MXP_NT, k_tiles = d.I / MX_BK;
+static int launch_mx_gemm_pair(long long R, int E, int n_feat, int k, const uint8_t* a_codes, const uint8_t* a_scales,
+                               const uint8_t* b_codes, const uint8_t* b_scales_pair, const int32_t* offsets, bf16* out,
+                               cudaStream_t s) {
+    const int n_tiles = (n_feat + MXP_NT - 1) / MXP_NT, k_tiles = k / MX_BK;
     CUtensorMap a, b, sfb, o;
-    if (!make_map_typed(&a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h_codes, d.I, R, MX_BK, MX_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_typed(&b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w_codes_t, d.I, (uint64_t)d.E * d.H, MX_BK, MXP_NT / 2,
+    if (!make_map_typed(&a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes, k, (uint64_t)R, MX_BK, MX_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_typed(&b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes, k, (uint64_t)E * n_feat, MX_BK, MXP_NT / 2,
                         CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_typed(&sfb, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, w_scales_pair, 256, (uint64_t)d.E * n_tiles * k_tiles, 256, 1,
+        !make_map_typed(&sfb, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, b_scales_pair, 256, (uint64_t)E * n_tiles * k_tiles, 256, 1,
                         CU_TENSOR_MAP_SWIZZLE_NONE) ||
-        !make_out_map(&o, y_perm, d.H, R))
+        !make_out_map(&o, out, n_feat, (uint64_t)R))
         return MOE_ERR_CUDA;
     MxPairParams p = {};
-    p.offsets = offsets; p.E = d.E; p.k_tiles = k_tiles; p.n_tiles = n_tiles; p.n_cols = d.H; p.R = (long long)R;
-    p.sa = reinterpret_cast<const uint32_t*>(h_scales); p.out = y_perm; p.ldo = d.H;
+    p.offsets = offsets; p.E = E; p.k_tiles = k_tiles; p.n_tiles = n_tiles; p.n_cols = n_feat; p.R = R;
+    p.sa = reinterpret_cast<const uint32_t*>(a_scales); p.out = out; p.ldo = n_feat;
     static int grid_of_device[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
@@ -890,20 +945,22 @@ static int launch_down_fwd_mxfp8_pair(const moe_dims_t& d, const uint8_t* h_code
     return check_launch();
 }
 
-int launch_down_fwd_mxfp8(const moe_dims_t& d, const uint8_t* h_codes, const uint8_t* h_scales, const uint8_t* w_codes_t,
-                          const uint8_t* w_scales, const int32_t* offsets, bf16* y_perm, cudaStream_t s) {
-    const uint64_t R = (uint64_t)d.T * d.K;
+// out[r, :] = dequant(a row r) . dequant(b[e])^T for the rows r of expert e: a [R, k] codes with scale words
+// [k/128][R], b [E, n_feat, k] codes with both scale tilings, out [R, n_feat] bf16.
+int launch_mx_gemm(long long R, int E, int n_feat, int k, const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
+                   const uint8_t* b_scales, const int32_t* offsets, bf16* out, cudaStream_t s) {
+    if (R >= kMxPairRows * E)
+        return launch_mx_gemm_pair(R, E, n_feat, k, a_codes, a_scales, b_codes, b_scales + mx_w_scale_single_bytes(E, n_feat, k),
+                                   offsets, out, s);
     CUtensorMap a, b, o;
-    if (!make_map_typed(&a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, h_codes, d.I, R, MX_BK, MX_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_map_typed(&b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, w_codes_t, d.I, (uint64_t)d.E * d.H, MX_BK, MX_BN,
+    if (!make_map_typed(&a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes, k, (uint64_t)R, MX_BK, MX_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_typed(&b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes, k, (uint64_t)E * n_feat, MX_BK, MX_BN,
                         CU_TENSOR_MAP_SWIZZLE_128B) ||
-        !make_out_map(&o, y_perm, d.H, R))
+        !make_out_map(&o, out, n_feat, (uint64_t)R))
         return MOE_ERR_CUDA;
     MxParams p = {};
-    p.offsets = offsets; p.E = d.E; p.k_tiles = d.I / MX_BK; p.n_tiles = d.H / MX_BN; p.n_cols = d.H; p.R = (long long)R;
-    p.sa = reinterpret_cast<const uint32_t*>(h_scales); p.sb = w_scales; p.out = y_perm; p.ldo = d.H;
-    if ((long long)R >= kMxPairRows * d.E)
-        return launch_down_fwd_mxfp8_pair(d, h_codes, h_scales, w_codes_t, w_scales + mx_w_scale_single_bytes(d), offsets, y_perm, s);
+    p.offsets = offsets; p.E = E; p.k_tiles = k / MX_BK; p.n_tiles = n_feat / MX_BN; p.n_cols = n_feat; p.R = R;
+    p.sa = reinterpret_cast<const uint32_t*>(a_scales); p.sb = b_scales; p.out = out; p.ldo = n_feat;
     static bool attr_set[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;

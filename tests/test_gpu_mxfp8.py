@@ -34,7 +34,7 @@ def _w_scales_from_layout(raw, E, H, I):
     return g.transpose(0, 1, 4, 3, 2, 5).reshape(E, H, I // 32)
 
 
-def _w_scales_pair_layout(scales, E, H, I):
+def _w_scales_pair_layout(scales, E, H, I):   # H = output features, I = contraction of the GEMM in question
     """[E, H, I/32] -> the second copy of the weight scales, in the tiling of the CTA-pair kernel:
     [E][ceil(H/208)][I/128][2 blocks][h' % 32][(h' % 128) / 32][b % 4] with h' = h % 208; also the mask of written bytes"""
     n_tiles = (H + 207) // 208
@@ -106,6 +106,57 @@ def test_quantisers_and_gemm_against_the_oracle(B, name):
     exact = O.down(h, w, ref["offsets"])
     rel = np.linalg.norm(Hh.to_np64(yp) - exact) / np.linalg.norm(exact)
     assert rel < 0.08
+
+
+def _w_scales_single_layout(scales, E, N, K):
+    """[E, N, K/32] -> [E][N/128][K/128][n % 32][(n % 128) / 32][b % 4] (the first copy of the weight scales)"""
+    g = scales.reshape(E, N // 128, 4, 32, K // 128, 4)          # [e, n/128, (n%128)/32, n%32, b/4, b%4]
+    return g.transpose(0, 1, 4, 3, 2, 5).reshape(-1)
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_down_dgrad_quantisers_and_gemm_against_the_oracle(B, name):
+    """dH_act = Q(dY_perm) . Q(W_down[e])^T with both operands quantised along H, on the same two GEMM kernels."""
+    counts, K, H, I = CASES[name]
+    cfg, host = Hh.ragged_workload(counts, K=K, H=H, I=I, seed=23)
+    ref = O.layer_fwd_bwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"], host["W_down"],
+                          host["dY"])
+    R, E = cfg.R, cfg.E
+    d = B.dims(cfg.T, H, I, E, K)
+    dy = W.round_to_bf16(ref["dY_perm"].astype(np.float32))
+    dy[0, :32] = 0.0
+    dy[R - 1, H - 32:] = np.linspace(-3000.0, 3000.0, 32, dtype=np.float32)
+    dy = W.round_to_bf16(dy)
+    w = host["W_down"].copy()
+    w[0, 0, :32] = 0.0
+    dy_dev, w_dev = Hh.to_dev_bf16(dy), Hh.to_dev_bf16(w)
+    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    dc, ds = u8(R * H), u8(B.moe_mxfp8_dy_scale_bytes(d))
+    wc, ws = u8(E * I * H), u8(B.moe_mxfp8_w_down_dgrad_scale_bytes(d))
+    n_single = E * (I // 128) * (H // 128) * 512
+    assert ds.numel() == (H // 128) * R * 4 and ws.numel() == n_single + E * ((I + 207) // 208) * (H // 128) * 1024
+    B.moe_mxfp8_quantize_dy_perm(d, dy_dev, dc, ds)
+    B.moe_mxfp8_quantize_w_down_dgrad(d, w_dev, wc, ws)
+    torch.cuda.synchronize()
+    o_dc, o_ds, _ = O.mxfp8_quantize(dy)
+    o_wc, o_ws, _ = O.mxfp8_quantize(w)              # [E, I, H]: along H as it lies
+    assert np.array_equal(_act_scales_from_layout(ds.cpu().numpy(), R, H), o_ds)
+    assert np.array_equal(dc.cpu().numpy().reshape(R, H), o_dc)
+    assert np.array_equal(wc.cpu().numpy().reshape(E, I, H), o_wc)
+    ws_host = ws.cpu().numpy()
+    assert np.array_equal(ws_host[:n_single], _w_scales_single_layout(o_ws, E, I, H))
+    want_pair, written = _w_scales_pair_layout(o_ws, E, I, H)
+    assert np.array_equal(ws_host[n_single:][written], want_pair[written])
+    assert np.all(ws_host[n_single:][~written] == 0xAB)
+    dh = torch.full((R, I), float("nan"), dtype=torch.bfloat16, device="cuda")
+    off = torch.from_numpy(ref["offsets"]).cuda()
+    B.moe_grouped_gemm_down_dgrad_mxfp8(d, dc, ds, wc, ws, off, dh)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    Hh.assert_close(Hh.to_np64(dh), O.down_dgrad_mxfp8(dy, w, ref["offsets"]), f"{name}: dH_act (MXFP8)",
+                    rel_fro=Hh.PER_CALL_FROBENIUS)
+    exact = O.down_bwd(dy, np.zeros((R, I)), w, ref["offsets"])[0]
+    assert np.linalg.norm(Hh.to_np64(dh) - exact) / np.linalg.norm(exact) < 0.08
 
 
 def test_shapes_the_block_scaled_path_does_not_take_are_refused(B):
