@@ -386,3 +386,22 @@ def down_dgrad_mxfp8(dY_perm, W_down, offsets):
         if hi > lo:
             out[lo:hi] = a_deq[lo:hi] @ b_deq[e].T
     return out
+
+
+def gateup_dgrad_mxfp8(dGU, W_gate, W_up, offsets):
+    """The data gradient of the gate/up projection with block-scaled FP8 operands along ITS contraction (the 2I gate
+    and up features): dXp[r,:] = Q(dGU[r,:I]) @ Q(Wg[e])^T + Q(dGU[r,I:]) @ Q(Wu[e])^T, where Q quantises dGU row-wise in
+    blocks of 32 along its 2I columns (I is a multiple of 32, so no block straddles the gate/up boundary) and Wg[e],
+    Wu[e] [H,I] row-wise in blocks of 32 along I; the products of the dequantised operands are taken exactly.
+    Returns dXp [R,H] float64."""
+    I = W_gate.shape[2]
+    assert I % MX_BLOCK == 0 and dGU.shape[1] == 2 * I
+    _, _, a_deq = mxfp8_quantize(dGU)
+    _, _, g_deq = mxfp8_quantize(_f64(W_gate))           # [E, H, I]: contraction last as it lies
+    _, _, u_deq = mxfp8_quantize(_f64(W_up))
+    out = np.zeros((a_deq.shape[0], W_gate.shape[1]), dtype=F64)
+    for e in range(W_gate.shape[0]):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        if hi > lo:
+            out[lo:hi] = a_deq[lo:hi, :I] @ g_deq[e].T + a_deq[lo:hi, I:] @ u_deq[e].T
+    return out

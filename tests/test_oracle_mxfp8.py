@@ -134,3 +134,31 @@ def test_down_dgrad_mxfp8_is_the_exact_product_of_the_dequantised_operands():
         lo, hi = offsets[e], offsets[e + 1]
         wrong[lo:hi] = O.mxfp8_quantize(dYp)[2][lo:hi] @ w_alt[e].T
     assert np.abs(wrong - got).max() > 1e-6
+
+
+def test_gateup_dgrad_mxfp8_is_the_exact_product_of_the_dequantised_operands():
+    rng = np.random.default_rng(5)
+    E, I, H = 2, 64, 12
+    counts = [4, 7]
+    offsets = np.concatenate([[0], np.cumsum(counts)])
+    dGU = rng.standard_normal((11, 2 * I)) * np.concatenate([np.full(I, 1.0), np.full(I, 37.0)])   # halves of different size
+    Wg = rng.standard_normal((E, H, I)) * 0.05
+    Wu = rng.standard_normal((E, H, I)) * 0.3
+    got = O.gateup_dgrad_mxfp8(dGU, Wg, Wu, offsets)
+    assert got.shape == (11, H)
+    for r, e in ((0, 0), (3, 0), (4, 1), (10, 1)):
+        ag = O.mxfp8_quantize(dGU[r, :I])[2]
+        au = O.mxfp8_quantize(dGU[r, I:])[2]
+        for h in (0, 5, 11):
+            bg = O.mxfp8_quantize(Wg[e, h, :])[2]
+            bu = O.mxfp8_quantize(Wu[e, h, :])[2]
+            assert abs(got[r, h] - float(ag @ bg + au @ bu)) <= 1e-10
+    # against the unquantised data gradient (the bf16 path's own oracle): a few per cent; equal for representable operands
+    ref = O.gateup_bwd_from_dgu(dGU, np.zeros((11, H)), Wg, Wu, offsets)[0]
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert 0.01 < rel < 0.06
+    dq, gq, uq = O.mxfp8_quantize(dGU)[2], O.mxfp8_quantize(Wg)[2], O.mxfp8_quantize(Wu)[2]
+    assert np.allclose(O.gateup_dgrad_mxfp8(dq, gq, uq, offsets), O.gateup_bwd_from_dgu(dq, np.zeros((11, H)), gq, uq, offsets)[0],
+                       rtol=0, atol=1e-12)
+    # swapping the two weight operands is a different result
+    assert np.abs(O.gateup_dgrad_mxfp8(dGU, Wu, Wg, offsets) - got).max() > 1e-3
