@@ -201,32 +201,19 @@ def make_step(B, b, wl, fused=False):
     return step
 
 
-def time_mxfp8_down(B, cfg, res, device, reps=20, min_seconds=0.3):
-    """The block-scaled FP8 twin of the down projection on this workload's own H_act, weights and offsets: the two
-    quantisers and the GEMM, each timed alone (back to back for at least `min_seconds`, events), beside the bf16 call
-    timed the same way."""
+def time_mxfp8(B, cfg, res, device, reps=20, min_seconds=0.3):
+    """The block-scaled FP8 twins of the three row-ragged GEMMs whose weight operand is (or can be stored)
+    contraction-contiguous -- down forward, down dgrad, gate/up dgrad -- on this workload's own activations, weights and
+    offsets: per GEMM the activation quantiser, the weight quantiser (once per optimizer step in training) and the GEMM,
+    each timed alone (back to back for at least `min_seconds`, events), beside the bf16 call timed the same way."""
     if cfg.H % 128 or cfg.I % 128:
         return None
     b, wl = res["buffers"], res["wl"]
     d = b.d
+    R, E, H, I = cfg.R, cfg.E, cfg.H, cfg.I
     u8 = lambda n: torch.empty(n, dtype=torch.uint8, device=device)
-    hc, hs = u8(cfg.R * cfg.I), u8(B.moe_mxfp8_act_scale_bytes(d))
-    wc, ws = u8(cfg.E * cfg.H * cfg.I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
-    yq = torch.empty_like(b.y_perm)
-    dc, ds = u8(cfg.R * cfg.H), u8(B.moe_mxfp8_dy_scale_bytes(d))
-    vc, vs = u8(cfg.E * cfg.I * cfg.H), u8(B.moe_mxfp8_w_down_dgrad_scale_bytes(d))
-    dhq = torch.empty_like(b.dh_act)
-    dh_ref = b.dh_act.clone()
-    fns = {"bf16_down_ms": lambda: B.moe_grouped_gemm_down(d, b.h_act, wl["W_down"], b.offsets, b.y_perm),
-           "quantize_h_act_ms": lambda: B.moe_mxfp8_quantize_h_act(d, b.h_act, hc, hs),
-           "quantize_w_down_ms": lambda: B.moe_mxfp8_quantize_w_down(d, wl["W_down"], wc, ws),
-           "mxfp8_down_ms": lambda: B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, b.offsets, yq),
-           "bf16_down_dgrad_ms": lambda: B.moe_grouped_gemm_down_dgrad(d, b.dy_perm, wl["W_down"], b.offsets, dh_ref),
-           "quantize_dy_perm_ms": lambda: B.moe_mxfp8_quantize_dy_perm(d, b.dy_perm, dc, ds),
-           "quantize_w_down_dgrad_ms": lambda: B.moe_mxfp8_quantize_w_down_dgrad(d, wl["W_down"], vc, vs),
-           "mxfp8_down_dgrad_ms": lambda: B.moe_grouped_gemm_down_dgrad_mxfp8(d, dc, ds, vc, vs, b.offsets, dhq)}
-    out = {}
-    for name, fn in fns.items():
+
+    def timed(fn):
         for _ in range(3):
             fn()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -240,17 +227,45 @@ def time_mxfp8_down(B, cfg, res, device, reps=20, min_seconds=0.3):
             fn()
         e1.record()
         torch.cuda.synchronize()
-        out[name] = e0.elapsed_time(e1) / n
-    fl = 2.0 * cfg.R * cfg.H * cfg.I
-    out["bf16_down_tflops"] = fl / (out["bf16_down_ms"] * 1e-3) / 1e12
-    out["mxfp8_down_tflops"] = fl / (out["mxfp8_down_ms"] * 1e-3) / 1e12
-    out["bf16_down_dgrad_tflops"] = fl / (out["bf16_down_dgrad_ms"] * 1e-3) / 1e12
-    out["mxfp8_down_dgrad_tflops"] = fl / (out["mxfp8_down_dgrad_ms"] * 1e-3) / 1e12
-    out["rel_frobenius_to_bf16_result"] = float((yq.float() - b.y_perm.float()).norm() / b.y_perm.float().norm())
-    out["dgrad_rel_frobenius_to_bf16_result"] = float((dhq.float() - dh_ref.float()).norm() / dh_ref.float().norm())
+        return e0.elapsed_time(e1) / n
+
+    def leg(flops, bf16_fn, q_act, q_w, fp8_fn, got, want):
+        o = {"bf16_ms": timed(bf16_fn), "quantize_act_ms": timed(q_act), "quantize_w_ms": timed(q_w), "fp8_ms": timed(fp8_fn)}
+        o["bf16_tflops"] = flops / (o["bf16_ms"] * 1e-3) / 1e12
+        o["fp8_tflops"] = flops / (o["fp8_ms"] * 1e-3) / 1e12
+        o["rel_frobenius_to_bf16_result"] = float((got.float() - want.float()).norm() / want.float().norm())
+        return o
+
+    out = {}
+    hc, hs = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    wc, ws = u8(E * H * I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
+    yq = torch.empty_like(b.y_perm)
+    out["down"] = leg(2.0 * R * H * I,
+                      lambda: B.moe_grouped_gemm_down(d, b.h_act, wl["W_down"], b.offsets, b.y_perm),
+                      lambda: B.moe_mxfp8_quantize_h_act(d, b.h_act, hc, hs),
+                      lambda: B.moe_mxfp8_quantize_w_down(d, wl["W_down"], wc, ws),
+                      lambda: B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, b.offsets, yq), yq, b.y_perm)
+    del hc, hs, wc, ws, yq
+    dc, ds = u8(R * H), u8(B.moe_mxfp8_dy_scale_bytes(d))
+    vc, vs = u8(E * I * H), u8(B.moe_mxfp8_w_down_dgrad_scale_bytes(d))
+    dhq, dh_ref = torch.empty_like(b.dh_act), torch.empty_like(b.dh_act)
+    out["down_dgrad"] = leg(2.0 * R * H * I,
+                            lambda: B.moe_grouped_gemm_down_dgrad(d, b.dy_perm, wl["W_down"], b.offsets, dh_ref),
+                            lambda: B.moe_mxfp8_quantize_dy_perm(d, b.dy_perm, dc, ds),
+                            lambda: B.moe_mxfp8_quantize_w_down_dgrad(d, wl["W_down"], vc, vs),
+                            lambda: B.moe_grouped_gemm_down_dgrad_mxfp8(d, dc, ds, vc, vs, b.offsets, dhq), dhq, dh_ref)
+    del dc, ds, vc, vs, dhq, dh_ref
+    gc, gs = u8(R * 2 * I), u8(B.moe_mxfp8_dgu_scale_bytes(d))
+    uc, us = u8(E * H * 2 * I), u8(B.moe_mxfp8_w_gateup_dgrad_scale_bytes(d))
+    dxq, dx_ref = torch.empty_like(b.dx_perm), torch.empty_like(b.dx_perm)
+    out["gateup_dgrad"] = leg(4.0 * R * H * I,
+                              lambda: B.moe_grouped_gemm_gateup_dgrad(d, b.dgu, wl["W_gate"], wl["W_up"], b.offsets, dx_ref),
+                              lambda: B.moe_mxfp8_quantize_dgu(d, b.dgu, gc, gs),
+                              lambda: B.moe_mxfp8_quantize_w_gateup_dgrad(d, wl["W_gate"], wl["W_up"], uc, us),
+                              lambda: B.moe_grouped_gemm_gateup_dgrad_mxfp8(d, gc, gs, uc, us, b.offsets, dxq), dxq, dx_ref)
     out["note"] = ("E4M3 elements, E8M0 scale per 32 along the contraction; tcgen05.mma kind::mxf8f6f4.block_scale on "
                    "256 x 208 CTA-pair tiles from 256 rows per expert on average, 128 x 128 single-CTA tiles below; "
-                   "the bf16 twin runs 256 x 256 CTA-pair tiles")
+                   "the bf16 twins run 256 x 256 CTA-pair tiles")
     if B.moe_device_status() != 0:
         raise RuntimeError("device status word is set after the MXFP8 calls")
     return out
@@ -705,7 +720,7 @@ def run_ours(args):
         out = {"workload": cfg.name, "steps": res["steps"], "ms_per_step": res["total_ms"] / res["steps"],
                "per_call_ms": {k: round(v, 5) for k, v in res["per_call_ms"].items()}}
         if args.with_mxfp8:
-            out["mxfp8_down"] = time_mxfp8_down(B, cfg, res, device, reps=2, min_seconds=0.0)
+            out["mxfp8"] = time_mxfp8(B, cfg, res, device, reps=2, min_seconds=0.0)
         print(json.dumps(out), flush=True)
         return
     res = time_config(B, cfg, device, args.steps, args.warmup, dist, min_seconds=args.min_seconds)
@@ -757,7 +772,7 @@ def run_ours(args):
         line["sustained"]["frac"] = fractions(line["sustained"]["value"], peaks)
         line["stream_calibration_in_step"] = stream_calibration_in_step(B, cfg, res, device)
         line["fused_dgrad_swiglu_bwd"] = time_fused_variant(B, cfg, res, device)
-        line["mxfp8_down"] = time_mxfp8_down(B, cfg, res, device)
+        line["mxfp8"] = time_mxfp8(B, cfg, res, device)
         del res
         torch.cuda.empty_cache()
         for name in args.also:
@@ -767,7 +782,7 @@ def run_ours(args):
             r2 = time_config(B, c2, device, 3, 3, None, sample_clocks=True, min_seconds=args.other_min_seconds)
             extra.append(summarize(c2, r2, peaks, peaks_kind, sms))
             extra[-1]["fused_dgrad_swiglu_bwd"] = time_fused_variant(B, c2, r2, device, seconds=0.5)
-            extra[-1]["mxfp8_down"] = time_mxfp8_down(B, c2, r2, device)
+            extra[-1]["mxfp8"] = time_mxfp8(B, c2, r2, device)
             del r2
             torch.cuda.empty_cache()
         if extra:

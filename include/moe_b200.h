@@ -274,6 +274,25 @@ int moe_grouped_gemm_down_dgrad_mxfp8(const moe_dims_t* dims, const void* dy_cod
                                       const void* w_codes, const void* w_scales, const int32_t* offsets,
                                       void* dh_act, moe_stream_t stream);
 
+/* The data gradient of the gate/up projection likewise: dx_perm[r,:] = dequant(dgu row r) . dequant([w_gate[e] |
+ * w_up[e]])^T, contraction over the 2I gate and up features (blocks of 32 never straddle the boundary: I is a
+ * multiple of 128).  w_gate, w_up [E,H,I] are contraction-contiguous as they lie; their codes go side by side:
+ *   moe_mxfp8_quantize_dgu             dgu [R,2I] bf16 -> codes [R,2I] bytes; scales: moe_mxfp8_dgu_scale_bytes(dims)
+ *                                      bytes laid out [2I/128][R][4].
+ *   moe_mxfp8_quantize_w_gateup_dgrad  w_gate, w_up -> codes [E,H,2I] bytes (gate columns first); scales:
+ *                                      moe_mxfp8_w_gateup_dgrad_scale_bytes(dims) bytes, the two tilings with
+ *                                      feature = h and 128-wide slices along the 2I columns.
+ *   moe_grouped_gemm_gateup_dgrad_mxfp8  dx_perm [R,H] bf16, overwritten.
+ * Same requirements, status codes and tolerance statement as the forward call. */
+size_t moe_mxfp8_dgu_scale_bytes(const moe_dims_t* dims);
+size_t moe_mxfp8_w_gateup_dgrad_scale_bytes(const moe_dims_t* dims);
+int moe_mxfp8_quantize_dgu(const moe_dims_t* dims, const void* dgu, void* codes, void* scales, moe_stream_t stream);
+int moe_mxfp8_quantize_w_gateup_dgrad(const moe_dims_t* dims, const void* w_gate, const void* w_up, void* codes,
+                                      void* scales, moe_stream_t stream);
+int moe_grouped_gemm_gateup_dgrad_mxfp8(const moe_dims_t* dims, const void* dgu_codes, const void* dgu_scales,
+                                        const void* w_codes, const void* w_scales, const int32_t* offsets,
+                                        void* dx_perm, moe_stream_t stream);
+
 /* ---- whole layer from HOST activations ------------------------------------------------------
  * One training step of the layer for a caller whose per-step tensors live in host memory:
  * copies x, topk_idx, topk_w, dy (HOST pointers; pinned memory makes the copies asynchronous)

@@ -27,6 +27,8 @@ EXPORTS = [
     "moe_grouped_gemm_down_mxfp8",
     "moe_mxfp8_dy_scale_bytes", "moe_mxfp8_w_down_dgrad_scale_bytes", "moe_mxfp8_quantize_dy_perm",
     "moe_mxfp8_quantize_w_down_dgrad", "moe_grouped_gemm_down_dgrad_mxfp8",
+    "moe_mxfp8_dgu_scale_bytes", "moe_mxfp8_w_gateup_dgrad_scale_bytes", "moe_mxfp8_quantize_dgu",
+    "moe_mxfp8_quantize_w_gateup_dgrad", "moe_grouped_gemm_gateup_dgrad_mxfp8",
 ]
 
 
@@ -58,7 +60,8 @@ def load_library() -> ctypes.CDLL:
         lib.moe_layer_arena_bytes.restype = ctypes.c_size_t
         lib.moe_layer_arena_bytes.argtypes = [ctypes.POINTER(MoeDims)]
         for name in ("moe_mxfp8_act_scale_bytes", "moe_mxfp8_w_down_scale_bytes", "moe_mxfp8_dy_scale_bytes",
-                     "moe_mxfp8_w_down_dgrad_scale_bytes"):
+                     "moe_mxfp8_w_down_dgrad_scale_bytes", "moe_mxfp8_dgu_scale_bytes",
+                     "moe_mxfp8_w_gateup_dgrad_scale_bytes"):
             getattr(lib, name).restype = ctypes.c_size_t
             getattr(lib, name).argtypes = [ctypes.POINTER(MoeDims)]
         lib.moe_device_status.restype = ctypes.c_int
@@ -90,6 +93,9 @@ def load_library() -> ctypes.CDLL:
             "moe_mxfp8_quantize_dy_perm": [dp, p, p, p, p],
             "moe_mxfp8_quantize_w_down_dgrad": [dp, p, p, p, p],
             "moe_grouped_gemm_down_dgrad_mxfp8": [dp, p, p, p, p, p, p, p],
+            "moe_mxfp8_quantize_dgu": [dp, p, p, p, p],
+            "moe_mxfp8_quantize_w_gateup_dgrad": [dp, p, p, p, p, p],
+            "moe_grouped_gemm_gateup_dgrad_mxfp8": [dp, p, p, p, p, p, p, p],
         }
         for name, argtypes in sigs.items():
             fn = getattr(lib, name)
@@ -265,6 +271,27 @@ def moe_mxfp8_quantize_w_down_dgrad(d, w_down, codes, scales):
 def moe_grouped_gemm_down_dgrad_mxfp8(d, dy_codes, dy_scales, w_codes, w_scales, offsets, dh_act):
     _call("moe_grouped_gemm_down_dgrad_mxfp8", ctypes.byref(d), _ptr(dy_codes), _ptr(dy_scales), _ptr(w_codes), _ptr(w_scales),
           _ptr(offsets), _ptr(dh_act), _stream())
+
+
+def moe_mxfp8_dgu_scale_bytes(d: MoeDims) -> int:
+    return int(load_library().moe_mxfp8_dgu_scale_bytes(ctypes.byref(d)))
+
+
+def moe_mxfp8_w_gateup_dgrad_scale_bytes(d: MoeDims) -> int:
+    return int(load_library().moe_mxfp8_w_gateup_dgrad_scale_bytes(ctypes.byref(d)))
+
+
+def moe_mxfp8_quantize_dgu(d, dgu, codes, scales):
+    _call("moe_mxfp8_quantize_dgu", ctypes.byref(d), _ptr(dgu), _ptr(codes), _ptr(scales), _stream())
+
+
+def moe_mxfp8_quantize_w_gateup_dgrad(d, w_gate, w_up, codes, scales):
+    _call("moe_mxfp8_quantize_w_gateup_dgrad", ctypes.byref(d), _ptr(w_gate), _ptr(w_up), _ptr(codes), _ptr(scales), _stream())
+
+
+def moe_grouped_gemm_gateup_dgrad_mxfp8(d, dgu_codes, dgu_scales, w_codes, w_scales, offsets, dx_perm):
+    _call("moe_grouped_gemm_gateup_dgrad_mxfp8", ctypes.byref(d), _ptr(dgu_codes), _ptr(dgu_scales), _ptr(w_codes),
+          _ptr(w_scales), _ptr(offsets), _ptr(dx_perm), _stream())
 
 
 def moe_layer_fwd_bwd_host(d, x_host, topk_idx_host, topk_w_host, dy_host, w_gate, w_up, w_down, y_host, dx_host,

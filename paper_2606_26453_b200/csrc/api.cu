@@ -331,7 +331,7 @@ int moe_mxfp8_quantize_w_down_dgrad(const moe_dims_t* dims, const void* w_down, 
     const void* const opt[] = {nullptr};
     s = check_ptrs(req, opt);
     if (s != MOE_OK) return s;
-    return launch_mx_quantize_w_rows(dims->E, dims->I, dims->H, cb(w_down), static_cast<uint8_t*>(codes),
+    return launch_mx_quantize_w_rows(dims->E, dims->I, dims->H, dims->H, 0, cb(w_down), static_cast<uint8_t*>(codes),
                                      static_cast<uint8_t*>(scales), st(stream));
 }
 
@@ -346,6 +346,56 @@ int moe_grouped_gemm_down_dgrad_mxfp8(const moe_dims_t* dims, const void* dy_cod
     return launch_mx_gemm((long long)dims->T * dims->K, dims->E, dims->I, dims->H, static_cast<const uint8_t*>(dy_codes),
                           static_cast<const uint8_t*>(dy_scales), static_cast<const uint8_t*>(w_codes),
                           static_cast<const uint8_t*>(w_scales), offsets, mb(dh_act), st(stream));
+}
+
+// ---- block-scaled FP8 data gradient of the gate/up projection (contraction over the 2I gate and up features) ----
+size_t moe_mxfp8_dgu_scale_bytes(const moe_dims_t* dims) {
+    if (check_mx_dims(dims) != MOE_OK) return 0;
+    return (size_t)(2 * dims->I / 128) * (size_t)dims->T * dims->K * 4;
+}
+
+size_t moe_mxfp8_w_gateup_dgrad_scale_bytes(const moe_dims_t* dims) {
+    if (check_mx_dims(dims) != MOE_OK) return 0;
+    return mx_w_scale_bytes(dims->E, dims->H, 2 * dims->I);
+}
+
+int moe_mxfp8_quantize_dgu(const moe_dims_t* dims, const void* dgu, void* codes, void* scales, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {dgu, codes, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_rows((long long)dims->T * dims->K, 2 * dims->I, cb(dgu), static_cast<uint8_t*>(codes),
+                                   static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_mxfp8_quantize_w_gateup_dgrad(const moe_dims_t* dims, const void* w_gate, const void* w_up, void* codes, void* scales,
+                                      moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {w_gate, w_up, codes, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    s = launch_mx_quantize_w_rows(dims->E, dims->H, dims->I, 2 * dims->I, 0, cb(w_gate), static_cast<uint8_t*>(codes),
+                                  static_cast<uint8_t*>(scales), st(stream));
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_w_rows(dims->E, dims->H, dims->I, 2 * dims->I, dims->I, cb(w_up), static_cast<uint8_t*>(codes),
+                                     static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_grouped_gemm_gateup_dgrad_mxfp8(const moe_dims_t* dims, const void* dgu_codes, const void* dgu_scales, const void* w_codes,
+                                        const void* w_scales, const int32_t* offsets, void* dx_perm, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {dgu_codes, dgu_scales, w_codes, w_scales, offsets, dx_perm};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_gemm((long long)dims->T * dims->K, dims->E, dims->H, 2 * dims->I, static_cast<const uint8_t*>(dgu_codes),
+                          static_cast<const uint8_t*>(dgu_scales), static_cast<const uint8_t*>(w_codes),
+                          static_cast<const uint8_t*>(w_scales), offsets, mb(dx_perm), st(stream));
 }
 
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).

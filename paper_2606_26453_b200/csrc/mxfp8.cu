@@ -758,11 +758,14 @@ __device__ __forceinline__ uint32_t mx_e4m3(float v) {
 // through two shuffles; two such loads are in flight per lane.  The 4 scale bytes of a (row, slice) are one 32-bit word:
 //   WEIGHTS = false (activations): word [slice][row];
 //   WEIGHTS = true  (weights whose contraction axis is contiguous, rows = E * n_feat, e.g. W_down read as [I, H] for the
-//                    data gradient): the word's place in each of the two weight-scale tilings.
+//                    data gradient): the word's place in each of the two weight-scale tilings.  The output may be a
+//                    column range of a wider operand (out_k_tiles slices per row, this input filling slices
+//                    out_kt0 .. out_kt0 + n/128): W_gate and W_up side by side along the contraction of the gate/up
+//                    data gradient.
 template <bool WEIGHTS>
 __global__ void __launch_bounds__(256) mx_quantize_rows_kernel(const uint4* __restrict__ x, long long rows, int n, int n_feat,
-                                                               uint2* __restrict__ codes, uint8_t* __restrict__ scales,
-                                                               uint8_t* __restrict__ scales_pair) {
+                                                               int out_k_tiles, int out_kt0, uint2* __restrict__ codes,
+                                                               uint8_t* __restrict__ scales, uint8_t* __restrict__ scales_pair) {
     constexpr int U = 2;
     const int lane = threadIdx.x & 31;
     const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -798,22 +801,22 @@ __global__ void __launch_bounds__(256) mx_quantize_rows_kernel(const uint4* __re
             uint2 out;
             out.x = mx_e4m3x2(v[0] * inv, v[1] * inv) | (mx_e4m3x2(v[2] * inv, v[3] * inv) << 16);
             out.y = mx_e4m3x2(v[4] * inv, v[5] * inv) | (mx_e4m3x2(v[6] * inv, v[7] * inv) << 16);
-            if (u < total) codes[(p0 + i) * 32 + lane] = out;
+            const long long r = u / k_tiles;
+            const int kt = (int)(u - r * k_tiles) + out_kt0;
+            if (u < total) codes[(r * out_k_tiles + kt) * 16 + (lane & 15)] = out;
             const uint32_t sbyte = (uint32_t)(se + 127);
             const int base = lane & 16;                       // first lane of this half-warp
             const uint32_t word = __shfl_sync(0xffffffffu, sbyte, base) | (__shfl_sync(0xffffffffu, sbyte, base + 4) << 8) |
                                   (__shfl_sync(0xffffffffu, sbyte, base + 8) << 16) | (__shfl_sync(0xffffffffu, sbyte, base + 12) << 24);
             if ((lane & 15) == 0 && u < total) {
-                const long long r = u / k_tiles;
-                const int kt = (int)(u - r * k_tiles);
                 if (!WEIGHTS) {
                     reinterpret_cast<uint32_t*>(scales)[(long long)kt * rows + r] = word;
                 } else {
                     const int e = (int)(r / n_feat), f = (int)(r - (long long)e * n_feat);
-                    *reinterpret_cast<uint32_t*>(scales + (((long long)e * (n_feat / 128) + f / 128) * k_tiles + kt) * 512 +
+                    *reinterpret_cast<uint32_t*>(scales + (((long long)e * (n_feat / 128) + f / 128) * out_k_tiles + kt) * 512 +
                                                  (f % 32) * 16 + ((f % 128) / 32) * 4) = word;
                     const int nt = f / MXP_NT, c = f % MXP_NT;
-                    *reinterpret_cast<uint32_t*>(scales_pair + (((long long)e * n_tiles_p + nt) * k_tiles + kt) * 1024 +
+                    *reinterpret_cast<uint32_t*>(scales_pair + (((long long)e * n_tiles_p + nt) * out_k_tiles + kt) * 1024 +
                                                  (c >> 7) * 512 + (c % 32) * 16 + ((c % 128) / 32) * 4) = word;
                 }
             }
@@ -880,7 +883,7 @@ static unsigned mx_row_quantiser_blocks(long long units) {
 
 int launch_mx_quantize_rows(long long rows, int n, const bf16* x, uint8_t* codes, uint8_t* scales, cudaStream_t s) {
     mx_quantize_rows_kernel<false><<<mx_row_quantiser_blocks(rows * (n / 128)), 256, 0, s>>>(
-        reinterpret_cast<const uint4*>(x), rows, n, 0, reinterpret_cast<uint2*>(codes), scales, nullptr);
+        reinterpret_cast<const uint4*>(x), rows, n, 0, n / 128, 0, reinterpret_cast<uint2*>(codes), scales, nullptr);
     return check_launch();
 }
 
@@ -891,11 +894,13 @@ int launch_mx_quantize_w_down(const moe_dims_t& d, const bf16* w_down, uint8_t* 
     return check_launch();
 }
 
-int launch_mx_quantize_w_rows(int E, int n_feat, int k, const bf16* w, uint8_t* codes, uint8_t* scales, cudaStream_t s) {
+// w [E * n_feat, k] -> columns [k_off, k_off + k) of the codes [E * n_feat, k_total] and the matching scale slices
+int launch_mx_quantize_w_rows(int E, int n_feat, int k, int k_total, int k_off, const bf16* w, uint8_t* codes, uint8_t* scales,
+                              cudaStream_t s) {
     const long long rows = (long long)E * n_feat;
     mx_quantize_rows_kernel<true><<<mx_row_quantiser_blocks(rows * (k / 128)), 256, 0, s>>>(
-        reinterpret_cast<const uint4*>(w), rows, k, n_feat, reinterpret_cast<uint2*>(codes), scales,
-        scales + mx_w_scale_single_bytes(E, n_feat, k));
+        reinterpret_cast<const uint4*>(w), rows, k, n_feat, k_total / 128, k_off / 128, reinterpret_cast<uint2*>(codes), scales,
+        scales + mx_w_scale_single_bytes(E, n_feat, k_total));
     return check_launch();
 }
 

@@ -159,6 +159,51 @@ def test_down_dgrad_quantisers_and_gemm_against_the_oracle(B, name):
     assert np.linalg.norm(Hh.to_np64(dh) - exact) / np.linalg.norm(exact) < 0.08
 
 
+@pytest.mark.parametrize("name", list(CASES))
+def test_gateup_dgrad_quantisers_and_gemm_against_the_oracle(B, name):
+    """dX_perm = Q(dGU) . Q([W_gate[e] | W_up[e]])^T, contraction over the 2I gate and up features."""
+    counts, K, H, I = CASES[name]
+    cfg, host = Hh.ragged_workload(counts, K=K, H=H, I=I, seed=25)
+    ref = O.layer_fwd_bwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"], host["W_down"],
+                          host["dY"])
+    R, E = cfg.R, cfg.E
+    d = B.dims(cfg.T, H, I, E, K)
+    dgu = W.round_to_bf16(ref["dGU"].astype(np.float32))
+    dgu[0, I - 32:I + 32] = 0.0                      # all-zero blocks on both sides of the gate/up boundary
+    dgu[R - 1, :32] = np.linspace(-9.0, 9.0, 32, dtype=np.float32)
+    dgu = W.round_to_bf16(dgu)
+    wg, wu = host["W_gate"].copy(), host["W_up"].copy() * 3.0
+    wu = W.round_to_bf16(wu)
+    dgu_dev, wg_dev, wu_dev = Hh.to_dev_bf16(dgu), Hh.to_dev_bf16(wg), Hh.to_dev_bf16(wu)
+    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    gc, gs = u8(R * 2 * I), u8(B.moe_mxfp8_dgu_scale_bytes(d))
+    wc, ws = u8(E * H * 2 * I), u8(B.moe_mxfp8_w_gateup_dgrad_scale_bytes(d))
+    n_single = E * (H // 128) * (2 * I // 128) * 512
+    assert gs.numel() == (2 * I // 128) * R * 4 and ws.numel() == n_single + E * ((H + 207) // 208) * (2 * I // 128) * 1024
+    B.moe_mxfp8_quantize_dgu(d, dgu_dev, gc, gs)
+    B.moe_mxfp8_quantize_w_gateup_dgrad(d, wg_dev, wu_dev, wc, ws)
+    torch.cuda.synchronize()
+    o_gc, o_gs, _ = O.mxfp8_quantize(dgu)
+    o_wc, o_ws, _ = O.mxfp8_quantize(np.concatenate([wg, wu], axis=2))     # [E, H, 2I]: blocks never straddle I
+    assert np.array_equal(_act_scales_from_layout(gs.cpu().numpy(), R, 2 * I), o_gs)
+    assert np.array_equal(gc.cpu().numpy().reshape(R, 2 * I), o_gc)
+    assert np.array_equal(wc.cpu().numpy().reshape(E, H, 2 * I), o_wc)
+    ws_host = ws.cpu().numpy()
+    assert np.array_equal(ws_host[:n_single], _w_scales_single_layout(o_ws, E, H, 2 * I))
+    want_pair, written = _w_scales_pair_layout(o_ws, E, H, 2 * I)
+    assert np.array_equal(ws_host[n_single:][written], want_pair[written])
+    assert np.all(ws_host[n_single:][~written] == 0xAB)
+    dx = torch.full((R, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    off = torch.from_numpy(ref["offsets"]).cuda()
+    B.moe_grouped_gemm_gateup_dgrad_mxfp8(d, gc, gs, wc, ws, off, dx)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    Hh.assert_close(Hh.to_np64(dx), O.gateup_dgrad_mxfp8(dgu, wg, wu, ref["offsets"]), f"{name}: dX_perm (MXFP8)",
+                    rel_fro=Hh.PER_CALL_FROBENIUS)
+    exact = O.gateup_bwd_from_dgu(dgu, np.zeros((R, H)), wg, wu, ref["offsets"])[0]
+    assert np.linalg.norm(Hh.to_np64(dx) - exact) / np.linalg.norm(exact) < 0.08
+
+
 def test_shapes_the_block_scaled_path_does_not_take_are_refused(B):
     d = B.dims(64, 192, 128, 2, 1)                   # H not a multiple of 128
     assert B.moe_mxfp8_act_scale_bytes(d) == 0
