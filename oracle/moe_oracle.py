@@ -405,3 +405,22 @@ def gateup_dgrad_mxfp8(dGU, W_gate, W_up, offsets):
         if hi > lo:
             out[lo:hi] = a_deq[lo:hi, :I] @ g_deq[e].T + a_deq[lo:hi, I:] @ u_deq[e].T
     return out
+
+
+def gateup_mxfp8(X_perm, W_gate, W_up, offsets):
+    """The gate/up projection with block-scaled FP8 operands along its contraction (H): g = Q(Xp[r,:]) @ Q(Wg[e]),
+    u = Q(Xp[r,:]) @ Q(Wu[e]), where Q quantises Xp row-wise in blocks of 32 along H and each weight column
+    Wg[e][:,i], Wu[e][:,i] in blocks of 32 along H (every gate / up feature has its own scales); the products of the
+    dequantised operands are taken exactly.  Returns the pre-activations GU [R,2I] = [g | u] float64."""
+    _, _, a_deq = mxfp8_quantize(X_perm)
+    g_deq = np.swapaxes(mxfp8_quantize(np.swapaxes(_f64(W_gate), 1, 2))[2], 1, 2)      # quantised along H, back to [E,H,I]
+    u_deq = np.swapaxes(mxfp8_quantize(np.swapaxes(_f64(W_up), 1, 2))[2], 1, 2)
+    return gateup_swiglu(a_deq, g_deq, u_deq, offsets)[1]
+
+
+def swiglu_fwd(GU):
+    """Hact = silu(g) * u with [g | u] = GU, silu(g) = g / (1 + exp(-g)).  Returns Hact [R,I] float64."""
+    GU = _f64(GU)
+    I = GU.shape[1] // 2
+    g, u = GU[:, :I], GU[:, I:]
+    return g / (1.0 + np.exp(-g)) * u

@@ -162,3 +162,33 @@ def test_gateup_dgrad_mxfp8_is_the_exact_product_of_the_dequantised_operands():
                        rtol=0, atol=1e-12)
     # swapping the two weight operands is a different result
     assert np.abs(O.gateup_dgrad_mxfp8(dGU, Wu, Wg, offsets) - got).max() > 1e-3
+
+
+def test_gateup_mxfp8_is_the_exact_product_of_the_dequantised_operands_and_swiglu_fwd_its_activation():
+    rng = np.random.default_rng(6)
+    E, I, H = 2, 10, 96
+    counts = [5, 8]
+    offsets = np.concatenate([[0], np.cumsum(counts)])
+    Xp = rng.standard_normal((13, H))
+    Wg = rng.standard_normal((E, H, I)) * 0.05
+    Wu = rng.standard_normal((E, H, I)) * 0.4
+    got = O.gateup_mxfp8(Xp, Wg, Wu, offsets)
+    assert got.shape == (13, 2 * I)
+    for r, e in ((0, 0), (4, 0), (5, 1), (12, 1)):
+        a = O.mxfp8_quantize(Xp[r])[2]
+        for i in (0, 3, 9):
+            assert abs(got[r, i] - float(a @ O.mxfp8_quantize(Wg[e, :, i])[2])) <= 1e-12        # gate column's own scales along H
+            assert abs(got[r, I + i] - float(a @ O.mxfp8_quantize(Wu[e, :, i])[2])) <= 1e-12
+    # against the unquantised projection: a few per cent; equal for representable operands
+    h_ref, gu_ref = O.gateup_swiglu(Xp, Wg, Wu, offsets)
+    rel = np.linalg.norm(got - gu_ref) / np.linalg.norm(gu_ref)
+    assert 0.01 < rel < 0.06
+    xq = O.mxfp8_quantize(Xp)[2]
+    gq = np.swapaxes(O.mxfp8_quantize(np.swapaxes(Wg, 1, 2))[2], 1, 2)
+    uq = np.swapaxes(O.mxfp8_quantize(np.swapaxes(Wu, 1, 2))[2], 1, 2)
+    assert np.array_equal(O.gateup_mxfp8(xq, gq, uq, offsets), O.gateup_swiglu(xq, gq, uq, offsets)[1])
+    # the activation of given pre-activations: the pinned forward's own H_act, and closed forms
+    assert np.array_equal(O.swiglu_fwd(gu_ref), h_ref)
+    assert np.allclose(O.swiglu_fwd(np.array([[0.0, 2.0, -2.0, 5.0, 7.0, 7.0]])), [[0.0, 2.0 / (1 + np.exp(-2.0)) * 7.0, -2.0 / (1 + np.exp(2.0)) * 7.0]])
+    t = torch.tensor(gu_ref)
+    assert np.allclose(O.swiglu_fwd(gu_ref), (torch.nn.functional.silu(t[:, :I]) * t[:, I:]).numpy(), rtol=1e-12, atol=1e-14)
