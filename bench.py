@@ -202,9 +202,8 @@ def make_step(B, b, wl, fused=False):
 
 
 def time_mxfp8(B, cfg, res, device, reps=20, min_seconds=0.3):
-    """The block-scaled FP8 twins of the three row-ragged GEMMs whose weight operand is (or can be stored)
-    contraction-contiguous -- down forward, down dgrad, gate/up dgrad -- on this workload's own activations, weights and
-    offsets: per GEMM the activation quantiser, the weight quantiser (once per optimizer step in training) and the GEMM,
+    """The block-scaled FP8 twins of the four row-ragged GEMMs -- down forward, down dgrad, gate/up dgrad, gate/up
+    forward (with its activation call) -- on this workload's own activations, weights and offsets: per GEMM the activation quantiser, the weight quantiser (once per optimizer step in training) and the GEMM,
     each timed alone (back to back for at least `min_seconds`, events), beside the bf16 call timed the same way."""
     if cfg.H % 128 or cfg.I % 128:
         return None
@@ -263,9 +262,27 @@ def time_mxfp8(B, cfg, res, device, reps=20, min_seconds=0.3):
                               lambda: B.moe_mxfp8_quantize_dgu(d, b.dgu, gc, gs),
                               lambda: B.moe_mxfp8_quantize_w_gateup_dgrad(d, wl["W_gate"], wl["W_up"], uc, us),
                               lambda: B.moe_grouped_gemm_gateup_dgrad_mxfp8(d, gc, gs, uc, us, b.offsets, dxq), dxq, dx_ref)
+    del gc, gs, uc, us, dxq, dx_ref
+    xc, xs = u8(R * H), u8(B.moe_mxfp8_x_scale_bytes(d))
+    tc, ts = u8(E * 2 * I * H), u8(B.moe_mxfp8_w_gateup_scale_bytes(d))
+    hc, hs = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    guq, hq, h_ref, gu_ref = torch.empty_like(b.gu), torch.empty_like(b.h_act), torch.empty_like(b.h_act), torch.empty_like(b.gu)
+
+    def gateup_fp8():   # the GEMM and the activation (which also emits the FP8 form the down projection reads)
+        B.moe_grouped_gemm_gateup_mxfp8(d, xc, xs, tc, ts, b.offsets, guq)
+        B.moe_swiglu_mxfp8(d, guq, hq, hc, hs)
+
+    out["gateup_swiglu"] = leg(4.0 * R * H * I,
+                               lambda: B.moe_grouped_gemm_gateup_swiglu(d, b.x_perm, wl["W_gate"], wl["W_up"], b.offsets, h_ref, gu_ref),
+                               lambda: B.moe_mxfp8_quantize_x_perm(d, b.x_perm, xc, xs),
+                               lambda: B.moe_mxfp8_quantize_w_gateup(d, wl["W_gate"], wl["W_up"], tc, ts),
+                               gateup_fp8, hq, h_ref)
+    out["gateup_swiglu"]["fp8_gemm_ms"] = timed(lambda: B.moe_grouped_gemm_gateup_mxfp8(d, xc, xs, tc, ts, b.offsets, guq))
+    out["gateup_swiglu"]["swiglu_and_quantize_ms"] = timed(lambda: B.moe_swiglu_mxfp8(d, guq, hq, hc, hs))
     out["note"] = ("E4M3 elements, E8M0 scale per 32 along the contraction; tcgen05.mma kind::mxf8f6f4.block_scale on "
                    "256 x 208 CTA-pair tiles from 256 rows per expert on average, 128 x 128 single-CTA tiles below; "
-                   "the bf16 twins run 256 x 256 CTA-pair tiles")
+                   "the bf16 twins run 256 x 256 CTA-pair tiles; the FP8 gate/up time is the GEMM plus the activation call, "
+                   "which also writes the FP8 form of H_act (so the down projection's quantize_act_ms is not paid in a chain)")
     if B.moe_device_status() != 0:
         raise RuntimeError("device status word is set after the MXFP8 calls")
     return out

@@ -293,6 +293,30 @@ int moe_grouped_gemm_gateup_dgrad_mxfp8(const moe_dims_t* dims, const void* dgu_
                                         const void* w_codes, const void* w_scales, const int32_t* offsets,
                                         void* dx_perm, moe_stream_t stream);
 
+/* The gate/up projection itself: gu[r,:] = [ dequant(x row r) . dequant(w_gate[e]) | dequant(x row r) . dequant(w_up[e]) ],
+ * contraction over H; every gate / up feature has its own scales along H.  The SwiGLU activation is a second call that
+ * also emits the block-scaled FP8 form of its result, so that the FP8 down projection needs no separate quantiser:
+ *   moe_mxfp8_quantize_x_perm    x_perm [R,H] bf16 -> codes [R,H] bytes; scales: moe_mxfp8_x_scale_bytes(dims) bytes,
+ *                                [H/128][R][4].
+ *   moe_mxfp8_quantize_w_gateup  w_gate, w_up [E,H,I] -> codes_t [E,2I,H] bytes (transposed: contraction contiguous;
+ *                                gate features first); scales: moe_mxfp8_w_gateup_scale_bytes(dims) bytes, the two
+ *                                tilings with feature = gate/up column and 128-wide slices along H.
+ *   moe_grouped_gemm_gateup_mxfp8  gu [R,2I] bf16 (gate columns [0,I), up columns [I,2I)), overwritten.
+ *   moe_swiglu_mxfp8             gu [R,2I] bf16 -> h_act [R,I] bf16 = silu(g)*u (fp32, rounded once), and h_codes /
+ *                                h_scales = the quantised form of exactly those bf16 values, laid out as
+ *                                moe_mxfp8_quantize_h_act writes them.  Elementwise, HBM-bound.
+ * Same requirements, status codes and tolerance statement as the other block-scaled calls. */
+size_t moe_mxfp8_x_scale_bytes(const moe_dims_t* dims);
+size_t moe_mxfp8_w_gateup_scale_bytes(const moe_dims_t* dims);
+int moe_mxfp8_quantize_x_perm(const moe_dims_t* dims, const void* x_perm, void* codes, void* scales, moe_stream_t stream);
+int moe_mxfp8_quantize_w_gateup(const moe_dims_t* dims, const void* w_gate, const void* w_up, void* codes_t, void* scales,
+                                moe_stream_t stream);
+int moe_grouped_gemm_gateup_mxfp8(const moe_dims_t* dims, const void* x_codes, const void* x_scales,
+                                  const void* w_codes_t, const void* w_scales, const int32_t* offsets, void* gu,
+                                  moe_stream_t stream);
+int moe_swiglu_mxfp8(const moe_dims_t* dims, const void* gu, void* h_act, void* h_codes, void* h_scales,
+                     moe_stream_t stream);
+
 /* ---- whole layer from HOST activations ------------------------------------------------------
  * One training step of the layer for a caller whose per-step tensors live in host memory:
  * copies x, topk_idx, topk_w, dy (HOST pointers; pinned memory makes the copies asynchronous)

@@ -29,6 +29,8 @@ EXPORTS = [
     "moe_mxfp8_quantize_w_down_dgrad", "moe_grouped_gemm_down_dgrad_mxfp8",
     "moe_mxfp8_dgu_scale_bytes", "moe_mxfp8_w_gateup_dgrad_scale_bytes", "moe_mxfp8_quantize_dgu",
     "moe_mxfp8_quantize_w_gateup_dgrad", "moe_grouped_gemm_gateup_dgrad_mxfp8",
+    "moe_mxfp8_x_scale_bytes", "moe_mxfp8_w_gateup_scale_bytes", "moe_mxfp8_quantize_x_perm", "moe_mxfp8_quantize_w_gateup",
+    "moe_grouped_gemm_gateup_mxfp8", "moe_swiglu_mxfp8",
 ]
 
 
@@ -61,7 +63,7 @@ def load_library() -> ctypes.CDLL:
         lib.moe_layer_arena_bytes.argtypes = [ctypes.POINTER(MoeDims)]
         for name in ("moe_mxfp8_act_scale_bytes", "moe_mxfp8_w_down_scale_bytes", "moe_mxfp8_dy_scale_bytes",
                      "moe_mxfp8_w_down_dgrad_scale_bytes", "moe_mxfp8_dgu_scale_bytes",
-                     "moe_mxfp8_w_gateup_dgrad_scale_bytes"):
+                     "moe_mxfp8_w_gateup_dgrad_scale_bytes", "moe_mxfp8_x_scale_bytes", "moe_mxfp8_w_gateup_scale_bytes"):
             getattr(lib, name).restype = ctypes.c_size_t
             getattr(lib, name).argtypes = [ctypes.POINTER(MoeDims)]
         lib.moe_device_status.restype = ctypes.c_int
@@ -96,6 +98,10 @@ def load_library() -> ctypes.CDLL:
             "moe_mxfp8_quantize_dgu": [dp, p, p, p, p],
             "moe_mxfp8_quantize_w_gateup_dgrad": [dp, p, p, p, p, p],
             "moe_grouped_gemm_gateup_dgrad_mxfp8": [dp, p, p, p, p, p, p, p],
+            "moe_mxfp8_quantize_x_perm": [dp, p, p, p, p],
+            "moe_mxfp8_quantize_w_gateup": [dp, p, p, p, p, p],
+            "moe_grouped_gemm_gateup_mxfp8": [dp, p, p, p, p, p, p, p],
+            "moe_swiglu_mxfp8": [dp, p, p, p, p, p],
         }
         for name, argtypes in sigs.items():
             fn = getattr(lib, name)
@@ -292,6 +298,31 @@ def moe_mxfp8_quantize_w_gateup_dgrad(d, w_gate, w_up, codes, scales):
 def moe_grouped_gemm_gateup_dgrad_mxfp8(d, dgu_codes, dgu_scales, w_codes, w_scales, offsets, dx_perm):
     _call("moe_grouped_gemm_gateup_dgrad_mxfp8", ctypes.byref(d), _ptr(dgu_codes), _ptr(dgu_scales), _ptr(w_codes),
           _ptr(w_scales), _ptr(offsets), _ptr(dx_perm), _stream())
+
+
+def moe_mxfp8_x_scale_bytes(d: MoeDims) -> int:
+    return int(load_library().moe_mxfp8_x_scale_bytes(ctypes.byref(d)))
+
+
+def moe_mxfp8_w_gateup_scale_bytes(d: MoeDims) -> int:
+    return int(load_library().moe_mxfp8_w_gateup_scale_bytes(ctypes.byref(d)))
+
+
+def moe_mxfp8_quantize_x_perm(d, x_perm, codes, scales):
+    _call("moe_mxfp8_quantize_x_perm", ctypes.byref(d), _ptr(x_perm), _ptr(codes), _ptr(scales), _stream())
+
+
+def moe_mxfp8_quantize_w_gateup(d, w_gate, w_up, codes_t, scales):
+    _call("moe_mxfp8_quantize_w_gateup", ctypes.byref(d), _ptr(w_gate), _ptr(w_up), _ptr(codes_t), _ptr(scales), _stream())
+
+
+def moe_grouped_gemm_gateup_mxfp8(d, x_codes, x_scales, w_codes_t, w_scales, offsets, gu):
+    _call("moe_grouped_gemm_gateup_mxfp8", ctypes.byref(d), _ptr(x_codes), _ptr(x_scales), _ptr(w_codes_t), _ptr(w_scales),
+          _ptr(offsets), _ptr(gu), _stream())
+
+
+def moe_swiglu_mxfp8(d, gu, h_act, h_codes, h_scales):
+    _call("moe_swiglu_mxfp8", ctypes.byref(d), _ptr(gu), _ptr(h_act), _ptr(h_codes), _ptr(h_scales), _stream())
 
 
 def moe_layer_fwd_bwd_host(d, x_host, topk_idx_host, topk_w_host, dy_host, w_gate, w_up, w_down, y_host, dx_host,

@@ -286,7 +286,8 @@ int moe_mxfp8_quantize_w_down(const moe_dims_t* dims, const void* w_down, void* 
     const void* const opt[] = {nullptr};
     s = check_ptrs(req, opt);
     if (s != MOE_OK) return s;
-    return launch_mx_quantize_w_down(*dims, cb(w_down), static_cast<uint8_t*>(codes_t), static_cast<uint8_t*>(scales), st(stream));
+    return launch_mx_quantize_w_transposed(dims->E, dims->I, dims->H, dims->H, 0, cb(w_down), static_cast<uint8_t*>(codes_t),
+                                           static_cast<uint8_t*>(scales), st(stream));
 }
 
 int moe_grouped_gemm_down_mxfp8(const moe_dims_t* dims, const void* h_codes, const void* h_scales, const void* w_codes_t,
@@ -396,6 +397,67 @@ int moe_grouped_gemm_gateup_dgrad_mxfp8(const moe_dims_t* dims, const void* dgu_
     return launch_mx_gemm((long long)dims->T * dims->K, dims->E, dims->H, 2 * dims->I, static_cast<const uint8_t*>(dgu_codes),
                           static_cast<const uint8_t*>(dgu_scales), static_cast<const uint8_t*>(w_codes),
                           static_cast<const uint8_t*>(w_scales), offsets, mb(dx_perm), st(stream));
+}
+
+// ---- block-scaled FP8 gate/up projection (contraction over H) and the SwiGLU activation with its quantiser ----
+size_t moe_mxfp8_x_scale_bytes(const moe_dims_t* dims) {
+    if (check_mx_dims(dims) != MOE_OK) return 0;
+    return (size_t)(dims->H / 128) * (size_t)dims->T * dims->K * 4;
+}
+
+size_t moe_mxfp8_w_gateup_scale_bytes(const moe_dims_t* dims) {
+    if (check_mx_dims(dims) != MOE_OK) return 0;
+    return mx_w_scale_bytes(dims->E, 2 * dims->I, dims->H);
+}
+
+int moe_mxfp8_quantize_x_perm(const moe_dims_t* dims, const void* x_perm, void* codes, void* scales, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {x_perm, codes, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_rows((long long)dims->T * dims->K, dims->H, cb(x_perm), static_cast<uint8_t*>(codes),
+                                   static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_mxfp8_quantize_w_gateup(const moe_dims_t* dims, const void* w_gate, const void* w_up, void* codes_t, void* scales,
+                                moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {w_gate, w_up, codes_t, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    s = launch_mx_quantize_w_transposed(dims->E, dims->H, dims->I, 2 * dims->I, 0, cb(w_gate), static_cast<uint8_t*>(codes_t),
+                                        static_cast<uint8_t*>(scales), st(stream));
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_w_transposed(dims->E, dims->H, dims->I, 2 * dims->I, dims->I, cb(w_up), static_cast<uint8_t*>(codes_t),
+                                           static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_grouped_gemm_gateup_mxfp8(const moe_dims_t* dims, const void* x_codes, const void* x_scales, const void* w_codes_t,
+                                  const void* w_scales, const int32_t* offsets, void* gu, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {x_codes, x_scales, w_codes_t, w_scales, offsets, gu};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_gemm((long long)dims->T * dims->K, dims->E, 2 * dims->I, dims->H, static_cast<const uint8_t*>(x_codes),
+                          static_cast<const uint8_t*>(x_scales), static_cast<const uint8_t*>(w_codes_t),
+                          static_cast<const uint8_t*>(w_scales), offsets, mb(gu), st(stream));
+}
+
+int moe_swiglu_mxfp8(const moe_dims_t* dims, const void* gu, void* h_act, void* h_codes, void* h_scales, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {gu, h_act, h_codes, h_scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_swiglu_quantize((long long)dims->T * dims->K, dims->I, cb(gu), mb(h_act), static_cast<uint8_t*>(h_codes),
+                                     static_cast<uint8_t*>(h_scales), st(stream));
 }
 
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).

@@ -61,9 +61,11 @@ int launch_gateup_wgrad(const moe_dims_t& d, const bf16* x_perm, const bf16* dgu
 size_t mx_w_scale_single_bytes(int E, int n_feat, int k);   // weight scales in the single-CTA tiling
 size_t mx_w_scale_bytes(int E, int n_feat, int k);          // both tilings, one after the other
 int launch_mx_quantize_rows(long long rows, int n, const bf16* x, uint8_t* codes, uint8_t* scales, cudaStream_t s);
-int launch_mx_quantize_w_down(const moe_dims_t& d, const bf16* w_down, uint8_t* codes_t, uint8_t* scales, cudaStream_t s);
+int launch_mx_quantize_w_transposed(int E, int k, int n, int n_total, int n_off, const bf16* w, uint8_t* codes_t, uint8_t* scales,
+                                    cudaStream_t s);
 int launch_mx_quantize_w_rows(int E, int n_feat, int k, int k_total, int k_off, const bf16* w, uint8_t* codes, uint8_t* scales,
                               cudaStream_t s);
+int launch_mx_swiglu_quantize(long long rows, int I, const bf16* gu, bf16* h_act, uint8_t* codes, uint8_t* scales, cudaStream_t s);
 int launch_mx_gemm(long long R, int E, int n_feat, int k, const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
                    const uint8_t* b_scales, const int32_t* offsets, bf16* out, cudaStream_t s);
 

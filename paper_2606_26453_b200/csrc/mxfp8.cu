@@ -824,25 +824,82 @@ __global__ void __launch_bounds__(256) mx_quantize_rows_kernel(const uint4* __re
     }
 }
 
-// w_down [E, I, H] bf16 -> codes [E, H, I] and scale blocks.  One thread per (expert, block of 32 along I, feature h):
-// consecutive lanes take consecutive h, so the 32 loads of a thread are coalesced across the warp; the thread keeps the
-// 32 values, picks the scale and writes 32 contiguous code bytes.
-__global__ void __launch_bounds__(256) mx_quantize_w_down_kernel(const bf16* __restrict__ w, int E, int I, int H,
-                                                                 uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
-                                                                 uint8_t* __restrict__ scales_pair) {
+// The SwiGLU activation of saved pre-activations with the activation quantiser fused in: GU [rows, 2I] bf16 ->
+// H_act [rows, I] bf16 (silu(g) * u in fp32, rounded once) and the block-scaled FP8 codes and scale words of exactly those
+// bf16 values, in the layouts of the activation quantiser.  Same lane mapping as mx_quantize_rows_kernel: a half-warp per
+// (row, 128-wide slice of I), 8 elements per lane.
+__global__ void __launch_bounds__(256) mx_swiglu_quantize_kernel(const uint4* __restrict__ gu, long long rows, int I,
+                                                                 uint4* __restrict__ h_act, uint2* __restrict__ codes,
+                                                                 uint32_t* __restrict__ scales) {
+    const int lane = threadIdx.x & 31;
+    const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const int k_tiles = I / 128;
+    const long long total = rows * k_tiles;
+    const long long pairs = (total + 1) / 2;
+    for (long long p0 = warp; p0 < pairs; p0 += n_warps) {
+        const long long u = 2 * p0 + (lane >> 4);
+        if (u >= total) continue;   // only the last pair can be half empty; no warp-wide operation below needs those lanes
+        const long long r = u / k_tiles;
+        const int kt = (int)(u - r * k_tiles);
+        const long long g_idx = (r * 2 * I + kt * 128) / 8 + (lane & 15);
+        const uint4 graw = __ldg(gu + g_idx), uraw = __ldg(gu + g_idx + I / 8);
+        const uint32_t* gw = reinterpret_cast<const uint32_t*>(&graw);
+        const uint32_t* uw = reinterpret_cast<const uint32_t*>(&uraw);
+        uint32_t hw[4];
+        float v[8];
+        float amax = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 g2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw[j]));
+            const float2 u2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&uw[j]));
+            const float h0 = __fdividef(g2.x, 1.f + __expf(-g2.x)) * u2.x;
+            const float h1 = __fdividef(g2.y, 1.f + __expf(-g2.y)) * u2.y;
+            hw[j] = pack_bf16(h0, h1);
+            const float2 hr = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&hw[j]));   // what H_act holds
+            v[2 * j] = hr.x; v[2 * j + 1] = hr.y;
+            amax = fmaxf(amax, fmaxf(fabsf(hr.x), fabsf(hr.y)));
+        }
+        const uint32_t half_mask = (lane & 16) ? 0xffff0000u : 0x0000ffffu;
+        amax = fmaxf(amax, __shfl_xor_sync(half_mask, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(half_mask, amax, 2));
+        const int se = mx_scale_exp(amax);
+        const float inv = mx_inv_scale(se);
+        uint2 out;
+        out.x = mx_e4m3x2(v[0] * inv, v[1] * inv) | (mx_e4m3x2(v[2] * inv, v[3] * inv) << 16);
+        out.y = mx_e4m3x2(v[4] * inv, v[5] * inv) | (mx_e4m3x2(v[6] * inv, v[7] * inv) << 16);
+        h_act[u * 16 + (lane & 15)] = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        codes[u * 16 + (lane & 15)] = out;
+        const uint32_t sbyte = (uint32_t)(se + 127);
+        const int base = lane & 16;
+        const uint32_t word = __shfl_sync(half_mask, sbyte, base) | (__shfl_sync(half_mask, sbyte, base + 4) << 8) |
+                              (__shfl_sync(half_mask, sbyte, base + 8) << 16) | (__shfl_sync(half_mask, sbyte, base + 12) << 24);
+        if ((lane & 15) == 0) scales[(long long)kt * rows + r] = word;
+    }
+}
+
+// Weights whose OUTPUT-feature axis is contiguous: w [E, k, n] bf16 (W_down [E, I, H]; W_gate, W_up [E, H, I]) -> codes
+// transposed, contraction contiguous, as rows n_off .. n_off + n of [E, n_total, k] (W_gate and W_up stacked along the 2I
+// output features of the gate/up projection), and the scale bytes in both tilings.  One thread per (expert, block of
+// 32 along k, feature): consecutive lanes take consecutive features, so the 32 loads of a thread are coalesced across
+// the warp; the thread keeps the 32 values, picks the scale and writes 32 contiguous code bytes.
+__global__ void __launch_bounds__(256) mx_quantize_w_transposed_kernel(const bf16* __restrict__ w, int E, int k, int n,
+                                                                       int n_total, int n_off, uint8_t* __restrict__ codes,
+                                                                       uint8_t* __restrict__ scales,
+                                                                       uint8_t* __restrict__ scales_pair) {
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const int blocks_i = I / 32;
-    const long long total = (long long)E * blocks_i * H;
+    const int blocks_k = k / 32;
+    const long long total = (long long)E * blocks_k * n;
     if (idx >= total) return;
-    const int h = (int)(idx % H);
-    const int ib = (int)((idx / H) % blocks_i);
-    const int e = (int)(idx / ((long long)H * blocks_i));
-    const bf16* src = w + ((long long)e * I + (long long)ib * 32) * H + h;
+    const int h = (int)(idx % n);
+    const int ib = (int)((idx / n) % blocks_k);
+    const int e = (int)(idx / ((long long)n * blocks_k));
+    const bf16* src = w + ((long long)e * k + (long long)ib * 32) * n + h;
     float v[32];
     float amax = 0.f;
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-        v[j] = __bfloat162float(src[(long long)j * H]);
+        v[j] = __bfloat162float(src[(long long)j * n]);
         amax = fmaxf(amax, fabsf(v[j]));
     }
     const int se = mx_scale_exp(amax);
@@ -850,17 +907,17 @@ __global__ void __launch_bounds__(256) mx_quantize_w_down_kernel(const bf16* __r
     uint32_t out[8];
 #pragma unroll
     for (int q = 0; q < 8; ++q)
-        out[q] = mx_e4m3(v[4 * q] * inv) | (mx_e4m3(v[4 * q + 1] * inv) << 8) | (mx_e4m3(v[4 * q + 2] * inv) << 16) |
-                 (mx_e4m3(v[4 * q + 3] * inv) << 24);
-    uint4* dst = reinterpret_cast<uint4*>(codes + ((long long)e * H + h) * I + (long long)ib * 32);
+        out[q] = mx_e4m3x2(v[4 * q] * inv, v[4 * q + 1] * inv) | (mx_e4m3x2(v[4 * q + 2] * inv, v[4 * q + 3] * inv) << 16);
+    const int f = n_off + h;   // output feature of the GEMM
+    uint4* dst = reinterpret_cast<uint4*>(codes + ((long long)e * n_total + f) * k + (long long)ib * 32);
     dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
     dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
-    const int k_tiles = I / 128;
-    scales[(((long long)e * (H / 128) + h / 128) * k_tiles + ib / 4) * 512 + (h % 32) * 16 + ((h % 128) / 32) * 4 + (ib % 4)] =
+    const int k_tiles = k / 128;
+    scales[(((long long)e * (n_total / 128) + f / 128) * k_tiles + ib / 4) * 512 + (f % 32) * 16 + ((f % 128) / 32) * 4 + (ib % 4)] =
         (uint8_t)(se + 127);
-    // the same byte in the tiling of the CTA-pair kernel: per (240-column tile, K slice) two 512-byte blocks
-    const int nt = h / MXP_NT, c = h % MXP_NT;
-    const int n_tiles_p = (H + MXP_NT - 1) / MXP_NT;
+    // the same byte in the tiling of the CTA-pair kernel: per (208-column tile, K slice) two 512-byte blocks
+    const int nt = f / MXP_NT, c = f % MXP_NT;
+    const int n_tiles_p = (n_total + MXP_NT - 1) / MXP_NT;
     scales_pair[(((long long)e * n_tiles_p + nt) * k_tiles + ib / 4) * 1024 + (c >> 7) * 512 + (c % 32) * 16 + ((c % 128) / 32) * 4 +
                 (ib % 4)] = (uint8_t)(se + 127);
 }
@@ -887,10 +944,24 @@ int launch_mx_quantize_rows(long long rows, int n, const bf16* x, uint8_t* codes
     return check_launch();
 }
 
-int launch_mx_quantize_w_down(const moe_dims_t& d, const bf16* w_down, uint8_t* codes_t, uint8_t* scales, cudaStream_t s) {
-    const long long total = (long long)d.E * (d.I / 32) * d.H;
-    mx_quantize_w_down_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(w_down, d.E, d.I, d.H, codes_t, scales,
-                                                                              scales + mx_w_scale_single_bytes(d.E, d.H, d.I));
+// w [E, k, n] -> rows [n_off, n_off + n) of the transposed codes [E, n_total, k] and the matching scale bytes
+int launch_mx_quantize_w_transposed(int E, int k, int n, int n_total, int n_off, const bf16* w, uint8_t* codes_t, uint8_t* scales,
+                                    cudaStream_t s) {
+    const long long total = (long long)E * (k / 32) * n;
+    mx_quantize_w_transposed_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
+        w, E, k, n, n_total, n_off, codes_t, scales, scales + mx_w_scale_single_bytes(E, n_total, k));
+    return check_launch();
+}
+
+int launch_mx_swiglu_quantize(long long rows, int I, const bf16* gu, bf16* h_act, uint8_t* codes, uint8_t* scales, cudaStream_t s) {
+    const long long units = rows * (I / 128);
+    long long blocks = (units + 15) / 16;   // 8 warps x 2 units per block and pass
+    const long long cap = (long long)sm_count() * 32;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    mx_swiglu_quantize_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const uint4*>(gu), rows, I,
+                                                             reinterpret_cast<uint4*>(h_act), reinterpret_cast<uint2*>(codes),
+                                                             reinterpret_cast<uint32_t*>(scales));
     return check_launch();
 }
 

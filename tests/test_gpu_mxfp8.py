@@ -204,6 +204,62 @@ def test_gateup_dgrad_quantisers_and_gemm_against_the_oracle(B, name):
     assert np.linalg.norm(Hh.to_np64(dx) - exact) / np.linalg.norm(exact) < 0.08
 
 
+@pytest.mark.parametrize("name", list(CASES))
+def test_gateup_forward_and_fused_swiglu_quantiser_against_the_oracle(B, name):
+    """GU = [Q(X_perm) . Q(W_gate[e]) | Q(X_perm) . Q(W_up[e])] (contraction over H), then H_act = silu(g) * u with its
+    block-scaled FP8 form from the same call, then the FP8 down projection fed by those codes: the forward chain."""
+    counts, K, H, I = CASES[name]
+    cfg, host = Hh.ragged_workload(counts, K=K, H=H, I=I, seed=27)
+    ref = O.layer_fwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"], host["W_down"])
+    R, E = cfg.R, cfg.E
+    d = B.dims(cfg.T, H, I, E, K)
+    x = W.round_to_bf16(ref["X_perm"].astype(np.float32))
+    x[0, :32] = 0.0
+    wg, wu = host["W_gate"].copy(), W.round_to_bf16(host["W_up"] * 2.0)
+    wg[0, :32, 0] = 0.0
+    x_dev, wg_dev, wu_dev = Hh.to_dev_bf16(x), Hh.to_dev_bf16(wg), Hh.to_dev_bf16(wu)
+    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    xc, xs = u8(R * H), u8(B.moe_mxfp8_x_scale_bytes(d))
+    wc, ws = u8(E * 2 * I * H), u8(B.moe_mxfp8_w_gateup_scale_bytes(d))
+    n_single = E * (2 * I // 128) * (H // 128) * 512
+    assert xs.numel() == (H // 128) * R * 4 and ws.numel() == n_single + E * ((2 * I + 207) // 208) * (H // 128) * 1024
+    B.moe_mxfp8_quantize_x_perm(d, x_dev, xc, xs)
+    B.moe_mxfp8_quantize_w_gateup(d, wg_dev, wu_dev, wc, ws)
+    torch.cuda.synchronize()
+    o_xc, o_xs, _ = O.mxfp8_quantize(x)
+    wt = np.concatenate([np.swapaxes(wg, 1, 2), np.swapaxes(wu, 1, 2)], axis=1)      # [E, 2I, H]: contraction last
+    o_wc, o_ws, _ = O.mxfp8_quantize(wt)
+    assert np.array_equal(_act_scales_from_layout(xs.cpu().numpy(), R, H), o_xs)
+    assert np.array_equal(xc.cpu().numpy().reshape(R, H), o_xc)
+    assert np.array_equal(wc.cpu().numpy().reshape(E, 2 * I, H), o_wc)
+    ws_host = ws.cpu().numpy()
+    assert np.array_equal(ws_host[:n_single], _w_scales_single_layout(o_ws, E, 2 * I, H))
+    want_pair, written = _w_scales_pair_layout(o_ws, E, 2 * I, H)
+    assert np.array_equal(ws_host[n_single:][written], want_pair[written])
+    assert np.all(ws_host[n_single:][~written] == 0xAB)
+    gu = torch.full((R, 2 * I), float("nan"), dtype=torch.bfloat16, device="cuda")
+    off = torch.from_numpy(ref["offsets"]).cuda()
+    B.moe_grouped_gemm_gateup_mxfp8(d, xc, xs, wc, ws, off, gu)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    Hh.assert_close(Hh.to_np64(gu), O.gateup_mxfp8(x, wg, wu, ref["offsets"]), f"{name}: GU (MXFP8)",
+                    rel_fro=Hh.PER_CALL_FROBENIUS)
+    # the activation of the CUDA side's own GU, and the quantised form of the CUDA side's own H_act (decided on exact values)
+    h = torch.full((R, I), float("nan"), dtype=torch.bfloat16, device="cuda")
+    hc, hs = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    B.moe_swiglu_mxfp8(d, gu, h, hc, hs)
+    torch.cuda.synchronize()
+    Hh.assert_close(Hh.to_np64(h), O.swiglu_fwd(Hh.to_np64(gu)), f"{name}: H_act from GU", rel_fro=Hh.PER_CALL_FROBENIUS)
+    o_hc, o_hs, _ = O.mxfp8_quantize(Hh.to_np64(h))
+    assert np.array_equal(hc.cpu().numpy().reshape(R, I), o_hc)
+    assert np.array_equal(_act_scales_from_layout(hs.cpu().numpy(), R, I), o_hs)
+    # ... which equals what the stand-alone activation quantiser makes of the same H_act
+    hc2, hs2 = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    B.moe_mxfp8_quantize_h_act(d, h, hc2, hs2)
+    torch.cuda.synchronize()
+    assert torch.equal(hc, hc2) and torch.equal(hs, hs2)
+
+
 def test_shapes_the_block_scaled_path_does_not_take_are_refused(B):
     d = B.dims(64, 192, 128, 2, 1)                   # H not a multiple of 128
     assert B.moe_mxfp8_act_scale_bytes(d) == 0
