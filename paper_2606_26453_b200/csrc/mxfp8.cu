@@ -1,5 +1,8 @@
-// Block-scaled FP8 (MXFP8) variant of the down projection: quantisers and a grouped GEMM on the block-scaled tensor-core
-// path (tcgen05.mma kind::mxf8f6f4 with block_scale).
+// Block-scaled FP8 (MXFP8) twins of the four row-ragged grouped GEMMs (gate/up forward, down forward, down dgrad,
+// gate/up dgrad) on the block-scaled tensor-core path (tcgen05.mma kind::mxf8f6f4 with block_scale): quantisers, one GEMM
+// in two tilings, and the SwiGLU activation with the activation quantiser fused in.  Every GEMM here is
+//   out[r, :] = dequant(a row r) . dequant(b[e])^T   for the rows r of expert e,
+// a [R, k] and b [E, n_feat, k] both contraction-contiguous; the callers choose which tensors play a and b.
 //
 // Format: E4M3 elements, one E8M0 scale (a power of two, 2^(s-127)) per 32 consecutive elements along the
 // contraction; scale of a block with largest magnitude a > 0: 2^(floor(log2 a) - 8); elements = v / scale rounded to
@@ -8,17 +11,19 @@
 // division by a power of two is exact in fp32, and the FP8 conversion instruction rounds to nearest even.
 //
 // Layouts (chosen so that the GEMM's scale factors reach tensor memory without per-element work):
-//   activation codes   [R, I] bytes, contraction contiguous
-//   activation scales  [I/128][R] 32-bit words: the 4 scale bytes of the 4 blocks of 32 inside one 128-wide slice of
+//   activation codes   [R, k] bytes, contraction contiguous
+//   activation scales  [k/128][R] 32-bit words: the 4 scale bytes of the 4 blocks of 32 inside one 128-wide slice of
 //                      the contraction, for one row -- rows of a tile start anywhere, so a warp gathers 128 words per
 //                      K slice and lays them out for the tensor-memory copy
-//   weight codes       [E, H, I] bytes: the down weights transposed, contraction contiguous
-//   weight scales      [E][H/128][I/128][512 bytes]: per 128 output features x 128 contraction elements, byte
-//                      (h % 32) * 16 + ((h % 128) / 32) * 4 + block -- the 32 x 16-byte pattern that
-//                      tcgen05.cp.32x128b.warpx4 copies from shared memory into 4 tensor-memory columns (lane = h % 32,
-//                      column = (h % 128) / 32, byte = block)
+//   weight codes       [E, n_feat, k] bytes, contraction contiguous (weights stored feature-contiguous are transposed by
+//                      their quantiser)
+//   weight scales      first [E][n_feat/128][k/128][512 bytes]: per 128 output features x 128 contraction elements, byte
+//                      (f % 32) * 16 + ((f % 128) / 32) * 4 + block -- the 32 x 16-byte pattern that
+//                      tcgen05.cp.32x128b.warpx4 copies from shared memory into 4 tensor-memory columns (lane = f % 32,
+//                      column = (f % 128) / 32, byte = block); then the same bytes in the tiling of the CTA-pair kernel
+//                      (see there)
 //
-// GEMM kernel: one CTA per SM, persistent over the same row-ragged tile list as the bf16 kernels (tiles of 128 rows x
+// Single-CTA kernel: one CTA per SM, persistent over the same row-ragged tile list as the bf16 kernels (tiles of 128 rows x
 // 128 output features), K slices of 128 (= 128 bytes per row: the same swizzled stage geometry as 64 bf16).
 //   warp 0      TMA producer: A and B code tiles, bulk copy of the weight-scale block
 //   warp 1      one thread: tcgen05.cp of both scale blocks into tensor memory, four tcgen05.mma (K = 32 each, scale
@@ -132,7 +137,7 @@ __device__ __forceinline__ MxTile mx_decode(const MxParams& p, const MxCtl* ctl,
 }
 
 __global__ void __launch_bounds__(MX_THREADS, 1)
-mx_down_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+mx_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_o, const MxParams p) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -464,7 +469,7 @@ __device__ __forceinline__ MxPairTile mxp_decode(const MxPairParams& p, const Mx
 }
 
 __global__ void __launch_bounds__(MXP_THREADS, 1)
-mx_down_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_sfb, const __grid_constant__ CUtensorMap map_o,
                     const MxPairParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -1004,20 +1009,20 @@ static int launch_mx_gemm_pair(long long R, int E, int n_feat, int k, const uint
     cfg.dynamicSmemBytes = MXP_SMEM_BYTES;
     cfg.attrs = attr; cfg.numAttrs = 1;
     if (grid_of_device[dev] == 0) {
-        if (cudaFuncSetAttribute(mx_down_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MXP_SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(mx_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MXP_SMEM_BYTES) != cudaSuccess)
             return MOE_ERR_CUDA;
         const int sms = sm_count();
         if (sms <= 0) return MOE_ERR_CUDA;
         // as many pairs as can be resident at once: a pair that had to wait for a free SM pair would double the duration
         cfg.gridDim = dim3(2 * (sms / 2));
         int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, mx_down_pair_kernel, &cfg) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
+        if (cudaOccupancyMaxActiveClusters(&clusters, mx_gemm_pair_kernel, &cfg) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
         if (clusters > sms / 2) clusters = sms / 2;
         grid_of_device[dev] = 2 * clusters;
     }
     cfg.gridDim = dim3(grid_of_device[dev]);
     cfg.stream = s;
-    if (cudaLaunchKernelEx(&cfg, mx_down_pair_kernel, a, b, sfb, o, p) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, mx_gemm_pair_kernel, a, b, sfb, o, p) != cudaSuccess) return MOE_ERR_CUDA;
     return check_launch();
 }
 
@@ -1041,13 +1046,13 @@ int launch_mx_gemm(long long R, int E, int n_feat, int k, const uint8_t* a_codes
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(mx_down_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MX_SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(mx_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MX_SMEM_BYTES) != cudaSuccess)
             return MOE_ERR_CUDA;
         attr_set[dev] = true;
     }
     const int sms = sm_count();
     if (sms <= 0) return MOE_ERR_CUDA;
-    mx_down_kernel<<<sms, MX_THREADS, MX_SMEM_BYTES, s>>>(a, b, o, p);
+    mx_gemm_kernel<<<sms, MX_THREADS, MX_SMEM_BYTES, s>>>(a, b, o, p);
     return check_launch();
 }
 
