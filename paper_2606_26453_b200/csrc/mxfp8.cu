@@ -743,7 +743,8 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 // scale exponent of a block with largest magnitude amax: floor(log2 amax) - 8, clamped to the E8M0 range; -127 for zero
 __device__ __forceinline__ int mx_scale_exp(float amax) {
     if (!(amax > 0.f)) return -127;
-    const int e = ilogbf(amax) - 8;
+    const int field = (__float_as_int(amax) >> 23) & 0xFF;             // amax is positive and finite
+    const int e = (field != 0 ? field - 127 : ilogbf(amax)) - 8;       // subnormal magnitudes take the library route
     return e < -127 ? -127 : (e > 127 ? 127 : e);
 }
 // 2^-s as a float (s in [-127, 127]; 2^-127 is a subnormal)
@@ -806,7 +807,7 @@ __global__ void __launch_bounds__(256) mx_quantize_rows_kernel(const uint4* __re
             uint2 out;
             out.x = mx_e4m3x2(v[0] * inv, v[1] * inv) | (mx_e4m3x2(v[2] * inv, v[3] * inv) << 16);
             out.y = mx_e4m3x2(v[4] * inv, v[5] * inv) | (mx_e4m3x2(v[6] * inv, v[7] * inv) << 16);
-            const long long r = u / k_tiles;
+            const long long r = (total >> 32) == 0 ? (long long)((uint32_t)u / (uint32_t)k_tiles) : u / k_tiles;
             const int kt = (int)(u - r * k_tiles) + out_kt0;
             if (u < total) codes[(r * out_k_tiles + kt) * 16 + (lane & 15)] = out;
             const uint32_t sbyte = (uint32_t)(se + 127);
@@ -845,7 +846,7 @@ __global__ void __launch_bounds__(256) mx_swiglu_quantize_kernel(const uint4* __
     for (long long p0 = warp; p0 < pairs; p0 += n_warps) {
         const long long u = 2 * p0 + (lane >> 4);
         if (u >= total) continue;   // only the last pair can be half empty; no warp-wide operation below needs those lanes
-        const long long r = u / k_tiles;
+        const long long r = (total >> 32) == 0 ? (long long)((uint32_t)u / (uint32_t)k_tiles) : u / k_tiles;
         const int kt = (int)(u - r * k_tiles);
         const long long g_idx = (r * 2 * I + kt * 128) / 8 + (lane & 15);
         const uint4 graw = __ldg(gu + g_idx), uraw = __ldg(gu + g_idx + I / 8);
