@@ -201,6 +201,90 @@ def make_step(B, b, wl, fused=False):
     return step
 
 
+def time_fp8_step(B, cfg, res, device, min_seconds=0.5):
+    """The layer step with the four row-ragged GEMMs replaced by their block-scaled FP8 twins (weight gradients, data
+    movement and SwiGLU backward unchanged): permute, quantise X_perm, FP8 gate/up, SwiGLU (+ FP8 form of H_act), FP8
+    down, combine | combine backward, quantise dY_perm, FP8 down dgrad, down wgrad, SwiGLU backward, quantise dGU, FP8
+    gate/up dgrad, gate/up wgrad, permute backward.  Timed back to back for at least `min_seconds`, once with the four
+    weight quantisations inside every step (weights change every optimizer step) and once with them outside (several
+    micro-batches per optimizer step)."""
+    if cfg.H % 128 or cfg.I % 128:
+        return None
+    b, wl = res["buffers"], res["wl"]
+    d = b.d
+    R, E, H, I = cfg.R, cfg.E, cfg.H, cfg.I
+    x, idx, w, dy = wl["X"], wl["topk_idx"], wl["topk_w"], wl["dY"]
+    wg, wu, wd = wl["W_gate"], wl["W_up"], wl["W_down"]
+    u8 = lambda n: torch.empty(n, dtype=torch.uint8, device=device)
+    xc, xs = u8(R * H), u8(B.moe_mxfp8_x_scale_bytes(d))            # also reused for dY_perm (same shape)
+    hc, hs = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    gc, gs = u8(R * 2 * I), u8(B.moe_mxfp8_dgu_scale_bytes(d))
+    w_gu, s_gu = u8(E * 2 * I * H), u8(B.moe_mxfp8_w_gateup_scale_bytes(d))
+    w_dn, s_dn = u8(E * H * I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
+    w_dd, s_dd = u8(E * I * H), u8(B.moe_mxfp8_w_down_dgrad_scale_bytes(d))
+    w_gd, s_gd = u8(E * H * 2 * I), u8(B.moe_mxfp8_w_gateup_dgrad_scale_bytes(d))
+
+    def quantise_weights():
+        B.moe_mxfp8_quantize_w_gateup(d, wg, wu, w_gu, s_gu)
+        B.moe_mxfp8_quantize_w_down(d, wd, w_dn, s_dn)
+        B.moe_mxfp8_quantize_w_down_dgrad(d, wd, w_dd, s_dd)
+        B.moe_mxfp8_quantize_w_gateup_dgrad(d, wg, wu, w_gd, s_gd)
+
+    def step():
+        B.moe_permute(d, x, idx, b.x_perm, b.counts, b.offsets, b.row_to_pair, b.pair_to_row, b.workspace)
+        B.moe_mxfp8_quantize_x_perm(d, b.x_perm, xc, xs)
+        B.moe_grouped_gemm_gateup_mxfp8(d, xc, xs, w_gu, s_gu, b.offsets, b.gu)
+        B.moe_swiglu_mxfp8(d, b.gu, b.h_act, hc, hs)
+        B.moe_grouped_gemm_down_mxfp8(d, hc, hs, w_dn, s_dn, b.offsets, b.y_perm)
+        B.moe_unpermute_combine(d, b.y_perm, w, b.pair_to_row, b.y)
+        B.moe_unpermute_combine_bwd(d, dy, b.y_perm, w, b.pair_to_row, b.dy_perm, b.dtopk_w)
+        B.moe_mxfp8_quantize_dy_perm(d, b.dy_perm, xc, xs)
+        B.moe_grouped_gemm_down_dgrad_mxfp8(d, xc, xs, w_dd, s_dd, b.offsets, b.dh_act)
+        B.moe_grouped_gemm_down_wgrad(d, b.h_act, b.dy_perm, b.offsets, b.dw_down)
+        B.moe_swiglu_bwd(d, b.dh_act, b.gu, b.dgu)
+        B.moe_mxfp8_quantize_dgu(d, b.dgu, gc, gs)
+        B.moe_grouped_gemm_gateup_dgrad_mxfp8(d, gc, gs, w_gd, s_gd, b.offsets, b.dx_perm)
+        B.moe_grouped_gemm_gateup_wgrad(d, b.x_perm, b.dgu, b.offsets, b.dw_gate, b.dw_up)
+        B.moe_permute_bwd(d, b.dx_perm, b.pair_to_row, b.dx)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        n = max(3, int(math.ceil(min_seconds * 1e3 / max(e0.elapsed_time(e1), 1e-3))))
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    quantise_weights()
+    ms_out = timed(step)
+    y_fp8, dx_fp8 = b.y.clone(), b.dx.clone()
+
+    def step_with_weights():
+        quantise_weights()
+        step()
+
+    ms_in = timed(step_with_weights)
+    # leave the buffers as the bf16 step leaves them, and measure the distance of the FP8 step's results from them
+    make_step(B, b, wl)()
+    torch.cuda.synchronize()
+    if B.moe_device_status() != 0:
+        raise RuntimeError("device status word is set after the FP8 step")
+    rel = lambda a, r: float((a.float() - r.float()).norm() / r.float().norm())
+    return {"ms_per_step_weights_quantised_outside": ms_out, "ms_per_step_weights_quantised_every_step": ms_in,
+            "bf16_ms_per_step": res["total_ms"] / res["steps"], "gpu_launches_per_step": 16,
+            "rel_frobenius_to_bf16_step": {"Y": rel(y_fp8, b.y), "dX": rel(dx_fp8, b.dx)},
+            "note": "15 library calls (permute is two launches); the three activation quantisers and the forward SwiGLU are "
+                    "separate HBM-bound launches here"}
+
+
 def time_mxfp8(B, cfg, res, device, reps=20, min_seconds=0.3, warm=3):
     """The block-scaled FP8 twins of the four row-ragged GEMMs -- down forward, down dgrad, gate/up dgrad, gate/up
     forward (with its activation call) -- on this workload's own activations, weights and offsets: per GEMM the activation quantiser, the weight quantiser (once per optimizer step in training) and the GEMM,
@@ -740,6 +824,8 @@ def run_ours(args):
                "per_call_ms": {k: round(v, 5) for k, v in res["per_call_ms"].items()}}
         if args.with_mxfp8:
             out["mxfp8"] = time_mxfp8(B, cfg, res, device, reps=1, min_seconds=0.0, warm=0)
+            if args.fp8_step:
+                out["fp8_step"] = time_fp8_step(B, cfg, res, device, min_seconds=0.3)
         print(json.dumps(out), flush=True)
         return
     res = time_config(B, cfg, device, args.steps, args.warmup, dist, min_seconds=args.min_seconds)
@@ -792,6 +878,7 @@ def run_ours(args):
         line["stream_calibration_in_step"] = stream_calibration_in_step(B, cfg, res, device)
         line["fused_dgrad_swiglu_bwd"] = time_fused_variant(B, cfg, res, device)
         line["mxfp8"] = time_mxfp8(B, cfg, res, device)
+        line["fp8_step"] = time_fp8_step(B, cfg, res, device)
         del res
         torch.cuda.empty_cache()
         for name in args.also:
@@ -802,6 +889,7 @@ def run_ours(args):
             extra.append(summarize(c2, r2, peaks, peaks_kind, sms))
             extra[-1]["fused_dgrad_swiglu_bwd"] = time_fused_variant(B, c2, r2, device, seconds=0.5)
             extra[-1]["mxfp8"] = time_mxfp8(B, c2, r2, device)
+            extra[-1]["fp8_step"] = time_fp8_step(B, c2, r2, device, min_seconds=0.3)
             del r2
             torch.cuda.empty_cache()
         if extra:
@@ -845,6 +933,7 @@ def main():
     ap.add_argument("--only-steps", action="store_true", help="profiling runs: warm-up and timed steps only")
     ap.add_argument("--fused", action="store_true", help="with --only-steps: the step form with the fused down-dgrad + SwiGLU-backward call")
     ap.add_argument("--with-mxfp8", action="store_true", help="with --only-steps: also run the block-scaled FP8 calls")
+    ap.add_argument("--fp8-step", action="store_true", help="with --only-steps --with-mxfp8: also time the FP8 form of the step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     args.also = [s for s in args.also.split(",") if s]
