@@ -186,6 +186,91 @@ def test_mxfp8_down_sampled_rows(full):
     assert torch.equal(yq, first)
 
 
+def test_mxfp8_other_gemms_sampled_rows(full):
+    """The other three block-scaled FP8 GEMMs at full size -- gate/up forward (with the SwiGLU call), down dgrad,
+    gate/up dgrad -- on sampled rows (first and last row of 4 experts + 4 inside each) against the exact products of the
+    dequantised operands; the oracle quantises the sampled rows and those experts' weights only."""
+    cfg, dev, b = full
+    if cfg.H % 128 or cfg.I % 128:
+        pytest.skip("the block-scaled path takes widths that are multiples of 128")
+    from paper_2606_26453_b200 import binding as B
+    d = b.d
+    R, E, H, I = cfg.R, cfg.E, cfg.H, cfg.I
+    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    nan = lambda *shape: torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    offsets = b.offsets.cpu().numpy()
+    rng = np.random.default_rng(cfg.cfg_id + 11)
+    nonempty = np.flatnonzero(np.diff(offsets) > 0)
+    experts = rng.choice(nonempty, size=min(4, nonempty.size), replace=False)
+    rows = []
+    for e in experts:
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        rows += [lo, hi - 1] + list(rng.integers(lo, hi, size=4))
+    rows = np.array(sorted(set(rows)))
+    expert_of = np.searchsorted(offsets, rows, side="right") - 1
+    rsel = torch.from_numpy(rows).cuda()
+    wg = {int(e): f32(dev["W_gate"][int(e)]) for e in experts}
+    wu = {int(e): f32(dev["W_up"][int(e)]) for e in experts}
+    wd = {int(e): f32(dev["W_down"][int(e)]) for e in experts}
+
+    # gate/up forward: GU rows, then H_act and its codes from the CUDA side's own GU
+    xc, xs = u8(R * H), u8(B.moe_mxfp8_x_scale_bytes(d))
+    tc, ts = u8(E * 2 * I * H), u8(B.moe_mxfp8_w_gateup_scale_bytes(d))
+    gu = nan(R, 2 * I)
+    B.moe_mxfp8_quantize_x_perm(d, b.x_perm, xc, xs)
+    B.moe_mxfp8_quantize_w_gateup(d, dev["W_gate"], dev["W_up"], tc, ts)
+    B.moe_grouped_gemm_gateup_mxfp8(d, xc, xs, tc, ts, b.offsets, gu)
+    h, hc, hs = nan(R, I), u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
+    B.moe_swiglu_mxfp8(d, gu, h, hc, hs)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0 and not bool(torch.isnan(gu).any()) and not bool(torch.isnan(h).any())
+    x_deq = O.mxfp8_quantize(f32(b.x_perm[rsel]))[2]
+    want = np.empty((rows.size, 2 * I))
+    for e in experts:
+        sel = expert_of == e
+        g_deq = O.mxfp8_quantize(wg[int(e)].T)[2]                # [I, H]: every gate feature's scales along H
+        u_deq = O.mxfp8_quantize(wu[int(e)].T)[2]
+        want[sel] = np.concatenate([x_deq[sel] @ g_deq.T, x_deq[sel] @ u_deq.T], axis=1)
+    Hh.assert_close(Hh.to_np64(gu[rsel]), want, f"{cfg.name}: GU rows (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    Hh.assert_close(Hh.to_np64(h[rsel]), O.swiglu_fwd(Hh.to_np64(gu[rsel])), f"{cfg.name}: H_act rows from GU",
+                    rel_fro=Hh.PER_CALL_FROBENIUS)
+    assert np.array_equal(hc.view(R, I)[rsel].cpu().numpy(), O.mxfp8_quantize(Hh.to_np64(h[rsel]))[0])
+    del xc, xs, tc, ts, gu, h, hc, hs
+
+    # down dgrad
+    dc, ds = u8(R * H), u8(B.moe_mxfp8_dy_scale_bytes(d))
+    vc, vs = u8(E * I * H), u8(B.moe_mxfp8_w_down_dgrad_scale_bytes(d))
+    dh = nan(R, I)
+    B.moe_mxfp8_quantize_dy_perm(d, b.dy_perm, dc, ds)
+    B.moe_mxfp8_quantize_w_down_dgrad(d, dev["W_down"], vc, vs)
+    B.moe_grouped_gemm_down_dgrad_mxfp8(d, dc, ds, vc, vs, b.offsets, dh)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0 and not bool(torch.isnan(dh).any())
+    dy_deq = O.mxfp8_quantize(f32(b.dy_perm[rsel]))[2]
+    want = np.empty((rows.size, I))
+    for e in experts:
+        sel = expert_of == e
+        want[sel] = dy_deq[sel] @ O.mxfp8_quantize(wd[int(e)])[2].T     # [I, H] as it lies
+    Hh.assert_close(Hh.to_np64(dh[rsel]), want, f"{cfg.name}: dH_act rows (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    del dc, ds, vc, vs, dh
+
+    # gate/up dgrad
+    gc, gs = u8(R * 2 * I), u8(B.moe_mxfp8_dgu_scale_bytes(d))
+    uc, us = u8(E * H * 2 * I), u8(B.moe_mxfp8_w_gateup_dgrad_scale_bytes(d))
+    dx = nan(R, H)
+    B.moe_mxfp8_quantize_dgu(d, b.dgu, gc, gs)
+    B.moe_mxfp8_quantize_w_gateup_dgrad(d, dev["W_gate"], dev["W_up"], uc, us)
+    B.moe_grouped_gemm_gateup_dgrad_mxfp8(d, gc, gs, uc, us, b.offsets, dx)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0 and not bool(torch.isnan(dx).any())
+    dgu_deq = O.mxfp8_quantize(f32(b.dgu[rsel]))[2]
+    want = np.empty((rows.size, H))
+    for e in experts:
+        sel = expert_of == e
+        want[sel] = dgu_deq[sel, :I] @ O.mxfp8_quantize(wg[int(e)])[2].T + dgu_deq[sel, I:] @ O.mxfp8_quantize(wu[int(e)])[2].T
+    Hh.assert_close(Hh.to_np64(dx[rsel]), want, f"{cfg.name}: dX_perm rows (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+
+
 # ------------------------------------------------------------------------------------------------
 # every element of every output, where the oracle can afford the whole layer (about 15 s and 45 s of host time)
 # ------------------------------------------------------------------------------------------------
