@@ -40,6 +40,15 @@ namespace moe {
 
 __device__ int g_mx_status = 0;
 
+#ifdef MOE_TEST_HOOKS
+// Test-only build: when set, every producer leaves out the loads and the barrier arrival of its first ring stage, so that
+// the bounded waits on that stage run out (see grouped_gemm.cu).
+__device__ int g_mx_test_withhold_first_stage = 0;
+extern "C" int moe_test_withhold_first_stage_mxfp8(int on) {
+    return cudaMemcpyToSymbol(g_mx_test_withhold_first_stage, &on, sizeof(int)) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+#endif
+
 int mx_read_and_clear_status(int* status_out) {
     int v = 0, zero = 0;
     if (cudaMemcpyFromSymbol(&v, g_mx_status, sizeof(int)) != cudaSuccess) return MOE_ERR_CUDA;
@@ -86,6 +95,8 @@ struct MxParams {
     long long ldo;
 };
 
+// (roles in which a whole warp waits take the verdict through __all_sync: a wait that runs out for one lane while the
+// barrier completes for another must not split the warp ahead of a warp-wide instruction)
 __device__ __forceinline__ bool mx_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     return mbar_wait_status(bar, parity, abort_flag, &g_mx_status);
 }
@@ -195,6 +206,13 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint8_t* sb_tile = p.sb + ((long long)tl.e * p.n_tiles + tl.n0 / MX_BN) * p.k_tiles * MX_SF_BYTES;
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
                     if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+#ifdef MOE_TEST_HOOKS
+                    if (g_mx_test_withhold_first_stage != 0 && issued == 0) {
+                        ++issued;
+                        if (++stage == MX_STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
+#endif
                     const uint32_t full = smem_u32(&ctl->full[stage]);
                     const uint32_t a_dst = stage_base(stage);
                     mbar_arrive_expect_tx(full, MX_A_BYTES + MX_B_BYTES + MX_SF_BYTES);
@@ -282,7 +300,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (kt >= p.k_tiles) break;
                     const uint4 cur = q[i];
                     if (kt + MX_SCALE_AHEAD < p.k_tiles) q[i] = load_slice(kt + MX_SCALE_AHEAD);
-                    if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag))) { ok = false; break; }
                     *reinterpret_cast<uint4*>(tiles_ptr + stage * MX_STAGE_BYTES + MX_A_BYTES + MX_B_BYTES + lane * 16) = cur;
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
@@ -299,7 +317,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t n_stores = 0, acc = 0, acc_phase = 0;
         for (long long t = blockIdx.x; t < n_tiles_total; t += gridDim.x) {
             const MxTile tl = mx_decode(p, ctl, t);
-            if (!mx_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag)) break;
+            if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag))) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + acc * MX_BN + ((uint32_t)(quarter * 32) << 16);
             const int slab0 = tl.row0 + quarter * 32;
@@ -535,6 +553,13 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 const int b_row = tl.e * p.n_cols + tl.n0 + (int)rank * (tl.width >> 1);
                 for (int kt = 0; kt < p.k_tiles; ++kt) {
                     if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+#ifdef MOE_TEST_HOOKS
+                    if (g_mx_test_withhold_first_stage != 0 && issued == 0) {
+                        ++issued;
+                        if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
+#endif
                     if (rank == 0) ctl->stage_n[stage] = tl.width;   // read by the MMA thread after its wait on full[stage]
                     const uint32_t bar = full0 + stage * (uint32_t)sizeof(unsigned long long);
                     const uint32_t dst = tiles_base + stage * MXP_STAGE_BYTES;
@@ -624,7 +649,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     if (kt >= p.k_tiles) break;
                     const uint4 cur = q[i];
                     if (kt + MX_SCALE_AHEAD < p.k_tiles) q[i] = load_slice(kt + MX_SCALE_AHEAD);
-                    if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag))) { ok = false; break; }
                     *reinterpret_cast<uint4*>(tiles_ptr + stage * MXP_STAGE_BYTES + MXP_SFA_OFF + lane * 16) = cur;
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
@@ -671,7 +696,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         uint32_t n_stores = 0, acc = 0, acc_phase = 0;
         for (long long t = first_tile; t < n_tiles_total; t += tile_stride) {
             const MxPairTile tl = mxp_decode(p, ctl, t);
-            if (!mx_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag)) break;
+            if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag))) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + acc * MXP_ACC_STRIDE + ((uint32_t)(quarter * 32) << 16);
             const int slab0 = tl.row0 + (int)rank * MX_BM + quarter * 32;
