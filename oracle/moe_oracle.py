@@ -424,3 +424,25 @@ def swiglu_fwd(GU):
     I = GU.shape[1] // 2
     g, u = GU[:, :I], GU[:, I:]
     return g / (1.0 + np.exp(-g)) * u
+
+
+def wgrad_mxfp8(A_rows, B_rows, offsets):
+    """A weight gradient with block-scaled FP8 operands along ITS contraction, the packed rows of each expert:
+    dW[e] = Q(A_e)^T @ Q(B_e) with A_e = A_rows[offsets[e]:offsets[e+1], :] ([n_e, M]) and B_e likewise ([n_e, N]), where Q
+    quantises every COLUMN in blocks of 32 consecutive rows counted from the expert's first row (a block never holds
+    rows of two experts; the expert's last block may be short and is scaled by the rows it has).  The product of the
+    dequantised operands is taken exactly; an expert without rows gives zeros.  Returns dW [E, M, N] float64.
+    (down projection: A = H_act, B = dY_perm; gate/up projection: A = X_perm, B = dGU, dW = [dW_gate | dW_up].)"""
+    A, B = _f64(A_rows), _f64(B_rows)
+    E = len(offsets) - 1
+    out = np.zeros((E, A.shape[1], B.shape[1]), dtype=F64)
+    for e in range(E):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        n = hi - lo
+        if n == 0:
+            continue
+        pad = (-n) % MX_BLOCK
+        at = np.concatenate([A[lo:hi].T, np.zeros((A.shape[1], pad))], axis=1)       # [M, n + pad]: contraction last
+        bt = np.concatenate([B[lo:hi].T, np.zeros((B.shape[1], pad))], axis=1)
+        out[e] = mxfp8_quantize(at)[2] @ mxfp8_quantize(bt)[2].T
+    return out

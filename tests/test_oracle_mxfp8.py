@@ -192,3 +192,42 @@ def test_gateup_mxfp8_is_the_exact_product_of_the_dequantised_operands_and_swigl
     assert np.allclose(O.swiglu_fwd(np.array([[0.0, 2.0, -2.0, 5.0, 7.0, 7.0]])), [[0.0, 2.0 / (1 + np.exp(-2.0)) * 7.0, -2.0 / (1 + np.exp(2.0)) * 7.0]])
     t = torch.tensor(gu_ref)
     assert np.allclose(O.swiglu_fwd(gu_ref), (torch.nn.functional.silu(t[:, :I]) * t[:, I:]).numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_wgrad_mxfp8_quantises_columns_in_expert_aligned_row_blocks():
+    rng = np.random.default_rng(7)
+    E, M, N = 4, 6, 5
+    counts = [40, 0, 32, 7]                       # a short last block, an empty expert, a whole block, less than a block
+    offsets = np.concatenate([[0], np.cumsum(counts)])
+    R = int(offsets[-1])
+    A = rng.standard_normal((R, M)) * np.exp2(rng.integers(-6, 6, size=(R, 1)))     # rows of very different size
+    B = rng.standard_normal((R, N))
+    got = O.wgrad_mxfp8(A, B, offsets)
+    assert got.shape == (E, M, N) and not got[1].any()
+    # by hand: expert 0 has the row blocks [0,32) and [32,40); expert 3 the block [72,79)
+    def col(x, lo, hi):                            # one column segment quantised as its own (zero-padded) block
+        seg = np.zeros(32)
+        seg[:hi - lo] = x[lo:hi]
+        return O.mxfp8_quantize(seg)[2][:hi - lo]
+    for (e, blocks) in ((0, [(0, 32), (32, 40)]), (2, [(40, 72)]), (3, [(72, 79)])):
+        for m in (0, 5):
+            for n in (0, 4):
+                want = sum(float(col(A[:, m], lo, hi) @ col(B[:, n], lo, hi)) for lo, hi in blocks)
+                assert abs(got[e, m, n] - want) <= 1e-10
+    # against the unquantised weight gradient (the bf16 path's own pinned oracle): a few per cent; equal for representable data
+    ref = O.down_bwd(B, A, np.zeros((E, M, N)), offsets)[1]          # dWd[e] = Hact_e^T dYp_e with Hact = A, dYp = B
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert 0.01 < rel < 0.08
+    Aq, Bq = np.zeros_like(A), np.zeros_like(B)
+    for e in range(E):                             # make both operands representable in the same blocks
+        lo, hi = offsets[e], offsets[e + 1]
+        for b0 in range(lo, hi, 32):
+            b1 = min(b0 + 32, hi)
+            for x, xq in ((A, Aq), (B, Bq)):
+                for c in range(x.shape[1]):
+                    xq[b0:b1, c] = col(x[:, c], b0, b1)
+    assert np.allclose(O.wgrad_mxfp8(Aq, Bq, offsets), O.down_bwd(Bq, Aq, np.zeros((E, M, N)), offsets)[1], rtol=0, atol=1e-12)
+    # the blocks are counted from the expert's first row, not from row 0 of the packed array: moving all rows by 8 changes nothing
+    shifted = np.concatenate([[0], np.cumsum([40, 0, 32, 7])])
+    A2, B2 = np.concatenate([np.zeros((8, M)), A]), np.concatenate([np.zeros((8, N)), B])     # same rows, moved by 8
+    assert np.allclose(O.wgrad_mxfp8(A2, B2, shifted + 8)[[0, 2, 3]], got[[0, 2, 3]])
