@@ -286,8 +286,9 @@ def time_fp8_step(B, cfg, res, device, min_seconds=0.5):
 
 
 def time_mxfp8(B, cfg, res, device, reps=20, min_seconds=0.3, warm=3):
-    """The block-scaled FP8 twins of the four row-ragged GEMMs -- down forward, down dgrad, gate/up dgrad, gate/up
-    forward (with its activation call) -- on this workload's own activations, weights and offsets: per GEMM the activation quantiser, the weight quantiser (once per optimizer step in training) and the GEMM,
+    """The block-scaled FP8 twins of the six grouped GEMMs -- down forward, down dgrad, gate/up dgrad, gate/up forward
+    (with its activation call), and the two weight gradients (both operands are activations there: `quantize_act_ms`
+    covers both, `quantize_w_ms` is empty) -- on this workload's own activations, weights and offsets: per GEMM the activation quantiser, the weight quantiser (once per optimizer step in training) and the GEMM,
     each timed alone (back to back for at least `min_seconds`, events), beside the bf16 call timed the same way."""
     if cfg.H % 128 or cfg.I % 128:
         return None
@@ -365,6 +366,35 @@ def time_mxfp8(B, cfg, res, device, reps=20, min_seconds=0.3, warm=3):
                                gateup_fp8, hq, h_ref)
     out["gateup_swiglu"]["fp8_gemm_ms"] = timed(lambda: B.moe_grouped_gemm_gateup_mxfp8(d, xc, xs, tc, ts, b.offsets, guq))
     out["gateup_swiglu"]["swiglu_and_quantize_ms"] = timed(lambda: B.moe_swiglu_mxfp8(d, guq, hq, hc, hs))
+    del xc, xs, tc, ts, hc, hs, guq, hq, h_ref, gu_ref
+    # the two weight gradients: operands quantised along the token axis (both are activations: no per-optimizer-step part)
+    tok = lambda n: (u8(B.moe_mxfp8_tokens_codes_bytes(d, n)), u8(B.moe_mxfp8_tokens_scale_bytes(d, n)))
+    (ac, asc), (bc, bsc) = tok(I), tok(H)
+    dwq, dw_ref = torch.empty_like(b.dw_down), torch.empty_like(b.dw_down)
+
+    def q_down_wgrad():
+        B.moe_mxfp8_quantize_tokens(d, b.h_act, I, 0, I, b.offsets, ac, asc)
+        B.moe_mxfp8_quantize_tokens(d, b.dy_perm, H, 0, H, b.offsets, bc, bsc)
+
+    out["down_wgrad"] = leg(2.0 * R * H * I,
+                            lambda: B.moe_grouped_gemm_down_wgrad(d, b.h_act, b.dy_perm, b.offsets, dw_ref),
+                            q_down_wgrad, lambda: None,
+                            lambda: B.moe_grouped_gemm_down_wgrad_mxfp8(d, ac, asc, bc, bsc, dwq), dwq, dw_ref)
+    del ac, asc, bc, bsc, dwq, dw_ref
+    (xc, xs), (gc, gs), (uc, us) = tok(H), tok(I), tok(I)
+    dgq, duq = torch.empty_like(b.dw_gate), torch.empty_like(b.dw_up)
+    dg_ref, du_ref = torch.empty_like(b.dw_gate), torch.empty_like(b.dw_up)
+
+    def q_gateup_wgrad():
+        B.moe_mxfp8_quantize_tokens(d, b.x_perm, H, 0, H, b.offsets, xc, xs)
+        B.moe_mxfp8_quantize_tokens(d, b.dgu, 2 * I, 0, I, b.offsets, gc, gs)
+        B.moe_mxfp8_quantize_tokens(d, b.dgu, 2 * I, I, I, b.offsets, uc, us)
+
+    out["gateup_wgrad"] = leg(4.0 * R * H * I,
+                              lambda: B.moe_grouped_gemm_gateup_wgrad(d, b.x_perm, b.dgu, b.offsets, dg_ref, du_ref),
+                              q_gateup_wgrad, lambda: None,
+                              lambda: B.moe_grouped_gemm_gateup_wgrad_mxfp8(d, xc, xs, gc, gs, uc, us, dgq, duq), dgq, dg_ref)
+    del xc, xs, gc, gs, uc, us, dgq, duq, dg_ref, du_ref
     out["note"] = ("E4M3 elements, E8M0 scale per 32 along the contraction; tcgen05.mma kind::mxf8f6f4.block_scale on "
                    "256 x 208 CTA-pair tiles from 256 rows per expert on average, 128 x 128 single-CTA tiles below; "
                    "the bf16 twins run 256 x 256 CTA-pair tiles; the FP8 gate/up time is the GEMM plus the activation call, "

@@ -317,6 +317,36 @@ int moe_grouped_gemm_gateup_mxfp8(const moe_dims_t* dims, const void* x_codes, c
 int moe_swiglu_mxfp8(const moe_dims_t* dims, const void* gu, void* h_act, void* h_codes, void* h_scales,
                      moe_stream_t stream);
 
+/* The two weight gradients, whose contraction runs over the packed rows of each expert (the paper's dW1 kernel is the
+ * bf16 form of the second; its section "Production Validation: VeOmni MoE" defines dW1_e = X_e^T G_e): both operands are
+ * quantised along the TOKEN axis, every column in blocks of 32 consecutive rows counted from the expert's first row (a
+ * block never holds rows of two experts; an expert's last block may be short), and stored transposed and padded:
+ *   moe_mxfp8_quantize_tokens  columns [col0, col0 + n_features) of x [R, ld] bf16 (ld, col0 multiples of 8; n_features a
+ *                              multiple of 128) -> codes_t [n_features, P] bytes with P = roundup(R,128) + 128*E:
+ *                              column slice_prefix[e]*128 + i holds row offsets[e] + i, each expert's columns padded with
+ *                              zero codes to a multiple of 128 (columns after the last expert's are not written);
+ *                              scales (moe_mxfp8_tokens_scale_bytes): slice_prefix[E+1] as int32 in the first 8192
+ *                              bytes, then the scale bytes as [P/128][n_features][4], then again tiled per 208 features
+ *                              [ceil(n/208)][P/128][1024] for use as the N-side operand.  Two launches.
+ *   moe_grouped_gemm_down_wgrad_mxfp8    dw_down [E,I,H] bf16 = Q(h_act)^T Q(dy_perm) per expert, from the token-
+ *                              quantised h_act (n_features = I) and dy_perm (n_features = H).
+ *   moe_grouped_gemm_gateup_wgrad_mxfp8  dw_gate, dw_up [E,H,I] bf16 from the token-quantised x_perm (n_features = H)
+ *                              and the two halves of dgu quantised separately (col0 = 0 and col0 = I, n_features = I,
+ *                              ld = 2I).  Two launches.
+ * Every expert's gradient is written, zeros for an expert without rows.  The row counts come from the slice_prefix in
+ * the first operand's scales (the offsets the quantiser was given).  Same requirements, status codes and tolerance
+ * statement as the other block-scaled calls. */
+size_t moe_mxfp8_tokens_codes_bytes(const moe_dims_t* dims, int n_features);
+size_t moe_mxfp8_tokens_scale_bytes(const moe_dims_t* dims, int n_features);
+int moe_mxfp8_quantize_tokens(const moe_dims_t* dims, const void* x, int ld, int col0, int n_features,
+                              const int32_t* offsets, void* codes_t, void* scales, moe_stream_t stream);
+int moe_grouped_gemm_down_wgrad_mxfp8(const moe_dims_t* dims, const void* h_codes_t, const void* h_scales,
+                                      const void* dy_codes_t, const void* dy_scales, void* dw_down,
+                                      moe_stream_t stream);
+int moe_grouped_gemm_gateup_wgrad_mxfp8(const moe_dims_t* dims, const void* x_codes_t, const void* x_scales,
+                                        const void* dg_codes_t, const void* dg_scales, const void* du_codes_t,
+                                        const void* du_scales, void* dw_gate, void* dw_up, moe_stream_t stream);
+
 /* ---- whole layer from HOST activations ------------------------------------------------------
  * One training step of the layer for a caller whose per-step tensors live in host memory:
  * copies x, topk_idx, topk_w, dy (HOST pointers; pinned memory makes the copies asynchronous)

@@ -31,6 +31,8 @@ EXPORTS = [
     "moe_mxfp8_quantize_w_gateup_dgrad", "moe_grouped_gemm_gateup_dgrad_mxfp8",
     "moe_mxfp8_x_scale_bytes", "moe_mxfp8_w_gateup_scale_bytes", "moe_mxfp8_quantize_x_perm", "moe_mxfp8_quantize_w_gateup",
     "moe_grouped_gemm_gateup_mxfp8", "moe_swiglu_mxfp8",
+    "moe_mxfp8_tokens_codes_bytes", "moe_mxfp8_tokens_scale_bytes", "moe_mxfp8_quantize_tokens",
+    "moe_grouped_gemm_down_wgrad_mxfp8", "moe_grouped_gemm_gateup_wgrad_mxfp8",
 ]
 
 
@@ -66,6 +68,9 @@ def load_library() -> ctypes.CDLL:
                      "moe_mxfp8_w_gateup_dgrad_scale_bytes", "moe_mxfp8_x_scale_bytes", "moe_mxfp8_w_gateup_scale_bytes"):
             getattr(lib, name).restype = ctypes.c_size_t
             getattr(lib, name).argtypes = [ctypes.POINTER(MoeDims)]
+        for name in ("moe_mxfp8_tokens_codes_bytes", "moe_mxfp8_tokens_scale_bytes"):
+            getattr(lib, name).restype = ctypes.c_size_t
+            getattr(lib, name).argtypes = [ctypes.POINTER(MoeDims), ctypes.c_int]
         lib.moe_device_status.restype = ctypes.c_int
         lib.moe_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
         p = ctypes.c_void_p
@@ -102,6 +107,9 @@ def load_library() -> ctypes.CDLL:
             "moe_mxfp8_quantize_w_gateup": [dp, p, p, p, p, p],
             "moe_grouped_gemm_gateup_mxfp8": [dp, p, p, p, p, p, p, p],
             "moe_swiglu_mxfp8": [dp, p, p, p, p, p],
+            "moe_mxfp8_quantize_tokens": [dp, p, ctypes.c_int, ctypes.c_int, ctypes.c_int, p, p, p, p],
+            "moe_grouped_gemm_down_wgrad_mxfp8": [dp, p, p, p, p, p, p],
+            "moe_grouped_gemm_gateup_wgrad_mxfp8": [dp, p, p, p, p, p, p, p, p, p],
         }
         for name, argtypes in sigs.items():
             fn = getattr(lib, name)
@@ -323,6 +331,29 @@ def moe_grouped_gemm_gateup_mxfp8(d, x_codes, x_scales, w_codes_t, w_scales, off
 
 def moe_swiglu_mxfp8(d, gu, h_act, h_codes, h_scales):
     _call("moe_swiglu_mxfp8", ctypes.byref(d), _ptr(gu), _ptr(h_act), _ptr(h_codes), _ptr(h_scales), _stream())
+
+
+def moe_mxfp8_tokens_codes_bytes(d: MoeDims, n_features: int) -> int:
+    return int(load_library().moe_mxfp8_tokens_codes_bytes(ctypes.byref(d), int(n_features)))
+
+
+def moe_mxfp8_tokens_scale_bytes(d: MoeDims, n_features: int) -> int:
+    return int(load_library().moe_mxfp8_tokens_scale_bytes(ctypes.byref(d), int(n_features)))
+
+
+def moe_mxfp8_quantize_tokens(d, x, ld, col0, n_features, offsets, codes_t, scales):
+    _call("moe_mxfp8_quantize_tokens", ctypes.byref(d), _ptr(x), int(ld), int(col0), int(n_features), _ptr(offsets),
+          _ptr(codes_t), _ptr(scales), _stream())
+
+
+def moe_grouped_gemm_down_wgrad_mxfp8(d, h_codes_t, h_scales, dy_codes_t, dy_scales, dw_down):
+    _call("moe_grouped_gemm_down_wgrad_mxfp8", ctypes.byref(d), _ptr(h_codes_t), _ptr(h_scales), _ptr(dy_codes_t),
+          _ptr(dy_scales), _ptr(dw_down), _stream())
+
+
+def moe_grouped_gemm_gateup_wgrad_mxfp8(d, x_codes_t, x_scales, dg_codes_t, dg_scales, du_codes_t, du_scales, dw_gate, dw_up):
+    _call("moe_grouped_gemm_gateup_wgrad_mxfp8", ctypes.byref(d), _ptr(x_codes_t), _ptr(x_scales), _ptr(dg_codes_t),
+          _ptr(dg_scales), _ptr(du_codes_t), _ptr(du_scales), _ptr(dw_gate), _ptr(dw_up), _stream())
 
 
 def moe_layer_fwd_bwd_host(d, x_host, topk_idx_host, topk_w_host, dy_host, w_gate, w_up, w_down, y_host, dx_host,

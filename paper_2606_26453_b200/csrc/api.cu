@@ -460,6 +460,66 @@ int moe_swiglu_mxfp8(const moe_dims_t* dims, const void* gu, void* h_act, void* 
                                      static_cast<uint8_t*>(h_scales), st(stream));
 }
 
+// ---- block-scaled FP8 weight gradients (contraction over the packed rows of each expert) ----
+static int check_tokens_args(const moe_dims_t* d, int n_features) {
+    const int s = check_mx_dims(d);
+    if (s != MOE_OK) return s;
+    return (n_features <= 0 || n_features % 128 != 0) ? MOE_ERR_UNSUPPORTED_SHAPE : MOE_OK;
+}
+
+size_t moe_mxfp8_tokens_codes_bytes(const moe_dims_t* dims, int n_features) {
+    if (check_tokens_args(dims, n_features) != MOE_OK) return 0;
+    return (size_t)n_features * (size_t)mx_tokens_pitch((long long)dims->T * dims->K, dims->E);
+}
+
+size_t moe_mxfp8_tokens_scale_bytes(const moe_dims_t* dims, int n_features) {
+    if (check_tokens_args(dims, n_features) != MOE_OK) return 0;
+    return mx_tokens_scale_bytes((long long)dims->T * dims->K, dims->E, n_features);
+}
+
+int moe_mxfp8_quantize_tokens(const moe_dims_t* dims, const void* x, int ld, int col0, int n_features, const int32_t* offsets,
+                              void* codes_t, void* scales, moe_stream_t stream) {
+    int s = check_tokens_args(dims, n_features);
+    if (s != MOE_OK) return s;
+    if (ld <= 0 || col0 < 0 || col0 % 8 != 0 || ld % 8 != 0 || col0 + n_features > ld) return MOE_ERR_DIMS;
+    const void* const req[] = {x, offsets, codes_t, scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_quantize_tokens((long long)dims->T * dims->K, dims->E, cb(x), ld, col0, n_features, offsets,
+                                     static_cast<uint8_t*>(codes_t), static_cast<uint8_t*>(scales), st(stream));
+}
+
+int moe_grouped_gemm_down_wgrad_mxfp8(const moe_dims_t* dims, const void* h_codes_t, const void* h_scales, const void* dy_codes_t,
+                                      const void* dy_scales, void* dw_down, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {h_codes_t, h_scales, dy_codes_t, dy_scales, dw_down};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_wgrad((long long)dims->T * dims->K, dims->E, dims->I, dims->H, static_cast<const uint8_t*>(h_codes_t),
+                           static_cast<const uint8_t*>(h_scales), static_cast<const uint8_t*>(dy_codes_t),
+                           static_cast<const uint8_t*>(dy_scales), mb(dw_down), st(stream));
+}
+
+int moe_grouped_gemm_gateup_wgrad_mxfp8(const moe_dims_t* dims, const void* x_codes_t, const void* x_scales,
+                                        const void* dg_codes_t, const void* dg_scales, const void* du_codes_t,
+                                        const void* du_scales, void* dw_gate, void* dw_up, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {x_codes_t, x_scales, dg_codes_t, dg_scales, du_codes_t, du_scales, dw_gate, dw_up};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    const long long R = (long long)dims->T * dims->K;
+    s = launch_mx_wgrad(R, dims->E, dims->H, dims->I, static_cast<const uint8_t*>(x_codes_t), static_cast<const uint8_t*>(x_scales),
+                        static_cast<const uint8_t*>(dg_codes_t), static_cast<const uint8_t*>(dg_scales), mb(dw_gate), st(stream));
+    if (s != MOE_OK) return s;
+    return launch_mx_wgrad(R, dims->E, dims->H, dims->I, static_cast<const uint8_t*>(x_codes_t), static_cast<const uint8_t*>(x_scales),
+                           static_cast<const uint8_t*>(du_codes_t), static_cast<const uint8_t*>(du_scales), mb(dw_up), st(stream));
+}
+
 // Arena layout of moe_layer_fwd_bwd_host (every block 256-byte aligned).
 namespace {
 // Two side streams (uploads, downloads) and a few events per device for moe_layer_fwd_bwd_host, created on first

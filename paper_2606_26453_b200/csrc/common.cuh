@@ -65,6 +65,12 @@ int launch_mx_quantize_w_transposed(int E, int k, int n, int n_total, int n_off,
                                     cudaStream_t s);
 int launch_mx_quantize_w_rows(int E, int n_feat, int k, int k_total, int k_off, const bf16* w, uint8_t* codes, uint8_t* scales,
                               cudaStream_t s);
+long long mx_tokens_pitch(long long R, int E);            // columns of a token-quantised (transposed) operand
+size_t mx_tokens_scale_bytes(long long R, int E, int n);
+int launch_mx_quantize_tokens(long long R, int E, const bf16* x, long long ld, int col0, int n, const int32_t* offsets,
+                              uint8_t* codes_t, uint8_t* scales, cudaStream_t s);
+int launch_mx_wgrad(long long R, int E, int M, int N, const uint8_t* a_codes_t, const uint8_t* a_scales, const uint8_t* b_codes_t,
+                    const uint8_t* b_scales, bf16* dw, cudaStream_t s);
 int launch_mx_swiglu_quantize(long long rows, int I, const bf16* gu, bf16* h_act, uint8_t* codes, uint8_t* scales, cudaStream_t s);
 int launch_mx_gemm(long long R, int E, int n_feat, int k, const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
                    const uint8_t* b_scales, const int32_t* offsets, bf16* out, cudaStream_t s);

@@ -764,6 +764,340 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     }
 }
 
+// ---- weight gradients on the pair kernel's machinery ------------------------------------------------------
+// dW[e] [M, N] = Q(A_e)^T Q(B_e) over the rows of expert e, both operands quantised along the token axis in blocks of 32
+// rows counted from the expert's first row and stored TRANSPOSED, contraction contiguous: codes [features, pitch] where
+// column slice_prefix[e] * 128 + i holds row offsets[e] + i of the packed tensor and every expert's columns are padded
+// with zero codes to a multiple of 128 -- so a K slice of 128 columns belongs to exactly one expert, both operands are
+// K-major like everywhere else in this file, and the ragged contraction needs no clearing of foreign rows in shared
+// memory.  The tile list is fixed (every expert x M tiles x N tiles); an expert's K slices are
+// [slice_prefix[e], slice_prefix[e+1]); a tile of an expert without rows skips the pipeline and its epilogue writes zeros.
+struct MxWgradCtl {
+    unsigned long long full[MXP_STAGES];
+    unsigned long long sf_full[MXP_STAGES];
+    unsigned long long empty[MXP_STAGES];
+    unsigned long long tmem_full[2];
+    unsigned long long tmem_empty[2];
+    unsigned long long drain;
+    unsigned long long drain_copy;
+    uint32_t tmem_base;
+    int abort_flag;
+    int stage_n[MXP_STAGES];
+    int32_t sp[MX_MAX_E + 1];   // slice_prefix
+};
+constexpr int MXW_SMEM_BYTES = MXP_STAGES * MXP_STAGE_BYTES + MXP_STAGING_BYTES + 1024 + (int)sizeof(MxWgradCtl);
+static_assert(MXW_SMEM_BYTES <= 232448, "exceeds the shared memory a CTA can opt in to");
+
+struct MxWgradParams {
+    const int32_t* slice_prefix;   // [E + 1], in 128-column slices
+    int E, M, m_tiles, n_tiles, n_cols, n_slices;   // n_slices: slices per row of the transposed codes (pitch / 128)
+    const uint32_t* sa;   // scale words of A [n_slices][M]
+    bf16* out;            // [E * M, n_cols]
+    long long ldo;
+};
+
+struct MxWgradTile {
+    int e, row0, n0, nt, width, k0, k_tiles;
+};
+__device__ __forceinline__ MxWgradTile mxw_decode(const MxWgradParams& p, const MxWgradCtl* ctl, long long t) {
+    const int per_e = p.m_tiles * p.n_tiles;
+    MxWgradTile tl;
+    tl.e = (int)(t / per_e);
+    const int local = (int)(t - (long long)tl.e * per_e);
+    tl.nt = local / p.m_tiles;   // column tile major inside an expert: the pairs running together share the B tile in L2
+    tl.row0 = (local - tl.nt * p.m_tiles) * MXP_ROWS;
+    tl.n0 = tl.nt * MXP_NT;
+    tl.width = min(MXP_NT, p.n_cols - tl.n0);
+    tl.k0 = ctl->sp[tl.e];
+    tl.k_tiles = ctl->sp[tl.e + 1] - tl.k0;
+    return tl;
+}
+
+__global__ void __launch_bounds__(MXP_THREADS, 1)
+mx_wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_sfb, const __grid_constant__ CUtensorMap map_o,
+                    const MxWgradParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
+    MxWgradCtl* ctl = reinterpret_cast<MxWgradCtl*>(tiles_ptr + MXP_STAGES * MXP_STAGE_BYTES + MXP_STAGING_BYTES);
+    volatile int* abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();   // 0 = the CTA that issues the MMAs
+    const long long first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;
+
+    for (int e = threadIdx.x; e <= p.E; e += MXP_THREADS) ctl->sp[e] = p.slice_prefix[e];
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MXP_STAGES; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 4);   // per CTA: the producer's arrive (with its byte count) + the scale warp's
+            mbar_init(smem_u32(&ctl->sf_full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
+            mbar_init(smem_u32(&ctl->tmem_empty[a]), 2 * MXP_EPI_WARPS);
+        }
+        mbar_init(smem_u32(&ctl->drain), 1);
+        mbar_init(smem_u32(&ctl->drain_copy), 1);
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tmap(&map_a);
+        prefetch_tmap(&map_b);
+        prefetch_tmap(&map_sfb);
+        prefetch_tmap(&map_o);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
+                     "r"((uint32_t)MX_TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();   // the other CTA's barriers and tensor memory exist from here on
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const long long n_tiles_total = (long long)p.E * p.m_tiles * p.n_tiles;
+    const uint32_t full0 = map_to_cta(smem_u32(&ctl->full[0]), 0);   // full[] of the MMA-issuing CTA
+
+    if (warp == 0) {
+        // ================= producer (both CTAs; each fills its own ring) =================
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, issued = 0;
+            bool ok = true;
+            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+                const MxWgradTile tl = mxw_decode(p, ctl, t);
+                const int sfb_row0 = tl.nt * p.n_slices + tl.k0;
+                const int b_row = tl.n0 + (int)rank * (tl.width >> 1);
+                for (int kt = 0; kt < tl.k_tiles; ++kt) {
+                    if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
+#ifdef MOE_TEST_HOOKS
+                    if (g_mx_test_withhold_first_stage != 0 && issued == 0) {
+                        ++issued;
+                        if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                        continue;
+                    }
+#endif
+                    if (rank == 0) ctl->stage_n[stage] = tl.width;   // read by the MMA thread after its wait on full[stage]
+                    const uint32_t bar = full0 + stage * (uint32_t)sizeof(unsigned long long);
+                    const uint32_t dst = tiles_base + stage * MXP_STAGE_BYTES;
+                    mbar_arrive_expect_tx_cluster(bar, MXP_TX_BYTES);
+                    tma_load_2d_pair(dst, &map_a, (tl.k0 + kt) * MX_BK, tl.row0 + (int)rank * MX_BM, bar);
+                    tma_load_2d_pair(dst + MXP_A_BYTES, &map_b, (tl.k0 + kt) * MX_BK, b_row, bar);
+                    tma_load_2d_pair(dst + MXP_SFB_OFF, &map_sfb, 0, sfb_row0 + kt, bar);
+                    ++issued;
+                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok && issued != 0) {
+                // leave no bulk copy in flight: the copies report to a barrier this thread cannot always poll (the other
+                // CTA's), so outwait them -- a copy that was issued completes within microseconds
+                const unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 2000000ull) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer: the first CTA's warp 1 =================
+        // The whole warp runs the loop and waits; one elected lane issues the tcgen05 instructions.  With the loop
+        // under `if (lane == 0)` every operand of a tcgen05 instruction (descriptors, addresses: uniform registers) is
+        // computed in the per-thread datapath and moved over, and the thread needed ~600 cycles per K slice against
+        // 448 of the tensor pipe; in converged code the values live in uniform registers from the start.
+        if (rank == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, n = MXP_NT;
+            bool ok = true;
+            const long long per_e = (long long)p.m_tiles * p.n_tiles;
+            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+                const int e_t = (int)(t / per_e);
+                const int k_tiles_t = ctl->sp[e_t + 1] - ctl->sp[e_t];
+                if (k_tiles_t == 0) continue;   // an expert without rows: the epilogue writes zeros on its own
+                if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * MXP_ACC_STRIDE;
+                for (int kt = 0; kt < k_tiles_t; ++kt) {
+                    if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->sf_full[stage]), phase, abort_flag))) { ok = false; break; }
+                    tc_fence_after();
+                    if (kt == 0) n = (uint32_t)ctl->stage_n[stage];
+                    const uint32_t s_base = tiles_base + stage * MXP_STAGE_BYTES;
+                    const uint32_t sfa_t = tmem_base + mxp_slot_col(stage), sfb_t = sfa_t + 4;
+                    const uint64_t a_desc = mx_operand_desc(s_base), b_desc = mx_operand_desc(s_base + MXP_A_BYTES);
+                    if (elect_one()) {
+#pragma unroll
+                        for (int k = 0; k < MX_BK / 32; ++k)
+                            mxp_mma(d_tmem, a_desc + (uint64_t)((k * 32) >> 4), b_desc + (uint64_t)((k * 32) >> 4), mxp_idesc(n, k),
+                                    sfa_t, sfb_t, (kt != 0 || k != 0) ? 1u : 0u);
+                        tc_commit<true>(smem_u32(&ctl->empty[stage]));
+                    }
+                    __syncwarp();
+                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (elect_one()) tc_commit<true>(smem_u32(&ctl->tmem_full[acc]));
+                __syncwarp();
+                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+            }
+            // all issued MMAs must have retired before tensor memory is released
+            if (lane == 0) {
+                tc_commit_local<true>(smem_u32(&ctl->drain));
+                const unsigned long long t0 = global_timer_ns();
+                while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
+            }
+        }
+        __syncwarp();
+    } else if (warp == 2) {
+        // ================= activation scales of this CTA's 128 rows =================
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+            const MxWgradTile tl = mxw_decode(p, ctl, t);
+            long long rows[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const long long r = (long long)tl.row0 + (int)rank * MX_BM + 32 * i + lane;
+                rows[i] = r < p.M ? r : p.M - 1;   // rows past the end are never stored; any valid address will do
+            }
+            // the words of MX_SCALE_AHEAD slices are in flight at any time: one slice per global-load round trip would
+            // bound the whole pipeline (the loads wait behind the operand traffic)
+            auto load_slice = [&](int kt) {
+                const uint32_t* s = p.sa + (long long)(tl.k0 + kt) * p.M;
+                return make_uint4(__ldg(s + rows[0]), __ldg(s + rows[1]), __ldg(s + rows[2]), __ldg(s + rows[3]));
+            };
+            uint4 q[MX_SCALE_AHEAD];
+#pragma unroll
+            for (int i = 0; i < MX_SCALE_AHEAD; ++i) q[i] = load_slice(min(i, max(tl.k_tiles - 1, 0)));
+            for (int kt0 = 0; ok && kt0 < tl.k_tiles; kt0 += MX_SCALE_AHEAD) {
+#pragma unroll
+                for (int i = 0; i < MX_SCALE_AHEAD; ++i) {
+                    const int kt = kt0 + i;
+                    if (kt >= tl.k_tiles) break;
+                    const uint4 cur = q[i];
+                    if (kt + MX_SCALE_AHEAD < tl.k_tiles) q[i] = load_slice(kt + MX_SCALE_AHEAD);
+                    if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag))) { ok = false; break; }
+                    *reinterpret_cast<uint4*>(tiles_ptr + stage * MXP_STAGE_BYTES + MXP_SFA_OFF + lane * 16) = cur;
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_remote(full0 + stage * (uint32_t)sizeof(unsigned long long));
+                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == MXP_COPY_WARP) {
+        // ================= scale copies: one thread of the first CTA =================
+        // Takes the three tcgen05.cp per K slice off the MMA thread (each tcgen05 instruction costs the issuing thread
+        // 60-85 cycles; with them the MMA thread needed ~770 cycles per slice).  Every ring stage has its own scale slot in
+        // tensor memory: full[stage] can only complete after the stage was released, i.e. after the MMAs that read the
+        // slot's previous contents have completed.
+        if (rank == 0 && lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            const long long per_e = (long long)p.m_tiles * p.n_tiles;
+            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
+                const int e_t = (int)(t / per_e);
+                const int k_tiles_t = ctl->sp[e_t + 1] - ctl->sp[e_t];
+                for (int kt = 0; kt < k_tiles_t; ++kt) {
+                    if (!mx_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t s_base = tiles_base + stage * MXP_STAGE_BYTES;
+                    const uint32_t sfa_t = tmem_base + mxp_slot_col(stage), sfb_t = sfa_t + 4;
+                    mxp_copy_scales(sfa_t, mx_scale_desc(s_base + MXP_SFA_OFF));
+                    mxp_copy_scales(sfb_t, mx_scale_desc(s_base + MXP_SFB_OFF));
+                    mxp_copy_scales(sfb_t + 4, mx_scale_desc(s_base + MXP_SFB_OFF + 512));
+                    tc_commit_local<true>(smem_u32(&ctl->sf_full[stage]));
+                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+            // all issued copies must have retired before tensor memory is released
+            tc_commit_local<true>(smem_u32(&ctl->drain_copy));
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(smem_u32(&ctl->drain_copy), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
+        }
+        __syncwarp();
+    } else {
+        // ================= epilogue (warps 3..10, both CTAs) =================
+        const int quarter = warp & 3;          // tensor-memory lanes [32 * quarter, 32 * quarter + 32)
+        const int half = (warp - 3) >> 2;      // 32-column blocks 0, 2, 4, 6 or 1, 3, 5 (+ the 16-column tail)
+        uint8_t* stage_ptr = tiles_ptr + MXP_STAGES * MXP_STAGE_BYTES + (warp - 3) * 2048;
+        const int sw = (lane >> 1) & 3;
+        const uint32_t empty0 = map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0);
+        uint32_t n_stores = 0, acc = 0, acc_phase = 0;
+        for (long long t = first_tile; t < n_tiles_total; t += tile_stride) {
+            const MxWgradTile tl = mxw_decode(p, ctl, t);
+            const bool have_acc = tl.k_tiles != 0;
+            if (have_acc) {
+                if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag))) break;
+                tc_fence_after();
+            }
+            const uint32_t taddr = tmem_base + acc * MXP_ACC_STRIDE + ((uint32_t)(quarter * 32) << 16);
+            const int slab_local = tl.row0 + (int)rank * MX_BM + quarter * 32;   // row of this expert's [M, N] gradient
+            const int rows_valid = max(0, min(32, p.M - slab_local));
+            const int slab0 = tl.e * p.M + slab_local;                           // row of the [E * M, N] output
+#pragma unroll 1
+            for (int c = half; c < 8; c += 2) {
+                const int left = tl.width - 32 * c;   // columns of the tile from this block on (warp-uniform)
+                if (left <= 0) break;
+                const int n = tl.n0 + c * 32;
+                uint32_t w[16];
+                if (!have_acc) {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) w[j] = 0u;
+                } else if (left >= 32) {
+                    uint32_t v[32];
+                    tc_ld32(taddr + c * 32, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                } else {
+                    uint32_t v[16];
+                    tc_ld16(taddr + c * 32, v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
+                }
+                if (rows_valid == 0) continue;
+                if (left >= 32 && rows_valid == 32) {
+                    if (n_stores != 0) {
+                        if (lane == 0) bulk_wait_read0();
+                        __syncwarp();
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j)
+                        *reinterpret_cast<uint4*>(stage_ptr + lane * 64 + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&map_o, n, slab0, smem_u32(stage_ptr));
+                        bulk_commit();
+                    }
+                    ++n_stores;
+                } else if (lane < rows_valid) {
+                    uint4* d4 = reinterpret_cast<uint4*>(p.out + ((long long)slab0 + lane) * p.ldo + n);
+                    d4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                    d4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    if (left >= 32) {
+                        d4[2] = make_uint4(w[8], w[9], w[10], w[11]);
+                        d4[3] = make_uint4(w[12], w[13], w[14], w[15]);
+                    }
+                }
+            }
+            if (!have_acc) continue;
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(empty0 + acc * (uint32_t)sizeof(unsigned long long));
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (n_stores != 0 && lane == 0) bulk_wait_all0();
+        __syncwarp();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();   // neither CTA's shared memory / barriers may go away while the other still uses them
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)MX_TMEM_COLS) : "memory");
+    }
+}
+
 // ---- quantisers ---------------------------------------------------------------------------------------
 // scale exponent of a block with largest magnitude amax: floor(log2 amax) - 8, clamped to the E8M0 range; -127 for zero
 __device__ __forceinline__ int mx_scale_exp(float amax) {
@@ -953,6 +1287,104 @@ __global__ void __launch_bounds__(256) mx_quantize_w_transposed_kernel(const bf1
                 (ib % 4)] = (uint8_t)(se + 127);
 }
 
+
+// ---- token-axis quantiser (operands of the weight gradients) ---------------------------------------------
+// slice_prefix[e] = number of 128-row slices of the experts before e, every expert's rows rounded up to whole slices
+__global__ void __launch_bounds__(1024) mx_slice_prefix_kernel(const int32_t* __restrict__ offsets, int E, int32_t* __restrict__ sp) {
+    __shared__ int32_t part[32];
+    const int e = threadIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int v = (e < E) ? (offsets[e + 1] - offsets[e] + 127) >> 7 : 0;
+    int incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += t;
+    }
+    if (lane == 31) part[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        int w = part[lane];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, w, d);
+            if (lane >= d) w += t;
+        }
+        part[lane] = w;
+    }
+    __syncthreads();
+    const int before = incl - v + (warp > 0 ? part[warp - 1] : 0);
+    if (e < E) sp[e] = before;
+    if (e == E - 1) sp[E] = before + v;
+}
+
+// x [R, ld] bf16, columns [col0, col0 + n) -> codes_t [n, pitch] (transposed, zero-padded per expert), scale words
+// [pitch/128][n] (the operand as the M side) and scale blocks in the pair tiling [ceil(n/208)][pitch/128][1024] (the
+// operand as the N side).  One thread per (padded block of 32 rows, group of 8 features): a 16-byte load per row and
+// thread, 512 contiguous bytes per warp; the thread keeps the 32 x 8 values as loaded, finds the 8 block maxima, then
+// writes 32 code bytes per feature.
+__global__ void __launch_bounds__(128) mx_quantize_tokens_kernel(const bf16* __restrict__ x, long long ld, int col0, int n,
+                                                                 const int32_t* __restrict__ offsets, const int32_t* __restrict__ sp,
+                                                                 int E, long long pitch, uint8_t* __restrict__ codes_t,
+                                                                 uint8_t* __restrict__ sa_words, uint8_t* __restrict__ sb_atoms) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int groups = n >> 3;
+    const int f0 = (int)(idx % groups) * 8;
+    const long long pb = idx / groups;                  // padded block of 32 rows
+    const int slice = (int)(pb >> 2);
+    if (slice >= sp[E]) return;
+    int lo = 0, hi = E;                                 // the expert whose slices hold `slice`: largest e with sp[e] <= slice
+    while (hi - lo > 1) {                               // (experts without rows share their successor's prefix)
+        const int mid = (lo + hi) >> 1;
+        if (sp[mid] <= slice) lo = mid; else hi = mid;
+    }
+    const int e = lo;
+    const int local_block = (int)(pb - 4ll * sp[e]);
+    const int n_e = offsets[e + 1] - offsets[e];
+    const int valid = max(0, min(32, n_e - 32 * local_block));
+    const uint4* src = reinterpret_cast<const uint4*>(x + ((long long)offsets[e] + 32ll * local_block) * ld + col0 + f0);
+    const long long ld16 = ld >> 3;
+    uint4 raw[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) raw[j] = j < valid ? __ldg(src + (long long)j * ld16) : make_uint4(0u, 0u, 0u, 0u);
+    float amax[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) amax[q] = 0.f;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw[j]);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[q]));
+            amax[2 * q] = fmaxf(amax[2 * q], fabsf(v.x));
+            amax[2 * q + 1] = fmaxf(amax[2 * q + 1], fabsf(v.y));
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int f = f0 + q;
+        const int se = mx_scale_exp(amax[q]);
+        const float inv = mx_inv_scale(se);
+        uint32_t out[8];
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {      // rows 4g .. 4g+3 of feature f
+            float v[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const uint32_t w = reinterpret_cast<const uint32_t*>(&raw[4 * g + t])[q >> 1];
+                v[t] = __uint_as_float((q & 1) ? (w & 0xffff0000u) : (w << 16));      // bf16 -> fp32 is a shift
+            }
+            out[g] = mx_e4m3x2(v[0] * inv, v[1] * inv) | (mx_e4m3x2(v[2] * inv, v[3] * inv) << 16);
+        }
+        uint4* dst = reinterpret_cast<uint4*>(codes_t + (long long)f * pitch + pb * 32);
+        dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+        dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+        const uint8_t sbyte = (uint8_t)(se + 127);
+        sa_words[((long long)slice * n + f) * 4 + (pb & 3)] = sbyte;
+        const int nt = f / MXP_NT, c = f % MXP_NT;
+        sb_atoms[((long long)nt * (pitch >> 7) + slice) * 1024 + (c >> 7) * 512 + (c % 32) * 16 + ((c % 128) / 32) * 4 + (pb & 3)] = sbyte;
+    }
+}
+
 }  // namespace
 
 // Weight scales of a GEMM with E experts, n_feat output features and a contraction of k: stored twice, in the tiling of
@@ -1003,6 +1435,75 @@ int launch_mx_quantize_w_rows(int E, int n_feat, int k, int k_total, int k_off, 
     mx_quantize_rows_kernel<true><<<mx_row_quantiser_blocks(rows * (k / 128)), 256, 0, s>>>(
         reinterpret_cast<const uint4*>(w), rows, k, n_feat, k_total / 128, k_off / 128, reinterpret_cast<uint2*>(codes), scales,
         scales + mx_w_scale_single_bytes(E, n_feat, k_total));
+    return check_launch();
+}
+
+// ---- weight-gradient operands and GEMM ----
+constexpr size_t MX_TOKENS_HEADER_BYTES = 8192;   // slice_prefix[E + 1] at the head of a token-quantised operand's scales
+long long mx_tokens_pitch(long long R, int E) { return ((R + 127) / 128) * 128 + 128ll * E; }
+size_t mx_tokens_scale_bytes(long long R, int E, int n) {
+    const long long slices = mx_tokens_pitch(R, E) / 128;
+    return MX_TOKENS_HEADER_BYTES + (size_t)slices * n * 4 + (size_t)((n + MXP_NT - 1) / MXP_NT) * slices * 1024;
+}
+
+int launch_mx_quantize_tokens(long long R, int E, const bf16* x, long long ld, int col0, int n, const int32_t* offsets,
+                              uint8_t* codes_t, uint8_t* scales, cudaStream_t s) {
+    const long long pitch = mx_tokens_pitch(R, E);
+    int32_t* sp = reinterpret_cast<int32_t*>(scales);
+    uint8_t* sa = scales + MX_TOKENS_HEADER_BYTES;
+    uint8_t* sb = sa + (size_t)(pitch / 128) * n * 4;
+    mx_slice_prefix_kernel<<<1, 1024, 0, s>>>(offsets, E, sp);
+    int st_ = check_launch();
+    if (st_ != MOE_OK) return st_;
+    const long long total = (pitch / 32) * (n / 8);
+    mx_quantize_tokens_kernel<<<(unsigned)((total + 127) / 128), 128, 0, s>>>(x, ld, col0, n, offsets, sp, E, pitch, codes_t, sa, sb);
+    return check_launch();
+}
+
+// dW [E, M, N] = Q(A)^T Q(B) per expert: a_* the M-side operand ([M, pitch] codes, scales with header and words),
+// b_* the N-side operand ([N, pitch] codes, its scales' pair-tiled blocks are used)
+int launch_mx_wgrad(long long R, int E, int M, int N, const uint8_t* a_codes_t, const uint8_t* a_scales, const uint8_t* b_codes_t,
+                    const uint8_t* b_scales, bf16* dw, cudaStream_t s) {
+    const long long pitch = mx_tokens_pitch(R, E);
+    const int n_slices = (int)(pitch / 128);
+    const int n_tiles = (N + MXP_NT - 1) / MXP_NT, m_tiles = (M + MXP_ROWS - 1) / MXP_ROWS;
+    const uint8_t* b_atoms = b_scales + MX_TOKENS_HEADER_BYTES + (size_t)n_slices * N * 4;
+    CUtensorMap a, b, sfb, o;
+    if (!make_map_typed(&a, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, a_codes_t, (uint64_t)pitch, (uint64_t)M, MX_BK, MX_BM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_typed(&b, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, b_codes_t, (uint64_t)pitch, (uint64_t)N, MX_BK, MXP_NT / 2,
+                        CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_typed(&sfb, CU_TENSOR_MAP_DATA_TYPE_UINT32, 4, b_atoms, 256, (uint64_t)n_tiles * n_slices, 256, 1,
+                        CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_out_map(&o, dw, N, (uint64_t)E * M))
+        return MOE_ERR_CUDA;
+    MxWgradParams p = {};
+    p.slice_prefix = reinterpret_cast<const int32_t*>(a_scales); p.E = E; p.M = M; p.m_tiles = m_tiles; p.n_tiles = n_tiles;
+    p.n_cols = N; p.n_slices = n_slices;
+    p.sa = reinterpret_cast<const uint32_t*>(a_scales + MX_TOKENS_HEADER_BYTES); p.out = dw; p.ldo = N;
+    static int grid_of_device[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return MOE_ERR_CUDA;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(MXP_THREADS);
+    cfg.dynamicSmemBytes = MXW_SMEM_BYTES;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (grid_of_device[dev] == 0) {
+        if (cudaFuncSetAttribute(mx_wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MXW_SMEM_BYTES) != cudaSuccess)
+            return MOE_ERR_CUDA;
+        const int sms = sm_count();
+        if (sms <= 0) return MOE_ERR_CUDA;
+        cfg.gridDim = dim3(2 * (sms / 2));
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, mx_wgrad_pair_kernel, &cfg) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
+        if (clusters > sms / 2) clusters = sms / 2;
+        grid_of_device[dev] = 2 * clusters;
+    }
+    cfg.gridDim = dim3(grid_of_device[dev]);
+    cfg.stream = s;
+    if (cudaLaunchKernelEx(&cfg, mx_wgrad_pair_kernel, a, b, sfb, o, p) != cudaSuccess) return MOE_ERR_CUDA;
     return check_launch();
 }
 

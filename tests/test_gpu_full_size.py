@@ -271,6 +271,62 @@ def test_mxfp8_other_gemms_sampled_rows(full):
     Hh.assert_close(Hh.to_np64(dx[rsel]), want, f"{cfg.name}: dX_perm rows (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
 
 
+def test_mxfp8_weight_gradients_sampled_experts(full):
+    """The block-scaled FP8 weight gradients at full size: the smallest expert with rows, a mid-sized one and every
+    expert without rows, on 256 output columns each, against the exact product of the token-quantised operands (the
+    oracle quantises those experts' rows only, in blocks of 32 counted from the expert's first row)."""
+    cfg, dev, b = full
+    if cfg.H % 128 or cfg.I % 128:
+        pytest.skip("the block-scaled path takes widths that are multiples of 128")
+    from paper_2606_26453_b200 import binding as B
+    d = b.d
+    R, E, H, I = cfg.R, cfg.E, cfg.H, cfg.I
+    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    tok = lambda n: (u8(B.moe_mxfp8_tokens_codes_bytes(d, n)), u8(B.moe_mxfp8_tokens_scale_bytes(d, n)))
+    offsets = b.offsets.cpu().numpy()
+    counts = np.diff(offsets)
+    order = np.argsort(counts, kind="stable")
+    nonempty = [int(e) for e in order if counts[e] > 0]
+    picks = [nonempty[0], nonempty[len(nonempty) // 2]]
+    cols = slice(128, 384)                                   # crosses a 208-column tile boundary
+
+    def expert_ref(a_rows, b_rows, e):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        one = np.array([0, hi - lo])
+        return O.wgrad_mxfp8(f32(a_rows[lo:hi]), f32(b_rows[lo:hi]), one)[0]
+
+    (hc, hs), (dc, ds) = tok(I), tok(H)
+    B.moe_mxfp8_quantize_tokens(d, b.h_act, I, 0, I, b.offsets, hc, hs)
+    B.moe_mxfp8_quantize_tokens(d, b.dy_perm, H, 0, H, b.offsets, dc, ds)
+    dwd = torch.full((E, I, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.moe_grouped_gemm_down_wgrad_mxfp8(d, hc, hs, dc, ds, dwd)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0 and not bool(torch.isnan(dwd).any())
+    for e in picks:
+        want = expert_ref(b.h_act, b.dy_perm[:, cols], e)
+        Hh.assert_close(Hh.to_np64(dwd[e][:, cols]), want, f"{cfg.name}: dW_down[{e}] (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    for e in np.flatnonzero(counts == 0):
+        assert not bool(dwd[int(e)].any())
+    del hc, hs, dc, ds, dwd
+
+    (xc, xs), (gc, gs), (uc, us) = tok(H), tok(I), tok(I)
+    B.moe_mxfp8_quantize_tokens(d, b.x_perm, H, 0, H, b.offsets, xc, xs)
+    B.moe_mxfp8_quantize_tokens(d, b.dgu, 2 * I, 0, I, b.offsets, gc, gs)
+    B.moe_mxfp8_quantize_tokens(d, b.dgu, 2 * I, I, I, b.offsets, uc, us)
+    dwg = torch.full((E, H, I), float("nan"), dtype=torch.bfloat16, device="cuda")
+    dwu = torch.full((E, H, I), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.moe_grouped_gemm_gateup_wgrad_mxfp8(d, xc, xs, gc, gs, uc, us, dwg, dwu)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0 and not bool(torch.isnan(dwg).any()) and not bool(torch.isnan(dwu).any())
+    for e in picks:
+        Hh.assert_close(Hh.to_np64(dwg[e][:, cols]), expert_ref(b.x_perm, b.dgu[:, :I][:, cols], e),
+                        f"{cfg.name}: dW_gate[{e}] (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+        Hh.assert_close(Hh.to_np64(dwu[e][:, cols]), expert_ref(b.x_perm, b.dgu[:, I:][:, cols], e),
+                        f"{cfg.name}: dW_up[{e}] (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    for e in np.flatnonzero(counts == 0):
+        assert not bool(dwg[int(e)].any()) and not bool(dwu[int(e)].any())
+
+
 # ------------------------------------------------------------------------------------------------
 # every element of every output, where the oracle can afford the whole layer (about 15 s and 45 s of host time)
 # ------------------------------------------------------------------------------------------------

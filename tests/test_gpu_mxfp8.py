@@ -260,6 +260,99 @@ def test_gateup_forward_and_fused_swiglu_quantiser_against_the_oracle(B, name):
     assert torch.equal(hc, hc2) and torch.equal(hs, hs2)
 
 
+def _oracle_tokens_layout(x, offsets):
+    """What moe_mxfp8_quantize_tokens must produce for x [R, n]: (codes_t [n, n_slices*128], scale bytes
+    [n_slices, n, 4], slice_prefix) -- every column quantised by the oracle in expert-aligned blocks of 32 rows."""
+    E = len(offsets) - 1
+    n = x.shape[1]
+    sp = np.concatenate([[0], np.cumsum([(offsets[e + 1] - offsets[e] + 127) // 128 for e in range(E)])]).astype(np.int64)
+    codes = np.zeros((n, int(sp[-1]) * 128), dtype=np.uint8)
+    scales = np.zeros((int(sp[-1]), n, 4), dtype=np.uint8)
+    for e in range(E):
+        lo, hi = int(offsets[e]), int(offsets[e + 1])
+        if hi == lo:
+            continue
+        width = int(sp[e + 1] - sp[e]) * 128
+        xt = np.zeros((n, width))
+        xt[:, :hi - lo] = x[lo:hi].T
+        c, sc, _ = O.mxfp8_quantize(xt)                      # along the padded token axis
+        codes[:, sp[e] * 128: sp[e] * 128 + width] = c
+        scales[sp[e]:sp[e + 1]] = sc.reshape(n, -1, 4).transpose(1, 0, 2)
+    return codes, scales, sp
+
+
+WGRAD_CASES = {
+    "one_slice": ([100], 1, 128, 128),
+    "ragged": ([0, 1, 127, 0, 129, 128, 300, 15, 0], 2, 256, 384),          # empty experts, short last blocks
+    "wide": ([200, 0, 31, 290, 1], 2, 384, 1408),                            # M and N tiles with remainders
+    "big_expert": ([1500, 513, 64], 1, 256, 256),                            # many K slices per tile
+}
+
+
+@pytest.mark.parametrize("name", list(WGRAD_CASES))
+def test_weight_gradients_token_quantiser_and_gemm_against_the_oracle(B, name):
+    """dW_down = Q(H_act)^T Q(dY_perm) and [dW_gate | dW_up] = Q(X_perm)^T Q(dGU) per expert, operands quantised along
+    the token axis in expert-aligned blocks of 32 rows."""
+    counts, K, H, I = WGRAD_CASES[name]
+    cfg, host = Hh.ragged_workload(counts, K=K, H=H, I=I, seed=29)
+    ref = O.layer_fwd_bwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"], host["W_down"],
+                          host["dY"])
+    R, E = cfg.R, cfg.E
+    offsets = ref["offsets"]
+    d = B.dims(cfg.T, H, I, E, K)
+    bf = lambda a: W.round_to_bf16(np.asarray(a, dtype=np.float32))
+    x, h, dy, dgu = bf(ref["X_perm"]), bf(ref["H_act"]), bf(ref["dY_perm"]), bf(ref["dGU"])
+    x[0, :] = 0.0                                              # a column block that starts with a zero row
+    off = torch.from_numpy(offsets).cuda()
+    P = ((R + 127) // 128) * 128 + 128 * E
+    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+
+    def quantise(t_host, col0, n):
+        t_dev = Hh.to_dev_bf16(t_host)
+        codes, scales = u8(B.moe_mxfp8_tokens_codes_bytes(d, n)), u8(B.moe_mxfp8_tokens_scale_bytes(d, n))
+        assert codes.numel() == n * P
+        B.moe_mxfp8_quantize_tokens(d, t_dev, t_host.shape[1], col0, n, off, codes, scales)
+        torch.cuda.synchronize()
+        o_codes, o_scales, sp = _oracle_tokens_layout(t_host[:, col0:col0 + n], offsets)
+        n_sl = int(sp[-1])
+        assert np.array_equal(scales[:4 * (E + 1)].cpu().numpy().view(np.int32), sp.astype(np.int32))
+        assert np.array_equal(codes.view(n, P)[:, :n_sl * 128].cpu().numpy(), o_codes)
+        words = scales[8192: 8192 + (P // 128) * n * 4].view(P // 128, n, 4)[:n_sl].cpu().numpy()
+        assert np.array_equal(words, o_scales)
+        # the same bytes in the pair tiling
+        atoms = scales[8192 + (P // 128) * n * 4:].view((n + 207) // 208, P // 128, 2, 32, 4, 4).cpu().numpy()
+        f = np.arange(n)
+        c = f % 208
+        got = atoms[f // 208, :n_sl, c >> 7, c % 32, (c % 128) // 32, :]          # [n, n_sl, 4]
+        assert np.array_equal(got.transpose(1, 0, 2), o_scales)
+        return codes, scales
+
+    hc, hs = quantise(h, 0, I)
+    dc, ds = quantise(dy, 0, H)
+    dwd = torch.full((E, I, H), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.moe_grouped_gemm_down_wgrad_mxfp8(d, hc, hs, dc, ds, dwd)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    want = O.wgrad_mxfp8(h, dy, offsets)
+    Hh.assert_close(Hh.to_np64(dwd), want, f"{name}: dW_down (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    for e in np.flatnonzero(np.diff(offsets) == 0):
+        assert not bool(dwd[e].any())                          # exact zeros for an expert without rows
+
+    xc, xs = quantise(x, 0, H)
+    gc, gs = quantise(dgu, 0, I)
+    uc, us = quantise(dgu, I, I)
+    dwg = torch.full((E, H, I), float("nan"), dtype=torch.bfloat16, device="cuda")
+    dwu = torch.full((E, H, I), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.moe_grouped_gemm_gateup_wgrad_mxfp8(d, xc, xs, gc, gs, uc, us, dwg, dwu)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    want = O.wgrad_mxfp8(x, dgu, offsets)                      # [E, H, 2I]
+    Hh.assert_close(Hh.to_np64(dwg), want[:, :, :I], f"{name}: dW_gate (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    Hh.assert_close(Hh.to_np64(dwu), want[:, :, I:], f"{name}: dW_up (MXFP8)", rel_fro=Hh.PER_CALL_FROBENIUS)
+    exact = O.gateup_bwd_from_dgu(dgu, x, host["W_gate"], host["W_up"], offsets)[1]
+    assert np.linalg.norm(Hh.to_np64(dwg) - exact) / np.linalg.norm(exact) < 0.08
+
+
 def test_shapes_the_block_scaled_path_does_not_take_are_refused(B):
     d = B.dims(64, 192, 128, 2, 1)                   # H not a multiple of 128
     assert B.moe_mxfp8_act_scale_bytes(d) == 0
