@@ -1,5 +1,5 @@
-// Block-scaled FP8 (MXFP8) twins of the four row-ragged grouped GEMMs (gate/up forward, down forward, down dgrad,
-// gate/up dgrad) on the block-scaled tensor-core path (tcgen05.mma kind::mxf8f6f4 with block_scale): quantisers, one GEMM
+// Block-scaled FP8 (MXFP8) twins of the six grouped GEMMs (gate/up forward, down forward, down dgrad, gate/up dgrad, and
+// the two weight gradients, further down) on the block-scaled tensor-core path (tcgen05.mma kind::mxf8f6f4 with block_scale): quantisers, one GEMM
 // in two tilings, and the SwiGLU activation with the activation quantiser fused in.  Every GEMM here is
 //   out[r, :] = dequant(a row r) . dequant(b[e])^T   for the rows r of expert e,
 // a [R, k] and b [E, n_feat, k] both contraction-contiguous; the callers choose which tensors play a and b.
