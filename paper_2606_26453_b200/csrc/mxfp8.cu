@@ -420,17 +420,24 @@ struct MxPairCtl {
     uint32_t tmem_base;
     int abort_flag;
     int stage_n[MXP_STAGES];   // columns of the tile a stage belongs to (published by the first CTA's producer)
-    int32_t offs[MX_MAX_E + 1];
-    int32_t tile_prefix[MX_MAX_E + 1];
+    int32_t offs[MX_MAX_E + 1];          // row-ragged form: offsets; weight gradients: slice_prefix
+    int32_t tile_prefix[MX_MAX_E + 1];   // row-ragged form: 256-row tiles of the experts before e
 };
 constexpr int MXP_SMEM_BYTES = MXP_STAGES * MXP_STAGE_BYTES + MXP_STAGING_BYTES + 1024 + (int)sizeof(MxPairCtl);
 static_assert(MXP_SMEM_BYTES <= 232448, "exceeds the shared memory a CTA can opt in to");
 
+// The pair kernel serves two problems (template parameter WGRAD):
+//   row-ragged GEMM   out[r, :] = a[r, :] . b[e]^T for the rows r of expert e: tiles of 256 rows from `offsets`, the
+//                     contraction is k_tiles slices for every tile, b and its scale blocks are indexed by expert;
+//   weight gradient   dW[e] [M, N] = A_e^T B_e with token-quantised, transposed operands (further down): a fixed tile
+//                     list (expert x M tiles x N tiles), the contraction of expert e is the slices
+//                     [slice_prefix[e], slice_prefix[e + 1]) of both operands, nothing is indexed by expert but the output.
 struct MxPairParams {
-    const int32_t* offsets;
-    int E, k_tiles, n_tiles, n_cols;
-    long long R;
-    const uint32_t* sa;   // activation scale words [k_tiles][R]
+    const int32_t* prefix;   // offsets [E + 1] / slice_prefix [E + 1]
+    int E, k_tiles, n_tiles, m_tiles, n_cols, n_slices;   // k_tiles: row-ragged form; m_tiles, n_slices: weight gradients
+    int M;                   // weight gradients: rows of one expert's output
+    long long sa_rows;       // rows per slice of the A-side scale words: R / M
+    const uint32_t* sa;      // scale words of the A side [slices][sa_rows]
     bf16* out;
     long long ldo;
 };
@@ -465,29 +472,61 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t v[16]) {
 }
 
 struct MxPairTile {
-    int e, row0, row_end, n0, nt, width;
+    int e, row0, row_end;   // first row of the tile and end of the valid rows, as the A operand counts them
+    int out_shift;          // output row = A row + out_shift
+    int n0, nt, width;      // first column, column-tile index, columns
+    int k0, k_tiles;        // K slices [k0, k0 + k_tiles) of both operands
+    int b_row, sfb_row0;    // first row of the tile in the B codes; row of its first scale block
 };
+template <bool WGRAD>
 __device__ __forceinline__ MxPairTile mxp_decode(const MxPairParams& p, const MxPairCtl* ctl, long long t) {
-    int lo = 0, hi = p.E;   // largest e with tile_prefix[e] * n_tiles <= t
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if ((long long)ctl->tile_prefix[mid] * p.n_tiles <= t) lo = mid; else hi = mid;
-    }
-    const int local = (int)(t - (long long)ctl->tile_prefix[lo] * p.n_tiles);
-    const int m_tiles_e = ctl->tile_prefix[lo + 1] - ctl->tile_prefix[lo];
     MxPairTile tl;
-    tl.e = lo;
-    tl.nt = local / m_tiles_e;   // column tile major inside an expert (the pairs running together share weight tiles in L2)
-    const int mt = local - tl.nt * m_tiles_e;
-    tl.row0 = ctl->offs[lo] + mt * MXP_ROWS;
-    tl.row_end = ctl->offs[lo + 1];
-    tl.n0 = tl.nt * MXP_NT;
+    if (WGRAD) {
+        const int per_e = p.m_tiles * p.n_tiles;
+        tl.e = (int)(t / per_e);
+        const int local = (int)(t - (long long)tl.e * per_e);
+        tl.nt = local / p.m_tiles;   // column tile major inside an expert: the pairs running together share the B tile in L2
+        tl.row0 = (local - tl.nt * p.m_tiles) * MXP_ROWS;
+        tl.row_end = p.M;
+        tl.out_shift = tl.e * p.M;
+        tl.k0 = ctl->offs[tl.e];
+        tl.k_tiles = ctl->offs[tl.e + 1] - tl.k0;
+        tl.n0 = tl.nt * MXP_NT;
+        tl.b_row = tl.n0;
+        tl.sfb_row0 = tl.nt * p.n_slices + tl.k0;
+    } else {
+        int lo = 0, hi = p.E;   // largest e with tile_prefix[e] * n_tiles <= t
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if ((long long)ctl->tile_prefix[mid] * p.n_tiles <= t) lo = mid; else hi = mid;
+        }
+        const int local = (int)(t - (long long)ctl->tile_prefix[lo] * p.n_tiles);
+        const int m_tiles_e = ctl->tile_prefix[lo + 1] - ctl->tile_prefix[lo];
+        tl.e = lo;
+        tl.nt = local / m_tiles_e;   // column tile major inside an expert (the pairs running together share weight tiles in L2)
+        tl.row0 = ctl->offs[lo] + (local - tl.nt * m_tiles_e) * MXP_ROWS;
+        tl.row_end = ctl->offs[lo + 1];
+        tl.out_shift = 0;
+        tl.k0 = 0;
+        tl.k_tiles = p.k_tiles;
+        tl.n0 = tl.nt * MXP_NT;
+        tl.b_row = lo * p.n_cols + tl.n0;
+        tl.sfb_row0 = (lo * p.n_tiles + tl.nt) * p.k_tiles;
+    }
     tl.width = min(MXP_NT, p.n_cols - tl.n0);
     return tl;
 }
+// K slices of tile t (the roles that do not need the rest of the tile)
+template <bool WGRAD>
+__device__ __forceinline__ int mxp_k_tiles(const MxPairParams& p, const MxPairCtl* ctl, long long t) {
+    if (!WGRAD) return p.k_tiles;
+    const int e = (int)(t / ((long long)p.m_tiles * p.n_tiles));
+    return ctl->offs[e + 1] - ctl->offs[e];
+}
 
+template <bool WGRAD>
 __global__ void __launch_bounds__(MXP_THREADS, 1)
-mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+mx_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_sfb, const __grid_constant__ CUtensorMap map_o,
                     const MxPairParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -499,7 +538,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const uint32_t rank = cluster_ctarank();   // 0 = the CTA that issues the MMAs
     const long long first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;
 
-    for (int e = threadIdx.x; e <= p.E; e += MXP_THREADS) ctl->offs[e] = p.offsets[e];
+    for (int e = threadIdx.x; e <= p.E; e += MXP_THREADS) ctl->offs[e] = p.prefix[e];
     if (threadIdx.x == 0) {
         for (int s = 0; s < MXP_STAGES; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 4);   // per CTA: the producer's arrive (with its byte count) + the scale warp's
@@ -520,7 +559,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         prefetch_tmap(&map_o);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (!WGRAD && threadIdx.x == 0) {   // row-ragged form: tiles of 256 rows per expert
         int run = 0;
         for (int e = 0; e < p.E; ++e) {
             ctl->tile_prefix[e] = run;
@@ -539,7 +578,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     cluster_sync_all();   // the other CTA's barriers and tensor memory exist from here on
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
-    const long long n_tiles_total = (long long)ctl->tile_prefix[p.E] * p.n_tiles;
+    const long long n_tiles_total = WGRAD ? (long long)p.E * p.m_tiles * p.n_tiles : (long long)ctl->tile_prefix[p.E] * p.n_tiles;
     const uint32_t full0 = map_to_cta(smem_u32(&ctl->full[0]), 0);   // full[] of the MMA-issuing CTA
 
     if (warp == 0) {
@@ -548,328 +587,9 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             uint32_t stage = 0, phase = 0, issued = 0;
             bool ok = true;
             for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
-                const MxPairTile tl = mxp_decode(p, ctl, t);
-                const int sfb_row0 = (tl.e * p.n_tiles + tl.nt) * p.k_tiles;
-                const int b_row = tl.e * p.n_cols + tl.n0 + (int)rank * (tl.width >> 1);
-                for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
-#ifdef MOE_TEST_HOOKS
-                    if (g_mx_test_withhold_first_stage != 0 && issued == 0) {
-                        ++issued;
-                        if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
-                        continue;
-                    }
-#endif
-                    if (rank == 0) ctl->stage_n[stage] = tl.width;   // read by the MMA thread after its wait on full[stage]
-                    const uint32_t bar = full0 + stage * (uint32_t)sizeof(unsigned long long);
-                    const uint32_t dst = tiles_base + stage * MXP_STAGE_BYTES;
-                    mbar_arrive_expect_tx_cluster(bar, MXP_TX_BYTES);
-                    tma_load_2d_pair(dst, &map_a, kt * MX_BK, tl.row0 + (int)rank * MX_BM, bar);
-                    tma_load_2d_pair(dst + MXP_A_BYTES, &map_b, kt * MX_BK, b_row, bar);
-                    tma_load_2d_pair(dst + MXP_SFB_OFF, &map_sfb, 0, sfb_row0 + kt, bar);
-                    ++issued;
-                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
-                }
-            }
-            if (!ok && issued != 0) {
-                // leave no bulk copy in flight: the copies report to a barrier this thread cannot always poll (the other
-                // CTA's), so outwait them -- a copy that was issued completes within microseconds
-                const unsigned long long t0 = global_timer_ns();
-                while (global_timer_ns() - t0 < 2000000ull) {}
-            }
-        }
-    } else if (warp == 1) {
-        // ================= MMA issuer: the first CTA's warp 1 =================
-        // The whole warp runs the loop and waits; one elected lane issues the tcgen05 instructions.  With the loop
-        // under `if (lane == 0)` every operand of a tcgen05 instruction (descriptors, addresses: uniform registers) is
-        // computed in the per-thread datapath and moved over, and the thread needed ~600 cycles per K slice against
-        // 448 of the tensor pipe; in converged code the values live in uniform registers from the start.
-        if (rank == 0) {
-            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, n = MXP_NT;
-            bool ok = true;
-            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
-                if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag))) break;
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * MXP_ACC_STRIDE;
-                for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->sf_full[stage]), phase, abort_flag))) { ok = false; break; }
-                    tc_fence_after();
-                    if (kt == 0) n = (uint32_t)ctl->stage_n[stage];
-                    const uint32_t s_base = tiles_base + stage * MXP_STAGE_BYTES;
-                    const uint32_t sfa_t = tmem_base + mxp_slot_col(stage), sfb_t = sfa_t + 4;
-                    const uint64_t a_desc = mx_operand_desc(s_base), b_desc = mx_operand_desc(s_base + MXP_A_BYTES);
-                    if (elect_one()) {
-#pragma unroll
-                        for (int k = 0; k < MX_BK / 32; ++k)
-                            mxp_mma(d_tmem, a_desc + (uint64_t)((k * 32) >> 4), b_desc + (uint64_t)((k * 32) >> 4), mxp_idesc(n, k),
-                                    sfa_t, sfb_t, (kt != 0 || k != 0) ? 1u : 0u);
-                        tc_commit<true>(smem_u32(&ctl->empty[stage]));
-                    }
-                    __syncwarp();
-                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
-                }
-                if (!ok) break;
-                if (elect_one()) tc_commit<true>(smem_u32(&ctl->tmem_full[acc]));
-                __syncwarp();
-                if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-            }
-            // all issued MMAs must have retired before tensor memory is released
-            if (lane == 0) {
-                tc_commit_local<true>(smem_u32(&ctl->drain));
-                const unsigned long long t0 = global_timer_ns();
-                while (!mbar_try_wait(smem_u32(&ctl->drain), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
-            }
-        }
-        __syncwarp();
-    } else if (warp == 2) {
-        // ================= activation scales of this CTA's 128 rows =================
-        uint32_t stage = 0, phase = 0;
-        bool ok = true;
-        for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
-            const MxPairTile tl = mxp_decode(p, ctl, t);
-            long long rows[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const long long r = (long long)tl.row0 + (int)rank * MX_BM + 32 * i + lane;
-                rows[i] = r < p.R ? r : p.R - 1;   // rows past the end are never stored; any valid address will do
-            }
-            // the words of MX_SCALE_AHEAD slices are in flight at any time: one slice per global-load round trip would
-            // bound the whole pipeline (the loads wait behind the operand traffic)
-            auto load_slice = [&](int kt) {
-                const uint32_t* s = p.sa + (long long)kt * p.R;
-                return make_uint4(__ldg(s + rows[0]), __ldg(s + rows[1]), __ldg(s + rows[2]), __ldg(s + rows[3]));
-            };
-            uint4 q[MX_SCALE_AHEAD];
-#pragma unroll
-            for (int i = 0; i < MX_SCALE_AHEAD; ++i) q[i] = load_slice(min(i, p.k_tiles - 1));
-            for (int kt0 = 0; ok && kt0 < p.k_tiles; kt0 += MX_SCALE_AHEAD) {
-#pragma unroll
-                for (int i = 0; i < MX_SCALE_AHEAD; ++i) {
-                    const int kt = kt0 + i;
-                    if (kt >= p.k_tiles) break;
-                    const uint4 cur = q[i];
-                    if (kt + MX_SCALE_AHEAD < p.k_tiles) q[i] = load_slice(kt + MX_SCALE_AHEAD);
-                    if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag))) { ok = false; break; }
-                    *reinterpret_cast<uint4*>(tiles_ptr + stage * MXP_STAGE_BYTES + MXP_SFA_OFF + lane * 16) = cur;
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_remote(full0 + stage * (uint32_t)sizeof(unsigned long long));
-                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
-                }
-            }
-        }
-    } else if (warp == MXP_COPY_WARP) {
-        // ================= scale copies: one thread of the first CTA =================
-        // Takes the three tcgen05.cp per K slice off the MMA thread (each tcgen05 instruction costs the issuing thread
-        // 60-85 cycles; with them the MMA thread needed ~770 cycles per slice).  Every ring stage has its own scale slot in
-        // tensor memory: full[stage] can only complete after the stage was released, i.e. after the MMAs that read the
-        // slot's previous contents have completed.
-        if (rank == 0 && lane == 0) {
-            uint32_t stage = 0, phase = 0;
-            bool ok = true;
-            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
-                for (int kt = 0; kt < p.k_tiles; ++kt) {
-                    if (!mx_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t s_base = tiles_base + stage * MXP_STAGE_BYTES;
-                    const uint32_t sfa_t = tmem_base + mxp_slot_col(stage), sfb_t = sfa_t + 4;
-                    mxp_copy_scales(sfa_t, mx_scale_desc(s_base + MXP_SFA_OFF));
-                    mxp_copy_scales(sfb_t, mx_scale_desc(s_base + MXP_SFB_OFF));
-                    mxp_copy_scales(sfb_t + 4, mx_scale_desc(s_base + MXP_SFB_OFF + 512));
-                    tc_commit_local<true>(smem_u32(&ctl->sf_full[stage]));
-                    if (++stage == MXP_STAGES) { stage = 0; phase ^= 1u; }
-                }
-            }
-            // all issued copies must have retired before tensor memory is released
-            tc_commit_local<true>(smem_u32(&ctl->drain_copy));
-            const unsigned long long t0 = global_timer_ns();
-            while (!mbar_try_wait(smem_u32(&ctl->drain_copy), 0) && global_timer_ns() - t0 < WAIT_LIMIT_NS) {}
-        }
-        __syncwarp();
-    } else {
-        // ================= epilogue (warps 3..10, both CTAs) =================
-        const int quarter = warp & 3;          // tensor-memory lanes [32 * quarter, 32 * quarter + 32)
-        const int half = (warp - 3) >> 2;      // 32-column blocks 0, 2, 4, 6 or 1, 3, 5 (+ the 16-column tail)
-        uint8_t* stage_ptr = tiles_ptr + MXP_STAGES * MXP_STAGE_BYTES + (warp - 3) * 2048;
-        const int sw = (lane >> 1) & 3;
-        const uint32_t empty0 = map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0);
-        uint32_t n_stores = 0, acc = 0, acc_phase = 0;
-        for (long long t = first_tile; t < n_tiles_total; t += tile_stride) {
-            const MxPairTile tl = mxp_decode(p, ctl, t);
-            if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag))) break;
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + acc * MXP_ACC_STRIDE + ((uint32_t)(quarter * 32) << 16);
-            const int slab0 = tl.row0 + (int)rank * MX_BM + quarter * 32;
-            const int rows_valid = max(0, min(32, tl.row_end - slab0));
-#pragma unroll 1
-            for (int c = half; c < 8; c += 2) {
-                const int left = tl.width - 32 * c;   // columns of the tile from this block on (warp-uniform)
-                if (left <= 0) break;
-                const int n = tl.n0 + c * 32;
-                uint32_t w[16];
-                if (left >= 32) {
-                    uint32_t v[32];
-                    tc_ld32(taddr + c * 32, v);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-                } else {
-                    uint32_t v[16];
-                    tc_ld16(taddr + c * 32, v);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) w[j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-                }
-                if (rows_valid == 0) continue;
-                if (left >= 32 && rows_valid == 32) {
-                    if (n_stores != 0) {
-                        if (lane == 0) bulk_wait_read0();
-                        __syncwarp();
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        *reinterpret_cast<uint4*>(stage_ptr + lane * 64 + ((j ^ sw) << 4)) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&map_o, n, slab0, smem_u32(stage_ptr));
-                        bulk_commit();
-                    }
-                    ++n_stores;
-                } else if (lane < rows_valid) {
-                    uint4* d4 = reinterpret_cast<uint4*>(p.out + ((long long)slab0 + lane) * p.ldo + n);
-                    d4[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                    d4[1] = make_uint4(w[4], w[5], w[6], w[7]);
-                    if (left >= 32) {
-                        d4[2] = make_uint4(w[8], w[9], w[10], w[11]);
-                        d4[3] = make_uint4(w[12], w[13], w[14], w[15]);
-                    }
-                }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_remote(empty0 + acc * (uint32_t)sizeof(unsigned long long));
-            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
-        }
-        if (n_stores != 0 && lane == 0) bulk_wait_all0();
-        __syncwarp();
-    }
-
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();   // neither CTA's shared memory / barriers may go away while the other still uses them
-    if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)MX_TMEM_COLS) : "memory");
-    }
-}
-
-// ---- weight gradients on the pair kernel's machinery ------------------------------------------------------
-// dW[e] [M, N] = Q(A_e)^T Q(B_e) over the rows of expert e, both operands quantised along the token axis in blocks of 32
-// rows counted from the expert's first row and stored TRANSPOSED, contraction contiguous: codes [features, pitch] where
-// column slice_prefix[e] * 128 + i holds row offsets[e] + i of the packed tensor and every expert's columns are padded
-// with zero codes to a multiple of 128 -- so a K slice of 128 columns belongs to exactly one expert, both operands are
-// K-major like everywhere else in this file, and the ragged contraction needs no clearing of foreign rows in shared
-// memory.  The tile list is fixed (every expert x M tiles x N tiles); an expert's K slices are
-// [slice_prefix[e], slice_prefix[e+1]); a tile of an expert without rows skips the pipeline and its epilogue writes zeros.
-struct MxWgradCtl {
-    unsigned long long full[MXP_STAGES];
-    unsigned long long sf_full[MXP_STAGES];
-    unsigned long long empty[MXP_STAGES];
-    unsigned long long tmem_full[2];
-    unsigned long long tmem_empty[2];
-    unsigned long long drain;
-    unsigned long long drain_copy;
-    uint32_t tmem_base;
-    int abort_flag;
-    int stage_n[MXP_STAGES];
-    int32_t sp[MX_MAX_E + 1];   // slice_prefix
-};
-constexpr int MXW_SMEM_BYTES = MXP_STAGES * MXP_STAGE_BYTES + MXP_STAGING_BYTES + 1024 + (int)sizeof(MxWgradCtl);
-static_assert(MXW_SMEM_BYTES <= 232448, "exceeds the shared memory a CTA can opt in to");
-
-struct MxWgradParams {
-    const int32_t* slice_prefix;   // [E + 1], in 128-column slices
-    int E, M, m_tiles, n_tiles, n_cols, n_slices;   // n_slices: slices per row of the transposed codes (pitch / 128)
-    const uint32_t* sa;   // scale words of A [n_slices][M]
-    bf16* out;            // [E * M, n_cols]
-    long long ldo;
-};
-
-struct MxWgradTile {
-    int e, row0, n0, nt, width, k0, k_tiles;
-};
-__device__ __forceinline__ MxWgradTile mxw_decode(const MxWgradParams& p, const MxWgradCtl* ctl, long long t) {
-    const int per_e = p.m_tiles * p.n_tiles;
-    MxWgradTile tl;
-    tl.e = (int)(t / per_e);
-    const int local = (int)(t - (long long)tl.e * per_e);
-    tl.nt = local / p.m_tiles;   // column tile major inside an expert: the pairs running together share the B tile in L2
-    tl.row0 = (local - tl.nt * p.m_tiles) * MXP_ROWS;
-    tl.n0 = tl.nt * MXP_NT;
-    tl.width = min(MXP_NT, p.n_cols - tl.n0);
-    tl.k0 = ctl->sp[tl.e];
-    tl.k_tiles = ctl->sp[tl.e + 1] - tl.k0;
-    return tl;
-}
-
-__global__ void __launch_bounds__(MXP_THREADS, 1)
-mx_wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                    const __grid_constant__ CUtensorMap map_sfb, const __grid_constant__ CUtensorMap map_o,
-                    const MxWgradParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t tiles_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* tiles_ptr = smem_raw + (tiles_base - smem_u32(smem_raw));
-    MxWgradCtl* ctl = reinterpret_cast<MxWgradCtl*>(tiles_ptr + MXP_STAGES * MXP_STAGE_BYTES + MXP_STAGING_BYTES);
-    volatile int* abort_flag = &ctl->abort_flag;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = cluster_ctarank();   // 0 = the CTA that issues the MMAs
-    const long long first_tile = blockIdx.x >> 1, tile_stride = gridDim.x >> 1;
-
-    for (int e = threadIdx.x; e <= p.E; e += MXP_THREADS) ctl->sp[e] = p.slice_prefix[e];
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < MXP_STAGES; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 4);   // per CTA: the producer's arrive (with its byte count) + the scale warp's
-            mbar_init(smem_u32(&ctl->sf_full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), 1);
-        }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(smem_u32(&ctl->tmem_full[a]), 1);
-            mbar_init(smem_u32(&ctl->tmem_empty[a]), 2 * MXP_EPI_WARPS);
-        }
-        mbar_init(smem_u32(&ctl->drain), 1);
-        mbar_init(smem_u32(&ctl->drain_copy), 1);
-        ctl->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        prefetch_tmap(&map_a);
-        prefetch_tmap(&map_b);
-        prefetch_tmap(&map_sfb);
-        prefetch_tmap(&map_o);
-    }
-    __syncthreads();
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
-                     "r"((uint32_t)MX_TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();   // the other CTA's barriers and tensor memory exist from here on
-    tc_fence_after();
-    const uint32_t tmem_base = ctl->tmem_base;
-    const long long n_tiles_total = (long long)p.E * p.m_tiles * p.n_tiles;
-    const uint32_t full0 = map_to_cta(smem_u32(&ctl->full[0]), 0);   // full[] of the MMA-issuing CTA
-
-    if (warp == 0) {
-        // ================= producer (both CTAs; each fills its own ring) =================
-        if (lane == 0) {
-            uint32_t stage = 0, phase = 0, issued = 0;
-            bool ok = true;
-            for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
-                const MxWgradTile tl = mxw_decode(p, ctl, t);
-                const int sfb_row0 = tl.nt * p.n_slices + tl.k0;
-                const int b_row = tl.n0 + (int)rank * (tl.width >> 1);
+                const MxPairTile tl = mxp_decode<WGRAD>(p, ctl, t);
+                const int sfb_row0 = tl.sfb_row0;
+                const int b_row = tl.b_row + (int)rank * (tl.width >> 1);
                 for (int kt = 0; kt < tl.k_tiles; ++kt) {
                     if (!mx_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag)) { ok = false; break; }
 #ifdef MOE_TEST_HOOKS
@@ -906,11 +626,9 @@ mx_wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (rank == 0) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, n = MXP_NT;
             bool ok = true;
-            const long long per_e = (long long)p.m_tiles * p.n_tiles;
             for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
-                const int e_t = (int)(t / per_e);
-                const int k_tiles_t = ctl->sp[e_t + 1] - ctl->sp[e_t];
-                if (k_tiles_t == 0) continue;   // an expert without rows: the epilogue writes zeros on its own
+                const int k_tiles_t = mxp_k_tiles<WGRAD>(p, ctl, t);
+                if (k_tiles_t == 0) continue;   // (weight gradients) an expert without rows: the epilogue writes zeros on its own
                 if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * MXP_ACC_STRIDE;
@@ -949,17 +667,17 @@ mx_wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
-            const MxWgradTile tl = mxw_decode(p, ctl, t);
+            const MxPairTile tl = mxp_decode<WGRAD>(p, ctl, t);
             long long rows[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const long long r = (long long)tl.row0 + (int)rank * MX_BM + 32 * i + lane;
-                rows[i] = r < p.M ? r : p.M - 1;   // rows past the end are never stored; any valid address will do
+                rows[i] = r < p.sa_rows ? r : p.sa_rows - 1;   // rows past the end are never stored; any valid address will do
             }
             // the words of MX_SCALE_AHEAD slices are in flight at any time: one slice per global-load round trip would
             // bound the whole pipeline (the loads wait behind the operand traffic)
             auto load_slice = [&](int kt) {
-                const uint32_t* s = p.sa + (long long)(tl.k0 + kt) * p.M;
+                const uint32_t* s = p.sa + (long long)(tl.k0 + kt) * p.sa_rows;
                 return make_uint4(__ldg(s + rows[0]), __ldg(s + rows[1]), __ldg(s + rows[2]), __ldg(s + rows[3]));
             };
             uint4 q[MX_SCALE_AHEAD];
@@ -990,10 +708,8 @@ mx_wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         if (rank == 0 && lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            const long long per_e = (long long)p.m_tiles * p.n_tiles;
             for (long long t = first_tile; ok && t < n_tiles_total; t += tile_stride) {
-                const int e_t = (int)(t / per_e);
-                const int k_tiles_t = ctl->sp[e_t + 1] - ctl->sp[e_t];
+                const int k_tiles_t = mxp_k_tiles<WGRAD>(p, ctl, t);
                 for (int kt = 0; kt < k_tiles_t; ++kt) {
                     if (!mx_wait(smem_u32(&ctl->full[stage]), phase, abort_flag)) { ok = false; break; }
                     tc_fence_after();
@@ -1021,16 +737,16 @@ mx_wgrad_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_con
         const uint32_t empty0 = map_to_cta(smem_u32(&ctl->tmem_empty[0]), 0);
         uint32_t n_stores = 0, acc = 0, acc_phase = 0;
         for (long long t = first_tile; t < n_tiles_total; t += tile_stride) {
-            const MxWgradTile tl = mxw_decode(p, ctl, t);
+            const MxPairTile tl = mxp_decode<WGRAD>(p, ctl, t);
             const bool have_acc = tl.k_tiles != 0;
             if (have_acc) {
                 if (!__all_sync(0xffffffffu, mx_wait(smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag))) break;
                 tc_fence_after();
             }
             const uint32_t taddr = tmem_base + acc * MXP_ACC_STRIDE + ((uint32_t)(quarter * 32) << 16);
-            const int slab_local = tl.row0 + (int)rank * MX_BM + quarter * 32;   // row of this expert's [M, N] gradient
-            const int rows_valid = max(0, min(32, p.M - slab_local));
-            const int slab0 = tl.e * p.M + slab_local;                           // row of the [E * M, N] output
+            const int slab_in = tl.row0 + (int)rank * MX_BM + quarter * 32;   // first row of this warp's slab, as the A operand counts rows
+            const int rows_valid = max(0, min(32, tl.row_end - slab_in));
+            const int slab0 = slab_in + tl.out_shift;                         // ... and as the output does
 #pragma unroll 1
             for (int c = half; c < 8; c += 2) {
                 const int left = tl.width - 32 * c;   // columns of the tile from this block on (warp-uniform)
@@ -1289,6 +1005,13 @@ __global__ void __launch_bounds__(256) mx_quantize_w_transposed_kernel(const bf1
 
 
 // ---- token-axis quantiser (operands of the weight gradients) ---------------------------------------------
+// dW[e] [M, N] = Q(A_e)^T Q(B_e) over the rows of expert e, both operands quantised along the token axis in blocks of 32
+// rows counted from the expert's first row and stored TRANSPOSED, contraction contiguous: codes [features, pitch] where
+// column slice_prefix[e] * 128 + i holds row offsets[e] + i of the packed tensor and every expert's columns are padded
+// with zero codes to a multiple of 128 -- so a K slice of 128 columns belongs to exactly one expert, both operands are
+// K-major like everywhere else in this file, and the ragged contraction needs no clearing of foreign rows in shared
+// memory.  The tile list is fixed (every expert x M tiles x N tiles); an expert's K slices are
+// [slice_prefix[e], slice_prefix[e+1]); a tile of an expert without rows skips the pipeline and its epilogue writes zeros.
 // slice_prefix[e] = number of 128-row slices of the experts before e, every expert's rows rounded up to whole slices
 __global__ void __launch_bounds__(1024) mx_slice_prefix_kernel(const int32_t* __restrict__ offsets, int E, int32_t* __restrict__ sp) {
     __shared__ int32_t part[32];
@@ -1476,9 +1199,9 @@ int launch_mx_wgrad(long long R, int E, int M, int N, const uint8_t* a_codes_t, 
                         CU_TENSOR_MAP_SWIZZLE_NONE) ||
         !make_out_map(&o, dw, N, (uint64_t)E * M))
         return MOE_ERR_CUDA;
-    MxWgradParams p = {};
-    p.slice_prefix = reinterpret_cast<const int32_t*>(a_scales); p.E = E; p.M = M; p.m_tiles = m_tiles; p.n_tiles = n_tiles;
-    p.n_cols = N; p.n_slices = n_slices;
+    MxPairParams p = {};
+    p.prefix = reinterpret_cast<const int32_t*>(a_scales); p.E = E; p.M = M; p.m_tiles = m_tiles; p.n_tiles = n_tiles;
+    p.n_cols = N; p.n_slices = n_slices; p.sa_rows = M;
     p.sa = reinterpret_cast<const uint32_t*>(a_scales + MX_TOKENS_HEADER_BYTES); p.out = dw; p.ldo = N;
     static int grid_of_device[64] = {};
     int dev = 0;
@@ -1488,22 +1211,22 @@ int launch_mx_wgrad(long long R, int E, int M, int N, const uint8_t* a_codes_t, 
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(MXP_THREADS);
-    cfg.dynamicSmemBytes = MXW_SMEM_BYTES;
+    cfg.dynamicSmemBytes = MXP_SMEM_BYTES;
     cfg.attrs = attr; cfg.numAttrs = 1;
     if (grid_of_device[dev] == 0) {
-        if (cudaFuncSetAttribute(mx_wgrad_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MXW_SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(mx_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, MXP_SMEM_BYTES) != cudaSuccess)
             return MOE_ERR_CUDA;
         const int sms = sm_count();
         if (sms <= 0) return MOE_ERR_CUDA;
         cfg.gridDim = dim3(2 * (sms / 2));
         int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, mx_wgrad_pair_kernel, &cfg) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
+        if (cudaOccupancyMaxActiveClusters(&clusters, mx_pair_kernel<true>, &cfg) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
         if (clusters > sms / 2) clusters = sms / 2;
         grid_of_device[dev] = 2 * clusters;
     }
     cfg.gridDim = dim3(grid_of_device[dev]);
     cfg.stream = s;
-    if (cudaLaunchKernelEx(&cfg, mx_wgrad_pair_kernel, a, b, sfb, o, p) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, mx_pair_kernel<true>, a, b, sfb, o, p) != cudaSuccess) return MOE_ERR_CUDA;
     return check_launch();
 }
 
@@ -1523,7 +1246,7 @@ static int launch_mx_gemm_pair(long long R, int E, int n_feat, int k, const uint
         !make_out_map(&o, out, n_feat, (uint64_t)R))
         return MOE_ERR_CUDA;
     MxPairParams p = {};
-    p.offsets = offsets; p.E = E; p.k_tiles = k_tiles; p.n_tiles = n_tiles; p.n_cols = n_feat; p.R = R;
+    p.prefix = offsets; p.E = E; p.k_tiles = k_tiles; p.n_tiles = n_tiles; p.n_cols = n_feat; p.sa_rows = R;
     p.sa = reinterpret_cast<const uint32_t*>(a_scales); p.out = out; p.ldo = n_feat;
     static int grid_of_device[64] = {};
     int dev = 0;
@@ -1536,20 +1259,20 @@ static int launch_mx_gemm_pair(long long R, int E, int n_feat, int k, const uint
     cfg.dynamicSmemBytes = MXP_SMEM_BYTES;
     cfg.attrs = attr; cfg.numAttrs = 1;
     if (grid_of_device[dev] == 0) {
-        if (cudaFuncSetAttribute(mx_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MXP_SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(mx_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, MXP_SMEM_BYTES) != cudaSuccess)
             return MOE_ERR_CUDA;
         const int sms = sm_count();
         if (sms <= 0) return MOE_ERR_CUDA;
         // as many pairs as can be resident at once: a pair that had to wait for a free SM pair would double the duration
         cfg.gridDim = dim3(2 * (sms / 2));
         int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, mx_gemm_pair_kernel, &cfg) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
+        if (cudaOccupancyMaxActiveClusters(&clusters, mx_pair_kernel<false>, &cfg) != cudaSuccess || clusters <= 0) return MOE_ERR_CUDA;
         if (clusters > sms / 2) clusters = sms / 2;
         grid_of_device[dev] = 2 * clusters;
     }
     cfg.gridDim = dim3(grid_of_device[dev]);
     cfg.stream = s;
-    if (cudaLaunchKernelEx(&cfg, mx_gemm_pair_kernel, a, b, sfb, o, p) != cudaSuccess) return MOE_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, mx_pair_kernel<false>, a, b, sfb, o, p) != cudaSuccess) return MOE_ERR_CUDA;
     return check_launch();
 }
 
