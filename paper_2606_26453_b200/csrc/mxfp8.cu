@@ -836,7 +836,7 @@ __device__ __forceinline__ uint32_t mx_e4m3(float v) {
 
 // rows x n bf16 -> codes (same layout) and scales.  A warp takes two (row, 128-wide slice) units per load: lane l holds
 // the 8 elements 8l..8l+7 of the 256 contiguous ones (one 16-byte load), the 4 lanes of a block of 32 agree on its scale
-// through two shuffles; two such loads are in flight per lane.  The 4 scale bytes of a (row, slice) are one 32-bit word:
+// through two shuffles; four such loads are in flight per lane.  The 4 scale bytes of a (row, slice) are one 32-bit word:
 //   WEIGHTS = false (activations): word [slice][row];
 //   WEIGHTS = true  (weights whose contraction axis is contiguous, rows = E * n_feat, e.g. W_down read as [I, H] for the
 //                    data gradient): the word's place in each of the two weight-scale tilings.  The output may be a
@@ -847,7 +847,7 @@ template <bool WEIGHTS>
 __global__ void __launch_bounds__(256) mx_quantize_rows_kernel(const uint4* __restrict__ x, long long rows, int n, int n_feat,
                                                                int out_k_tiles, int out_kt0, uint2* __restrict__ codes,
                                                                uint8_t* __restrict__ scales, uint8_t* __restrict__ scales_pair) {
-    constexpr int U = 2;
+    constexpr int U = 4;
     const int lane = threadIdx.x & 31;
     const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -1118,7 +1118,7 @@ size_t mx_w_scale_bytes(int E, int n_feat, int k) {
 }
 
 static unsigned mx_row_quantiser_blocks(long long units) {
-    long long blocks = (units + 31) / 32;   // 8 warps x 4 units per block and pass
+    long long blocks = (units + 63) / 64;   // 8 warps x 8 units per block and pass
     const long long cap = (long long)sm_count() * 16;
     if (blocks > cap) blocks = cap;
     return (unsigned)(blocks < 1 ? 1 : blocks);
