@@ -376,10 +376,10 @@ __global__ void __launch_bounds__(kThreads) gather_sum_kernel(const uint4* __res
 // dy_perm[row_k, :] = w_k * dy[t, :]; dtopk_w[t,k] = <dy[t,:], y_perm[row_k,:]> (warp shuffles, then a
 // fixed-order sum over the block's warps: deterministic).  y_perm pieces are fetched four slots at a time
 // (three blocks per SM: with the 80 registers that allows nothing spills; at five blocks per SM the K = 8 kernel
-// spilled and ran 16 % slower inside a step).
+// spilled and ran 16 % slower inside a step; the instance for a run-time K keeps 32 accumulators and takes two blocks).
 // ------------------------------------------------------------------------------------------------
 template <int KT, bool WITH_DW>
-__global__ void __launch_bounds__(kThreads, 3) combine_bwd_kernel(const uint4* __restrict__ dy,
+__global__ void __launch_bounds__(kThreads, KT > 0 ? 3 : 2) combine_bwd_kernel(const uint4* __restrict__ dy,
                                                                   const uint4* __restrict__ y_perm,
                                                                   const float* __restrict__ topk_w,
                                                                   const int32_t* __restrict__ pair_to_row,
