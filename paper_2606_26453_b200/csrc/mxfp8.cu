@@ -830,9 +830,6 @@ __device__ __forceinline__ float mx_inv_scale(int s) {
 __device__ __forceinline__ uint32_t mx_e4m3x2(float lo, float hi) {
     return (uint32_t)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, __NV_E4M3);
 }
-__device__ __forceinline__ uint32_t mx_e4m3(float v) {
-    return (uint32_t)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
-}
 
 // rows x n bf16 -> codes (same layout) and scales.  A warp takes two (row, 128-wide slice) units per load: lane l holds
 // the 8 elements 8l..8l+7 of the 256 contiguous ones (one 16-byte load), the 4 lanes of a block of 32 agree on its scale
