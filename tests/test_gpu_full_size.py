@@ -144,7 +144,7 @@ def test_mxfp8_down_sampled_rows(full):
         pytest.skip("the block-scaled path takes widths that are multiples of 128")
     from paper_2606_26453_b200 import binding as B
     d = b.d
-    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
     hc, hs = u8(cfg.R * cfg.I), u8(B.moe_mxfp8_act_scale_bytes(d))
     wc, ws = u8(cfg.E * cfg.H * cfg.I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
     B.moe_mxfp8_quantize_h_act(d, b.h_act, hc, hs)
@@ -196,7 +196,7 @@ def test_mxfp8_other_gemms_sampled_rows(full):
     from paper_2606_26453_b200 import binding as B
     d = b.d
     R, E, H, I = cfg.R, cfg.E, cfg.H, cfg.I
-    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
     nan = lambda *shape: torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda")
     offsets = b.offsets.cpu().numpy()
     rng = np.random.default_rng(cfg.cfg_id + 11)
@@ -281,7 +281,7 @@ def test_mxfp8_weight_gradients_sampled_experts(full):
     from paper_2606_26453_b200 import binding as B
     d = b.d
     R, E, H, I = cfg.R, cfg.E, cfg.H, cfg.I
-    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
     tok = lambda n: (u8(B.moe_mxfp8_tokens_codes_bytes(d, n)), u8(B.moe_mxfp8_tokens_scale_bytes(d, n)))
     offsets = b.offsets.cpu().numpy()
     counts = np.diff(offsets)

@@ -1,4 +1,7 @@
-"""Block-scaled FP8 (MXFP8) down projection through the C ABI against the oracle's quantiser and quantised product.
+"""Block-scaled FP8 (MXFP8) calls through the C ABI against the oracle's quantiser and quantised products.
+
+Code and scale buffers start out as 0xFF bytes: as a scale that is NaN, so a kernel that consumed a byte its quantiser
+never wrote would poison its output.
 
 Integer results (element codes, scale bytes) are compared bit for bit: both sides decide them on exact values.  The GEMM
 is held to the per-call bound of the bf16 kernels against the EXACT product of the dequantised operands (products of
@@ -75,7 +78,7 @@ def test_quantisers_and_gemm_against_the_oracle(B, name):
     w = host["W_down"].copy()
     w[0, :32, 0] = 0.0
     h_dev, w_dev = Hh.to_dev_bf16(h), Hh.to_dev_bf16(w)
-    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
     hc, hs = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
     wc, ws = u8(E * H * I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
     n_single = E * (H // 128) * (I // 128) * 512
@@ -92,7 +95,7 @@ def test_quantisers_and_gemm_against_the_oracle(B, name):
     assert np.array_equal(_w_scales_from_layout(ws_host[:n_single], E, H, I), o_ws)
     want_pair, written = _w_scales_pair_layout(o_ws, E, H, I)
     assert np.array_equal(ws_host[n_single:][written], want_pair[written])
-    assert np.all(ws_host[n_single:][~written] == 0xAB)          # bytes no column owns are left alone
+    assert np.all(ws_host[n_single:][~written] == 0xFF)          # bytes no column owns are left alone
     assert np.array_equal(wc.cpu().numpy().reshape(E, H, I), o_wc)
     # the GEMM on the quantised operands
     yp = torch.full((R, H), float("nan"), dtype=torch.bfloat16, device="cuda")
@@ -130,7 +133,7 @@ def test_down_dgrad_quantisers_and_gemm_against_the_oracle(B, name):
     w = host["W_down"].copy()
     w[0, 0, :32] = 0.0
     dy_dev, w_dev = Hh.to_dev_bf16(dy), Hh.to_dev_bf16(w)
-    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
     dc, ds = u8(R * H), u8(B.moe_mxfp8_dy_scale_bytes(d))
     wc, ws = u8(E * I * H), u8(B.moe_mxfp8_w_down_dgrad_scale_bytes(d))
     n_single = E * (I // 128) * (H // 128) * 512
@@ -147,7 +150,7 @@ def test_down_dgrad_quantisers_and_gemm_against_the_oracle(B, name):
     assert np.array_equal(ws_host[:n_single], _w_scales_single_layout(o_ws, E, I, H))
     want_pair, written = _w_scales_pair_layout(o_ws, E, I, H)
     assert np.array_equal(ws_host[n_single:][written], want_pair[written])
-    assert np.all(ws_host[n_single:][~written] == 0xAB)
+    assert np.all(ws_host[n_single:][~written] == 0xFF)
     dh = torch.full((R, I), float("nan"), dtype=torch.bfloat16, device="cuda")
     off = torch.from_numpy(ref["offsets"]).cuda()
     B.moe_grouped_gemm_down_dgrad_mxfp8(d, dc, ds, wc, ws, off, dh)
@@ -175,7 +178,7 @@ def test_gateup_dgrad_quantisers_and_gemm_against_the_oracle(B, name):
     wg, wu = host["W_gate"].copy(), host["W_up"].copy() * 3.0
     wu = W.round_to_bf16(wu)
     dgu_dev, wg_dev, wu_dev = Hh.to_dev_bf16(dgu), Hh.to_dev_bf16(wg), Hh.to_dev_bf16(wu)
-    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
     gc, gs = u8(R * 2 * I), u8(B.moe_mxfp8_dgu_scale_bytes(d))
     wc, ws = u8(E * H * 2 * I), u8(B.moe_mxfp8_w_gateup_dgrad_scale_bytes(d))
     n_single = E * (H // 128) * (2 * I // 128) * 512
@@ -192,7 +195,7 @@ def test_gateup_dgrad_quantisers_and_gemm_against_the_oracle(B, name):
     assert np.array_equal(ws_host[:n_single], _w_scales_single_layout(o_ws, E, H, 2 * I))
     want_pair, written = _w_scales_pair_layout(o_ws, E, H, 2 * I)
     assert np.array_equal(ws_host[n_single:][written], want_pair[written])
-    assert np.all(ws_host[n_single:][~written] == 0xAB)
+    assert np.all(ws_host[n_single:][~written] == 0xFF)
     dx = torch.full((R, H), float("nan"), dtype=torch.bfloat16, device="cuda")
     off = torch.from_numpy(ref["offsets"]).cuda()
     B.moe_grouped_gemm_gateup_dgrad_mxfp8(d, gc, gs, wc, ws, off, dx)
@@ -218,7 +221,7 @@ def test_gateup_forward_and_fused_swiglu_quantiser_against_the_oracle(B, name):
     wg, wu = host["W_gate"].copy(), W.round_to_bf16(host["W_up"] * 2.0)
     wg[0, :32, 0] = 0.0
     x_dev, wg_dev, wu_dev = Hh.to_dev_bf16(x), Hh.to_dev_bf16(wg), Hh.to_dev_bf16(wu)
-    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
     xc, xs = u8(R * H), u8(B.moe_mxfp8_x_scale_bytes(d))
     wc, ws = u8(E * 2 * I * H), u8(B.moe_mxfp8_w_gateup_scale_bytes(d))
     n_single = E * (2 * I // 128) * (H // 128) * 512
@@ -236,7 +239,7 @@ def test_gateup_forward_and_fused_swiglu_quantiser_against_the_oracle(B, name):
     assert np.array_equal(ws_host[:n_single], _w_scales_single_layout(o_ws, E, 2 * I, H))
     want_pair, written = _w_scales_pair_layout(o_ws, E, 2 * I, H)
     assert np.array_equal(ws_host[n_single:][written], want_pair[written])
-    assert np.all(ws_host[n_single:][~written] == 0xAB)
+    assert np.all(ws_host[n_single:][~written] == 0xFF)
     gu = torch.full((R, 2 * I), float("nan"), dtype=torch.bfloat16, device="cuda")
     off = torch.from_numpy(ref["offsets"]).cuda()
     B.moe_grouped_gemm_gateup_mxfp8(d, xc, xs, wc, ws, off, gu)
@@ -305,7 +308,7 @@ def test_weight_gradients_token_quantiser_and_gemm_against_the_oracle(B, name):
     x[0, :] = 0.0                                              # a column block that starts with a zero row
     off = torch.from_numpy(offsets).cuda()
     P = ((R + 127) // 128) * 128 + 128 * E
-    u8 = lambda n: torch.full((n,), 0xAB, dtype=torch.uint8, device="cuda")
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
 
     def quantise(t_host, col0, n):
         t_dev = Hh.to_dev_bf16(t_host)
