@@ -484,6 +484,46 @@ def time_config(B, cfg, device, steps, warmup, dist=None, sample_clocks=True, mi
     return dict(wl=wl, buffers=b, total_ms=total_ms, per_call_ms=per_call, clocks=clocks, steps=steps)
 
 
+def time_permute_alone(B, device, names, reps=15):
+    """`moe_permute` outside the step, the way a data-movement kernel is usually judged: the chip idle for two seconds
+    first (boost clocks, no power cap), L2 flushed before every call (a 256 MiB fill), median of `reps` calls, per
+    workload.  Inside a step the same call runs at the SM clock the power cap leaves after a GEMM (per-call figures of
+    the step, `stream_calibration_in_step`)."""
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    out = {}
+    time.sleep(2.0)
+    for name in names:
+        cfg = W.CONFIGS[name]
+        idx, _ = W.make_routing(cfg)
+        idx = torch.from_numpy(idx).to(device)
+        x = torch.randn(cfg.T, cfg.H, device=device).to(torch.bfloat16)
+        d = B.dims(cfg.T, cfg.H, cfg.I, cfg.E, cfg.K)
+        xp = torch.empty((cfg.R, cfg.H), dtype=torch.bfloat16, device=device)
+        i32 = lambda n: torch.empty(n, dtype=torch.int32, device=device)
+        counts, offsets, r2p, p2r = i32(cfg.E), i32(cfg.E + 1), i32(cfg.R), i32(cfg.R)
+        ws = torch.empty(max(B.moe_permute_workspace_bytes(d), 16), dtype=torch.uint8, device=device)
+        call = lambda: B.moe_permute(d, x, idx, xp, counts, offsets, r2p, p2r, ws)
+        for _ in range(3):
+            call()
+        times = []
+        for _ in range(reps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            call()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = statistics.median(times)
+        gbs = call_bytes(cfg)["permute"] / (ms * 1e-3) / 1e9
+        out[name] = {"us": ms * 1e3, "gbs": gbs, "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS}
+        del x, xp, idx
+        torch.cuda.empty_cache()
+    if B.moe_device_status() != 0:
+        raise RuntimeError("device status word is set after the isolated permute calls")
+    return out
+
+
 def time_router(B, cfg, device, reps=30):
     """The router in front of the layer (outside the step the headline metric times): logits of the workload's own
     draw -> top-k indices and weights, and the backward to the logits.  Timed alone with CUDA events after
@@ -929,6 +969,7 @@ def run_ours(args):
         if router is not None:
             router["workload"] = router_cfg.name
             line["router"] = router
+        line["permute_alone"] = time_permute_alone(B, device, [cfg.name] + [n for n in args.also if n != cfg.name])
         line["stream_calibration"] = stream_calibration(device)
         line["gemm_calibration"] = gemm_calibration(device)
         if wl_host is not None:
