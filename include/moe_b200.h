@@ -221,9 +221,10 @@ int moe_router_topk(const moe_dims_t* dims, const float* logits, int32_t* topk_i
 int moe_router_topk_bwd(const moe_dims_t* dims, const int32_t* topk_idx, const float* topk_w,
                         const float* dtopk_w, float* dlogits, moe_stream_t stream);
 
-/* ---- block-scaled FP8 (MXFP8) down projection -------------------------------------------------
- * A lower-precision twin of moe_grouped_gemm_down on the block-scaled tensor-core path (the paper only names FP8
- * tensor-core paths among its micro-profiling tools; the format is the OCP Microscaling MXFP8 one): both operands
+/* ---- block-scaled FP8 (MXFP8) twins of the six grouped GEMMs ------------------------------------
+ * Lower-precision forms of the grouped GEMMs on the block-scaled tensor-core path (the paper only names FP8
+ * tensor-core paths among its micro-profiling tools; the format is the OCP Microscaling MXFP8 one).  Every call works
+ * on caller-owned code and scale buffers; outputs stay bf16, accumulation fp32.  First the down projection: both operands
  * as FP8 E4M3 codes with one E8M0 scale byte s (value 2^(s-127)) per 32 consecutive elements ALONG THE CONTRACTION
  * (I).  Scale of a block with largest magnitude a > 0: 2^(floor(log2 a) - 8), clamped to the E8M0 range; elements:
  * value / scale rounded to nearest even onto the E4M3 grid, magnitudes above 448 saturating; an all-zero block has
