@@ -1039,9 +1039,10 @@ __global__ void __launch_bounds__(1024) mx_slice_prefix_kernel(const int32_t* __
 
 // x [R, ld] bf16, columns [col0, col0 + n) -> codes_t [n, pitch] (transposed, zero-padded per expert), scale words
 // [pitch/128][n] (the operand as the M side) and scale blocks in the pair tiling [ceil(n/208)][pitch/128][1024] (the
-// operand as the N side).  One thread per (padded block of 32 rows, group of 8 features): a 16-byte load per row and
-// thread, 512 contiguous bytes per warp; the thread keeps the 32 x 8 values as loaded, finds the 8 block maxima, then
-// writes 32 code bytes per feature.
+// operand as the N side).  One thread per (128-column slice, group of 8 features): the slice's four blocks of 32 rows one
+// after the other -- a 16-byte load per row, 512 contiguous bytes per warp; the thread keeps the 32 x 8 values as
+// loaded, finds the 8 block maxima, writes 32 code bytes per feature -- then the four scale bytes of each feature as
+// one word into each of the two scale layouts.
 __global__ void __launch_bounds__(128) mx_quantize_tokens_kernel(const bf16* __restrict__ x, long long ld, int col0, int n,
                                                                  const int32_t* __restrict__ offsets, const int32_t* __restrict__ sp,
                                                                  int E, long long pitch, uint8_t* __restrict__ codes_t,
@@ -1049,8 +1050,7 @@ __global__ void __launch_bounds__(128) mx_quantize_tokens_kernel(const bf16* __r
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int groups = n >> 3;
     const int f0 = (int)(idx % groups) * 8;
-    const long long pb = idx / groups;                  // padded block of 32 rows
-    const int slice = (int)(pb >> 2);
+    const int slice = (int)(idx / groups);
     if (slice >= sp[E]) return;
     int lo = 0, hi = E;                                 // the expert whose slices hold `slice`: largest e with sp[e] <= slice
     while (hi - lo > 1) {                               // (experts without rows share their successor's prefix)
@@ -1058,50 +1058,61 @@ __global__ void __launch_bounds__(128) mx_quantize_tokens_kernel(const bf16* __r
         if (sp[mid] <= slice) lo = mid; else hi = mid;
     }
     const int e = lo;
-    const int local_block = (int)(pb - 4ll * sp[e]);
     const int n_e = offsets[e + 1] - offsets[e];
-    const int valid = max(0, min(32, n_e - 32 * local_block));
-    const uint4* src = reinterpret_cast<const uint4*>(x + ((long long)offsets[e] + 32ll * local_block) * ld + col0 + f0);
     const long long ld16 = ld >> 3;
-    uint4 raw[32];
+    uint32_t words[8];
 #pragma unroll
-    for (int j = 0; j < 32; ++j) raw[j] = j < valid ? __ldg(src + (long long)j * ld16) : make_uint4(0u, 0u, 0u, 0u);
-    float amax[8];
+    for (int q = 0; q < 8; ++q) words[q] = 0u;
+#pragma unroll 1
+    for (int blk = 0; blk < 4; ++blk) {
+        const int local_block = 4 * (slice - sp[e]) + blk;
+        const long long pb = 4ll * slice + blk;         // padded block of 32 rows
+        const int valid = max(0, min(32, n_e - 32 * local_block));
+        const uint4* src = reinterpret_cast<const uint4*>(x + ((long long)offsets[e] + 32ll * local_block) * ld + col0 + f0);
+        uint4 raw[32];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) amax[q] = 0.f;
+        for (int j = 0; j < 32; ++j) raw[j] = j < valid ? __ldg(src + (long long)j * ld16) : make_uint4(0u, 0u, 0u, 0u);
+        float amax[8];
 #pragma unroll
-    for (int j = 0; j < 32; ++j) {
-        const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw[j]);
+        for (int q = 0; q < 8; ++q) amax[q] = 0.f;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[q]));
-            amax[2 * q] = fmaxf(amax[2 * q], fabsf(v.x));
-            amax[2 * q + 1] = fmaxf(amax[2 * q + 1], fabsf(v.y));
+        for (int j = 0; j < 32; ++j) {
+            const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw[j]);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[q]));
+                amax[2 * q] = fmaxf(amax[2 * q], fabsf(v.x));
+                amax[2 * q + 1] = fmaxf(amax[2 * q + 1], fabsf(v.y));
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int se = mx_scale_exp(amax[q]);
+            const float inv = mx_inv_scale(se);
+            uint32_t out[8];
+#pragma unroll
+            for (int g = 0; g < 8; ++g) {      // rows 4g .. 4g+3 of feature f0 + q
+                float v[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const uint32_t w = reinterpret_cast<const uint32_t*>(&raw[4 * g + t])[q >> 1];
+                    v[t] = __uint_as_float((q & 1) ? (w & 0xffff0000u) : (w << 16));      // bf16 -> fp32 is a shift
+                }
+                out[g] = mx_e4m3x2(v[0] * inv, v[1] * inv) | (mx_e4m3x2(v[2] * inv, v[3] * inv) << 16);
+            }
+            uint4* dst = reinterpret_cast<uint4*>(codes_t + (long long)(f0 + q) * pitch + pb * 32);
+            dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
+            dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
+            words[q] |= (uint32_t)(se + 127) << (8 * blk);
         }
     }
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
         const int f = f0 + q;
-        const int se = mx_scale_exp(amax[q]);
-        const float inv = mx_inv_scale(se);
-        uint32_t out[8];
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {      // rows 4g .. 4g+3 of feature f
-            float v[4];
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                const uint32_t w = reinterpret_cast<const uint32_t*>(&raw[4 * g + t])[q >> 1];
-                v[t] = __uint_as_float((q & 1) ? (w & 0xffff0000u) : (w << 16));      // bf16 -> fp32 is a shift
-            }
-            out[g] = mx_e4m3x2(v[0] * inv, v[1] * inv) | (mx_e4m3x2(v[2] * inv, v[3] * inv) << 16);
-        }
-        uint4* dst = reinterpret_cast<uint4*>(codes_t + (long long)f * pitch + pb * 32);
-        dst[0] = make_uint4(out[0], out[1], out[2], out[3]);
-        dst[1] = make_uint4(out[4], out[5], out[6], out[7]);
-        const uint8_t sbyte = (uint8_t)(se + 127);
-        sa_words[((long long)slice * n + f) * 4 + (pb & 3)] = sbyte;
+        *reinterpret_cast<uint32_t*>(sa_words + ((long long)slice * n + f) * 4) = words[q];
         const int nt = f / MXP_NT, c = f % MXP_NT;
-        sb_atoms[((long long)nt * (pitch >> 7) + slice) * 1024 + (c >> 7) * 512 + (c % 32) * 16 + ((c % 128) / 32) * 4 + (pb & 3)] = sbyte;
+        *reinterpret_cast<uint32_t*>(sb_atoms + ((long long)nt * (pitch >> 7) + slice) * 1024 + (c >> 7) * 512 + (c % 32) * 16 +
+                                     ((c % 128) / 32) * 4) = words[q];
     }
 }
 
@@ -1175,7 +1186,7 @@ int launch_mx_quantize_tokens(long long R, int E, const bf16* x, long long ld, i
     mx_slice_prefix_kernel<<<1, 1024, 0, s>>>(offsets, E, sp);
     int st_ = check_launch();
     if (st_ != MOE_OK) return st_;
-    const long long total = (pitch / 32) * (n / 8);
+    const long long total = (pitch / 128) * (n / 8);
     mx_quantize_tokens_kernel<<<(unsigned)((total + 127) / 128), 128, 0, s>>>(x, ld, col0, n, offsets, sp, E, pitch, codes_t, sa, sb);
     return check_launch();
 }
