@@ -278,7 +278,8 @@ def time_fp8_step(B, cfg, res, device, min_seconds=0.5):
     if B.moe_device_status() != 0:
         raise RuntimeError("device status word is set after the FP8 step")
     rel = lambda a, r: float((a.float() - r.float()).norm() / r.float().norm())
-    return {"ms_per_step_weights_quantised_outside": ms_out, "ms_per_step_weights_quantised_every_step": ms_in,
+    return {"layer_tflops_weights_quantised_outside": cfg.flops_fwd_bwd / (ms_out * 1e-3) / 1e12,
+            "ms_per_step_weights_quantised_outside": ms_out, "ms_per_step_weights_quantised_every_step": ms_in,
             "bf16_ms_per_step": res["total_ms"] / res["steps"], "gpu_launches_per_step": 16,
             "rel_frobenius_to_bf16_step": {"Y": rel(y_fp8, b.y), "dX": rel(dx_fp8, b.dx)},
             "note": "15 library calls (permute is two launches); the three activation quantisers and the forward SwiGLU are "
