@@ -619,10 +619,9 @@ mx_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (warp == 1) {
         // ================= MMA issuer: the first CTA's warp 1 =================
-        // The whole warp runs the loop and waits; one elected lane issues the tcgen05 instructions.  With the loop
-        // under `if (lane == 0)` every operand of a tcgen05 instruction (descriptors, addresses: uniform registers) is
-        // computed in the per-thread datapath and moved over, and the thread needed ~600 cycles per K slice against
-        // 448 of the tensor pipe; in converged code the values live in uniform registers from the start.
+        // The whole warp runs the loop and takes every wait's verdict together; one elected lane issues the tcgen05
+        // instructions.  (Measured against the same loop under `if (lane == 0)`: no difference in time -- the 60-85
+        // cycles a tcgen05 instruction costs its issuer are not operand marshalling.)
         if (rank == 0) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0, n = MXP_NT;
             bool ok = true;
