@@ -389,7 +389,9 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // What bounds it (cycle counters, throw-away builds): every tcgen05 instruction costs its issuing thread 60-85 cycles
 // whatever its size, so a K slice (wait, four MMAs, commit) takes the MMA warp ~470 cycles -- more than the ~420 the
 // tensor pipe needs for four N = 208 MMAs.  With the three scale copies in the same thread it was ~770; with two or four
-// scale slots the chain MMA -> stage released -> copies -> MMA set the pace instead (~510).
+// scale slots the chain MMA -> stage released -> copies -> MMA set the pace instead (~510).  In the full kernel a slice
+// takes ~590 cycles: operand reads by the tensor core and fills by the TMA unit together ask shared memory for ~140 bytes
+// per cycle at this tile width (halving the waits and commits per slice changed nothing).
 constexpr int MXP_NT = 208;                 // tile columns over the pair
 constexpr int MXP_ROWS = 2 * MX_BM;         // tile rows over the pair
 constexpr int MXP_STAGES = 6;
