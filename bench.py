@@ -54,6 +54,12 @@ NCU_TRAFFIC = {
     ("imbalanced", "down_wgrad"): (4209.6e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
     ("imbalanced", "gateup_dgrad"): (6412.4e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
     ("imbalanced", "gateup_wgrad"): (8502.4e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("few_large", "gateup_swiglu"): (3594.8e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("few_large", "down"): (2325.6e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("few_large", "down_dgrad"): (1500.0e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("few_large", "down_wgrad"): (1607.2e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("few_large", "gateup_dgrad"): (4612.4e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
+    ("few_large", "gateup_wgrad"): (2831.6e6, "ncu on a 1/4 copy (tokens and experts divided by 4), scaled x 4"),
     ("fine_grained", "gateup_swiglu"): (1029.0e6, "ncu capture of the full-size workload"),
     ("fine_grained", "down"): (525.0e6, "ncu capture of the full-size workload"),
     ("fine_grained", "down_wgrad"): (497.6e6, "ncu capture of the full-size workload"),
