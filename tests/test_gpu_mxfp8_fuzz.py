@@ -115,3 +115,41 @@ def test_random_shapes_all_six_fp8_gemms(seed):
     close(dwu, want[:, :, I:], "dW_up")
     for e in np.flatnonzero(np.diff(offsets) == 0):
         assert not bool(dwd[e].any()) and not bool(dwg[e].any()) and not bool(dwu[e].any()), tag
+
+
+def test_many_tiny_experts():
+    """1024 experts (the largest count the library takes) with 0..5 rows each, and a single expert holding everything:
+    the expert tables, the slice prefix and the fixed tile list of the weight gradients at their limits."""
+    from paper_2606_26453_b200 import binding as B
+    B.load_library()
+    rng = np.random.default_rng(99)
+    for counts in (list(rng.integers(0, 6, size=1024)), [777]):
+        H, I, K = 128, 256, 1
+        cfg, host = Hh.ragged_workload(counts, K=K, H=H, I=I, seed=77)
+        dev = Hh.device_workload(host)
+        b = Hh.run_cuda_layer(dev, cfg.E)
+        d = b.d
+        R, E = cfg.R, cfg.E
+        offsets = b.offsets.cpu().numpy()
+        u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
+        nan = lambda *shape: torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+        hc, hs = u8(R * I), u8(B.moe_mxfp8_act_scale_bytes(d))
+        wc, ws = u8(E * H * I), u8(B.moe_mxfp8_w_down_scale_bytes(d))
+        yq = nan(R, H)
+        B.moe_mxfp8_quantize_h_act(d, b.h_act, hc, hs)
+        B.moe_mxfp8_quantize_w_down(d, dev["W_down"], wc, ws)
+        B.moe_grouped_gemm_down_mxfp8(d, hc, hs, wc, ws, b.offsets, yq)
+        tok = lambda n: (u8(B.moe_mxfp8_tokens_codes_bytes(d, n)), u8(B.moe_mxfp8_tokens_scale_bytes(d, n)))
+        (ac, asc), (bc, bsc) = tok(I), tok(H)
+        B.moe_mxfp8_quantize_tokens(d, b.h_act, I, 0, I, b.offsets, ac, asc)
+        B.moe_mxfp8_quantize_tokens(d, b.dy_perm, H, 0, H, b.offsets, bc, bsc)
+        dwd = nan(E, I, H)
+        B.moe_grouped_gemm_down_wgrad_mxfp8(d, ac, asc, bc, bsc, dwd)
+        torch.cuda.synchronize()
+        assert B.moe_device_status() == 0
+        Hh.assert_close(Hh.to_np64(yq), O.down_mxfp8(Hh.to_np64(b.h_act), host["W_down"], offsets), f"Y_perm (MXFP8), E={E}",
+                        rel_fro=Hh.PER_CALL_FROBENIUS)
+        Hh.assert_close(Hh.to_np64(dwd), O.wgrad_mxfp8(Hh.to_np64(b.h_act), Hh.to_np64(b.dy_perm), offsets),
+                        f"dW_down (MXFP8), E={E}", rel_fro=Hh.PER_CALL_FROBENIUS)
+        for e in np.flatnonzero(np.diff(offsets) == 0):
+            assert not bool(dwd[e].any())
