@@ -31,8 +31,11 @@ permute/unpermute, empty-expert zeros; for the router: a per-row selection loop,
 shift invariance, the all-ties closed form, finite differences; for the fused down-dgrad + SwiGLU backward:
 autograd with respect to the saved pre-activations; for the block-scaled FP8 quantiser: the round trip of all 254
 finite codes, a library FP8 cast inside the range, hand-built blocks for the scale choice, ties and saturation,
-the half-ulp error bound, idempotence, and per-element products written out by hand.  No function here is
-"parity unpinned".
+the half-ulp error bound, idempotence; for the six quantised GEMMs (`gateup_mxfp8`, `down_mxfp8`, `down_dgrad_mxfp8`,
+`gateup_dgrad_mxfp8`, `wgrad_mxfp8`) and `swiglu_fwd`: per-element products with the quantiser applied by hand to each
+operand vector (expert-aligned row blocks for the weight gradients), equality with the pinned bf16-path function on
+representable operands, detectably different results for a transposed or swapped operand, a library SiLU.  No function
+here is "parity unpinned".
 """
 from __future__ import annotations
 
