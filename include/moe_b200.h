@@ -293,6 +293,10 @@ int moe_mxfp8_quantize_w_gateup_dgrad(const moe_dims_t* dims, const void* w_gate
 int moe_grouped_gemm_gateup_dgrad_mxfp8(const moe_dims_t* dims, const void* dgu_codes, const void* dgu_scales,
                                         const void* w_codes, const void* w_scales, const int32_t* offsets,
                                         void* dx_perm, moe_stream_t stream);
+/* moe_swiglu_bwd with the quantiser of its result fused in: dgu exactly as moe_swiglu_bwd writes it, and dgu_codes /
+ * dgu_scales = what moe_mxfp8_quantize_dgu makes of that dgu (one pass over the data instead of two). */
+int moe_swiglu_bwd_mxfp8(const moe_dims_t* dims, const void* dh_act, const void* gu_saved, void* dgu, void* dgu_codes,
+                         void* dgu_scales, moe_stream_t stream);
 
 /* The gate/up projection itself: gu[r,:] = [ dequant(x row r) . dequant(w_gate[e]) | dequant(x row r) . dequant(w_up[e]) ],
  * contraction over H; every gate / up feature has its own scales along H.  The SwiGLU activation is a second call that

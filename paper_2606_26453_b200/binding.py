@@ -32,7 +32,7 @@ EXPORTS = [
     "moe_mxfp8_x_scale_bytes", "moe_mxfp8_w_gateup_scale_bytes", "moe_mxfp8_quantize_x_perm", "moe_mxfp8_quantize_w_gateup",
     "moe_grouped_gemm_gateup_mxfp8", "moe_swiglu_mxfp8",
     "moe_mxfp8_tokens_codes_bytes", "moe_mxfp8_tokens_scale_bytes", "moe_mxfp8_quantize_tokens",
-    "moe_grouped_gemm_down_wgrad_mxfp8", "moe_grouped_gemm_gateup_wgrad_mxfp8",
+    "moe_grouped_gemm_down_wgrad_mxfp8", "moe_grouped_gemm_gateup_wgrad_mxfp8", "moe_swiglu_bwd_mxfp8",
 ]
 
 
@@ -107,6 +107,7 @@ def load_library() -> ctypes.CDLL:
             "moe_mxfp8_quantize_w_gateup": [dp, p, p, p, p, p],
             "moe_grouped_gemm_gateup_mxfp8": [dp, p, p, p, p, p, p, p],
             "moe_swiglu_mxfp8": [dp, p, p, p, p, p],
+            "moe_swiglu_bwd_mxfp8": [dp, p, p, p, p, p, p],
             "moe_mxfp8_quantize_tokens": [dp, p, ctypes.c_int, ctypes.c_int, ctypes.c_int, p, p, p, p],
             "moe_grouped_gemm_down_wgrad_mxfp8": [dp, p, p, p, p, p, p],
             "moe_grouped_gemm_gateup_wgrad_mxfp8": [dp, p, p, p, p, p, p, p, p, p],
@@ -354,6 +355,11 @@ def moe_grouped_gemm_down_wgrad_mxfp8(d, h_codes_t, h_scales, dy_codes_t, dy_sca
 def moe_grouped_gemm_gateup_wgrad_mxfp8(d, x_codes_t, x_scales, dg_codes_t, dg_scales, du_codes_t, du_scales, dw_gate, dw_up):
     _call("moe_grouped_gemm_gateup_wgrad_mxfp8", ctypes.byref(d), _ptr(x_codes_t), _ptr(x_scales), _ptr(dg_codes_t),
           _ptr(dg_scales), _ptr(du_codes_t), _ptr(du_scales), _ptr(dw_gate), _ptr(dw_up), _stream())
+
+
+def moe_swiglu_bwd_mxfp8(d, dh_act, gu_saved, dgu, dgu_codes, dgu_scales):
+    _call("moe_swiglu_bwd_mxfp8", ctypes.byref(d), _ptr(dh_act), _ptr(gu_saved), _ptr(dgu), _ptr(dgu_codes), _ptr(dgu_scales),
+          _stream())
 
 
 def moe_layer_fwd_bwd_host(d, x_host, topk_idx_host, topk_w_host, dy_host, w_gate, w_up, w_down, y_host, dx_host,

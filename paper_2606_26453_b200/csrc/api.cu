@@ -460,6 +460,18 @@ int moe_swiglu_mxfp8(const moe_dims_t* dims, const void* gu, void* h_act, void* 
                                      static_cast<uint8_t*>(h_scales), st(stream));
 }
 
+int moe_swiglu_bwd_mxfp8(const moe_dims_t* dims, const void* dh_act, const void* gu_saved, void* dgu, void* dgu_codes,
+                         void* dgu_scales, moe_stream_t stream) {
+    int s = check_mx_dims(dims);
+    if (s != MOE_OK) return s;
+    const void* const req[] = {dh_act, gu_saved, dgu, dgu_codes, dgu_scales};
+    const void* const opt[] = {nullptr};
+    s = check_ptrs(req, opt);
+    if (s != MOE_OK) return s;
+    return launch_mx_swiglu_bwd_quantize((long long)dims->T * dims->K, dims->I, cb(dh_act), cb(gu_saved), mb(dgu),
+                                         static_cast<uint8_t*>(dgu_codes), static_cast<uint8_t*>(dgu_scales), st(stream));
+}
+
 // ---- block-scaled FP8 weight gradients (contraction over the packed rows of each expert) ----
 static int check_tokens_args(const moe_dims_t* d, int n_features) {
     const int s = check_mx_dims(d);

@@ -72,6 +72,8 @@ int launch_mx_quantize_tokens(long long R, int E, const bf16* x, long long ld, i
 int launch_mx_wgrad(long long R, int E, int M, int N, const uint8_t* a_codes_t, const uint8_t* a_scales, const uint8_t* b_codes_t,
                     const uint8_t* b_scales, bf16* dw, cudaStream_t s);
 int launch_mx_swiglu_quantize(long long rows, int I, const bf16* gu, bf16* h_act, uint8_t* codes, uint8_t* scales, cudaStream_t s);
+int launch_mx_swiglu_bwd_quantize(long long rows, int I, const bf16* dh_act, const bf16* gu, bf16* dgu, uint8_t* codes,
+                                  uint8_t* scales, cudaStream_t s);
 int launch_mx_gemm(long long R, int E, int n_feat, int k, const uint8_t* a_codes, const uint8_t* a_scales, const uint8_t* b_codes,
                    const uint8_t* b_scales, const int32_t* offsets, bf16* out, cudaStream_t s);
 

@@ -957,6 +957,68 @@ __global__ void __launch_bounds__(256) mx_swiglu_quantize_kernel(const uint4* __
     }
 }
 
+// The SwiGLU backward (elementwise part of the gate/up backward) with the row quantiser of its result fused in:
+// dGU = [dg | du] [rows, 2I] bf16 exactly as moe_swiglu_bwd computes it, and the block-scaled FP8 codes and scale words of
+// those bf16 values along the 2I columns (the A operand of the FP8 gate/up dgrad).  One thread per 8 columns of a row
+// (its 8 gate and its 8 up columns), a half-warp per 128-wide slice of each half.
+__global__ void __launch_bounds__(256) mx_swiglu_bwd_quantize_kernel(const uint4* __restrict__ dh_act, const uint4* __restrict__ gu,
+                                                                     long long rows, int I, uint4* __restrict__ dgu,
+                                                                     uint2* __restrict__ codes, uint32_t* __restrict__ scales) {
+    const int lane = threadIdx.x & 31;
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int iv = I >> 3;                       // 16-byte pieces per half row (a multiple of 16)
+    if (i >= rows * iv) return;                  // whole half-warps leave together
+    const long long r = (rows * iv >> 32) == 0 ? (long long)((uint32_t)i / (uint32_t)iv) : i / iv;
+    const int c = (int)(i - r * iv);
+    const uint4 dhv = __ldg(dh_act + i), gv = __ldg(gu + r * (2 * iv) + c), uv = __ldg(gu + r * (2 * iv) + iv + c);
+    const uint32_t* dw = reinterpret_cast<const uint32_t*>(&dhv);
+    const uint32_t* gw = reinterpret_cast<const uint32_t*>(&gv);
+    const uint32_t* uw = reinterpret_cast<const uint32_t*>(&uv);
+    uint32_t og[4], ou[4];
+    float vg[8], vu[8], amax_g = 0.f, amax_u = 0.f;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float2 d2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&dw[j]));
+        const float2 g2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw[j]));
+        const float2 u2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&uw[j]));
+        const float s0 = __fdividef(1.f, 1.f + __expf(-g2.x)), s1 = __fdividef(1.f, 1.f + __expf(-g2.y));
+        og[j] = pack_bf16(d2.x * u2.x * s0 * (1.f + g2.x * (1.f - s0)), d2.y * u2.y * s1 * (1.f + g2.y * (1.f - s1)));
+        ou[j] = pack_bf16(d2.x * g2.x * s0, d2.y * g2.y * s1);
+        const float2 rg = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&og[j]));   // what dGU holds
+        const float2 ru = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&ou[j]));
+        vg[2 * j] = rg.x; vg[2 * j + 1] = rg.y; vu[2 * j] = ru.x; vu[2 * j + 1] = ru.y;
+        amax_g = fmaxf(amax_g, fmaxf(fabsf(rg.x), fabsf(rg.y)));
+        amax_u = fmaxf(amax_u, fmaxf(fabsf(ru.x), fabsf(ru.y)));
+    }
+    dgu[r * (2 * iv) + c] = make_uint4(og[0], og[1], og[2], og[3]);
+    dgu[r * (2 * iv) + iv + c] = make_uint4(ou[0], ou[1], ou[2], ou[3]);
+    const uint32_t half_mask = (lane & 16) ? 0xffff0000u : 0x0000ffffu;
+    amax_g = fmaxf(amax_g, __shfl_xor_sync(half_mask, amax_g, 1));
+    amax_g = fmaxf(amax_g, __shfl_xor_sync(half_mask, amax_g, 2));
+    amax_u = fmaxf(amax_u, __shfl_xor_sync(half_mask, amax_u, 1));
+    amax_u = fmaxf(amax_u, __shfl_xor_sync(half_mask, amax_u, 2));
+    const int se_g = mx_scale_exp(amax_g), se_u = mx_scale_exp(amax_u);
+    const float inv_g = mx_inv_scale(se_g), inv_u = mx_inv_scale(se_u);
+    uint2 cg, cu;
+    cg.x = mx_e4m3x2(vg[0] * inv_g, vg[1] * inv_g) | (mx_e4m3x2(vg[2] * inv_g, vg[3] * inv_g) << 16);
+    cg.y = mx_e4m3x2(vg[4] * inv_g, vg[5] * inv_g) | (mx_e4m3x2(vg[6] * inv_g, vg[7] * inv_g) << 16);
+    cu.x = mx_e4m3x2(vu[0] * inv_u, vu[1] * inv_u) | (mx_e4m3x2(vu[2] * inv_u, vu[3] * inv_u) << 16);
+    cu.y = mx_e4m3x2(vu[4] * inv_u, vu[5] * inv_u) | (mx_e4m3x2(vu[6] * inv_u, vu[7] * inv_u) << 16);
+    codes[r * (2 * iv) + c] = cg;
+    codes[r * (2 * iv) + iv + c] = cu;
+    const int base = lane & 16;
+    const uint32_t bg = (uint32_t)(se_g + 127), bu = (uint32_t)(se_u + 127);
+    const uint32_t word_g = __shfl_sync(half_mask, bg, base) | (__shfl_sync(half_mask, bg, base + 4) << 8) |
+                            (__shfl_sync(half_mask, bg, base + 8) << 16) | (__shfl_sync(half_mask, bg, base + 12) << 24);
+    const uint32_t word_u = __shfl_sync(half_mask, bu, base) | (__shfl_sync(half_mask, bu, base + 4) << 8) |
+                            (__shfl_sync(half_mask, bu, base + 8) << 16) | (__shfl_sync(half_mask, bu, base + 12) << 24);
+    if ((lane & 15) == 0) {
+        const int kt = c >> 4;                   // 128-wide slice inside the half
+        scales[(long long)kt * rows + r] = word_g;
+        scales[(long long)((I >> 7) + kt) * rows + r] = word_u;
+    }
+}
+
 // Weights whose OUTPUT-feature axis is contiguous: w [E, k, n] bf16 (W_down [E, I, H]; W_gate, W_up [E, H, I]) -> codes
 // transposed, contraction contiguous, as rows n_off .. n_off + n of [E, n_total, k] (W_gate and W_up stacked along the 2I
 // output features of the gate/up projection), and the scale bytes in both tilings.  One thread per (expert, block of
@@ -1157,6 +1219,15 @@ int launch_mx_swiglu_quantize(long long rows, int I, const bf16* gu, bf16* h_act
     mx_swiglu_quantize_kernel<<<(unsigned)blocks, 256, 0, s>>>(reinterpret_cast<const uint4*>(gu), rows, I,
                                                              reinterpret_cast<uint4*>(h_act), reinterpret_cast<uint2*>(codes),
                                                              reinterpret_cast<uint32_t*>(scales));
+    return check_launch();
+}
+
+int launch_mx_swiglu_bwd_quantize(long long rows, int I, const bf16* dh_act, const bf16* gu, bf16* dgu, uint8_t* codes,
+                                  uint8_t* scales, cudaStream_t s) {
+    const long long total = rows * (I / 8);
+    mx_swiglu_bwd_quantize_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(
+        reinterpret_cast<const uint4*>(dh_act), reinterpret_cast<const uint4*>(gu), rows, I, reinterpret_cast<uint4*>(dgu),
+        reinterpret_cast<uint2*>(codes), reinterpret_cast<uint32_t*>(scales));
     return check_launch();
 }
 

@@ -356,6 +356,31 @@ def test_weight_gradients_token_quantiser_and_gemm_against_the_oracle(B, name):
     assert np.linalg.norm(Hh.to_np64(dwg) - exact) / np.linalg.norm(exact) < 0.08
 
 
+@pytest.mark.parametrize("name", ["ragged", "wide", "pair_wide"])
+def test_swiglu_backward_with_fused_quantiser_equals_the_two_calls(B, name):
+    """moe_swiglu_bwd_mxfp8 = moe_swiglu_bwd followed by moe_mxfp8_quantize_dgu, bit for bit (dGU, codes, scales); dGU is
+    also held to the oracle's SwiGLU backward like the unfused call."""
+    counts, K, H, I = CASES[name]
+    cfg, host = Hh.ragged_workload(counts, K=K, H=H, I=I, seed=33)
+    ref = O.layer_fwd_bwd(host["X"], host["topk_idx"], host["topk_w"], host["W_gate"], host["W_up"], host["W_down"],
+                          host["dY"])
+    R = cfg.R
+    d = B.dims(cfg.T, H, I, cfg.E, K)
+    dh = Hh.to_dev_bf16(W.round_to_bf16(ref["dH_act"].astype(np.float32)))
+    gu = Hh.to_dev_bf16(W.round_to_bf16(ref["GU"].astype(np.float32)))
+    u8 = lambda n: torch.full((n,), 0xFF, dtype=torch.uint8, device="cuda")
+    nan = lambda *shape: torch.full(shape, float("nan"), dtype=torch.bfloat16, device="cuda")
+    dgu1, c1, s1 = nan(R, 2 * I), u8(R * 2 * I), u8(B.moe_mxfp8_dgu_scale_bytes(d))
+    B.moe_swiglu_bwd(d, dh, gu, dgu1)
+    B.moe_mxfp8_quantize_dgu(d, dgu1, c1, s1)
+    dgu2, c2, s2 = nan(R, 2 * I), u8(R * 2 * I), u8(B.moe_mxfp8_dgu_scale_bytes(d))
+    B.moe_swiglu_bwd_mxfp8(d, dh, gu, dgu2, c2, s2)
+    torch.cuda.synchronize()
+    assert B.moe_device_status() == 0
+    assert torch.equal(dgu1, dgu2) and torch.equal(c1, c2) and torch.equal(s1, s2)
+    Hh.assert_close(Hh.to_np64(dgu2), O.swiglu_bwd(Hh.to_np64(dh), Hh.to_np64(gu)), f"{name}: dGU", rel_fro=Hh.PER_CALL_FROBENIUS)
+
+
 def test_shapes_the_block_scaled_path_does_not_take_are_refused(B):
     d = B.dims(64, 192, 128, 2, 1)                   # H not a multiple of 128
     assert B.moe_mxfp8_act_scale_bytes(d) == 0
